@@ -191,7 +191,7 @@ def test_integer_log():
         e = v.bit_length() - 1
         frac = Fraction(v, 2 ** e) - 1                  # in [0,1)
         assert oracle.ilog(a) == 4 * e + math.floor(4 * frac)
-        assert 0 <= math.log2(v) - oracle.ilog(a) / 4 < 0.25 + 1e-9     # under-estimates log2 by < 1/4
+        assert 0 <= math.log2(v) - oracle.ilog(a) / 4 < 0.34             # under-estimates log2 by < 1/4 + 0.086
     ls = [oracle.ilog(a) for a in range(0, 5000)]
     assert all(b >= a for a, b in zip(ls, ls[1:]))     # monotone
 
