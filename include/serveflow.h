@@ -1,0 +1,273 @@
+/*
+ * serveflow.h - C ABI of the B200 (sm_100a) fast-slow flow-serving library.
+ *
+ * The library runs the data-parallel hot path of the fast-slow serving
+ * architecture of "ServeFlow: A Fast-Slow Model Architecture for Network Traffic
+ * Analysis": every flow is first answered by a cheap model on its first few
+ * packets; an uncertainty score decides which flows are assigned to a slow model
+ * that sees more packets of the same flow (Sec. 3.1, Fig. 4; Sec. 3.2).
+ *
+ * Conventions
+ *  - Every call returns an int status: SF_OK (0) or a negative SF_ERR_* code;
+ *    sf_strerror() names it.  Nothing aborts or throws across this boundary.
+ *  - Unless a parameter says "host", data pointers are DEVICE pointers owned by
+ *    the caller, read-only unless named *_out.  Outputs documented as nullable
+ *    are skipped when NULL.
+ *  - Calls enqueue work on the caller's stream (a cudaStream_t passed as void*,
+ *    NULL = the default stream) and do not synchronise, except where stated.
+ *  - Handles (sf_ctx, sf_forest, sf_slow, sf_table) are owned by the library,
+ *    built from HOST arrays that are copied and re-laid-out inside, and released
+ *    by the matching *_destroy.  A handle belongs to the device of its context.
+ *  - Arguments are validated on the host before anything is launched.  Device-side
+ *    conditions (capacity overflow, a full hash table, a wait that ran out) are
+ *    recorded in a device error word that sf_ctx_poll() reads; no kernel traps.
+ *  - There is no CPU fallback: without a CUDA device every compute call fails.
+ */
+#ifndef SERVEFLOW_H
+#define SERVEFLOW_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SF_OK                  0
+#define SF_ERR_ARG            -1   /* NULL where not allowed, size out of range, misaligned pointer */
+#define SF_ERR_ALLOC          -2   /* device or host allocation failed */
+#define SF_ERR_CUDA           -3   /* a CUDA runtime/driver call failed (sf_last_cuda_error) */
+#define SF_ERR_CAPACITY       -4   /* more flows were assigned than `capacity`; the list was clamped */
+#define SF_ERR_TABLE_FULL     -5   /* a key found no slot within the probe limit; its packet was dropped */
+#define SF_ERR_UNSUPPORTED    -6   /* shape outside what the kernels implement */
+#define SF_ERR_DEVICE_TIMEOUT -7   /* a bounded device-side wait gave up */
+
+/* enums passed as int */
+#define SF_RF           0          /* random forest: mean of leaf class-probability vectors */
+#define SF_GBDT         1          /* boosted trees, binary logistic: sum of leaf scalars (margin) */
+#define SF_LC_GT        0          /* assign iff 1 - max_c prob[c] > tau[argmax]  (Sec. 3.2, least confidence) */
+#define SF_ABSMARGIN_LT 1          /* assign iff |margin| < tau[0]  (|p-0.5| < 0.2  <=>  |margin| < ln(7/3)) */
+#define SF_MLP16        0          /* wide row = P packets x 16 fields */
+#define SF_CNN8         1          /* wide row = P positions x 8 channels (channels last) */
+#define SF_F32          0
+#define SF_BF16         1
+
+/* |margin| threshold equivalent to |sigmoid(margin) - 0.5| < 0.2: fp32(ln(0.7/0.3)) */
+#define SF_TAU_MARGIN_DEFAULT 0x1.b1d106p-1f
+
+typedef struct sf_ctx sf_ctx;
+typedef struct sf_forest sf_forest;
+typedef struct sf_slow sf_slow;
+typedef struct sf_table sf_table;
+
+const char* sf_strerror(int status);
+/* Text of the last CUDA error seen by this thread's last failing call (host string, never NULL). */
+const char* sf_last_cuda_error(void);
+/* Library version and the SM architecture it was compiled for ("sm_100a"). */
+const char* sf_version(void);
+
+/* ---- context ------------------------------------------------------------ */
+/* Creates a context on `device`: a device workspace of `workspace_bytes` (scan
+ * scratch, intermediates of sf_serve_batch; grown with a synchronising
+ * reallocation if a later call needs more), device counters and the error word.
+ * Fails with SF_ERR_CUDA when no device is present. */
+int  sf_ctx_create(sf_ctx** out, int device, size_t workspace_bytes);
+void sf_ctx_destroy(sf_ctx* ctx);
+
+typedef struct {
+    uint64_t n_flows;                  /* flows seen by sf_route / sf_serve_batch / the table */
+    uint64_t n_fast_done;              /* answered by the fast model */
+    uint64_t n_escalated;              /* assigned to the slow model */
+    uint64_t n_slow_done;              /* answered by the slow model */
+    uint64_t n_missed;                 /* dropped: table full */
+    uint64_t n_dropped_after_decision; /* packets of flows that already have their answer */
+    int32_t  device_error;             /* first SF_ERR_* recorded on the device, or 0 */
+    int32_t  reserved;
+} sf_counters;
+/* Synchronises `stream`, copies the counters to host memory and returns
+ * device_error (SF_OK if none).  `reset` != 0 clears counters and error word. */
+int  sf_ctx_poll(sf_ctx* ctx, sf_counters* host_out, int reset, void* stream);
+
+/* ---- packet planes -------------------------------------------------------- */
+/* Header planes of n_flows flows with a row pitch of pitch_pkts packets:
+ *   size     uint16[n][pitch]          packet length in bytes
+ *   iat_us   uint32[n][pitch]          inter-arrival time before the packet, microseconds
+ *   dir_bits uint32[n][ceil(pitch/32)] bit (i%32) of word (i/32) = direction of packet i
+ *   hdr      uint8 [n][pitch][hdr_bytes]  raw header bytes (only the wide rows use them; may be NULL otherwise)
+ *   n_valid  uint8 [n] or NULL         packets actually present (NULL = all)
+ * Rows must be 16-byte aligned: pitch*2 and pitch*4 multiples of 16 or the planes
+ * are read with narrower loads (any pitch is accepted; base pointers must be
+ * aligned to 16 bytes). */
+typedef struct {
+    const uint16_t* size;
+    const uint32_t* iat_us;
+    const uint32_t* dir_bits;
+    const uint8_t*  hdr;
+    const uint8_t*  n_valid;
+    uint32_t n_flows, pitch_pkts, hdr_bytes;
+} sf_packets;
+
+/* ---- S1: feature extraction ----------------------------------------------- */
+/* The pipeline's "feature computation" step (Sec. 1, Fig. 1) for a batch.  For
+ * each flow, F = 8*G statistics of the first min(N, n_valid) packets, feature
+ * 8g+k: group g = quantity x subset (g0 size/all, g1 iat/all, g2 size/fwd,
+ * g3 size/bwd, g4 iat/fwd, g5 iat/bwd, g6 size/turn, g7 iat/turn; fwd = dir bit 0,
+ * turn = direction differs from the previous packet), slot k = cnt, sum, min, max,
+ * mean, var (population), first, last.  Sums are exact integers (128-bit for the
+ * variance numerator) converted to fp32 once, round-to-nearest-even; mean =
+ * fp32(sum)/fp32(cnt); var = fp32(cnt*S2 - S1^2)/fp32(cnt^2); empty subset = zeros.
+ * feat_out: fp32[n_flows][F] row-major.  N in 1..32, N <= pitch, F in {8,16,..,64}. */
+int  sf_extract_features(sf_ctx* ctx, const sf_packets* pk, uint32_t N, uint32_t F,
+                         float* feat_out, void* stream);
+
+/* ---- S2: fast model (tree ensemble) ---------------------------------------- */
+/* Builds an ensemble of T complete binary trees of depth `depth` (heap order:
+ * children of node i are 2i+1, 2i+2) from HOST arrays fid uint16[T][2^d-1],
+ * thr fp32[T][2^d-1], leaf fp32[T][2^d][C] (SF_RF) or fp32[T][2^d] (SF_GBDT, C
+ * ignored and treated as 2 classes).  depth 1..12, F <= 64, C <= 16. */
+int  sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t depth, uint32_t F, uint32_t C,
+                      const uint16_t* fid_host, const float* thr_host, const float* leaf_host,
+                      sf_forest** out);
+void sf_forest_destroy(sf_forest* forest);
+/* The fast model of the cascade (Sec. 3.1) on n feature rows fp32[n][F].  At a
+ * node a flow goes LEFT iff x[fid] <= thr.  SF_RF: prob[c] = (sum over trees
+ * t = 0..T-1, in that order, fp32) of leaf[t][l_t][c], divided by fp32(T) ->
+ * out fp32[n][C].  SF_GBDT: margin = sum of leaf[t][l_t] in tree order ->
+ * out fp32[n].  leaf_idx_out (nullable): uint16[n][T]. */
+int  sf_fast_infer(sf_ctx* ctx, const sf_forest* forest, const float* feat, uint32_t n,
+                   float* prob_or_margin_out, uint16_t* leaf_idx_out, void* stream);
+
+/* ---- S3: uncertainty score, threshold, compaction, wide rows --------------- */
+typedef struct {
+    int rule;               /* SF_LC_GT | SF_ABSMARGIN_LT */
+    const float* tau;       /* device: fp32[C] per predicted class (all equal = universal threshold) for
+                               SF_LC_GT; fp32[1] for SF_ABSMARGIN_LT */
+    int wide_layout;        /* SF_MLP16 | SF_CNN8 */
+    int row_dtype;          /* SF_BF16 | SF_F32 */
+    uint32_t P;             /* packets per wide row (row width D = 16*P or 8*P) */
+    uint32_t P_real;        /* packets taken from the planes; positions P_real..P-1 are zero (0 = P) */
+    uint32_t capacity;      /* rows available in esc_ids_out / rows_out */
+} sf_route_cfg;
+/* Flow assignment (Sec. 3.2): score = LC(x) = 1 - max_y P(y|x) (or |margin|),
+ * fast label = argmax (lowest index on ties; margin > 0 for SF_GBDT), a flow is
+ * assigned to the slow model iff the score passes the threshold (strict
+ * comparison).  Assigned flow ids are written in ascending order to
+ * esc_ids_out[0..n_esc) and their count to *n_esc_out (device).  If `wide` and
+ * rows_out are given, each assigned flow's wide row is gathered and converted:
+ * per packet size*2^-11, L(iat)*2^-7 (L = integer piecewise-linear log2 of iat+1,
+ * 0..128), direction 0/1, header bytes*2^-8 (13 for SF_MLP16, 5 for SF_CNN8),
+ * rounded to bf16 (RNE) or kept fp32.  If more than `capacity` flows qualify the
+ * count saturates at capacity and the error word gets SF_ERR_CAPACITY.
+ * Nullable: rows_out (with wide), decision_out uint8[n], label_fast_out uint8[n],
+ * score_out fp32[n]. */
+int  sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* prob_or_margin, uint32_t n, uint32_t C,
+              const sf_packets* wide, uint32_t* esc_ids_out, uint32_t* n_esc_out, void* rows_out,
+              uint8_t* decision_out, uint8_t* label_fast_out, float* score_out, void* stream);
+
+/* Algorithm 1 (universal uncertainty thresholds) on HOST data: sorts a copy of
+ * the n validation scores ascending and returns, for each quantile
+ * q = q_num[j]/q_den, the score at 1-based index ceil(q*n).  Host-only helper. */
+int  sf_universal_thresholds(const float* scores_host, uint64_t n, const uint32_t* q_num_host,
+                             uint32_t q_den, uint32_t n_q, float* thresholds_host_out);
+
+/* ---- S4: slow model -------------------------------------------------------- */
+/* MLP h_{k+1} = ReLU(W_k h_k + b_k), logits = W_L h_L + b_L.  dims_host has
+ * n_layers+1 entries; W_host[k] is fp32 [dims[k+1]][dims[k]] (HOST), b_host[k]
+ * fp32[dims[k+1]].  SF_BF16: weights and hidden activations are bf16 (RNE),
+ * products accumulate in fp32 on the tensor cores, biases and logits fp32; needs
+ * hidden widths that are multiples of 64 and dims[0] a multiple of 64.  SF_F32:
+ * plain fp32.  The last layer may have any width up to 16 classes. */
+int  sf_mlp_create(sf_ctx* ctx, int dtype, uint32_t n_layers, const uint32_t* dims_host,
+                   const float* const* W_host, const float* const* b_host, sf_slow** out);
+/* 1-D CNN over L positions x Cin channels (channels last): conv(k) Cin->C1 + ReLU,
+ * conv(k) C1->C2 + ReLU (stride 1, zero "same" padding), mean over positions,
+ * linear C2->n_cls.  w1 [C1][k][Cin], w2 [C2][k][C1], w3 [n_cls][C2] (HOST, fp32).
+ * Implemented shape: L=128, Cin=8, C1=64, C2=128, k=5, n_cls<=16, SF_BF16. */
+int  sf_cnn_create(sf_ctx* ctx, int dtype, uint32_t L, uint32_t Cin, uint32_t C1, uint32_t C2, uint32_t k,
+                   uint32_t n_cls, const float* w1_host, const float* b1_host, const float* w2_host,
+                   const float* b2_host, const float* w3_host, const float* b3_host, sf_slow** out);
+void sf_slow_destroy(sf_slow* slow);
+/* The slow model of the cascade (Sec. 3.1) on the first *n_rows_dev rows (a DEVICE
+ * count, read by the kernels: no host round trip) of rows[capacity][D] (bf16 or
+ * fp32 as the model's dtype).  logits_out fp32[capacity][n_cls]; label_out
+ * uint8[capacity] (nullable) = argmax, lowest index on ties.  Rows at or beyond
+ * the count are not written. */
+int  sf_slow_infer(sf_ctx* ctx, const sf_slow* slow, const void* rows, const uint32_t* n_rows_dev,
+                   uint32_t capacity, float* logits_out, uint8_t* label_out, void* stream);
+
+/* ---- S1..S5: the whole cascade on one batch -------------------------------- */
+/* Features of fast_ctx (first N packets) -> fast model -> assignment -> wide rows
+ * of slow_ctx -> slow model -> merge: label_out[f] = slow label if assigned else
+ * fast label; stage_out[f] = 1 (fast) or 2 (slow); *n_esc_out (device, nullable)
+ * = number assigned.  Intermediates live in the context's workspace.  fast_ctx
+ * and slow_ctx may be the same planes.  Results equal the staged calls'. */
+int  sf_serve_batch(sf_ctx* ctx, const sf_forest* forest, const sf_slow* slow, const sf_packets* fast_ctx,
+                    uint32_t N, uint32_t F, const sf_packets* slow_ctx, const sf_route_cfg* cfg,
+                    uint8_t* label_out, uint8_t* stage_out, uint32_t* n_esc_out, void* stream);
+/* Same, but every plane pointer of fast_ctx / slow_ctx, cfg->tau, label_out,
+ * stage_out and n_esc_out are HOST pointers (pinned memory recommended): the
+ * planes are copied to device staging buffers owned by the context, the cascade
+ * runs, the three outputs are copied back, and the call returns after
+ * synchronising the stream. */
+int  sf_serve_batch_host(sf_ctx* ctx, const sf_forest* forest, const sf_slow* slow, const sf_packets* fast_ctx_host,
+                         uint32_t N, uint32_t F, const sf_packets* slow_ctx_host, const sf_route_cfg* cfg_host_tau,
+                         uint8_t* label_host_out, uint8_t* stage_host_out, uint32_t* n_esc_host_out, void* stream);
+/* Pointers into the workspace to the intermediates of the last sf_serve_batch on
+ * this context (for inspection and tests): any out pointer may be NULL. */
+int  sf_serve_batch_intermediates(sf_ctx* ctx, const float** feat, const float** fast_out, const uint32_t** esc_ids,
+                                  const void** rows, const float** logits, const uint8_t** label_fast,
+                                  const uint8_t** label_slow);
+
+/* ---- streaming: device-resident per-flow state table ----------------------- */
+/* One batch of interleaved packets, struct of arrays (device), n <= 65536. */
+typedef struct {
+    const uint32_t* src; const uint32_t* dst;     /* addresses */
+    const uint16_t* sport; const uint16_t* dport; /* ports */
+    const uint8_t*  proto;
+    const uint8_t*  dir;                          /* 0/1 */
+    const uint16_t* size;
+    const uint32_t* iat_us;
+    const uint8_t*  hdr;                          /* uint8[n][13] */
+    uint32_t n;
+} sf_pkt_batch;
+typedef struct {
+    uint32_t n_new_flows;        /* keys first seen in this batch */
+    uint32_t n_fast_fired;       /* flows that reached fast_pkts packets and were scored */
+    uint32_t n_fast_done;        /* ... of which answered by the fast model */
+    uint32_t n_escalated;        /* ... of which assigned to the slow model */
+    uint32_t n_slow_fired;       /* assigned flows that reached slow_pkts packets and were answered */
+    uint32_t n_dropped_after_decision;
+    uint32_t n_missed;           /* packets dropped because no slot was found */
+    uint32_t reserved;
+} sf_batch_result;
+typedef struct { uint32_t src, dst; uint16_t sport, dport; uint8_t proto; uint8_t pad[3]; } sf_key;
+typedef struct {
+    uint8_t found;      /* key present */
+    uint8_t stage;      /* 0 collecting, 1 answered by the fast model, 2 assigned and waiting, 3 answered by the slow model */
+    uint8_t label_fast, label_slow;
+    uint32_t n_pkts;    /* packets recorded */
+    float score;
+} sf_flow_result;
+/* The queues of Sec. 3.1 / 4.1 (first-packet features, later packets joined by
+ * flow id, escalations) replaced by one device hash table keyed by the 5-tuple:
+ * 2^log2_slots slots, linear probing with a bounded probe count; every flow keeps
+ * its first fast_pkts packets; flows assigned to the slow model get one of
+ * `slow_slabs` slabs holding slow_pkts packets. */
+int  sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_pkts, uint32_t slow_pkts,
+                     uint32_t slow_slabs, sf_table** out);
+void sf_table_destroy(sf_table* table);
+/* Ingests one batch in arrival order: look up / insert each key, append the packet
+ * to its flow's context, run S1-S3 (F features of the first fast_pkts packets) for
+ * flows that just reached fast_pkts packets, and S4 for assigned flows that just
+ * reached slow_pkts packets (wide row = slow_pkts real packets zero-padded to
+ * cfg->P).  *result_dev (device) receives the batch's counts. */
+int  sf_table_ingest(sf_ctx* ctx, sf_table* table, const sf_pkt_batch* batch, const sf_forest* forest,
+                     uint32_t F, const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_dev,
+                     void* stream);
+int  sf_table_lookup(sf_ctx* ctx, const sf_table* table, const sf_key* keys_dev, uint32_t n,
+                     sf_flow_result* out_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SERVEFLOW_H */

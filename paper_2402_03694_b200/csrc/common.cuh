@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of libserveflow.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/serveflow.h"
+
+#define SF_NUM_SMS_DEFAULT 148
+
+// Device-visible block: counters first (mirrors sf_counters), then scratch words.
+struct sf_dev_state {
+    sf_counters counters;
+    uint32_t    scan_total;      // number of assigned flows found by the last route
+    uint32_t    pad[15];
+};
+
+struct sf_ctx {
+    int device;
+    int num_sms;
+    // general workspace (bump-allocated per call)
+    char*  ws;
+    size_t ws_bytes;
+    size_t ws_used;
+    // fixed small state
+    sf_dev_state* d_state;
+    // staging for the host-pointer entry point
+    char*  stage;
+    size_t stage_bytes;
+    // intermediates of the last sf_serve_batch
+    const float* last_feat; const float* last_fast_out; const uint32_t* last_esc_ids;
+    const void* last_rows; const float* last_logits; const uint8_t* last_label_fast;
+    const uint8_t* last_label_slow;
+};
+
+struct sf_forest {
+    sf_ctx* ctx;
+    int kind;
+    uint32_t T, depth, F, C;
+    // nodes: per tree 2^depth entries of 8 bytes {thr, fid}, 1-based heap (entry 0 unused)
+    uint2* d_nodes;
+    // leaves: RF fp32[T][2^d][C]; GBDT fp32[T][2^d]
+    float* d_leaf;
+};
+
+enum { SF_SLOW_MLP = 0, SF_SLOW_CNN = 1 };
+
+struct sf_slow {
+    sf_ctx* ctx;
+    int arch;                 // SF_SLOW_MLP | SF_SLOW_CNN
+    int dtype;                // SF_F32 | SF_BF16
+    uint32_t n_layers;
+    uint32_t dims[9];
+    void*  d_W[8];            // bf16 or fp32 [out][in]
+    float* d_b[8];
+    // CNN
+    uint32_t L, Cin, C1, C2, k, n_cls;
+    void* d_w1; void* d_w2; void* d_w3;      // re-laid-out bf16 operands
+    float* d_b1; float* d_b2; float* d_b3;
+};
+
+// ---- helpers ---------------------------------------------------------------
+int  sf_set_cuda_error(cudaError_t e, const char* where);      // records text, returns SF_ERR_CUDA
+#define SF_CUDA(call) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) return sf_set_cuda_error(e__, #call); } while (0)
+#define SF_LAUNCH_CHECK(name) do { cudaError_t e__ = cudaGetLastError(); if (e__ != cudaSuccess) return sf_set_cuda_error(e__, name); } while (0)
+
+// workspace: reset at the start of a composite call, then bump-allocate (256-byte aligned)
+int   sf_ws_reserve(sf_ctx* ctx, size_t bytes);     // ensure capacity (may reallocate, synchronising)
+void  sf_ws_reset(sf_ctx* ctx);
+void* sf_ws_alloc(sf_ctx* ctx, size_t bytes);       // NULL if the reservation was too small
+static inline size_t sf_align256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+// ---- internal launchers (each validates nothing; callers did) ---------------
+int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st);
+int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st);
+// route scratch: block_counts uint32[ceil(n/1024)+1], decision bytes if the caller gave none
+size_t sf_route_scratch_bytes(uint32_t n);
+int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,
+                    const sf_packets* wide, uint32_t* esc_ids, uint32_t* n_esc, void* rows,
+                    uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st);
+size_t sf_slow_scratch_bytes(const sf_slow* s, uint32_t capacity);
+int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
+                   float* logits, uint8_t* label, void* scratch, cudaStream_t st);
+int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t n, const uint32_t* esc_ids,
+                    const uint32_t* n_esc, uint32_t capacity, const uint8_t* label_slow,
+                    uint8_t* label, uint8_t* stage, cudaStream_t st);
+
+// bf16 tensor-core layers (gemm_tc.cu)
+int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
+                        float* logits, uint8_t* label, void* scratch, cudaStream_t st);
+int sf_cnn_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
+                        float* logits, uint8_t* label, void* scratch, cudaStream_t st);
+int sf_cnn_prepare(sf_slow* s, const float* w1, const float* b1, const float* w2, const float* b2,
+                   const float* w3, const float* b3);
+
+// record a device-side condition once (first error wins)
+__device__ __forceinline__ void sf_dev_set_error(sf_dev_state* st, int code) {
+    atomicCAS(&st->counters.device_error, 0, code);
+}

@@ -1,0 +1,326 @@
+// S4 (bf16 MLP): hidden layers as tcgen05 GEMMs with TMEM accumulators fed by
+// TMA, and the narrow last layer (<= 16 classes) as a CUDA-core dot-product head.
+//
+// Hidden layer: out[r][o] = bf16( ReLU( sum_k A[r][k] * W[o][k] + b[o] ) ), r < *n_rows.
+// Persistent kernel, one CTA per SM, tile 128 x BN, K slices of 64 bf16 (one 128-byte
+// swizzled row per matrix row).  Warp roles:
+//   warp 0      TMA producer: loads the A and W slices of a ring of stages
+//   warp 1      allocates TMEM; one lane issues tcgen05.mma (4 per stage, K = 16 each)
+//   warps 2..5  epilogue: tcgen05.ld the fp32 accumulators (one TMEM lane quarter per
+//               warp), add bias, ReLU, round to bf16, 16-byte stores
+// Two accumulator buffers in TMEM (2 x BN columns) let the MMAs of tile i+1 overlap
+// the epilogue of tile i.  The row count lives in device memory, so routing and the
+// slow model need no host round trip; tiles past the count are never scheduled and
+// rows past it are never stored.  Every barrier wait is bounded: on a timeout the
+// block records SF_ERR_DEVICE_TIMEOUT, lets its copies land, frees TMEM and returns.
+#include "tc_common.cuh"
+
+namespace sftc {
+
+int encode_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
+                        uint32_t box_rows, uint32_t box_cols)
+{
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) return sf_set_cuda_error(e != cudaSuccess ? e : cudaErrorUnknown, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
+        fn = (encode_fn)p;
+    }
+    cuuint64_t gdim[2] = {cols, rows};
+    cuuint64_t gstride[1] = {cols * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return sf_set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return SF_OK;
+}
+
+}  // namespace sftc
+
+namespace {
+using namespace sftc;
+
+constexpr uint32_t BM = 128;
+constexpr uint32_t BK = 64;
+constexpr uint32_t kGemmThreads = 192;
+
+template <uint32_t BN> struct GemmCfg {
+    static constexpr uint32_t kStageBytesA = BM * BK * 2;
+    static constexpr uint32_t kStageBytesB = BN * BK * 2;
+    static constexpr uint32_t kStageBytes = kStageBytesA + kStageBytesB;
+    static constexpr uint32_t kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr uint32_t kTmemCols = 2 * BN;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct GemmBars {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <uint32_t BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                           const float* __restrict__ bias, const uint32_t* __restrict__ n_rows_dev,
+                           uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out, sf_dev_state* st)
+{
+    using Cfg = GemmCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* tiles = smem_raw + (base_u32 - smem_u32(smem_raw));
+    GemmBars* bars = reinterpret_cast<GemmBars*>(tiles + Cfg::kStages * Cfg::kStageBytes);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t n_rows = *n_rows_dev;
+    const uint32_t tiles_m = (n_rows + BM - 1) / BM;
+    const uint32_t tiles_n = N / BN;
+    const uint32_t n_tiles = tiles_m * tiles_n;
+    const uint32_t k_blocks = K / BK;
+
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < Cfg::kStages; s++) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        for (uint32_t b = 0; b < 2; b++) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], 4); }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&bars->tmem_base, Cfg::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmW);
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const uint32_t tm = tile / tiles_n, tn = tile - tm * tiles_n;
+                for (uint32_t kb = 0; kb < k_blocks; kb++) {
+                    if (!mbar_wait(&bars->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t* sA = tiles + stage * Cfg::kStageBytes;
+                    uint8_t* sB = sA + Cfg::kStageBytesA;
+                    mbar_expect_tx(&bars->full[stage], Cfg::kStageBytes);
+                    tma_load_2d(sA, &tmA, (int32_t)(kb * BK), (int32_t)(tm * BM), &bars->full[stage]);
+                    tma_load_2d(sB, &tmW, (int32_t)(kb * BK), (int32_t)(tn * BN), &bars->full[stage]);
+                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+            uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
+            bool ok = true;
+            for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(&bars->tmem_empty[buf], bphase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (uint32_t kb = 0; kb < k_blocks; kb++) {
+                    if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t aaddr = base_u32 + stage * Cfg::kStageBytes;
+                    const uint32_t baddr = aaddr + Cfg::kStageBytesA;
+#pragma unroll
+                    for (uint32_t k = 0; k < BK / 16; k++) {
+                        // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row
+                        const uint64_t adesc = make_smem_desc(aaddr + k * 32u, 16, 1024, 2);
+                        const uint64_t bdesc = make_smem_desc(baddr + k * 32u, 16, 1024, 2);
+                        umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&bars->empty[stage]);            // stage reusable once these MMAs retire
+                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(&bars->tmem_full[buf]);              // accumulator complete
+                buf ^= 1u; if (buf == 0) bphase ^= 1u;
+            }
+        }
+    } else {
+        const uint32_t quarter = warp & 3u;                        // TMEM lanes [32q, 32q+32)
+        uint32_t buf = 0, bphase = 0;
+        bool ok = true;
+        for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            const uint32_t tm = tile / tiles_n, tn = tile - tm * tiles_n;
+            // the whole warp takes the same way out: the TMEM loads below are warp-collective
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->tmem_full[buf], bphase, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t row = tm * BM + quarter * 32u + lane;
+            const uint32_t col0 = tn * BN;
+            const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BN;
+            __nv_bfloat16* orow = out + (size_t)row * N + col0;
+#pragma unroll 1
+            for (uint32_t c = 0; c < BN; c += 32) {
+                uint32_t v[32];
+                tmem_ld32(taddr + c, v);
+                tmem_ld_wait();
+                if (row < n_rows) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int j = 0; j < 16; j++) {
+                        float x0 = __uint_as_float(v[2 * j]) + __ldg(bias + col0 + c + 2 * j);
+                        float x1 = __uint_as_float(v[2 * j + 1]) + __ldg(bias + col0 + c + 2 * j + 1);
+                        __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(x0, 0.0f), fmaxf(x1, 0.0f));
+                        packed[j] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(orow + c);
+#pragma unroll
+                    for (int q = 0; q < 4; q++)
+                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+            buf ^= 1u; if (buf == 0) bphase ^= 1u;
+        }
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait ran out somewhere in this block: give copies in flight time to land
+        if (threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT);
+        __nanosleep(200000);
+        __syncthreads();
+    }
+    tc_fence_after();
+    if (warp == 1) { __syncwarp(); tmem_dealloc(tmem_base, Cfg::kTmemCols); }
+}
+
+// Last layer: logits[r][c] = sum_k h[r][k] * W[c][k] + b[c], c < C <= 16; one warp per row,
+// weights staged in shared memory, 16-byte loads, fp32 accumulation, warp-shuffle reduce.
+__global__ void __launch_bounds__(256)
+head_bf16_kernel(const __nv_bfloat16* __restrict__ h, const __nv_bfloat16* __restrict__ W, const float* __restrict__ b,
+                 const uint32_t* __restrict__ n_rows_dev, uint32_t K, uint32_t C,
+                 float* __restrict__ logits, uint8_t* __restrict__ label)
+{
+    extern __shared__ __align__(16) uint8_t smem_w[];
+    __nv_bfloat16* sW = reinterpret_cast<__nv_bfloat16*>(smem_w);
+    const uint32_t n_rows = *n_rows_dev;
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(W);
+        uint4* dst = reinterpret_cast<uint4*>(sW);
+        const uint32_t vecs = C * K / 8;
+        for (uint32_t v = threadIdx.x; v < vecs; v += blockDim.x) dst[v] = __ldg(src + v);
+    }
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rows; r += warps) {
+        float acc[16];
+#pragma unroll
+        for (int c = 0; c < 16; c++) acc[c] = 0.0f;
+        const __nv_bfloat16* hr = h + (size_t)r * K;
+        for (uint32_t k = lane * 8; k < K; k += 256) {
+            uint4 hv = __ldg(reinterpret_cast<const uint4*>(hr + k));
+            const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+            float2 x[4];
+#pragma unroll
+            for (int j = 0; j < 4; j++) x[j] = __bfloat1622float2(hp[j]);
+#pragma unroll
+            for (int c = 0; c < 16; c++) {
+                if ((uint32_t)c < C) {
+                    uint4 wv = *reinterpret_cast<const uint4*>(sW + (size_t)c * K + k);
+                    const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        float2 w = __bfloat1622float2(wp[j]);
+                        acc[c] = fmaf(x[j].x, w.x, acc[c]);
+                        acc[c] = fmaf(x[j].y, w.y, acc[c]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < 16; c++) {
+            if ((uint32_t)c < C) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xFFFFFFFFu, acc[c], o);
+            }
+        }
+        if (lane == 0) {
+            uint32_t a = 0; float mx = 0.0f;
+#pragma unroll
+            for (int c = 0; c < 16; c++) {
+                if ((uint32_t)c < C) {
+                    float v = acc[c] + b[c];
+                    logits[(size_t)r * C + c] = v;
+                    if (c == 0 || v > mx) { mx = v; a = c; }
+                }
+            }
+            if (label) label[r] = (uint8_t)a;
+        }
+    }
+}
+
+template <uint32_t BN>
+int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, const uint32_t* n_rows_dev,
+                uint32_t capacity, uint32_t N, uint32_t K, void* out, cudaStream_t st)
+{
+    using Cfg = GemmCfg<BN>;
+    CUtensorMap tmA, tmW;
+    int rc = encode_tmap_bf16_2d(&tmA, A, capacity, K, BM, BK);
+    if (rc != SF_OK) return rc;
+    rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
+    if (rc != SF_OK) return rc;
+    auto k = gemm_bias_relu_bf16_kernel<BN>;
+    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes));
+    uint32_t max_tiles = ((capacity + BM - 1) / BM) * (N / BN);
+    uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
+    k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
+                                                  reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state);
+    SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel");
+    return SF_OK;
+}
+
+}  // namespace
+
+int sf_launch_head_bf16(sf_ctx* ctx, const void* h, const void* W, const float* b, const uint32_t* n_rows_dev,
+                        uint32_t capacity, uint32_t K, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
+{
+    size_t smem = (size_t)C * K * 2;
+    SF_CUDA(cudaFuncSetAttribute(head_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    uint32_t blocks = (capacity + 7) / 8;
+    uint32_t maxb = (uint32_t)ctx->num_sms * 4;
+    if (blocks > maxb) blocks = maxb;
+    head_bf16_kernel<<<blocks, 256, smem, st>>>(reinterpret_cast<const __nv_bfloat16*>(h),
+                                                reinterpret_cast<const __nv_bfloat16*>(W), b, n_rows_dev, K, C, logits, label);
+    SF_LAUNCH_CHECK("head_bf16_kernel");
+    return SF_OK;
+}
+
+int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
+                        float* logits, uint8_t* label, void* scratch, cudaStream_t st)
+{
+    uint32_t maxh = 0;
+    for (uint32_t l = 1; l < s->n_layers; l++) if (s->dims[l] > maxh) maxh = s->dims[l];
+    char* h0 = reinterpret_cast<char*>(scratch);
+    char* h1 = h0 + sf_align256((size_t)capacity * maxh * 2);
+    const void* in = rows;
+    for (uint32_t l = 0; l + 1 < s->n_layers; l++) {
+        void* out = (l & 1) ? h1 : h0;
+        const uint32_t K = s->dims[l], N = s->dims[l + 1];
+        int rc;
+        if (N % 256 == 0)      rc = launch_gemm<256>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st);
+        else if (N % 128 == 0) rc = launch_gemm<128>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st);
+        else                   rc = launch_gemm<64>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st);
+        if (rc != SF_OK) return rc;
+        in = out;
+    }
+    const uint32_t L = s->n_layers - 1;
+    return sf_launch_head_bf16(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st);
+}

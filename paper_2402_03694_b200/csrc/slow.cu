@@ -1,0 +1,222 @@
+// S4: slow-model handles, the fp32 MLP path (plain FFMA tiles) and dispatch to
+// the bf16 tensor-core paths.
+#include "common.cuh"
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+namespace {
+
+// out[r][o] = act( sum_k in[r][k] * W[o][k] + b[o] ),  r < *n_rows_dev
+// 64x64 output tile, 16-deep K slices, 256 threads with 4x4 register tiles.
+template <bool RELU>
+__global__ void __launch_bounds__(256)
+dense_f32_kernel(const float* __restrict__ in, const float* __restrict__ W, const float* __restrict__ b,
+                 const uint32_t* __restrict__ n_rows_dev, uint32_t K, uint32_t N, float* __restrict__ out)
+{
+    __shared__ float As[16][64 + 4];
+    __shared__ float Bs[16][64 + 4];
+    const uint32_t n_rows = *n_rows_dev;
+    const uint32_t r0 = blockIdx.x * 64, o0 = blockIdx.y * 64;
+    if (r0 >= n_rows) return;
+    const uint32_t tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) acc[i][j] = 0.0f;
+    const uint32_t lr = threadIdx.x >> 2;          // 0..63: tile row loaded by this thread
+    const uint32_t lk = (threadIdx.x & 3) * 4;     // 0,4,8,12
+    for (uint32_t k0 = 0; k0 < K; k0 += 16) {
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            uint32_t k = k0 + lk + j;
+            uint32_t r = r0 + lr, o = o0 + lr;
+            As[lk + j][lr] = (r < n_rows && k < K) ? in[(size_t)r * K + k] : 0.0f;
+            Bs[lk + j][lr] = (o < N && k < K) ? W[(size_t)o * K + k] : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 16; k++) {
+            float a[4], w[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) a[i] = As[k][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; j++) w[j] = Bs[k][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; i++)
+#pragma unroll
+                for (int j = 0; j < 4; j++) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        uint32_t r = r0 + ty * 4 + i;
+        if (r >= n_rows) continue;
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            uint32_t o = o0 + tx * 4 + j;
+            if (o >= N) continue;
+            float v = acc[i][j] + b[o];
+            if (RELU) v = fmaxf(v, 0.0f);
+            out[(size_t)r * N + o] = v;
+        }
+    }
+}
+
+__global__ void argmax_kernel(const float* __restrict__ logits, const uint32_t* __restrict__ n_rows_dev,
+                              uint32_t C, uint8_t* __restrict__ label)
+{
+    const uint32_t n_rows = *n_rows_dev;
+    for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < n_rows; r += gridDim.x * blockDim.x) {
+        const float* p = logits + (size_t)r * C;
+        uint32_t a = 0; float mx = p[0];
+        for (uint32_t c = 1; c < C; c++) if (p[c] > mx) { mx = p[c]; a = c; }
+        label[r] = (uint8_t)a;
+    }
+}
+
+__global__ void count_slow_kernel(const uint32_t* __restrict__ n_rows_dev, sf_dev_state* st) {
+    atomicAdd((unsigned long long*)&st->counters.n_slow_done, (unsigned long long)*n_rows_dev);
+}
+
+void f32_to_bf16_host(const float* src, uint16_t* dst, size_t n) {
+    for (size_t i = 0; i < n; i++) {
+        uint32_t u; memcpy(&u, src + i, 4);
+        uint32_t low = u & 0xFFFFu, up = u >> 16;
+        if (low > 0x8000u || (low == 0x8000u && (up & 1u))) up++;
+        dst[i] = (uint16_t)up;
+    }
+}
+
+}  // namespace
+
+size_t sf_slow_scratch_bytes(const sf_slow* s, uint32_t capacity) {
+    if (s->arch == SF_SLOW_CNN) return sf_align256((size_t)capacity * s->C2 * sizeof(float)) + 256;
+    uint32_t maxh = 0;
+    for (uint32_t l = 1; l < s->n_layers; l++) if (s->dims[l] > maxh) maxh = s->dims[l];
+    size_t esz = s->dtype == SF_BF16 ? 2 : 4;
+    return 2 * sf_align256((size_t)capacity * maxh * esz) + 256;
+}
+
+int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
+                   float* logits, uint8_t* label, void* scratch, cudaStream_t st)
+{
+    if (capacity == 0) return SF_OK;
+    int rc;
+    if (s->arch == SF_SLOW_CNN) {
+        rc = sf_cnn_bf16_forward(ctx, s, rows, n_rows_dev, capacity, logits, label, scratch, st);
+    } else if (s->dtype == SF_BF16) {
+        rc = sf_mlp_bf16_forward(ctx, s, rows, n_rows_dev, capacity, logits, label, scratch, st);
+    } else {
+        uint32_t maxh = 0;
+        for (uint32_t l = 1; l < s->n_layers; l++) if (s->dims[l] > maxh) maxh = s->dims[l];
+        float* h0 = reinterpret_cast<float*>(scratch);
+        float* h1 = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + sf_align256((size_t)capacity * maxh * 4));
+        const float* in = reinterpret_cast<const float*>(rows);
+        for (uint32_t l = 0; l < s->n_layers; l++) {
+            const bool last = (l + 1 == s->n_layers);
+            float* out = last ? logits : ((l & 1) ? h1 : h0);
+            dim3 grid((capacity + 63) / 64, (s->dims[l + 1] + 63) / 64);
+            if (last) dense_f32_kernel<false><<<grid, 256, 0, st>>>(in, (const float*)s->d_W[l], s->d_b[l], n_rows_dev, s->dims[l], s->dims[l + 1], out);
+            else      dense_f32_kernel<true><<<grid, 256, 0, st>>>(in, (const float*)s->d_W[l], s->d_b[l], n_rows_dev, s->dims[l], s->dims[l + 1], out);
+            SF_LAUNCH_CHECK("dense_f32_kernel");
+            in = out;
+        }
+        if (label) {
+            uint32_t blocks = (capacity + 255) / 256; if (blocks > 1184) blocks = 1184;
+            argmax_kernel<<<blocks, 256, 0, st>>>(logits, n_rows_dev, s->dims[s->n_layers], label);
+            SF_LAUNCH_CHECK("argmax_kernel");
+        }
+        rc = SF_OK;
+    }
+    if (rc != SF_OK) return rc;
+    count_slow_kernel<<<1, 1, 0, st>>>(n_rows_dev, ctx->d_state);
+    SF_LAUNCH_CHECK("count_slow_kernel");
+    return SF_OK;
+}
+
+extern "C" int sf_mlp_create(sf_ctx* ctx, int dtype, uint32_t n_layers, const uint32_t* dims,
+                             const float* const* W, const float* const* b, sf_slow** out)
+{
+    if (!ctx || !dims || !W || !b || !out) return SF_ERR_ARG;
+    if (dtype != SF_F32 && dtype != SF_BF16) return SF_ERR_ARG;
+    if (n_layers < 1 || n_layers > 8) return SF_ERR_ARG;
+    for (uint32_t l = 0; l <= n_layers; l++) if (dims[l] == 0 || dims[l] > 65536) return SF_ERR_ARG;
+    for (uint32_t l = 0; l < n_layers; l++) if (!W[l] || !b[l]) return SF_ERR_ARG;
+    if (dims[n_layers] > 16) return SF_ERR_UNSUPPORTED;
+    if (dtype == SF_BF16) {
+        if (n_layers < 2) return SF_ERR_UNSUPPORTED;
+        for (uint32_t l = 0; l < n_layers; l++) if (dims[l] % 64 != 0) return SF_ERR_UNSUPPORTED;
+    }
+    SF_CUDA(cudaSetDevice(ctx->device));
+    sf_slow* s = new (std::nothrow) sf_slow();
+    if (!s) return SF_ERR_ALLOC;
+    memset(s, 0, sizeof(*s));
+    s->ctx = ctx; s->arch = SF_SLOW_MLP; s->dtype = dtype; s->n_layers = n_layers;
+    for (uint32_t l = 0; l <= n_layers; l++) s->dims[l] = dims[l];
+    cudaError_t e = cudaSuccess;
+    for (uint32_t l = 0; l < n_layers && e == cudaSuccess; l++) {
+        size_t cnt = (size_t)dims[l] * dims[l + 1];
+        e = cudaMalloc(&s->d_b[l], sizeof(float) * dims[l + 1]);
+        if (e == cudaSuccess) e = cudaMemcpy(s->d_b[l], b[l], sizeof(float) * dims[l + 1], cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) break;
+        if (dtype == SF_BF16) {
+            uint16_t* h = (uint16_t*)malloc(cnt * 2);
+            if (!h) { sf_slow_destroy(s); return SF_ERR_ALLOC; }
+            f32_to_bf16_host(W[l], h, cnt);
+            e = cudaMalloc(&s->d_W[l], cnt * 2);
+            if (e == cudaSuccess) e = cudaMemcpy(s->d_W[l], h, cnt * 2, cudaMemcpyHostToDevice);
+            free(h);
+        } else {
+            e = cudaMalloc(&s->d_W[l], cnt * 4);
+            if (e == cudaSuccess) e = cudaMemcpy(s->d_W[l], W[l], cnt * 4, cudaMemcpyHostToDevice);
+        }
+    }
+    if (e != cudaSuccess) { sf_slow_destroy(s); return sf_set_cuda_error(e, "sf_mlp_create"); }
+    *out = s;
+    return SF_OK;
+}
+
+extern "C" int sf_cnn_create(sf_ctx* ctx, int dtype, uint32_t L, uint32_t Cin, uint32_t C1, uint32_t C2, uint32_t k,
+                             uint32_t n_cls, const float* w1, const float* b1, const float* w2, const float* b2,
+                             const float* w3, const float* b3, sf_slow** out)
+{
+    if (!ctx || !w1 || !b1 || !w2 || !b2 || !w3 || !b3 || !out) return SF_ERR_ARG;
+    if (dtype != SF_BF16) return SF_ERR_UNSUPPORTED;
+    if (L != 128 || Cin != 8 || C1 != 64 || C2 != 128 || k != 5 || n_cls < 1 || n_cls > 16) return SF_ERR_UNSUPPORTED;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    sf_slow* s = new (std::nothrow) sf_slow();
+    if (!s) return SF_ERR_ALLOC;
+    memset(s, 0, sizeof(*s));
+    s->ctx = ctx; s->arch = SF_SLOW_CNN; s->dtype = dtype;
+    s->L = L; s->Cin = Cin; s->C1 = C1; s->C2 = C2; s->k = k; s->n_cls = n_cls;
+    int rc = sf_cnn_prepare(s, w1, b1, w2, b2, w3, b3);
+    if (rc != SF_OK) { sf_slow_destroy(s); return rc; }
+    *out = s;
+    return SF_OK;
+}
+
+extern "C" void sf_slow_destroy(sf_slow* s) {
+    if (!s) return;
+    for (int l = 0; l < 8; l++) { if (s->d_W[l]) cudaFree(s->d_W[l]); if (s->d_b[l]) cudaFree(s->d_b[l]); }
+    if (s->d_w1) cudaFree(s->d_w1); if (s->d_w2) cudaFree(s->d_w2); if (s->d_w3) cudaFree(s->d_w3);
+    if (s->d_b1) cudaFree(s->d_b1); if (s->d_b2) cudaFree(s->d_b2); if (s->d_b3) cudaFree(s->d_b3);
+    delete s;
+}
+
+extern "C" int sf_slow_infer(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev,
+                             uint32_t capacity, float* logits_out, uint8_t* label_out, void* stream)
+{
+    if (!ctx || !s || !rows || !n_rows_dev || !logits_out) return SF_ERR_ARG;
+    if (((uintptr_t)rows & 127) != 0) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    size_t need = sf_slow_scratch_bytes(s, capacity);
+    int rc = sf_ws_reserve(ctx, need);
+    if (rc != SF_OK) return rc;
+    sf_ws_reset(ctx);
+    void* scratch = sf_ws_alloc(ctx, need);
+    if (!scratch) return SF_ERR_ALLOC;
+    return sf_launch_slow(ctx, s, rows, n_rows_dev, capacity, logits_out, label_out, scratch, (cudaStream_t)stream);
+}

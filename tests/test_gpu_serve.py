@@ -1,0 +1,112 @@
+"""GPU parity of the whole cascade (sf_serve_batch and its host-pointer variant)
+against the oracle's staged evaluation."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import flowgen
+import oracle
+from workload import make_workload
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2402_03694_b200 import build, binding as sf, harness as hz
+    build.build()
+    ctx = sf.sf_ctx_create(0, 0)
+    yield sf, hz, ctx
+    sf.sf_ctx_destroy(ctx)
+
+
+def bits(a):
+    return np.ascontiguousarray(a, np.float32).view(np.uint32)
+
+
+def run_and_check(sf, hz, ctx, wl, capacity=None):
+    cfg, n = wl["cfg"], wl["n"]
+    tol = 2e-2 if cfg.slow_dtype == "bf16" else 1e-4
+    ref = oracle.serve_batch(cfg, wl["fast"], wl["wide"], wl["forest"], wl["slow"], wl["tau"], threads=8)
+    forest = hz.make_forest(ctx, wl["forest"])
+    slow = hz.make_slow(ctx, cfg, wl["slow"])
+    fast_d = hz.upload_packets(wl["fast"], with_hdr=False)
+    wide_d = hz.upload_packets(wl["wide"])
+    cap = n if capacity is None else capacity
+    rcfg = hz.route_cfg_for(cfg, hz.dev(wl["tau"]), cap)
+    label = torch.full((n,), 255, dtype=torch.uint8, device="cuda")
+    stage = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_serve_batch(ctx, forest, slow, fast_d["struct"], cfg.N, cfg.F, wide_d["struct"], rcfg, label, stage, n_esc)
+    torch.cuda.synchronize()
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    k = int(n_esc.cpu().numpy()[0])
+    assert k == ref["n_esc"] and c.n_flows == n and c.n_escalated == k and c.n_slow_done == k
+    p = sf.sf_serve_batch_intermediates(ctx)
+    Cf = 1 if cfg.kind == "gbdt" else cfg.C
+    feat = hz.ptr_tensor(p["feat"], (n, cfg.F), torch.float32).cpu().numpy()
+    fo = hz.ptr_tensor(p["fast_out"], (n, Cf), torch.float32).cpu().numpy()
+    ids = hz.ptr_tensor(p["esc_ids"], (k,), torch.uint32).cpu().numpy()
+    D = cfg.D
+    rows = hz.ptr_tensor(p["rows"], (k, D), torch.bfloat16 if cfg.slow_dtype == "bf16" else torch.float32).float().cpu().numpy()
+    logits = hz.ptr_tensor(p["logits"], (k, cfg.n_slow_classes), torch.float32).cpu().numpy()
+    assert np.array_equal(bits(feat), bits(ref["feat"]))
+    assert np.array_equal(bits(fo.reshape(ref["fast_out"].shape)), bits(ref["fast_out"]))
+    assert np.array_equal(ids, ref["esc_ids"])
+    assert np.array_equal(bits(rows), bits(ref["rows"]))
+    assert np.max(np.abs(logits - ref["logits"])) <= tol
+    st = stage.cpu().numpy()
+    lab = label.cpu().numpy()
+    assert np.array_equal(st, ref["stage"])
+    fastm = st == 1
+    assert np.array_equal(lab[fastm], ref["label_final"][fastm])
+    s = np.sort(ref["logits"], axis=1)
+    clear = (s[:, -1] - s[:, -2]) >= 2 * tol
+    assert np.array_equal(lab[ref["esc_ids"]][clear], ref["label_slow"][clear])
+    assert np.array_equal(lab[ref["esc_ids"]], hz.ptr_tensor(p["label_slow"], (k,), torch.uint8).cpu().numpy())
+    # host-pointer entry point gives the same answers
+    fast_h = hz.pinned_packets(wl["fast"], with_hdr=False)
+    wide_h = hz.pinned_packets(wl["wide"])
+    rcfg_h = hz.route_cfg_for(cfg, np.ascontiguousarray(wl["tau"]), cap)
+    lab_h = np.zeros(n, np.uint8); st_h = np.zeros(n, np.uint8); ne_h = np.zeros(1, np.uint32)
+    sf.sf_serve_batch_host(ctx, forest, slow, fast_h["struct"], cfg.N, cfg.F, wide_h["struct"], rcfg_h, lab_h, st_h, ne_h)
+    assert int(ne_h[0]) == k and np.array_equal(lab_h, lab) and np.array_equal(st_h, st)
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_slow_destroy(slow)
+    sf.sf_forest_destroy(forest)
+    return ref
+
+
+def test_c1_full(env):
+    sf, hz, ctx = env
+    wl = make_workload(flowgen.get_config(1))
+    ref = run_and_check(sf, hz, ctx, wl)
+    assert 0.2 < ref["n_esc"] / wl["n"] < 0.3
+
+
+def test_c2_shapes_reduced_flow_count(env):
+    """Config 2's model shapes (100 depth-12 trees, 2048-wide bf16 MLP) on 6,000 flows:
+    several 512-flow tiles plus a ragged tail, ~1,400 assigned rows (11 GEMM row tiles)."""
+    sf, hz, ctx = env
+    wl = make_workload(flowgen.get_config(2), n=6000)
+    run_and_check(sf, hz, ctx, wl)
+
+
+def test_c3_shapes_reduced_flow_count(env):
+    sf, hz, ctx = env
+    wl = make_workload(flowgen.get_config(3), n=9000)
+    run_and_check(sf, hz, ctx, wl)
+
+
+def test_shared_planes_and_ragged_sizes(env):
+    """fast_ctx and slow_ctx alias the same wide planes (pitch = P), odd flow count."""
+    sf, hz, ctx = env
+    cfg = dataclasses.replace(flowgen.get_config(1), n=1237)
+    wl = make_workload(cfg, n=1237)
+    wl["fast"] = wl["wide"]
+    run_and_check(sf, hz, ctx, wl)

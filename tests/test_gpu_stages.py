@@ -1,0 +1,328 @@
+"""GPU parity: each stage of the CUDA library, called through the C ABI, against the
+CPU oracle on the same seeded inputs.  Integer / index / fast-model outputs must be
+bit-exact; slow-model logits within 1e-4 (fp32) or 2e-2 (bf16) absolute."""
+import numpy as np
+import pytest
+
+import flowgen
+import oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2402_03694_b200 import build, binding as sf, harness as hz
+    build.build()
+    ctx = sf.sf_ctx_create(0, 1 << 20)
+    yield sf, hz, ctx
+    sf.sf_ctx_poll(ctx, raise_on_error=False)
+    sf.sf_ctx_destroy(ctx)
+
+
+def bits(a):
+    return np.ascontiguousarray(a, np.float32).view(np.uint32)
+
+
+# ------------------------------------------------------------------ S1 -------
+@pytest.mark.parametrize("N,F,n,pitch", [
+    (8, 24, 4096, 8), (16, 48, 5003, 16), (32, 64, 3001, 32), (8, 32, 777, 8),
+    (8, 24, 1000, 64),      # window shorter than the row pitch (wide planes)
+    (5, 16, 300, 12),       # pitch not a multiple of 8: scalar-load path
+    (1, 8, 129, 8), (8, 64, 1, 8),
+])
+def test_extract_bit_exact(env, N, F, n, pitch):
+    sf, hz, ctx = env
+    pk = flowgen.gen_packets(500 + N + F, n, pitch, H=0)
+    pk["iat_us"][0, :] = 2 ** 32 - 1
+    if n > 2:
+        pk["iat_us"][1, ::2] = 0
+        pk["iat_us"][1, 1::2] = 2 ** 32 - 1
+        pk["size"][2, :] = 65535
+    ref = oracle.extract_features(pk, N, F)
+    d = hz.upload_packets(pk, with_hdr=False)
+    out = torch.empty((n, F), dtype=torch.float32, device="cuda")
+    sf.sf_extract_features(ctx, d["struct"], N, F, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(out.cpu().numpy()), bits(ref))
+
+
+def test_extract_short_flows(env):
+    sf, hz, ctx = env
+    n, N, F = 2500, 16, 48
+    pk = flowgen.gen_packets(41, n, 16, H=0)
+    nv = np.random.default_rng(2).integers(0, 20, size=n).astype(np.uint8)
+    ref = oracle.extract_features(pk, N, F, n_valid=nv)
+    d = hz.upload_packets(pk, n_valid=nv, with_hdr=False)
+    out = torch.empty((n, F), dtype=torch.float32, device="cuda")
+    sf.sf_extract_features(ctx, d["struct"], N, F, out)
+    assert np.array_equal(bits(out.cpu().numpy()), bits(ref))
+
+
+def test_extract_rejects_bad_arguments(env):
+    sf, hz, ctx = env
+    pk = flowgen.gen_packets(1, 16, 8, H=0)
+    d = hz.upload_packets(pk, with_hdr=False)
+    out = torch.empty((16, 24), dtype=torch.float32, device="cuda")
+    for N, F in ((0, 24), (33, 24), (9, 24), (8, 20), (8, 72)):
+        with pytest.raises(sf.SfError) as e:
+            sf.sf_extract_features(ctx, d["struct"], N, F, out)
+        assert e.value.status == sf.SF_ERR_ARG
+
+
+# ------------------------------------------------------------------ S2 -------
+def _features(n, N, F, seed):
+    pk = flowgen.gen_packets(seed, n, N, H=0)
+    return oracle.extract_features(pk, N, F, threads=4)
+
+
+@pytest.mark.parametrize("kind,T,d,F,C,n", [
+    ("rf", 16, 8, 24, 4, 4096),
+    ("rf", 10, 12, 48, 8, 3000),     # depth-12 trees: one tree per shared-memory chunk
+    ("rf", 7, 10, 64, 16, 1500),
+    ("rf", 5, 3, 8, 3, 600),         # class count that is not a multiple of 4
+    ("gbdt", 70, 6, 32, 2, 5001),    # 64 trees per chunk + a ragged second chunk
+    ("gbdt", 3, 1, 8, 2, 33),
+])
+def test_forest_bit_exact(env, kind, T, d, F, C, n):
+    sf, hz, ctx = env
+    N = {8: 8, 24: 8, 32: 8, 48: 16, 64: 32}[F]
+    feat = _features(n, N, F, 600 + T)
+    fo = flowgen.gen_forest(700 + T, kind, T, d, F, C, feat)
+    ref, ref_li = oracle.forest_infer(fo, feat, want_leaf_idx=True)
+    h = hz.make_forest(ctx, fo)
+    fd = hz.dev(feat)
+    out = torch.empty((n, C) if kind == "rf" else (n,), dtype=torch.float32, device="cuda")
+    li = torch.empty((n, T), dtype=torch.uint16, device="cuda")
+    sf.sf_fast_infer(ctx, h, fd, n, out, li)
+    torch.cuda.synchronize()
+    assert np.array_equal(li.cpu().numpy(), ref_li)
+    assert np.array_equal(bits(out.cpu().numpy()), bits(ref))
+    out2 = torch.empty_like(out)
+    sf.sf_fast_infer(ctx, h, fd, n, out2, None)           # leaf indices are optional
+    assert torch.equal(out, out2)
+    sf.sf_forest_destroy(h)
+
+
+def test_forest_summation_order_is_tree_order(env):
+    sf, hz, ctx = env
+    vals = [2.0 ** 24, 1.0, 1.0, -(2.0 ** 24)]
+    fo = {"kind": "gbdt", "T": 4, "depth": 1, "F": 8, "C": 2, "fid": np.zeros((4, 1), np.uint16),
+          "thr": np.zeros((4, 1), np.float32), "leaf": np.array([[v, v] for v in vals], np.float32)}
+    h = hz.make_forest(ctx, fo)
+    out = torch.empty(5, dtype=torch.float32, device="cuda")
+    sf.sf_fast_infer(ctx, h, torch.zeros((5, 8), device="cuda"), 5, out)
+    assert np.all(out.cpu().numpy() == 0.0)
+    sf.sf_forest_destroy(h)
+
+
+# ------------------------------------------------------------------ S3 -------
+def test_route_least_confidence_bit_exact(env):
+    sf, hz, ctx = env
+    sf.sf_ctx_poll(ctx, reset=True)
+    n, C = 10007, 8
+    rng = np.random.default_rng(11)
+    prob = rng.dirichlet([0.5] * C, size=n).astype(np.float32)
+    prob[5] = 1.0 / C                                            # all-equal row: label 0
+    tau = rng.uniform(0.3, 0.6, size=C).astype(np.float32)
+    prob[7] = 0; prob[7, 3] = 1 - tau[3]; prob[7, 0] = tau[3]    # near the threshold
+    ref = oracle.route_lc(prob, tau)
+    P, H = 64, 13
+    wide = flowgen.gen_packets(12, n, P, H)
+    nv = np.full(n, 255, np.uint8); nv[ref["esc_ids"][:50]] = 17
+    w = hz.upload_packets(wide, n_valid=nv)
+    for dtype in (sf.SF_BF16, sf.SF_F32):
+        cfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, dtype, P, n)
+        ids = torch.full((n,), 0xFFFFFFFF, dtype=torch.uint32, device="cuda")
+        n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+        rows = torch.zeros((n, P * 16), dtype=torch.bfloat16 if dtype == sf.SF_BF16 else torch.float32, device="cuda")
+        dec = torch.empty(n, dtype=torch.uint8, device="cuda")
+        lab = torch.empty(n, dtype=torch.uint8, device="cuda")
+        sc = torch.empty(n, dtype=torch.float32, device="cuda")
+        sf.sf_route(ctx, cfg, hz.dev(prob), n, C, w["struct"], ids, n_esc, rows, dec, lab, sc)
+        torch.cuda.synchronize()
+        k = int(n_esc.cpu().numpy()[0])
+        assert k == ref["n_esc"]
+        assert np.array_equal(ids.cpu().numpy()[:k], ref["esc_ids"])
+        assert np.array_equal(dec.cpu().numpy(), ref["decision"])
+        assert np.array_equal(lab.cpu().numpy(), ref["label"])
+        assert np.array_equal(bits(sc.cpu().numpy()), bits(ref["score"]))
+        ref_rows = oracle.wide_rows(0, ref["esc_ids"], wide, P, dtype == sf.SF_BF16, n_valid=nv, threads=4)
+        got = rows[:k].float().cpu().numpy()
+        assert np.array_equal(bits(got), bits(ref_rows))
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert c.n_flows == 2 * n and c.n_escalated == 2 * ref["n_esc"] and c.n_fast_done == 2 * (n - ref["n_esc"])
+
+
+def test_route_absmargin_and_cnn_layout(env):
+    sf, hz, ctx = env
+    n, P, H = 6001, 128, 5
+    rng = np.random.default_rng(13)
+    margin = (rng.normal(size=n) * 2.24).astype(np.float32)
+    margin[3] = np.float32(oracle.TAU_MARGIN)          # equal to the threshold: strict < keeps it
+    margin[4] = -np.float32(oracle.TAU_MARGIN)
+    ref = oracle.route_absmargin(margin)
+    wide = flowgen.gen_packets(14, n, P, H)
+    w = hz.upload_packets(wide)
+    tau = hz.dev(np.array([sf.SF_TAU_MARGIN_DEFAULT], np.float32))
+    assert np.float32(sf.SF_TAU_MARGIN_DEFAULT) == np.float32(oracle.TAU_MARGIN)
+    cfg = sf.make_route_cfg(sf.SF_ABSMARGIN_LT, tau, sf.SF_CNN8, sf.SF_BF16, P, n)
+    ids = torch.zeros(n, dtype=torch.uint32, device="cuda")
+    n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    rows = torch.zeros((n, P * 8), dtype=torch.bfloat16, device="cuda")
+    dec = torch.empty(n, dtype=torch.uint8, device="cuda")
+    lab = torch.empty(n, dtype=torch.uint8, device="cuda")
+    sf.sf_route(ctx, cfg, hz.dev(margin), n, 2, w["struct"], ids, n_esc, rows, dec, lab, None)
+    k = int(n_esc.cpu().numpy()[0])
+    assert k == ref["n_esc"] and ref["decision"][3] == 0 and ref["decision"][4] == 0
+    assert np.array_equal(ids.cpu().numpy()[:k], ref["esc_ids"])
+    assert np.array_equal(dec.cpu().numpy(), ref["decision"]) and np.array_equal(lab.cpu().numpy(), ref["label"])
+    ref_rows = oracle.wide_rows(1, ref["esc_ids"], wide, P, True, threads=4)
+    assert np.array_equal(bits(rows[:k].float().cpu().numpy()), bits(ref_rows))
+    sf.sf_ctx_poll(ctx, reset=True)
+
+
+def test_route_zero_padding_and_empty_and_overflow(env):
+    sf, hz, ctx = env
+    n, C = 3000, 4
+    rng = np.random.default_rng(15)
+    prob = rng.dirichlet([0.5] * C, size=n).astype(np.float32)
+    tau = np.full(C, 0.4, np.float32)
+    ref = oracle.route_lc(prob, tau)
+    wide = flowgen.gen_packets(16, n, 64, 13)
+    w = hz.upload_packets(wide)
+    # 64 real packets in a 128-packet row
+    cfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, 128, n, P_real=64)
+    ids = torch.zeros(n, dtype=torch.uint32, device="cuda")
+    n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    rows = torch.ones((n, 2048), dtype=torch.bfloat16, device="cuda")
+    sf.sf_route(ctx, cfg, hz.dev(prob), n, C, w["struct"], ids, n_esc, rows)
+    k = int(n_esc.cpu().numpy()[0])
+    ref_rows = oracle.wide_rows(0, ref["esc_ids"], wide, 128, True, P_real=64, threads=4)
+    assert k == ref["n_esc"] and np.array_equal(bits(rows[:k].float().cpu().numpy()), bits(ref_rows))
+    # nothing assigned
+    cfg0 = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(np.full(C, 2.0, np.float32)), sf.SF_MLP16, sf.SF_BF16, 64, n)
+    sf.sf_route(ctx, cfg0, hz.dev(prob), n, C, None, ids, n_esc)
+    assert int(n_esc.cpu().numpy()[0]) == 0
+    # empty batch
+    sf.sf_route(ctx, cfg0, hz.dev(prob), 0, C, None, ids, n_esc)
+    assert int(n_esc.cpu().numpy()[0]) == 0
+    assert sf.sf_ctx_poll(ctx, reset=True).device_error == 0
+    # capacity overflow: count saturates, the prefix is still right, the error word says so
+    cap = ref["n_esc"] // 2
+    cfgc = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, 64, cap)
+    ids2 = torch.full((n,), 0xFFFFFFFF, dtype=torch.uint32, device="cuda")
+    sf.sf_route(ctx, cfgc, hz.dev(prob), n, C, None, ids2, n_esc)
+    assert int(n_esc.cpu().numpy()[0]) == cap
+    got = ids2.cpu().numpy()
+    assert np.array_equal(got[:cap], ref["esc_ids"][:cap]) and np.all(got[cap:] == 0xFFFFFFFF)
+    c = sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    assert c.device_error == sf.SF_ERR_CAPACITY
+    assert sf.sf_ctx_poll(ctx).device_error == 0
+
+
+# ------------------------------------------------------------------ S4 -------
+def _run_slow(sf, hz, ctx, handle, rows_t, n_rows, cap, n_cls):
+    cnt = hz.dev(np.array([n_rows], np.uint32))
+    logits = torch.full((cap, n_cls), float("nan"), dtype=torch.float32, device="cuda")
+    label = torch.full((cap,), 255, dtype=torch.uint8, device="cuda")
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_slow_infer(ctx, handle, rows_t, cnt, cap, logits, label)
+    torch.cuda.synchronize()
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert c.device_error == 0 and c.n_slow_done == n_rows
+    return logits.cpu().numpy(), label.cpu().numpy()
+
+
+def _check_labels(ref_logits, ref_label, got_label, tol):
+    s = np.sort(ref_logits, axis=1)
+    clear = (s[:, -1] - s[:, -2]) >= 2 * tol if ref_logits.shape[1] > 1 else np.ones(len(ref_label), bool)
+    assert np.array_equal(got_label[clear], ref_label[clear])
+
+
+def test_mlp_fp32(env):
+    sf, hz, ctx = env
+    m = flowgen.gen_mlp(21, (1024, 256, 256, 4))
+    n_rows, cap = 1000, 1100
+    rows = np.random.default_rng(3).uniform(0, 1, size=(cap, 1024)).astype(np.float32)
+    ref, ref_label = oracle.mlp(m, rows[:n_rows], False, threads=8)
+    h = sf.sf_mlp_create(ctx, sf.SF_F32, m["dims"], m["W"], m["b"])
+    logits, label = _run_slow(sf, hz, ctx, h, hz.dev(rows), n_rows, cap, 4)
+    assert np.max(np.abs(logits[:n_rows] - ref)) <= TOL_F32
+    assert np.all(np.isnan(logits[n_rows:])) and np.all(label[n_rows:] == 255)     # rows past the count untouched
+    _check_labels(ref, ref_label, label[:n_rows], TOL_F32)
+    sf.sf_slow_destroy(h)
+
+
+@pytest.mark.parametrize("dims,n_rows,cap", [
+    ((64, 64, 4), 128, 128),              # one tile, one K slice
+    ((128, 128, 8), 300, 384),            # ragged last tile
+    ((256, 256, 256, 2), 130, 1000),      # BN = 256, count far below capacity
+    ((192, 320, 64, 16), 515, 600),       # BN = 64 path, K not a power of two
+])
+def test_mlp_bf16_small_integers_are_exact(env, dims, n_rows, cap):
+    """Integer-valued bf16 operands with small sums: every product and partial sum is
+    exactly representable, so the tensor-core result must equal integer arithmetic."""
+    sf, hz, ctx = env
+    rng = np.random.default_rng(sum(dims))
+    nl = len(dims) - 1
+    W = [rng.integers(-2, 3, size=(dims[l + 1], dims[l])).astype(np.float32) for l in range(nl)]
+    b = [rng.integers(-3, 4, size=dims[l + 1]).astype(np.float32) for l in range(nl)]
+    # sparsify so that activations stay below 256 (exact in bf16)
+    for l in range(nl):
+        W[l] *= (rng.random(W[l].shape) < 8.0 / dims[l])
+    x = rng.integers(0, 3, size=(cap, dims[0])).astype(np.float32)
+    h = x[:n_rows].astype(np.int64)
+    for l in range(nl):
+        h = h @ W[l].astype(np.int64).T + b[l].astype(np.int64)
+        if l + 1 < nl:
+            h = np.maximum(h, 0)
+            assert h.max() < 256
+    m = {"dims": dims, "W": W, "b": b}
+    o_logits, _ = oracle.mlp(m, x[:n_rows], True, threads=4)
+    assert np.array_equal(o_logits, h.astype(np.float32))
+    hd = sf.sf_mlp_create(ctx, sf.SF_BF16, dims, W, b)
+    logits, label = _run_slow(sf, hz, ctx, hd, hz.dev(x).to(torch.bfloat16), n_rows, cap, dims[-1])
+    assert np.array_equal(logits[:n_rows], h.astype(np.float32))
+    assert np.array_equal(label[:n_rows], np.argmax(h, axis=1).astype(np.uint8))
+    assert np.all(np.isnan(logits[n_rows:]))
+    sf.sf_slow_destroy(hd)
+
+
+@pytest.mark.parametrize("dims,n_rows", [((1024, 512, 512, 2), 700), ((2048, 1024, 1024, 1024, 8), 400)])
+def test_mlp_bf16_within_tolerance(env, dims, n_rows):
+    sf, hz, ctx = env
+    m = flowgen.gen_mlp(33, dims)
+    wide = flowgen.gen_packets(34, n_rows, dims[0] // 16, 13)
+    rows = oracle.wide_rows(0, np.arange(n_rows, dtype=np.uint32), wide, dims[0] // 16, True, threads=4)
+    ref, ref_label = oracle.mlp(m, rows, True, threads=8)
+    hd = sf.sf_mlp_create(ctx, sf.SF_BF16, m["dims"], m["W"], m["b"])
+    cap = n_rows + 57
+    rt = torch.zeros((cap, dims[0]), dtype=torch.bfloat16, device="cuda")
+    rt[:n_rows] = hz.dev(rows).to(torch.bfloat16)
+    logits, label = _run_slow(sf, hz, ctx, hd, rt, n_rows, cap, dims[-1])
+    assert np.max(np.abs(logits[:n_rows] - ref)) <= TOL_BF16
+    _check_labels(ref, ref_label, label[:n_rows], TOL_BF16)
+    # zero rows: nothing is written
+    logits0, _ = _run_slow(sf, hz, ctx, hd, rt, 0, cap, dims[-1])
+    assert np.all(np.isnan(logits0))
+    sf.sf_slow_destroy(hd)
+
+
+def test_create_rejects_unsupported_shapes(env):
+    sf, hz, ctx = env
+    W = [np.zeros((48, 100), np.float32), np.zeros((4, 48), np.float32)]
+    b = [np.zeros(48, np.float32), np.zeros(4, np.float32)]
+    with pytest.raises(sf.SfError) as e:
+        sf.sf_mlp_create(ctx, sf.SF_BF16, (100, 48, 4), W, b)
+    assert e.value.status == sf.SF_ERR_UNSUPPORTED
+    with pytest.raises(sf.SfError):
+        sf.sf_forest_create(ctx, sf.SF_RF, 1, 13, 8, 2, np.zeros((1, 8191)), np.zeros((1, 8191)), np.zeros((1, 8192, 2)))
+    with pytest.raises(sf.SfError):      # feature id out of range
+        sf.sf_forest_create(ctx, sf.SF_RF, 1, 1, 8, 2, np.full((1, 1), 9), np.zeros((1, 1)), np.zeros((1, 2, 2)))
