@@ -55,14 +55,16 @@ def route_cfg_for(cfg, tau_dev, capacity, P_real=0):
     return sf.make_route_cfg(rule, tau_dev, layout, dt, cfg.P, capacity, P_real)
 
 
+class _DevPtr:
+    def __init__(self, ptr, n, typestr):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (int(ptr), False), "version": 2}
+
+
 def ptr_tensor(ptr, shape, dtype, device="cuda:0"):
-    """View library-owned device memory as a torch tensor (copy of it, for inspection)."""
-    import ctypes
+    """Copy of library-owned device memory as a torch tensor (for inspection)."""
     n = int(np.prod(shape))
-    out = torch.empty(n, dtype=dtype, device=device)
-    nbytes = n * out.element_size()
-    if nbytes:
-        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), ptr, nbytes, 3)   # cudaMemcpyDeviceToDevice
-        if int(rc) != 0:
-            raise RuntimeError("cudaMemcpy failed: %s" % rc)
-    return out.view(*shape)
+    esz = torch.empty(0, dtype=dtype).element_size()
+    if n == 0:
+        return torch.empty(shape, dtype=dtype, device=device)
+    raw = torch.as_tensor(_DevPtr(ptr, n * esz, "|u1"), device=device)
+    return raw.clone().view(dtype).view(*shape)
