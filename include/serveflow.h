@@ -88,6 +88,23 @@ typedef struct {
  * device_error (SF_OK if none).  `reset` != 0 clears counters and error word. */
 int  sf_ctx_poll(sf_ctx* ctx, sf_counters* host_out, int reset, void* stream);
 
+/* Per-kernel timing (off by default).  When enabled, every compute call records
+ * CUDA events on its stream around each kernel class and keeps the last 64 calls'
+ * records.  sf_ctx_get_timing synchronises `stream` and writes SF_N_TIMERS
+ * elapsed times in milliseconds (0 for classes the call did not run) of the call
+ * made `back` calls ago (0 = the most recent) to host memory. */
+#define SF_T_EXTRACT 0   /* S1 feature kernel */
+#define SF_T_FOREST  1   /* S2 tree-ensemble kernel */
+#define SF_T_SCORE   2   /* S3 score + scan + scatter kernels */
+#define SF_T_GATHER  3   /* S3 wide-row gather kernel */
+#define SF_T_GEMM    4   /* S4 hidden layers (tensor-core GEMMs, the fp32 dense kernels, or the fused CNN kernel) */
+#define SF_T_HEAD    5   /* S4 last layer + argmax */
+#define SF_T_MERGE   6   /* S5 merge kernels */
+#define SF_T_TABLE   7   /* streaming table kernels */
+#define SF_N_TIMERS  8
+int  sf_ctx_set_timing(sf_ctx* ctx, int enable);
+int  sf_ctx_get_timing(sf_ctx* ctx, uint32_t back, float* ms_host_out, void* stream);
+
 /* ---- packet planes -------------------------------------------------------- */
 /* Header planes of n_flows flows with a row pitch of pitch_pkts packets:
  *   size     uint16[n][pitch]          packet length in bytes

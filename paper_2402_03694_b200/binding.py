@@ -78,6 +78,7 @@ FLOW_RESULT_DTYPE = np.dtype([("found", "u1"), ("stage", "u1"), ("label_fast", "
 
 EXPORTS = [
     "sf_strerror", "sf_last_cuda_error", "sf_version", "sf_ctx_create", "sf_ctx_destroy", "sf_ctx_poll",
+    "sf_ctx_set_timing", "sf_ctx_get_timing",
     "sf_extract_features", "sf_forest_create", "sf_forest_destroy", "sf_fast_infer", "sf_route",
     "sf_universal_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
     "sf_serve_batch", "sf_serve_batch_host", "sf_serve_batch_intermediates",
@@ -105,6 +106,8 @@ def _lib():
         V, U32, I = C.c_void_p, C.c_uint32, C.c_int
         L.sf_ctx_create.argtypes = [C.POINTER(V), I, C.c_size_t]
         L.sf_ctx_poll.argtypes = [V, C.POINTER(sf_counters), I, V]
+        L.sf_ctx_set_timing.argtypes = [V, I]
+        L.sf_ctx_get_timing.argtypes = [V, U32, V, V]
         L.sf_extract_features.argtypes = [V, C.POINTER(sf_packets), U32, U32, V, V]
         L.sf_forest_create.argtypes = [V, I, U32, U32, U32, U32, V, V, V, C.POINTER(V)]
         L.sf_fast_infer.argtypes = [V, V, V, U32, V, V, V]
@@ -190,6 +193,20 @@ def sf_ctx_poll(ctx, reset=False, stream=None, raise_on_error=True):
     if raise_on_error:
         _check(st, "sf_ctx_poll")
     return c
+
+
+SF_TIMER_NAMES = ("extract", "forest", "score", "gather", "gemm", "head", "merge", "table")
+
+
+def sf_ctx_set_timing(ctx, enable):
+    _check(_lib().sf_ctx_set_timing(ctx, int(enable)), "sf_ctx_set_timing")
+
+
+def sf_ctx_get_timing(ctx, back=0, stream=None):
+    """dict name -> milliseconds for the call made `back` calls ago."""
+    out = np.zeros(len(SF_TIMER_NAMES), np.float32)
+    _check(_lib().sf_ctx_get_timing(ctx, back, out.ctypes.data, _stream(stream)), "sf_ctx_get_timing")
+    return {k: float(v) for k, v in zip(SF_TIMER_NAMES, out)}
 
 
 def sf_extract_features(ctx, pk, N, F, feat_out, stream=None):

@@ -34,6 +34,52 @@ extern "C" const char* sf_strerror(int status) {
     return "unknown status";
 }
 
+// ---- timing ----------------------------------------------------------------------
+void sf_time_new_record(sf_ctx* ctx) {
+    if (!ctx->timing) return;
+    ctx->t_rec++;
+    memset(ctx->t_used[(ctx->t_rec - 1) & 63], 0, SF_N_TIMERS);
+}
+void sf_time_begin(sf_ctx* ctx, int slot, cudaStream_t st) {
+    if (!ctx->timing || ctx->t_rec == 0) return;
+    uint32_t r = (ctx->t_rec - 1) & 63;
+    if (ctx->t_used[r][slot]) return;                // a class that runs in several pieces keeps its first start
+    cudaEventRecord(ctx->t_ev[r][slot][0], st);
+    ctx->t_used[r][slot] = 1;
+}
+void sf_time_end(sf_ctx* ctx, int slot, cudaStream_t st) {
+    if (!ctx->timing || ctx->t_rec == 0) return;
+    uint32_t r = (ctx->t_rec - 1) & 63;
+    cudaEventRecord(ctx->t_ev[r][slot][1], st);
+    ctx->t_used[r][slot] = 2;
+}
+
+extern "C" int sf_ctx_set_timing(sf_ctx* ctx, int enable) {
+    if (!ctx) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    if (enable && !ctx->t_ev[0][0][0]) {
+        for (int r = 0; r < 64; r++)
+            for (int s = 0; s < SF_N_TIMERS; s++)
+                for (int k = 0; k < 2; k++) SF_CUDA(cudaEventCreate(&ctx->t_ev[r][s][k]));
+    }
+    ctx->timing = enable ? 1 : 0;
+    ctx->t_rec = 0;
+    return SF_OK;
+}
+
+extern "C" int sf_ctx_get_timing(sf_ctx* ctx, uint32_t back, float* ms_out, void* stream) {
+    if (!ctx || !ms_out || back >= 64) return SF_ERR_ARG;
+    if (!ctx->timing || ctx->t_rec <= back) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    SF_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    uint32_t r = (ctx->t_rec - 1 - back) & 63;
+    for (int s = 0; s < SF_N_TIMERS; s++) {
+        ms_out[s] = 0.0f;
+        if (ctx->t_used[r][s] == 2) SF_CUDA(cudaEventElapsedTime(&ms_out[s], ctx->t_ev[r][s][0], ctx->t_ev[r][s][1]));
+    }
+    return SF_OK;
+}
+
 // ---- workspace ---------------------------------------------------------------
 int sf_ws_reserve(sf_ctx* ctx, size_t bytes) {
     if (bytes <= ctx->ws_bytes) return SF_OK;
@@ -85,6 +131,10 @@ extern "C" void sf_ctx_destroy(sf_ctx* c) {
     if (c->ws) cudaFree(c->ws);
     if (c->stage) cudaFree(c->stage);
     if (c->d_state) cudaFree(c->d_state);
+    if (c->t_ev[0][0][0])
+        for (int r = 0; r < 64; r++)
+            for (int s = 0; s < SF_N_TIMERS; s++)
+                for (int k = 0; k < 2; k++) cudaEventDestroy(c->t_ev[r][s][k]);
     delete c;
 }
 
@@ -189,16 +239,23 @@ int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf
     uint8_t* label_slow = reinterpret_cast<uint8_t*>(base + p.label_slow);
     uint32_t* n_esc_dev = &ctx->d_state->scan_total;
 
+    sf_time_new_record(ctx);
+    sf_time_begin(ctx, SF_T_EXTRACT, st);
     rc = sf_launch_extract(fast, N, F, feat, st);
+    sf_time_end(ctx, SF_T_EXTRACT, st);
     if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_FOREST, st);
     rc = sf_launch_forest(fo, feat, n, fast_out, nullptr, st);
+    sf_time_end(ctx, SF_T_FOREST, st);
     if (rc != SF_OK) return rc;
     rc = sf_launch_route(ctx, cfg, fast_out, n, fo->C, wide, esc_ids, n_esc_out, rows, decision, label_fast, nullptr,
                          base + p.route_scratch, st);
     if (rc != SF_OK) return rc;
     rc = sf_launch_slow(ctx, s, rows, n_esc_dev, cfg->capacity, logits, label_slow, base + p.slow_scratch, st);
     if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_MERGE, st);
     rc = sf_launch_merge(label_fast, decision, n, esc_ids, n_esc_dev, cfg->capacity, label_slow, label_out, stage_out, st);
+    sf_time_end(ctx, SF_T_MERGE, st);
     if (rc != SF_OK) return rc;
     ctx->last_feat = feat; ctx->last_fast_out = fast_out; ctx->last_esc_ids = esc_ids; ctx->last_rows = rows;
     ctx->last_logits = logits; ctx->last_label_fast = label_fast; ctx->last_label_slow = label_slow;

@@ -27,6 +27,11 @@ struct sf_ctx {
     // staging for the host-pointer entry point
     char*  stage;
     size_t stage_bytes;
+    // optional per-kernel-class timing: ring of event pairs
+    int timing;
+    uint32_t t_rec;                               // records started so far
+    cudaEvent_t t_ev[64][SF_N_TIMERS][2];
+    uint8_t t_used[64][SF_N_TIMERS];
     // intermediates of the last sf_serve_batch
     const float* last_feat; const float* last_fast_out; const uint32_t* last_esc_ids;
     const void* last_rows; const float* last_logits; const uint8_t* last_label_fast;
@@ -63,6 +68,11 @@ struct sf_slow {
 int  sf_set_cuda_error(cudaError_t e, const char* where);      // records text, returns SF_ERR_CUDA
 #define SF_CUDA(call) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) return sf_set_cuda_error(e__, #call); } while (0)
 #define SF_LAUNCH_CHECK(name) do { cudaError_t e__ = cudaGetLastError(); if (e__ != cudaSuccess) return sf_set_cuda_error(e__, name); } while (0)
+
+// timing: sf_time_new_record at the start of a public compute call, begin/end around kernels
+void sf_time_new_record(sf_ctx* ctx);
+void sf_time_begin(sf_ctx* ctx, int slot, cudaStream_t st);
+void sf_time_end(sf_ctx* ctx, int slot, cudaStream_t st);
 
 // workspace: reset at the start of a composite call, then bump-allocate (256-byte aligned)
 int   sf_ws_reserve(sf_ctx* ctx, size_t bytes);     // ensure capacity (may reallocate, synchronising)

@@ -187,5 +187,9 @@ extern "C" int sf_extract_features(sf_ctx* ctx, const sf_packets* pk, uint32_t N
     if (N < 1 || N > 32 || N > pk->pitch_pkts) return SF_ERR_ARG;
     if (F < 8 || F > 64 || (F % 8) != 0) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
-    return sf_launch_extract(pk, N, F, feat_out, (cudaStream_t)stream);
+    sf_time_new_record(ctx);
+    sf_time_begin(ctx, SF_T_EXTRACT, (cudaStream_t)stream);
+    int rc = sf_launch_extract(pk, N, F, feat_out, (cudaStream_t)stream);
+    sf_time_end(ctx, SF_T_EXTRACT, (cudaStream_t)stream);
+    return rc;
 }

@@ -227,5 +227,9 @@ extern "C" int sf_fast_infer(sf_ctx* ctx, const sf_forest* fo, const float* feat
     if (!ctx || !fo || !feat || !out) return SF_ERR_ARG;
     if (((uintptr_t)feat & 15) != 0) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
-    return sf_launch_forest(fo, feat, n, out, leaf_idx_out, (cudaStream_t)stream);
+    sf_time_new_record(ctx);
+    sf_time_begin(ctx, SF_T_FOREST, (cudaStream_t)stream);
+    int rc = sf_launch_forest(fo, feat, n, out, leaf_idx_out, (cudaStream_t)stream);
+    sf_time_end(ctx, SF_T_FOREST, (cudaStream_t)stream);
+    return rc;
 }

@@ -311,6 +311,7 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     char* h0 = reinterpret_cast<char*>(scratch);
     char* h1 = h0 + sf_align256((size_t)capacity * maxh * 2);
     const void* in = rows;
+    sf_time_begin(ctx, SF_T_GEMM, st);
     for (uint32_t l = 0; l + 1 < s->n_layers; l++) {
         void* out = (l & 1) ? h1 : h0;
         const uint32_t K = s->dims[l], N = s->dims[l + 1];
@@ -321,6 +322,10 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
         if (rc != SF_OK) return rc;
         in = out;
     }
+    sf_time_end(ctx, SF_T_GEMM, st);
     const uint32_t L = s->n_layers - 1;
-    return sf_launch_head_bf16(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st);
+    sf_time_begin(ctx, SF_T_HEAD, st);
+    int rc = sf_launch_head_bf16(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st);
+    sf_time_end(ctx, SF_T_HEAD, st);
+    return rc;
 }

@@ -215,6 +215,7 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
     uint32_t* block_counts = reinterpret_cast<uint32_t*>(scratch);
     uint8_t* dec = decision ? decision
                             : reinterpret_cast<uint8_t*>(scratch) + sf_align256(((size_t)nb + 1) * sizeof(uint32_t));
+    sf_time_begin(ctx, SF_T_SCORE, st);
     if (n > 0) {
         if (cfg->rule == SF_ABSMARGIN_LT)
             score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts);
@@ -228,6 +229,7 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
         scatter_kernel<<<nb, kScoreBlock, 0, st>>>(dec, n, block_counts, cfg->capacity, esc_ids);
         SF_LAUNCH_CHECK("scatter_kernel");
     }
+    sf_time_end(ctx, SF_T_SCORE, st);
     if (wide && rows && n > 0 && cfg->capacity > 0) {
         const uint32_t P = cfg->P, P_real = cfg->P_real ? cfg->P_real : cfg->P;
         // enough warps to cover the capacity, at most a few waves of resident blocks
@@ -235,12 +237,14 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
         uint32_t max_blocks = (uint32_t)ctx->num_sms * 32;
         if (blocks > max_blocks) blocks = max_blocks;
         const uint32_t* cnt = &ctx->d_state->scan_total;
+        sf_time_begin(ctx, SF_T_GATHER, st);
 #define SF_GATHER(Wv, BF) gather_kernel<Wv, BF><<<blocks, 256, 0, st>>>(esc_ids, cnt, wide->size, wide->iat_us, wide->dir_bits, \
             wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, P, P_real, rows)
         if (cfg->wide_layout == SF_MLP16) { if (cfg->row_dtype == SF_BF16) SF_GATHER(16, true); else SF_GATHER(16, false); }
         else                              { if (cfg->row_dtype == SF_BF16) SF_GATHER(8, true);  else SF_GATHER(8, false); }
 #undef SF_GATHER
         SF_LAUNCH_CHECK("gather_kernel");
+        sf_time_end(ctx, SF_T_GATHER, st);
     }
     return SF_OK;
 }
@@ -284,6 +288,7 @@ extern "C" int sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_
     sf_ws_reset(ctx);
     void* scratch = sf_ws_alloc(ctx, sf_route_scratch_bytes(n));
     if (!scratch) return SF_ERR_ALLOC;
+    sf_time_new_record(ctx);
     return sf_launch_route(ctx, cfg, fast_out, n, C, rows_out ? wide : nullptr, esc_ids_out, n_esc_out, rows_out,
                            decision_out, label_fast_out, score_out, scratch, (cudaStream_t)stream);
 }

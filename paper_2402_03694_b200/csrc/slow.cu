@@ -115,8 +115,10 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
         float* h0 = reinterpret_cast<float*>(scratch);
         float* h1 = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + sf_align256((size_t)capacity * maxh * 4));
         const float* in = reinterpret_cast<const float*>(rows);
+        sf_time_begin(ctx, SF_T_GEMM, st);
         for (uint32_t l = 0; l < s->n_layers; l++) {
             const bool last = (l + 1 == s->n_layers);
+            if (last) { sf_time_end(ctx, SF_T_GEMM, st); sf_time_begin(ctx, SF_T_HEAD, st); }
             float* out = last ? logits : ((l & 1) ? h1 : h0);
             dim3 grid((capacity + 63) / 64, (s->dims[l + 1] + 63) / 64);
             if (last) dense_f32_kernel<false><<<grid, 256, 0, st>>>(in, (const float*)s->d_W[l], s->d_b[l], n_rows_dev, s->dims[l], s->dims[l + 1], out);
@@ -129,6 +131,7 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
             argmax_kernel<<<blocks, 256, 0, st>>>(logits, n_rows_dev, s->dims[s->n_layers], label);
             SF_LAUNCH_CHECK("argmax_kernel");
         }
+        sf_time_end(ctx, SF_T_HEAD, st);
         rc = SF_OK;
     }
     if (rc != SF_OK) return rc;
@@ -218,5 +221,6 @@ extern "C" int sf_slow_infer(sf_ctx* ctx, const sf_slow* s, const void* rows, co
     sf_ws_reset(ctx);
     void* scratch = sf_ws_alloc(ctx, need);
     if (!scratch) return SF_ERR_ALLOC;
+    sf_time_new_record(ctx);
     return sf_launch_slow(ctx, s, rows, n_rows_dev, capacity, logits_out, label_out, scratch, (cudaStream_t)stream);
 }
