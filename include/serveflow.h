@@ -41,6 +41,7 @@ extern "C" {
 #define SF_ERR_TABLE_FULL     -5   /* a key found no slot within the probe limit; its packet was dropped */
 #define SF_ERR_UNSUPPORTED    -6   /* shape outside what the kernels implement */
 #define SF_ERR_DEVICE_TIMEOUT -7   /* a bounded device-side wait gave up */
+#define SF_ERR_STATIC_LIMIT   -8   /* sf_route_noalloc: more flows than its built-in scratch holds */
 
 /* enums passed as int */
 #define SF_RF           0          /* random forest: mean of leaf class-probability vectors */
@@ -180,6 +181,40 @@ typedef struct {
 int  sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* prob_or_margin, uint32_t n, uint32_t C,
               const sf_packets* wide, uint32_t* esc_ids_out, uint32_t* n_esc_out, void* rows_out,
               uint8_t* decision_out, uint8_t* label_fast_out, float* score_out, void* stream);
+
+/* Assignment without any allocation.  (The paper has no counterpart to this call: it
+ * exists for the way some programs have to use a GPU library.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated or freed - a
+ * serving loop whose memory was handed out once at start-up and is now fixed, a plug-in
+ * running inside another framework's memory pool, a real-time thread that must not take
+ * the driver's allocator lock.  Such callers cannot create an sf_ctx (that allocates),
+ * so this call takes no context.
+ *
+ * It does what sf_route does up to the list of assigned flows - score, fast label,
+ * strict threshold, ascending ids, count - and gathers no wide rows.  The per-block
+ * counts and, when decision_out is NULL, the per-flow decisions go to a fixed array
+ * built into the library image (about 4 MB; every GPU that loads the library keeps it
+ * until the process ends), so n may be at most SF_NOALLOC_MAX_FLOWS; a larger n is
+ * refused with SF_ERR_STATIC_LIMIT before anything is launched.  The call performs no
+ * cudaMalloc/cudaFree and calls nothing that allocates.
+ *
+ * All outputs are device pointers of the caller: esc_ids_out uint32[cfg->capacity],
+ * n_esc_out uint32[1]; nullable: decision_out uint8[n], label_fast_out uint8[n],
+ * score_out fp32[n], status_out int32[1] (0, or SF_ERR_CAPACITY when more flows
+ * qualified than cfg->capacity; the count then saturates as in sf_route).
+ * cfg->wide_layout, row_dtype, P and P_real are ignored.
+ *
+ * The first call on a device looks up the array's device address (a one-time set-up
+ * with that device current); make that first call before starting any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents
+ * (the call clears the part that must start at zero), so two calls whose GPU work
+ * overlaps - different streams, or different threads - race; run them one after the
+ * other on a stream, or order them with events. */
+#define SF_NOALLOC_MAX_FLOWS 4194304u
+int  sf_route_noalloc(int device, const sf_route_cfg* cfg, const float* prob_or_margin, uint32_t n, uint32_t C,
+                      uint32_t* esc_ids_out, uint32_t* n_esc_out, uint8_t* decision_out, uint8_t* label_fast_out,
+                      float* score_out, int32_t* status_out, void* stream);
 
 /* Algorithm 1 (universal uncertainty thresholds) on HOST data: sorts a copy of
  * the n validation scores ascending and returns, for each quantile

@@ -16,6 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libserveflow.so")
 SF_OK = 0
 SF_ERR_ARG, SF_ERR_ALLOC, SF_ERR_CUDA, SF_ERR_CAPACITY = -1, -2, -3, -4
 SF_ERR_TABLE_FULL, SF_ERR_UNSUPPORTED, SF_ERR_DEVICE_TIMEOUT = -5, -6, -7
+SF_ERR_STATIC_LIMIT = -8
+SF_NOALLOC_MAX_FLOWS = 4194304
 SF_RF, SF_GBDT = 0, 1
 SF_LC_GT, SF_ABSMARGIN_LT = 0, 1
 SF_MLP16, SF_CNN8 = 0, 1
@@ -80,6 +82,7 @@ EXPORTS = [
     "sf_strerror", "sf_last_cuda_error", "sf_version", "sf_ctx_create", "sf_ctx_destroy", "sf_ctx_poll",
     "sf_ctx_set_timing", "sf_ctx_get_timing",
     "sf_extract_features", "sf_forest_create", "sf_forest_destroy", "sf_fast_infer", "sf_route",
+    "sf_route_noalloc",
     "sf_universal_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
     "sf_serve_batch", "sf_serve_batch_host", "sf_serve_batch_intermediates",
     "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_lookup",
@@ -112,6 +115,7 @@ def _lib():
         L.sf_forest_create.argtypes = [V, I, U32, U32, U32, U32, V, V, V, C.POINTER(V)]
         L.sf_fast_infer.argtypes = [V, V, V, U32, V, V, V]
         L.sf_route.argtypes = [V, C.POINTER(sf_route_cfg), V, U32, U32, C.POINTER(sf_packets), V, V, V, V, V, V, V]
+        L.sf_route_noalloc.argtypes = [I, C.POINTER(sf_route_cfg), V, U32, U32, V, V, V, V, V, V, V]
         L.sf_universal_thresholds.argtypes = [V, C.c_uint64, V, U32, U32, V]
         L.sf_mlp_create.argtypes = [V, I, U32, V, C.POINTER(V), C.POINTER(V), C.POINTER(V)]
         L.sf_cnn_create.argtypes = [V, I, U32, U32, U32, U32, U32, U32, V, V, V, V, V, V, C.POINTER(V)]
@@ -237,6 +241,15 @@ def sf_route(ctx, cfg, fast_out, n, Cn, wide, esc_ids_out, n_esc_out, rows_out=N
     _check(_lib().sf_route(ctx, C.byref(cfg), _dp(fast_out), n, Cn, C.byref(wide) if wide is not None else None,
                            _dp(esc_ids_out), _dp(n_esc_out), _dp(rows_out), _dp(decision_out), _dp(label_fast_out),
                            _dp(score_out), _stream(stream)), "sf_route")
+
+
+def sf_route_noalloc(device, cfg, fast_out, n, Cn, esc_ids_out, n_esc_out, decision_out=None, label_fast_out=None,
+                     score_out=None, status_out=None, stream=None):
+    """Assignment (score, threshold, ascending ids, count) for callers that may not allocate
+    device memory: no context, scratch built into the library, n <= SF_NOALLOC_MAX_FLOWS."""
+    _check(_lib().sf_route_noalloc(device, C.byref(cfg), _dp(fast_out), n, Cn, _dp(esc_ids_out), _dp(n_esc_out),
+                                   _dp(decision_out), _dp(label_fast_out), _dp(score_out), _dp(status_out),
+                                   _stream(stream)), "sf_route_noalloc")
 
 
 def sf_universal_thresholds(scores, q_num, q_den=100):

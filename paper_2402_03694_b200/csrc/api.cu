@@ -30,6 +30,7 @@ extern "C" const char* sf_strerror(int status) {
     case SF_ERR_TABLE_FULL: return "flow table full";
     case SF_ERR_UNSUPPORTED: return "unsupported shape";
     case SF_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    case SF_ERR_STATIC_LIMIT: return "more flows than the built-in scratch of sf_route_noalloc holds (SF_NOALLOC_MAX_FLOWS)";
     }
     return "unknown status";
 }

@@ -292,3 +292,70 @@ extern "C" int sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_
     return sf_launch_route(ctx, cfg, fast_out, n, C, rows_out ? wide : nullptr, esc_ids_out, n_esc_out, rows_out,
                            decision_out, label_fast_out, score_out, scratch, (cudaStream_t)stream);
 }
+
+// ---- allocation-free variant of the assignment step --------------------------------
+// Scratch for sf_route_noalloc: one state block, the per-block counts and one decision
+// byte per flow.  It lives in the library image, so every GPU that loads the library
+// holds these bytes until the process exits.
+namespace {
+constexpr uint32_t kNoAllocBlocks = SF_NOALLOC_MAX_FLOWS / kScoreBlock;
+struct NoAllocScratch {
+    sf_dev_state state;
+    uint32_t block_counts[kNoAllocBlocks + 64];
+    uint8_t decision[SF_NOALLOC_MAX_FLOWS];
+};
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+namespace {
+constexpr int kMaxDevices = 64;
+NoAllocScratch* g_noalloc_ptr[kMaxDevices] = {};
+
+__global__ void noalloc_report_kernel(const sf_dev_state* st, int32_t* status_out) {
+    *status_out = st->counters.device_error;
+}
+}  // namespace
+
+extern "C" int sf_route_noalloc(int device, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,
+                                uint32_t* esc_ids_out, uint32_t* n_esc_out, uint8_t* decision_out,
+                                uint8_t* label_fast_out, float* score_out, int32_t* status_out, void* stream)
+{
+    if (!cfg || !fast_out || !esc_ids_out || !n_esc_out || !cfg->tau) return SF_ERR_ARG;
+    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT) return SF_ERR_ARG;
+    if (cfg->rule == SF_LC_GT && (C < 1 || C > 256)) return SF_ERR_ARG;
+    if (device < 0 || device >= kMaxDevices) return SF_ERR_ARG;
+    if (n > SF_NOALLOC_MAX_FLOWS) return SF_ERR_STATIC_LIMIT;
+    SF_CUDA(cudaSetDevice(device));
+    if (!g_noalloc_ptr[device]) {
+        // In host code the array's name is only a handle; the device address has to be asked for,
+        // once per device, with that device current.
+        void* p = nullptr;
+        SF_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        g_noalloc_ptr[device] = reinterpret_cast<NoAllocScratch*>(p);
+    }
+    NoAllocScratch* sc = g_noalloc_ptr[device];
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left: the state block must start at zero
+    SF_CUDA(cudaMemsetAsync(&sc->state, 0, sizeof(sf_dev_state), st));
+    const uint32_t nb = (n + kScoreBlock - 1) / kScoreBlock;
+    uint8_t* dec = decision_out ? decision_out : sc->decision;
+    if (n > 0) {
+        if (cfg->rule == SF_ABSMARGIN_LT)
+            score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast_out, score_out, sc->block_counts);
+        else
+            score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast_out, score_out, sc->block_counts);
+        SF_LAUNCH_CHECK("score_kernel");
+    }
+    scan_kernel<<<1, 1024, 0, st>>>(sc->block_counts, nb, n, cfg->capacity, n_esc_out, &sc->state);
+    SF_LAUNCH_CHECK("scan_kernel");
+    if (n > 0) {
+        scatter_kernel<<<nb, kScoreBlock, 0, st>>>(dec, n, sc->block_counts, cfg->capacity, esc_ids_out);
+        SF_LAUNCH_CHECK("scatter_kernel");
+    }
+    if (status_out) {
+        noalloc_report_kernel<<<1, 1, 0, st>>>(&sc->state, status_out);
+        SF_LAUNCH_CHECK("noalloc_report_kernel");
+    }
+    return SF_OK;
+}
