@@ -42,8 +42,10 @@ struct sf_forest {
     sf_ctx* ctx;
     int kind;
     uint32_t T, depth, F, C;
-    // nodes: per tree 2^depth entries of 8 bytes {thr, fid}, 1-based heap (entry 0 unused)
-    uint2* d_nodes;
+    // per-tree image of tree_stride bytes: 2^depth node entries of 8 bytes {thr bits, byte offset of the
+    // feature's row in the kernel's shared-memory tile}, 1-based heap (entry 0 unused), then (GBDT) 2^depth leaf scalars
+    unsigned char* d_image;
+    uint32_t tree_stride;
     // leaves: RF fp32[T][2^d][C]; GBDT fp32[T][2^d]
     float* d_leaf;
 };

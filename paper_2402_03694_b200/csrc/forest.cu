@@ -1,13 +1,18 @@
 // S2: tree-ensemble inference (the cascade's fast model).
 //
-// One thread per flow; a block owns a tile of flows whose feature rows sit in
-// shared memory transposed ([feature][flow], so a lane's read of x[fid] hits bank
-// = lane whatever fid is).  The ensemble streams through shared memory in chunks
-// of whole trees (8-byte nodes {thr, fid}, 1-based heap), double-buffered with
-// cp.async so the next chunk loads while the block walks the current one.  A
-// thread adds its leaf payloads in tree order t = 0..T-1, which fixes the fp32
-// summation order; random-forest leaf vectors are gathered from L2 one tree ahead
-// of their use so the gather latency hides behind the next tree's walk.
+// One thread per flow, 512 flows per block.  The block's feature rows sit in shared
+// memory transposed ([feature][flow], so a lane's read of x[fid] hits bank = lane
+// whatever fid is).  The ensemble streams through shared memory in chunks of whole
+// trees, double-buffered with cp.async so the next chunk loads while the block walks
+// the current one.  A node is 8 bytes {threshold bits, byte offset of its feature's
+// row in the tile}; trees are 1-based heaps.  A walk keeps the node's shared-memory
+// ADDRESS as its state (addr' = 2*addr + (go right ? 8 : 0) - base), so a level costs
+// six instructions: node load, feature address, feature load, compare, select, shift-add.
+// Each thread walks NCH trees of the chunk at once (independent dependency chains
+// hide the shared-memory latency), then adds their leaf payloads in tree order
+// t = 0..T-1, which fixes the fp32 summation order.  Random-forest leaf vectors are
+// gathered from L2 one group ahead of their use; boosted-tree leaf scalars travel
+// with their tree's nodes in the shared-memory image.
 #include "common.cuh"
 #include <new>
 #include <stdlib.h>
@@ -15,165 +20,241 @@
 
 namespace {
 
-constexpr int kChunkBytes = 32 * 1024;     // one depth-12 tree of 8-byte nodes
+constexpr uint32_t kB = 512;                       // flows (= threads) per block
+constexpr uint32_t kMaxSmem = 232448;              // 227 KB
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t saddr, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(saddr), "l"(gmem) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ uint32_t walk_tree(const uint2* __restrict__ nodes, const float* __restrict__ xcol,
-                                              uint32_t B, uint32_t depth) {
-    uint32_t i = 1;
-    for (uint32_t l = 0; l < depth; l++) {
-        uint2 nd = nodes[i];
-        float x = xcol[nd.y * B];
-        i = 2 * i + ((x <= __uint_as_float(nd.x)) ? 0u : 1u);
-    }
-    return i - (1u << depth);
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ float lds32f(uint32_t a) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(a));
+    return v;
 }
 
-// KIND: SF_RF (leaf = C-vector of class probabilities) or SF_GBDT (leaf = scalar, C = 1).
-template <int KIND, int C>
-__global__ void forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
-                              const uint2* __restrict__ nodes, const float* __restrict__ leaf,
-                              uint32_t T, uint32_t depth, uint32_t trees_per_chunk,
-                              float* __restrict__ out, uint16_t* __restrict__ leaf_idx)
+// Walk NCH consecutive trees (shared-memory images at base, base+stride, ...) for the
+// flow whose feature column starts at xbase; returns leaf indices.
+template <int NCH>
+__device__ __forceinline__ void walk(uint32_t base, uint32_t stride, uint32_t xbase, uint32_t depth, uint32_t (&leaf)[NCH]) {
+    uint32_t a[NCH], left[NCH], right[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; c++) {
+        const uint32_t b = base + c * stride;
+        a[c] = b + 8u;                 // node 1
+        left[c] = 0u - b;              // addr' = 2*addr - base      (child 2i)
+        right[c] = 8u - b;             // addr' = 2*addr - base + 8  (child 2i+1)
+    }
+    for (uint32_t l = 0; l < depth; l++) {
+        uint2 nd[NCH];
+        float x[NCH];
+#pragma unroll
+        for (int c = 0; c < NCH; c++) nd[c] = lds64(a[c]);
+#pragma unroll
+        for (int c = 0; c < NCH; c++) x[c] = lds32f(xbase + nd[c].y);
+#pragma unroll
+        for (int c = 0; c < NCH; c++) a[c] = 2u * a[c] + ((x[c] <= __uint_as_float(nd[c].x)) ? left[c] : right[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < NCH; c++) leaf[c] = ((a[c] - (base + c * stride)) >> 3) - (1u << depth);
+}
+
+template <int C>
+__device__ __forceinline__ void load_leaf_vec(const float* __restrict__ lv, float (&p)[C]) {
+    if ((C & 3) == 0) {
+#pragma unroll
+        for (int c = 0; c < C; c += 4) {
+            float4 v = __ldg(reinterpret_cast<const float4*>(lv + c));
+            p[c] = v.x; p[c + 1] = v.y; p[c + 2] = v.z; p[c + 3] = v.w;
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < C; c++) p[c] = __ldg(lv + c);
+    }
+}
+
+// KIND: SF_RF (leaf = C-vector of class probabilities in global memory) or SF_GBDT (leaf =
+// scalar stored behind the tree's nodes in the image, C = 1).  NCH: trees walked at once.
+template <int KIND, int C, int NCH>
+__global__ void __launch_bounds__(kB, 1)
+forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
+              const unsigned char* __restrict__ image, const float* __restrict__ leaf,
+              uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
+              float* __restrict__ out, uint16_t* __restrict__ leaf_idx)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const uint32_t B = blockDim.x;
-    uint2* buf0 = reinterpret_cast<uint2*>(smem_raw);
-    uint2* buf1 = reinterpret_cast<uint2*>(smem_raw + kChunkBytes);
-    float* xs = reinterpret_cast<float*>(smem_raw + 2 * kChunkBytes);       // [F][B]
-    const uint32_t f0 = blockIdx.x * B;
-    const uint32_t f = f0 + threadIdx.x;
+    const uint32_t sbuf0 = smem_u32(smem_raw);
+    float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][kB]
+    const uint32_t xbase = smem_u32(xs) + threadIdx.x * 4u;
+    const uint32_t f = blockIdx.x * kB + threadIdx.x;
     const bool live = f < n;
-    const uint32_t tree_nodes = 1u << depth;                 // entries per tree (entry 0 unused)
+    const uint32_t n_leaf = 1u << depth;
     const uint32_t n_chunks = (T + trees_per_chunk - 1) / trees_per_chunk;
 
-    auto issue_chunk = [&](uint32_t ck, uint2* dst) {
-        uint32_t t0 = ck * trees_per_chunk;
-        uint32_t nt = min(trees_per_chunk, T - t0);
-        uint32_t vecs = nt * tree_nodes / 2;                 // 16-byte units
-        const uint4* src = reinterpret_cast<const uint4*>(nodes + (size_t)t0 * tree_nodes);
-        uint4* d4 = reinterpret_cast<uint4*>(dst);
-        for (uint32_t v = threadIdx.x; v < vecs; v += B) cp_async16(d4 + v, src + v);
+    auto issue_chunk = [&](uint32_t ck) {
+        const uint32_t t0 = ck * trees_per_chunk;
+        const uint32_t nt = min(trees_per_chunk, T - t0);
+        const uint32_t vecs = nt * (tree_stride >> 4);
+        const uint4* src = reinterpret_cast<const uint4*>(image + (size_t)t0 * tree_stride);
+        const uint32_t dst = sbuf0 + (ck & 1u) * chunk_bytes;
+        for (uint32_t v = threadIdx.x; v < vecs; v += kB) cp_async16(dst + v * 16u, src + v);
         cp_async_commit();
     };
 
-    issue_chunk(0, buf0);
-    // feature tile, transposed
+    issue_chunk(0);
     if (live) {
         const float* row = feat + (size_t)f * F;
         if ((F & 3) == 0) {
             for (uint32_t j = 0; j < F; j += 4) {
                 float4 v = __ldg(reinterpret_cast<const float4*>(row + j));
-                xs[(j + 0) * B + threadIdx.x] = v.x; xs[(j + 1) * B + threadIdx.x] = v.y;
-                xs[(j + 2) * B + threadIdx.x] = v.z; xs[(j + 3) * B + threadIdx.x] = v.w;
+                xs[(j + 0) * kB + threadIdx.x] = v.x; xs[(j + 1) * kB + threadIdx.x] = v.y;
+                xs[(j + 2) * kB + threadIdx.x] = v.z; xs[(j + 3) * kB + threadIdx.x] = v.w;
             }
         } else {
-            for (uint32_t j = 0; j < F; j++) xs[j * B + threadIdx.x] = row[j];
+            for (uint32_t j = 0; j < F; j++) xs[j * kB + threadIdx.x] = row[j];
         }
     } else {
-        for (uint32_t j = 0; j < F; j++) xs[j * B + threadIdx.x] = 0.0f;
+        for (uint32_t j = 0; j < F; j++) xs[j * kB + threadIdx.x] = 0.0f;
     }
 
     float acc[C];
-    float pend[C];
+    float pend[NCH][C];
 #pragma unroll
-    for (int c = 0; c < C; c++) { acc[c] = 0.0f; pend[c] = 0.0f; }
-    bool have_pend = false;
-    const float* xcol = xs + threadIdx.x;
+    for (int c = 0; c < C; c++) acc[c] = 0.0f;
+    int n_pend = 0;                                   // leaf vectors in flight (RF)
+
+    auto flush_pending = [&]() {
+#pragma unroll
+        for (int k = 0; k < NCH; k++)
+            if (k < n_pend) {
+#pragma unroll
+                for (int c = 0; c < C; c++) acc[c] = __fadd_rn(acc[c], pend[k][c]);
+            }
+        n_pend = 0;
+    };
 
     for (uint32_t ck = 0; ck < n_chunks; ck++) {
-        uint2* cur = (ck & 1) ? buf1 : buf0;
-        if (ck + 1 < n_chunks) { issue_chunk(ck + 1, (ck & 1) ? buf0 : buf1); cp_async_wait<1>(); }
+        if (ck + 1 < n_chunks) { issue_chunk(ck + 1); cp_async_wait<1>(); }
         else cp_async_wait<0>();
         __syncthreads();
+        const uint32_t cur = sbuf0 + (ck & 1u) * chunk_bytes;
         const uint32_t t0 = ck * trees_per_chunk;
         const uint32_t nt = min(trees_per_chunk, T - t0);
-        for (uint32_t tt = 0; tt < nt; tt++) {
-            const uint32_t t = t0 + tt;
-            const uint32_t l = walk_tree(cur + (size_t)tt * tree_nodes, xcol, B, depth);
-            if (leaf_idx && live) leaf_idx[(size_t)f * T + t] = (uint16_t)l;
+        uint32_t tt = 0;
+        for (; tt + NCH <= nt; tt += NCH) {
+            uint32_t l[NCH];
+            walk<NCH>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
+            if (leaf_idx && live) {
+#pragma unroll
+                for (int k = 0; k < NCH; k++) leaf_idx[(size_t)f * T + t0 + tt + k] = (uint16_t)l[k];
+            }
             if (KIND == SF_GBDT) {
-                acc[0] = __fadd_rn(acc[0], __ldg(leaf + (size_t)t * tree_nodes + l));
+                float v[NCH];
+#pragma unroll
+                for (int k = 0; k < NCH; k++) v[k] = lds32f(cur + (tt + k) * tree_stride + n_leaf * 8u + l[k] * 4u);
+#pragma unroll
+                for (int k = 0; k < NCH; k++) acc[0] = __fadd_rn(acc[0], v[k]);
             } else {
-                // add the previous tree's vector (already in flight), then fetch this one
-                if (have_pend) {
+                flush_pending();                      // the previous group's vectors have landed by now
 #pragma unroll
-                    for (int c = 0; c < C; c++) acc[c] = __fadd_rn(acc[c], pend[c]);
-                }
-                const float* lv = leaf + ((size_t)t * tree_nodes + l) * C;
-                if ((C & 3) == 0) {
-#pragma unroll
-                    for (int c = 0; c < C; c += 4) {
-                        float4 v = __ldg(reinterpret_cast<const float4*>(lv + c));
-                        pend[c] = v.x; pend[c + 1] = v.y; pend[c + 2] = v.z; pend[c + 3] = v.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < C; c++) pend[c] = __ldg(lv + c);
-                }
-                have_pend = true;
+                for (int k = 0; k < NCH; k++)
+                    load_leaf_vec<C>(leaf + ((size_t)(t0 + tt + k) * n_leaf + l[k]) * C, pend[k]);
+                n_pend = NCH;
             }
         }
-        __syncthreads();          // everyone is done with `cur` before it is refilled
+        for (; tt < nt; tt++) {                       // ragged end of the chunk: one tree at a time
+            uint32_t l[1];
+            walk<1>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
+            if (leaf_idx && live) leaf_idx[(size_t)f * T + t0 + tt] = (uint16_t)l[0];
+            if (KIND == SF_GBDT) {
+                acc[0] = __fadd_rn(acc[0], lds32f(cur + tt * tree_stride + n_leaf * 8u + l[0] * 4u));
+            } else {
+                flush_pending();
+                load_leaf_vec<C>(leaf + ((size_t)(t0 + tt) * n_leaf + l[0]) * C, pend[0]);
+                n_pend = 1;
+            }
+        }
+        __syncthreads();          // everyone is done with this buffer before it is refilled
     }
+    if (KIND == SF_RF) flush_pending();
     if (!live) return;
     if (KIND == SF_GBDT) {
         out[f] = acc[0];
     } else {
         const float fT = __uint2float_rn(T);
 #pragma unroll
-        for (int c = 0; c < C; c++) {
-            float a = have_pend ? __fadd_rn(acc[c], pend[c]) : acc[c];
-            out[(size_t)f * C + c] = __fdiv_rn(a, fT);
-        }
+        for (int c = 0; c < C; c++) out[(size_t)f * C + c] = __fdiv_rn(acc[c], fT);
     }
 }
 
-template <int KIND, int C>
-int launch(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
-    const uint32_t tree_bytes = (1u << fo->depth) * 8u;
-    const uint32_t tpc = kChunkBytes / tree_bytes;                 // >= 1 for depth <= 12
-    // block of 512 flows while the feature tile fits, else 256
-    uint32_t B = 512;
-    size_t smem = 2 * (size_t)kChunkBytes + (size_t)fo->F * B * sizeof(float);
-    if (smem > 200 * 1024) { B = 256; smem = 2 * (size_t)kChunkBytes + (size_t)fo->F * B * sizeof(float); }
-    auto k = forest_kernel<KIND, C>;
-    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const uint32_t grid = (n + B - 1) / B;
-    k<<<grid, B, smem, st>>>(feat, n, fo->F, fo->d_nodes, fo->d_leaf, fo->T, fo->depth, tpc, out, leaf_idx);
+struct Plan { uint32_t chunk_bytes, tpc, nch; size_t smem; };
+
+Plan make_plan(const sf_forest* fo) {
+    Plan p;
+    const size_t feat_bytes = (size_t)fo->F * kB * sizeof(float);
+    p.chunk_bytes = (feat_bytes + 2 * 65536 <= kMaxSmem) ? 65536u : 32768u;
+    p.tpc = p.chunk_bytes / fo->tree_stride;          // >= 1: a depth-12 tree is 32 KB
+    if (p.tpc > fo->T) p.tpc = fo->T;
+    p.nch = (fo->kind == SF_GBDT) ? (p.tpc >= 4 ? 4u : (p.tpc >= 2 ? 2u : 1u)) : (p.tpc >= 2 ? 2u : 1u);
+    p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes;
+    return p;
+}
+
+template <int KIND, int C, int NCH>
+int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+    auto k = forest_kernel<KIND, C, NCH>;
+    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
+    const uint32_t grid = (n + kB - 1) / kB;
+    k<<<grid, kB, p.smem, st>>>(feat, n, fo->F, fo->d_image, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
+                                p.chunk_bytes, out, leaf_idx);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
+}
+
+template <int C>
+int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+    const Plan p = make_plan(fo);
+    if (p.nch == 2) return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st);
+    return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st);
+}
+
+int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+    const Plan p = make_plan(fo);
+    if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st);
+    if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st);
+    return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st);
 }
 
 }  // namespace
 
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
     if (n == 0) return SF_OK;
-    if (fo->kind == SF_GBDT) return launch<SF_GBDT, 1>(fo, feat, n, out, leaf_idx, st);
+    if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st);
     switch (fo->C) {
-    case 1:  return launch<SF_RF, 1>(fo, feat, n, out, leaf_idx, st);
-    case 2:  return launch<SF_RF, 2>(fo, feat, n, out, leaf_idx, st);
-    case 3:  return launch<SF_RF, 3>(fo, feat, n, out, leaf_idx, st);
-    case 4:  return launch<SF_RF, 4>(fo, feat, n, out, leaf_idx, st);
-    case 5:  return launch<SF_RF, 5>(fo, feat, n, out, leaf_idx, st);
-    case 6:  return launch<SF_RF, 6>(fo, feat, n, out, leaf_idx, st);
-    case 7:  return launch<SF_RF, 7>(fo, feat, n, out, leaf_idx, st);
-    case 8:  return launch<SF_RF, 8>(fo, feat, n, out, leaf_idx, st);
-    case 9:  return launch<SF_RF, 9>(fo, feat, n, out, leaf_idx, st);
-    case 10: return launch<SF_RF, 10>(fo, feat, n, out, leaf_idx, st);
-    case 11: return launch<SF_RF, 11>(fo, feat, n, out, leaf_idx, st);
-    case 12: return launch<SF_RF, 12>(fo, feat, n, out, leaf_idx, st);
-    case 13: return launch<SF_RF, 13>(fo, feat, n, out, leaf_idx, st);
-    case 14: return launch<SF_RF, 14>(fo, feat, n, out, leaf_idx, st);
-    case 15: return launch<SF_RF, 15>(fo, feat, n, out, leaf_idx, st);
-    case 16: return launch<SF_RF, 16>(fo, feat, n, out, leaf_idx, st);
+    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st);
+    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st);
+    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st);
+    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st);
+    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st);
+    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st);
+    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st);
+    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st);
+    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st);
+    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st);
+    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st);
+    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st);
+    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st);
+    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st);
+    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st);
+    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st);
     }
     return SF_ERR_UNSUPPORTED;
 }
@@ -191,22 +272,29 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     sf_forest* fo = new (std::nothrow) sf_forest();
     if (!fo) return SF_ERR_ALLOC;
     fo->ctx = ctx; fo->kind = kind; fo->T = T; fo->depth = depth; fo->F = F; fo->C = (kind == SF_GBDT) ? 1 : C;
-    fo->d_nodes = nullptr; fo->d_leaf = nullptr;
-    // 1-based heap: host node i (0-based, children 2i+1 / 2i+2) becomes entry i+1 (children 2j, 2j+1)
-    uint2* h = (uint2*)malloc(sizeof(uint2) * (size_t)T * n_ent);
+    fo->d_image = nullptr; fo->d_leaf = nullptr;
+    // Image of one tree: 2^d node entries of 8 bytes in a 1-based heap (host node i, children
+    // 2i+1 / 2i+2, becomes entry i+1, children 2j / 2j+1; entry 0 unused), then for boosted
+    // trees the 2^d leaf scalars; padded to a multiple of 16 bytes for the 16-byte copies.
+    uint32_t stride = n_ent * 8u + (kind == SF_GBDT ? n_ent * 4u : 0u);
+    stride = (stride + 15u) & ~15u;
+    fo->tree_stride = stride;
+    unsigned char* h = (unsigned char*)calloc((size_t)T, stride);
     if (!h) { delete fo; return SF_ERR_ALLOC; }
     for (uint32_t t = 0; t < T; t++) {
-        h[(size_t)t * n_ent] = make_uint2(0u, 0u);
+        uint32_t* ent = reinterpret_cast<uint32_t*>(h + (size_t)t * stride);
         for (uint32_t i = 0; i < n_int; i++) {
             uint32_t bits; float v = thr[(size_t)t * n_int + i];
             memcpy(&bits, &v, 4);
-            h[(size_t)t * n_ent + i + 1] = make_uint2(bits, (uint32_t)fid[(size_t)t * n_int + i]);
+            ent[2 * (i + 1)] = bits;
+            ent[2 * (i + 1) + 1] = (uint32_t)fid[(size_t)t * n_int + i] * kB * 4u;     // byte offset of the feature's row
         }
+        if (kind == SF_GBDT) memcpy(h + (size_t)t * stride + n_ent * 8u, leaf + (size_t)t * n_ent, n_ent * 4u);
     }
-    size_t leaf_count = (size_t)T * n_ent * fo->C;
-    cudaError_t e = cudaMalloc(&fo->d_nodes, sizeof(uint2) * (size_t)T * n_ent);
+    const size_t leaf_count = (size_t)T * n_ent * fo->C;
+    cudaError_t e = cudaMalloc(&fo->d_image, (size_t)T * stride);
     if (e == cudaSuccess) e = cudaMalloc(&fo->d_leaf, sizeof(float) * leaf_count);
-    if (e == cudaSuccess) e = cudaMemcpy(fo->d_nodes, h, sizeof(uint2) * (size_t)T * n_ent, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(fo->d_image, h, (size_t)T * stride, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(fo->d_leaf, leaf, sizeof(float) * leaf_count, cudaMemcpyHostToDevice);
     free(h);
     if (e != cudaSuccess) { sf_forest_destroy(fo); return sf_set_cuda_error(e, "sf_forest_create"); }
@@ -216,7 +304,7 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
 
 extern "C" void sf_forest_destroy(sf_forest* fo) {
     if (!fo) return;
-    if (fo->d_nodes) cudaFree(fo->d_nodes);
+    if (fo->d_image) cudaFree(fo->d_image);
     if (fo->d_leaf) cudaFree(fo->d_leaf);
     delete fo;
 }

@@ -55,25 +55,29 @@ template <uint32_t BN> struct GemmCfg {
     static constexpr uint32_t kStageBytesA = BM * BK * 2;
     static constexpr uint32_t kStageBytesB = BN * BK * 2;
     static constexpr uint32_t kStageBytes = kStageBytesA + kStageBytesB;
-    static constexpr uint32_t kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr uint32_t kTmemCols = 2 * BN;
+    static constexpr uint32_t kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : (BN == 64 ? 8 : 10));
+    static constexpr uint32_t kTmemCols = 2 * BN;             // a power of two >= 32
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct GemmBars {
-    uint64_t full[8];
-    uint64_t empty[8];
+    uint64_t full[10];
+    uint64_t empty[10];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
 
-template <uint32_t BN>
+// HEAD = false: hidden layer, out = bf16(ReLU(acc + bias)) [rows][N].
+// HEAD = true (BN = 16): last layer, W zero-padded to 16 rows; logits[r][c] = acc + bias for
+// c < C (fp32, no activation) and label[r] = argmax (lowest index on ties).
+template <uint32_t BN, bool HEAD>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                            const float* __restrict__ bias, const uint32_t* __restrict__ n_rows_dev,
-                           uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out, sf_dev_state* st)
+                           uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out, sf_dev_state* st,
+                           float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C)
 {
     using Cfg = GemmCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
@@ -162,6 +166,23 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             const uint32_t row = tm * BM + quarter * 32u + lane;
             const uint32_t col0 = tn * BN;
             const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BN;
+            if constexpr (HEAD) {
+                uint32_t v[16];
+                tmem_ld16(taddr, v);
+                tmem_ld_wait();
+                if (row < n_rows) {
+                    uint32_t a = 0; float mx = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < 16; c++) {
+                        if ((uint32_t)c < C) {
+                            float x = __uint_as_float(v[c]) + __ldg(bias + c);
+                            logits[(size_t)row * C + c] = x;
+                            if (c == 0 || x > mx) { mx = x; a = c; }
+                        }
+                    }
+                    if (label) label[row] = (uint8_t)a;
+                }
+            } else {
             __nv_bfloat16* orow = out + (size_t)row * N + col0;
 #pragma unroll 1
             for (uint32_t c = 0; c < BN; c += 32) {
@@ -182,6 +203,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                     for (int q = 0; q < 4; q++)
                         dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
                 }
+            }
             }
             tc_fence_before();
             __syncwarp();
@@ -277,13 +299,32 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     if (rc != SF_OK) return rc;
     rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
     if (rc != SF_OK) return rc;
-    auto k = gemm_bias_relu_bf16_kernel<BN>;
+    auto k = gemm_bias_relu_bf16_kernel<BN, false>;
     SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes));
     uint32_t max_tiles = ((capacity + BM - 1) / BM) * (N / BN);
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
-                                                  reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state);
+                                                  reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state, nullptr, nullptr, 0);
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel");
+    return SF_OK;
+}
+
+// last layer on the tensor cores: one 128 x 16 tile per 128 rows, W padded to 16 rows
+int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bias, const uint32_t* n_rows_dev,
+                   uint32_t capacity, uint32_t K, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
+{
+    using Cfg = GemmCfg<16>;
+    CUtensorMap tmA, tmW;
+    int rc = encode_tmap_bf16_2d(&tmA, A, capacity, K, BM, BK);
+    if (rc != SF_OK) return rc;
+    rc = encode_tmap_bf16_2d(&tmW, W16, 16, K, 16, BK);
+    if (rc != SF_OK) return rc;
+    auto k = gemm_bias_relu_bf16_kernel<16, true>;
+    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes));
+    uint32_t max_tiles = (capacity + BM - 1) / BM;
+    uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
+    k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C);
+    SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(head)");
     return SF_OK;
 }
 
@@ -325,7 +366,7 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     sf_time_end(ctx, SF_T_GEMM, st);
     const uint32_t L = s->n_layers - 1;
     sf_time_begin(ctx, SF_T_HEAD, st);
-    int rc = sf_launch_head_bf16(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st);
+    int rc = launch_head_tc(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st);
     sf_time_end(ctx, SF_T_HEAD, st);
     return rc;
 }

@@ -166,11 +166,14 @@ extern "C" int sf_mlp_create(sf_ctx* ctx, int dtype, uint32_t n_layers, const ui
         if (e == cudaSuccess) e = cudaMemcpy(s->d_b[l], b[l], sizeof(float) * dims[l + 1], cudaMemcpyHostToDevice);
         if (e != cudaSuccess) break;
         if (dtype == SF_BF16) {
-            uint16_t* h = (uint16_t*)malloc(cnt * 2);
+            // the last layer runs as a 128 x 16 tensor-core tile: pad its rows to 16 with zeros
+            const size_t rows_pad = (l + 1 == n_layers) ? 16 : dims[l + 1];
+            const size_t cnt_pad = rows_pad * dims[l];
+            uint16_t* h = (uint16_t*)calloc(cnt_pad, 2);
             if (!h) { sf_slow_destroy(s); return SF_ERR_ALLOC; }
             f32_to_bf16_host(W[l], h, cnt);
-            e = cudaMalloc(&s->d_W[l], cnt * 2);
-            if (e == cudaSuccess) e = cudaMemcpy(s->d_W[l], h, cnt * 2, cudaMemcpyHostToDevice);
+            e = cudaMalloc(&s->d_W[l], cnt_pad * 2);
+            if (e == cudaSuccess) e = cudaMemcpy(s->d_W[l], h, cnt_pad * 2, cudaMemcpyHostToDevice);
             free(h);
         } else {
             e = cudaMalloc(&s->d_W[l], cnt * 4);
