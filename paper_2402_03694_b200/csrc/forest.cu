@@ -3,8 +3,9 @@
 // One thread per flow, 512 flows per block.  The block's feature rows sit in shared
 // memory transposed ([feature][flow], so a lane's read of x[fid] hits bank = lane
 // whatever fid is).  The ensemble streams through shared memory in chunks of whole
-// trees, double-buffered with cp.async so the next chunk loads while the block walks
-// the current one.  A node is 8 bytes {threshold bits, byte offset of its feature's
+// trees: one thread issues a bulk copy (cp.async.bulk, completion on an mbarrier) of the
+// next chunk into the other buffer while the block walks the current one, so the copy
+// costs no load/store instructions.  A node is 8 bytes {threshold bits, byte offset of its feature's
 // row in the tile}; trees are 1-based heaps.  A walk keeps the node's shared-memory
 // ADDRESS as its state (addr' = 2*addr + (go right ? 8 : 0) - base), so a level costs
 // six instructions: node load, feature address, feature load, compare, select, shift-add.
@@ -13,7 +14,7 @@
 // t = 0..T-1, which fixes the fp32 summation order.  Random-forest leaf vectors are
 // gathered from L2 one group ahead of their use; boosted-tree leaf scalars travel
 // with their tree's nodes in the shared-memory image.
-#include "common.cuh"
+#include "tc_common.cuh"
 #include <new>
 #include <stdlib.h>
 #include <string.h>
@@ -24,12 +25,6 @@ constexpr uint32_t kB = 512;                       // flows (= threads) per bloc
 constexpr uint32_t kMaxSmem = 232448;              // 227 KB
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(uint32_t saddr, const void* gmem) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(saddr), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 __device__ __forceinline__ uint2 lds64(uint32_t a) {
     uint2 v;
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
@@ -69,7 +64,15 @@ __device__ __forceinline__ void walk(uint32_t base, uint32_t stride, uint32_t xb
 
 template <int C>
 __device__ __forceinline__ void load_leaf_vec(const float* __restrict__ lv, float (&p)[C]) {
-    if ((C & 3) == 0) {
+    if ((C & 7) == 0) {
+        // 32-byte vectors: one 256-bit load touches one sector per lane
+#pragma unroll
+        for (int c = 0; c < C; c += 8)
+            asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                         : "=f"(p[c]), "=f"(p[c + 1]), "=f"(p[c + 2]), "=f"(p[c + 3]),
+                           "=f"(p[c + 4]), "=f"(p[c + 5]), "=f"(p[c + 6]), "=f"(p[c + 7])
+                         : "l"(lv + c));
+    } else if ((C & 3) == 0) {
 #pragma unroll
         for (int c = 0; c < C; c += 4) {
             float4 v = __ldg(reinterpret_cast<const float4*>(lv + c));
@@ -88,28 +91,35 @@ __global__ void __launch_bounds__(kB, 1)
 forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
               const unsigned char* __restrict__ image, const float* __restrict__ leaf,
               uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
-              float* __restrict__ out, uint16_t* __restrict__ leaf_idx)
+              float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t sbuf0 = smem_u32(smem_raw);
     float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][kB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * kB * 4);   // [2] + flag
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2);
     const uint32_t xbase = smem_u32(xs) + threadIdx.x * 4u;
     const uint32_t f = blockIdx.x * kB + threadIdx.x;
     const bool live = f < n;
     const uint32_t n_leaf = 1u << depth;
     const uint32_t n_chunks = (T + trees_per_chunk - 1) / trees_per_chunk;
 
+    // called by thread 0 only; the buffer's previous readers have passed a __syncthreads
     auto issue_chunk = [&](uint32_t ck) {
         const uint32_t t0 = ck * trees_per_chunk;
         const uint32_t nt = min(trees_per_chunk, T - t0);
-        const uint32_t vecs = nt * (tree_stride >> 4);
-        const uint4* src = reinterpret_cast<const uint4*>(image + (size_t)t0 * tree_stride);
-        const uint32_t dst = sbuf0 + (ck & 1u) * chunk_bytes;
-        for (uint32_t v = threadIdx.x; v < vecs; v += kB) cp_async16(dst + v * 16u, src + v);
-        cp_async_commit();
+        const uint32_t bytes = nt * tree_stride;                         // a multiple of 16
+        sftc::mbar_expect_tx(&bars[ck & 1u], bytes);
+        sftc::bulk_load(smem_raw + (size_t)(ck & 1u) * chunk_bytes, image + (size_t)t0 * tree_stride, bytes, &bars[ck & 1u]);
     };
 
-    issue_chunk(0);
+    if (threadIdx.x == 0) {
+        sftc::mbar_init(&bars[0], 1);
+        sftc::mbar_init(&bars[1], 1);
+        *abort_flag = 0;
+        sftc::fence_barrier_init();
+        issue_chunk(0);
+    }
     if (live) {
         const float* row = feat + (size_t)f * F;
         if ((F & 3) == 0) {
@@ -142,9 +152,10 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
     };
 
     for (uint32_t ck = 0; ck < n_chunks; ck++) {
-        if (ck + 1 < n_chunks) { issue_chunk(ck + 1); cp_async_wait<1>(); }
-        else cp_async_wait<0>();
-        __syncthreads();
+        if (ck == 0) __syncthreads();             // barriers initialised, feature tile written
+        if (threadIdx.x == 0 && ck + 1 < n_chunks) issue_chunk(ck + 1);
+        // every thread waits for this chunk's bytes (bounded: all give up together if they never land)
+        if (!sftc::mbar_wait(&bars[ck & 1u], (ck >> 1) & 1u, abort_flag)) break;
         const uint32_t cur = sbuf0 + (ck & 1u) * chunk_bytes;
         const uint32_t t0 = ck * trees_per_chunk;
         const uint32_t nt = min(trees_per_chunk, T - t0);
@@ -185,6 +196,7 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         __syncthreads();          // everyone is done with this buffer before it is refilled
     }
     if (KIND == SF_RF) flush_pending();
+    if (*abort_flag) { if (threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT); return; }
     if (!live) return;
     if (KIND == SF_GBDT) {
         out[f] = acc[0];
@@ -200,11 +212,11 @@ struct Plan { uint32_t chunk_bytes, tpc, nch; size_t smem; };
 Plan make_plan(const sf_forest* fo) {
     Plan p;
     const size_t feat_bytes = (size_t)fo->F * kB * sizeof(float);
-    p.chunk_bytes = (feat_bytes + 2 * 65536 <= kMaxSmem) ? 65536u : 32768u;
+    p.chunk_bytes = (feat_bytes + 2 * 65536 + 32 <= kMaxSmem) ? 65536u : 32768u;
     p.tpc = p.chunk_bytes / fo->tree_stride;          // >= 1: a depth-12 tree is 32 KB
     if (p.tpc > fo->T) p.tpc = fo->T;
     p.nch = (fo->kind == SF_GBDT) ? (p.tpc >= 4 ? 4u : (p.tpc >= 2 ? 2u : 1u)) : (p.tpc >= 2 ? 2u : 1u);
-    p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes;
+    p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes + 32;       // + two mbarriers and the abort flag
     return p;
 }
 
@@ -214,7 +226,7 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
     SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
     const uint32_t grid = (n + kB - 1) / kB;
     k<<<grid, kB, p.smem, st>>>(feat, n, fo->F, fo->d_image, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
-                                p.chunk_bytes, out, leaf_idx);
+                                p.chunk_bytes, out, leaf_idx, fo->ctx->d_state);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
 }
