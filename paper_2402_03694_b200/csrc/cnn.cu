@@ -1,9 +1,342 @@
-// S4 (1-D CNN): placeholder translation unit until the fused tcgen05 kernel lands.
+// S4 (1-D CNN slow model), one fused kernel per batch of assigned flows:
+//   conv1 (k=5, 8 -> 64) + ReLU -> conv2 (k=5, 64 -> 128) + ReLU -> mean over the 128
+//   positions -> linear 128 -> n_cls -> argmax.
+// Both convolutions run on the tcgen05 tensor cores as implicit GEMMs with one flow's
+// 128 positions as the M = 128 rows of a tile; nothing but the 2 KB input row and the
+// logits ever touches global memory.
+//
+// How the shifted ("same" padded) operands are expressed without im2col.  Activations
+// are kept in shared memory in the un-swizzled core-matrix layout: for every group of
+// 8 channels a column of 16-byte rows, one row per position, with two zero rows above
+// and below.  In that layout a matrix descriptor's start address may be moved by whole
+// rows, so tap t of a convolution is the same buffer started t rows further down; the
+// zero rows supply the padding.  For conv1 (8 input channels = one 16-byte row per
+// position) consecutive taps are consecutive rows, so a K = 16 step (two taps) uses a
+// K-direction stride of 16 bytes: the im2col matrix is never materialised.
+//
+// Persistent CTAs, one per SM, loop over flows.  Warp 0 streams input rows with bulk
+// copies into a ring; warp 1 issues the MMAs (3 for conv1, 20 for conv2 per flow) in the
+// order conv1(i+1), conv2(i) so that the first epilogue of the next flow overlaps the
+// second convolution of this one; warps 2..5 are the epilogues: E1 turns the conv1
+// accumulators (TMEM) into bf16 activations in shared memory (conv2's A operand), E2
+// applies bias + ReLU + bf16 rounding to the conv2 accumulators, reduces over positions
+// with a fixed shuffle tree (deterministic), and evaluates the linear head.
+// Accumulators, activations and input rows are all double (or more) buffered.
+// Every wait is bounded; on a timeout the block records SF_ERR_DEVICE_TIMEOUT and leaves.
 #include "tc_common.cuh"
+#include <stdlib.h>
+#include <string.h>
 
-int sf_cnn_prepare(sf_slow*, const float*, const float*, const float*, const float*, const float*, const float*) {
-    return SF_ERR_UNSUPPORTED;
+namespace {
+using namespace sftc;
+
+constexpr uint32_t L = 128, CIN = 8, C1 = 64, C2 = 128, KW = 5, NCLS_MAX = 16;
+constexpr uint32_t kThreads = 192;
+constexpr uint32_t XS = 4;                                  // input-row ring depth
+constexpr uint32_t X_STAGE = (2 + L + 3) * 16;              // 2 zero rows, 128 rows, 3 zero rows (tap 5 is a zero tap)
+constexpr uint32_t H1_COL = (2 + L + 2) * 16;               // one 8-channel column of conv1's output: 2112 bytes
+constexpr uint32_t H1_BYTES = (C1 / 8) * H1_COL;            // 16,896
+// weight blob (device and shared memory share this layout)
+constexpr uint32_t W2_OFF = 0;                              // [5 taps][8 k-chunks][128 n][8] bf16
+constexpr uint32_t W2_BYTES = KW * (C1 / 8) * C2 * 16;      // 81,920
+constexpr uint32_t W1_OFF = W2_OFF + W2_BYTES;              // [6 taps][64 n][8] bf16 (tap 5 = 0)
+constexpr uint32_t W1_BYTES = 6 * C1 * 16;                  // 6,144
+constexpr uint32_t W3_OFF = W1_OFF + W1_BYTES;              // fp32 [16][128]
+constexpr uint32_t W3_BYTES = NCLS_MAX * C2 * 4;            // 8,192
+constexpr uint32_t B1_OFF = W3_OFF + W3_BYTES;              // fp32 [64]
+constexpr uint32_t B2_OFF = B1_OFF + C1 * 4;                // fp32 [128]
+constexpr uint32_t B3_OFF = B2_OFF + C2 * 4;                // fp32 [16]
+constexpr uint32_t BLOB_BYTES = B3_OFF + NCLS_MAX * 4;      // 97,088
+// shared memory map
+constexpr uint32_t SM_BLOB = 0;
+constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // 2 buffers
+constexpr uint32_t SM_X = SM_H1 + 2 * H1_BYTES;             // XS stages
+constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // fp32 [4 warps][128] column partial sums
+constexpr uint32_t SM_LOGIT = SM_PART + 4 * C2 * 4;         // fp32 [16]
+constexpr uint32_t SM_BARS = SM_LOGIT + 64;
+constexpr uint32_t SM_TOTAL = SM_BARS + 256;
+static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_X % 16 == 0 && SM_BARS % 8 == 0, "alignment");
+
+struct Bars {
+    uint64_t w_full;
+    uint64_t x_full[XS], x_empty[XS];
+    uint64_t d1_full[2], d1_empty[2], h1_full[2], h1_empty[2], d2_full[2], d2_empty[2];
+    uint32_t tmem_base, abort_flag;
+};
+static_assert(sizeof(Bars) <= 256, "barrier block");
+
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
-int sf_cnn_bf16_forward(sf_ctx*, const sf_slow*, const void*, const uint32_t*, uint32_t, float*, uint8_t*, void*, cudaStream_t) {
-    return SF_ERR_UNSUPPORTED;
+
+// sum over the 32 lanes of each of 32 per-lane values; lane l ends up with column l's total.
+// The order of additions is a fixed tree, so the result is reproducible run to run.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], uint32_t lane) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const bool up = (lane & off) != 0;
+#pragma unroll
+        for (int j = 0; j < off; j++) {
+            const float keep = up ? v[j + off] : v[j];
+            const float send = up ? v[j] : v[j + off];
+            v[j] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
+        }
+    }
+    return v[0];
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restrict__ n_rows_dev,
+                 const unsigned char* __restrict__ blob, uint32_t n_cls,
+                 float* __restrict__ logits, uint8_t* __restrict__ label, sf_dev_state* st)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    Bars* bars = reinterpret_cast<Bars*>(smem + SM_BARS);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t n_rows = *n_rows_dev;
+    // flows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+    const uint32_t n_mine = (n_rows > blockIdx.x) ? (n_rows - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    // zero everything that acts as padding (and the rest of the activation buffers)
+    for (uint32_t i = threadIdx.x; i < (2 * H1_BYTES + XS * X_STAGE) / 16; i += kThreads)
+        reinterpret_cast<uint4*>(smem + SM_H1)[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) {
+        mbar_init(&bars->w_full, 1);
+        for (uint32_t s = 0; s < XS; s++) { mbar_init(&bars->x_full[s], 1); mbar_init(&bars->x_empty[s], 1); }
+        for (uint32_t b = 0; b < 2; b++) {
+            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], 4);
+            mbar_init(&bars->h1_full[b], 4); mbar_init(&bars->h1_empty[b], 1);
+            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], 4);
+        }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+    }
+    fence_proxy_async();                       // the zero fill must be visible to the tensor-core reads
+    if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0 && n_mine > 0) {
+            mbar_expect_tx(&bars->w_full, BLOB_BYTES);
+            bulk_load(smem + SM_BLOB, blob, BLOB_BYTES, &bars->w_full);
+            for (uint32_t i = 0; i < n_mine; i++) {
+                const uint32_t s = i % XS, ph = (i / XS) & 1u;
+                if (!mbar_wait(&bars->x_empty[s], ph ^ 1u, abort_flag)) break;
+                const uint32_t r = blockIdx.x + i * gridDim.x;
+                mbar_expect_tx(&bars->x_full[s], L * CIN * 2);
+                bulk_load(smem + SM_X + s * X_STAGE + 32, rows + (size_t)r * L * CIN, L * CIN * 2, &bars->x_full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && n_mine > 0) {
+            constexpr uint32_t idesc1 = make_idesc_bf16(128, C1);
+            constexpr uint32_t idesc2 = make_idesc_bf16(128, C2);
+            bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
+            auto conv1 = [&](uint32_t i) -> bool {
+                const uint32_t s = i % XS, xph = (i / XS) & 1u, b = i & 1u, ph = (i >> 1) & 1u;
+                if (!mbar_wait(&bars->x_full[s], xph, abort_flag)) return false;
+                if (!mbar_wait(&bars->d1_empty[b], ph ^ 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t xa = sbase + SM_X + s * X_STAGE;
+#pragma unroll
+                for (uint32_t k = 0; k < 3; k++) {           // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
+                    const uint64_t ad = make_smem_desc(xa + k * 32u, 16, 128, 0);
+                    const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W1_OFF + k * 2u * (C1 * 16u), C1 * 16u, 128, 0);
+                    umma_bf16(tmem_base + b * C1, ad, bd, idesc1, k != 0 ? 1u : 0u);
+                }
+                umma_commit(&bars->x_empty[s]);
+                umma_commit(&bars->d1_full[b]);
+                return true;
+            };
+            auto conv2 = [&](uint32_t i) -> bool {
+                const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
+                if (!mbar_wait(&bars->h1_full[b], ph, abort_flag)) return false;
+                if (!mbar_wait(&bars->d2_empty[b], ph ^ 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t ha = sbase + SM_H1 + b * H1_BYTES;
+#pragma unroll
+                for (uint32_t t = 0; t < KW; t++) {
+#pragma unroll
+                    for (uint32_t k = 0; k < C1 / 16; k++) {
+                        const uint64_t ad = make_smem_desc(ha + (2u * k) * H1_COL + t * 16u, H1_COL, 128, 0);
+                        const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W2_OFF + t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u),
+                                                           C2 * 16u, 128, 0);
+                        umma_bf16(tmem_base + 128u + b * C2, ad, bd, idesc2, (t | k) != 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(&bars->h1_empty[b]);
+                umma_commit(&bars->d2_full[b]);
+                return true;
+            };
+            if (ok) ok = conv1(0);
+            for (uint32_t i = 0; i < n_mine && ok; i++) {
+                if (i + 1 < n_mine) ok = conv1(i + 1);
+                if (ok) ok = conv2(i);
+            }
+        }
+    } else if (n_mine > 0) {
+        const uint32_t q = warp & 3u;                    // TMEM lane quarter of this warp
+        const uint32_t p = q * 32u + lane;               // position handled by this thread
+        const uint32_t et = (warp - 2u) * 32u + lane;    // 0..127 among the epilogue threads
+        const float* b1 = reinterpret_cast<const float*>(smem + SM_BLOB + B1_OFF);
+        const float* b2 = reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF);
+        const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
+        const float* w3 = reinterpret_cast<const float*>(smem + SM_BLOB + W3_OFF);
+        float* part = reinterpret_cast<float*>(smem + SM_PART);
+        float* slog = reinterpret_cast<float*>(smem + SM_LOGIT);
+        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
+
+        auto E1 = [&](uint32_t i) -> bool {
+            const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
+            bool w = mbar_wait(&bars->d1_full[b], ph, abort_flag) && mbar_wait(&bars->h1_empty[b], ph ^ 1u, abort_flag);
+            if (!__all_sync(0xFFFFFFFFu, w)) return false;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + b * C1;
+            uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (p + 2u) * 16u;
+#pragma unroll
+            for (uint32_t c0 = 0; c0 < C1; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(taddr + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 4; j++) {            // 4 columns of 8 channels
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int e = 0; e < 4; e++) {
+                        const int c = j * 8 + e * 2;
+                        float x0 = fmaxf(__uint_as_float(v[c]) + b1[c0 + c], 0.0f);
+                        float x1 = fmaxf(__uint_as_float(v[c + 1]) + b1[c0 + c + 1], 0.0f);
+                        __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                        pk[e] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(hrow + ((c0 >> 3) + j) * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            fence_proxy_async();                         // activations -> visible to the MMA's shared-memory reads
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(&bars->d1_empty[b]); mbar_arrive(&bars->h1_full[b]); }
+            return true;
+        };
+        auto E2 = [&](uint32_t i) -> bool {
+            const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&bars->d2_full[b], ph, abort_flag))) return false;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 128u + b * C2;
+#pragma unroll 1
+            for (uint32_t c0 = 0; c0 < C2; c0 += 32) {
+                uint32_t v[32];
+                float x[32];
+                tmem_ld32(taddr + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c = 0; c < 32; c++)
+                    x[c] = __bfloat162float(__float2bfloat16_rn(fmaxf(__uint_as_float(v[c]) + b2[c0 + c], 0.0f)));
+                const float colsum = transpose_reduce32(x, lane);     // over this warp's 32 positions
+                part[(warp - 2u) * C2 + c0 + lane] = colsum;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->d2_empty[b]);
+            named_barrier_sync(1, 128);
+            // linear head: thread et -> class et/8, channels (et%8)*16 .. +16
+            {
+                const uint32_t cls = et >> 3, seg = et & 7u;
+                float acc = 0.0f;
+#pragma unroll
+                for (uint32_t k = 0; k < 16; k++) {
+                    const uint32_t ch = seg * 16u + k;
+                    const float pooled = (((part[ch] + part[C2 + ch]) + part[2 * C2 + ch]) + part[3 * C2 + ch]) * (1.0f / 128.0f);
+                    acc = fmaf(w3[cls * C2 + ch], pooled, acc);
+                }
+                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 4);
+                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
+                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
+                if (seg == 0) slog[cls] = acc + b3[cls];
+            }
+            named_barrier_sync(1, 128);
+            const uint32_t r = blockIdx.x + i * gridDim.x;
+            if (et < n_cls) logits[(size_t)r * n_cls + et] = slog[et];
+            if (et == 32 && label) {
+                uint32_t a = 0; float mx = slog[0];
+                for (uint32_t c = 1; c < n_cls; c++) if (slog[c] > mx) { mx = slog[c]; a = c; }
+                label[r] = (uint8_t)a;
+            }
+            named_barrier_sync(1, 128);                  // slog / part are free again
+            return true;
+        };
+        if (ok) ok = E1(0);
+        for (uint32_t i = 0; i < n_mine && ok; i++) {
+            if (i + 1 < n_mine) ok = E1(i + 1);
+            if (ok) ok = E2(i);
+        }
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT);
+        __nanosleep(200000);
+        __syncthreads();
+    }
+    tc_fence_after();
+    if (warp == 1) { __syncwarp(); tmem_dealloc(tmem_base, 512); }
+}
+
+uint16_t bf16_bits(float x) {
+    uint32_t u; memcpy(&u, &x, 4);
+    uint32_t low = u & 0xFFFFu, up = u >> 16;
+    if (low > 0x8000u || (low == 0x8000u && (up & 1u))) up++;
+    return (uint16_t)up;
+}
+float bf16_value(float x) { uint32_t u = (uint32_t)bf16_bits(x) << 16; float f; memcpy(&f, &u, 4); return f; }
+
+}  // namespace
+
+int sf_cnn_prepare(sf_slow* s, const float* w1, const float* b1, const float* w2, const float* b2,
+                   const float* w3, const float* b3)
+{
+    unsigned char* h = (unsigned char*)calloc(1, BLOB_BYTES);
+    if (!h) return SF_ERR_ALLOC;
+    uint16_t* W2 = reinterpret_cast<uint16_t*>(h + W2_OFF);
+    for (uint32_t t = 0; t < KW; t++)
+        for (uint32_t j = 0; j < C1 / 8; j++)
+            for (uint32_t n = 0; n < C2; n++)
+                for (uint32_t e = 0; e < 8; e++)
+                    W2[((t * (C1 / 8) + j) * C2 + n) * 8 + e] = bf16_bits(w2[((size_t)n * KW + t) * C1 + j * 8 + e]);
+    uint16_t* W1 = reinterpret_cast<uint16_t*>(h + W1_OFF);
+    for (uint32_t t = 0; t < KW; t++)
+        for (uint32_t n = 0; n < C1; n++)
+            for (uint32_t e = 0; e < CIN; e++)
+                W1[(t * C1 + n) * 8 + e] = bf16_bits(w1[((size_t)n * KW + t) * CIN + e]);
+    float* W3 = reinterpret_cast<float*>(h + W3_OFF);
+    for (uint32_t c = 0; c < s->n_cls; c++)
+        for (uint32_t k = 0; k < C2; k++) W3[c * C2 + k] = bf16_value(w3[(size_t)c * C2 + k]);
+    memcpy(h + B1_OFF, b1, C1 * 4);
+    memcpy(h + B2_OFF, b2, C2 * 4);
+    memcpy(h + B3_OFF, b3, s->n_cls * 4);
+    cudaError_t e = cudaMalloc(&s->d_w1, BLOB_BYTES);
+    if (e == cudaSuccess) e = cudaMemcpy(s->d_w1, h, BLOB_BYTES, cudaMemcpyHostToDevice);
+    free(h);
+    if (e != cudaSuccess) return sf_set_cuda_error(e, "sf_cnn_prepare");
+    return SF_OK;
+}
+
+int sf_cnn_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
+                        float* logits, uint8_t* label, void* scratch, cudaStream_t st)
+{
+    (void)scratch;
+    SF_CUDA(cudaFuncSetAttribute(cnn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL));
+    uint32_t grid = (uint32_t)ctx->num_sms < capacity ? (uint32_t)ctx->num_sms : capacity;
+    sf_time_begin(ctx, SF_T_GEMM, st);
+    cnn_fused_kernel<<<grid, kThreads, SM_TOTAL, st>>>(reinterpret_cast<const __nv_bfloat16*>(rows), n_rows_dev,
+                                                     reinterpret_cast<const unsigned char*>(s->d_w1), s->n_cls,
+                                                     logits, label, ctx->d_state);
+    sf_time_end(ctx, SF_T_GEMM, st);
+    SF_LAUNCH_CHECK("cnn_fused_kernel");
+    return SF_OK;
 }

@@ -326,3 +326,44 @@ def test_create_rejects_unsupported_shapes(env):
         sf.sf_forest_create(ctx, sf.SF_RF, 1, 13, 8, 2, np.zeros((1, 8191)), np.zeros((1, 8191)), np.zeros((1, 8192, 2)))
     with pytest.raises(sf.SfError):      # feature id out of range
         sf.sf_forest_create(ctx, sf.SF_RF, 1, 1, 8, 2, np.full((1, 1), 9), np.zeros((1, 1)), np.zeros((1, 2, 2)))
+
+
+# ------------------------------------------------------------------ S4: CNN --
+def _cnn_rows(n_rows, seed):
+    wide = flowgen.gen_packets(seed, n_rows, 128, 5)
+    return oracle.wide_rows(1, np.arange(n_rows, dtype=np.uint32), wide, 128, True, threads=4)
+
+
+def test_cnn_tap_alignment_with_delta_kernels(env):
+    """conv kernels that are a single shifted tap: any error in how the shifted operands
+    are addressed (row shift, zero padding at both ends) shows up at once."""
+    sf, hz, ctx = env
+    n_rows, cap = 5, 8
+    rows = _cnn_rows(cap, 71)
+    for t1, t2 in ((2, 2), (0, 2), (4, 2), (2, 0), (2, 4), (1, 3)):
+        m = flowgen.gen_cnn(72, 128, 8, 64, 128, 5, 16)
+        mix1 = m["w1"][:, 2, :].copy(); mix2 = m["w2"][:, 2, :].copy()
+        m["w1"][:] = 0; m["w1"][:, t1, :] = mix1
+        m["w2"][:] = 0; m["w2"][:, t2, :] = mix2
+        ref, _ = oracle.cnn(m, rows[:n_rows], True)
+        h = sf.sf_cnn_create(ctx, sf.SF_BF16, m)
+        logits, _ = _run_slow(sf, hz, ctx, h, hz.dev(rows).to(torch.bfloat16), n_rows, cap, 16)
+        assert np.max(np.abs(logits[:n_rows] - ref)) <= TOL_BF16, (t1, t2)
+        sf.sf_slow_destroy(h)
+
+
+@pytest.mark.parametrize("n_rows,cap,n_cls", [(1, 1, 16), (300, 333, 16), (1000, 1000, 7)])
+def test_cnn_within_tolerance(env, n_rows, cap, n_cls):
+    sf, hz, ctx = env
+    m = flowgen.gen_cnn(73, 128, 8, 64, 128, 5, n_cls)
+    rows = _cnn_rows(cap, 74)
+    ref, ref_label = oracle.cnn(m, rows[:n_rows], True, threads=8)
+    h = sf.sf_cnn_create(ctx, sf.SF_BF16, m)
+    rt = hz.dev(rows).to(torch.bfloat16)
+    logits, label = _run_slow(sf, hz, ctx, h, rt, n_rows, cap, n_cls)
+    assert np.max(np.abs(logits[:n_rows] - ref)) <= TOL_BF16
+    assert np.all(np.isnan(logits[n_rows:]))
+    _check_labels(ref, ref_label, label[:n_rows], TOL_BF16)
+    logits2, label2 = _run_slow(sf, hz, ctx, h, rt, n_rows, cap, n_cls)      # run-to-run identical bits
+    assert np.array_equal(logits[:n_rows], logits2[:n_rows]) and np.array_equal(label[:n_rows], label2[:n_rows])
+    sf.sf_slow_destroy(h)

@@ -110,3 +110,10 @@ def test_shared_planes_and_ragged_sizes(env):
     wl = make_workload(cfg, n=1237)
     wl["fast"] = wl["wide"]
     run_and_check(sf, hz, ctx, wl)
+
+
+def test_c4_shapes_reduced_flow_count(env):
+    """Config 4: 64 depth-10 trees over 64 features of 32 packets, 16 classes, fused 1-D CNN."""
+    sf, hz, ctx = env
+    wl = make_workload(flowgen.get_config(4), n=5000)
+    run_and_check(sf, hz, ctx, wl)
