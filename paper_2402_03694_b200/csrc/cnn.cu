@@ -17,7 +17,7 @@
 // Persistent CTAs, one per SM, loop over flows.  Warp 0 streams input rows with bulk
 // copies into a ring; warp 1 issues the MMAs (3 for conv1, 20 for conv2 per flow) in the
 // order conv1(i+1), conv2(i) so that the first epilogue of the next flow overlaps the
-// second convolution of this one; warps 2..5 are the epilogues: E1 turns the conv1
+// second convolution of this one; warps 2..17 are the epilogues (lane quarter = warp % 4, four column groups each): E1 turns the conv1
 // accumulators (TMEM) into bf16 activations in shared memory (conv2's A operand), E2
 // applies bias + ReLU + bf16 rounding to the conv2 accumulators, reduces over positions
 // with a fixed shuffle tree (deterministic), and evaluates the linear head.
@@ -31,7 +31,9 @@ namespace {
 using namespace sftc;
 
 constexpr uint32_t L = 128, CIN = 8, C1 = 64, C2 = 128, KW = 5, NCLS_MAX = 16;
-constexpr uint32_t kThreads = 192;
+constexpr uint32_t kEpiWarps = 16;                          // 4 TMEM lane quarters x 4 column groups
+constexpr uint32_t kEpiThreads = kEpiWarps * 32;
+constexpr uint32_t kThreads = 64 + kEpiThreads;
 constexpr uint32_t XS = 4;                                  // input-row ring depth
 constexpr uint32_t X_STAGE = (2 + L + 3) * 16;              // 2 zero rows, 128 rows, 3 zero rows (tap 5 is a zero tap)
 constexpr uint32_t H1_COL = (2 + L + 2) * 16;               // one 8-channel column of conv1's output: 2112 bytes
@@ -106,9 +108,9 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
         mbar_init(&bars->w_full, 1);
         for (uint32_t s = 0; s < XS; s++) { mbar_init(&bars->x_full[s], 1); mbar_init(&bars->x_empty[s], 1); }
         for (uint32_t b = 0; b < 2; b++) {
-            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], 4);
-            mbar_init(&bars->h1_full[b], 4); mbar_init(&bars->h1_empty[b], 1);
-            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], 4);
+            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kEpiWarps);
+            mbar_init(&bars->h1_full[b], kEpiWarps); mbar_init(&bars->h1_empty[b], 1);
+            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], kEpiWarps);
         }
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -182,7 +184,8 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     } else if (n_mine > 0) {
         const uint32_t q = warp & 3u;                    // TMEM lane quarter of this warp
         const uint32_t p = q * 32u + lane;               // position handled by this thread
-        const uint32_t et = (warp - 2u) * 32u + lane;    // 0..127 among the epilogue threads
+        const uint32_t g = (warp - 2u) >> 2;             // column group handled by this warp (0..3)
+        const uint32_t et = (warp - 2u) * 32u + lane;    // 0..511 among the epilogue threads
         const float* b1 = reinterpret_cast<const float*>(smem + SM_BLOB + B1_OFF);
         const float* b2 = reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF);
         const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
@@ -196,15 +199,15 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             bool w = mbar_wait(&bars->d1_full[b], ph, abort_flag) && mbar_wait(&bars->h1_empty[b], ph ^ 1u, abort_flag);
             if (!__all_sync(0xFFFFFFFFu, w)) return false;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + b * C1;
+            const uint32_t c0 = g * 16u;                 // this warp's 16 of the 64 conv1 channels
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + b * C1 + c0;
             uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (p + 2u) * 16u;
-#pragma unroll
-            for (uint32_t c0 = 0; c0 < C1; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(taddr + c0, v);
+            {
+                uint32_t v[16];
+                tmem_ld16(taddr, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 4; j++) {            // 4 columns of 8 channels
+                for (int j = 0; j < 2; j++) {            // 2 columns of 8 channels
                     uint32_t pk[4];
 #pragma unroll
                     for (int e = 0; e < 4; e++) {
@@ -227,39 +230,38 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&bars->d2_full[b], ph, abort_flag))) return false;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 128u + b * C2;
-#pragma unroll 1
-            for (uint32_t c0 = 0; c0 < C2; c0 += 32) {
+            const uint32_t c0 = g * 32u;                 // this warp's 32 of the 128 conv2 channels
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 128u + b * C2 + c0;
+            {
                 uint32_t v[32];
                 float x[32];
-                tmem_ld32(taddr + c0, v);
+                tmem_ld32(taddr, v);
                 tmem_ld_wait();
 #pragma unroll
                 for (int c = 0; c < 32; c++)
                     x[c] = __bfloat162float(__float2bfloat16_rn(fmaxf(__uint_as_float(v[c]) + b2[c0 + c], 0.0f)));
                 const float colsum = transpose_reduce32(x, lane);     // over this warp's 32 positions
-                part[(warp - 2u) * C2 + c0 + lane] = colsum;
+                part[q * C2 + c0 + lane] = colsum;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->d2_empty[b]);
-            named_barrier_sync(1, 128);
-            // linear head: thread et -> class et/8, channels (et%8)*16 .. +16
+            named_barrier_sync(1, kEpiThreads);
+            // linear head: epilogue warp w -> class w, lane -> channels 4*lane .. 4*lane+3
             {
-                const uint32_t cls = et >> 3, seg = et & 7u;
+                const uint32_t cls = et >> 5;
                 float acc = 0.0f;
 #pragma unroll
-                for (uint32_t k = 0; k < 16; k++) {
-                    const uint32_t ch = seg * 16u + k;
+                for (uint32_t k = 0; k < 4; k++) {
+                    const uint32_t ch = lane * 4u + k;
                     const float pooled = (((part[ch] + part[C2 + ch]) + part[2 * C2 + ch]) + part[3 * C2 + ch]) * (1.0f / 128.0f);
                     acc = fmaf(w3[cls * C2 + ch], pooled, acc);
                 }
-                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 4);
-                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
-                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
-                if (seg == 0) slog[cls] = acc + b3[cls];
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                if (lane == 0) slog[cls] = acc + b3[cls];
             }
-            named_barrier_sync(1, 128);
+            named_barrier_sync(1, kEpiThreads);
             const uint32_t r = blockIdx.x + i * gridDim.x;
             if (et < n_cls) logits[(size_t)r * n_cls + et] = slog[et];
             if (et == 32 && label) {
@@ -267,7 +269,7 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 for (uint32_t c = 1; c < n_cls; c++) if (slog[c] > mx) { mx = slog[c]; a = c; }
                 label[r] = (uint8_t)a;
             }
-            named_barrier_sync(1, 128);                  // slog / part are free again
+            named_barrier_sync(1, kEpiThreads);          // slog / part are free again
             return true;
         };
         if (ok) ok = E1(0);
