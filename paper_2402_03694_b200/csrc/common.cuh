@@ -83,13 +83,19 @@ void* sf_ws_alloc(sf_ctx* ctx, size_t bytes);       // NULL if the reservation w
 static inline size_t sf_align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 // ---- internal launchers (each validates nothing; callers did) ---------------
-int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st);
-int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st);
+int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st,
+                      const uint32_t* n_dev = nullptr);   // n_dev: optional device-side flow count (<= pk->n_flows)
+int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st,
+                     const uint32_t* n_dev = nullptr);
 // route scratch: block_counts uint32[ceil(n/1024)+1], decision bytes if the caller gave none
 size_t sf_route_scratch_bytes(uint32_t n);
 int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,
                     const sf_packets* wide, uint32_t* esc_ids, uint32_t* n_esc, void* rows,
                     uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st);
+int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C, uint8_t* decision,
+                    uint8_t* label, float* score, uint32_t* block_counts, const uint32_t* n_dev, cudaStream_t st);
+int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wide, const uint32_t* ids,
+                     const uint32_t* n_ids_dev, uint32_t capacity, void* rows, cudaStream_t st);
 size_t sf_slow_scratch_bytes(const sf_slow* s, uint32_t capacity);
 int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
                    float* logits, uint8_t* label, void* scratch, cudaStream_t st);

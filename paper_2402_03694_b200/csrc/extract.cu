@@ -101,12 +101,14 @@ template <int G, bool VEC>
 __global__ void __launch_bounds__(kFlowsPerBlock)
 extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ iat,
                const uint32_t* __restrict__ dir_bits, const uint8_t* __restrict__ n_valid,
-               uint32_t n, uint32_t pitch, uint32_t N, float* __restrict__ feat)
+               uint32_t n, uint32_t pitch, uint32_t N, float* __restrict__ feat, const uint32_t* __restrict__ n_dev)
 {
     constexpr int F = 8 * G;
     constexpr int STRIDE = F + 1;                  // odd stride: conflict-free row writes
     extern __shared__ float tile[];                // [kFlowsPerBlock][STRIDE]
+    if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
     const uint32_t f0 = blockIdx.x * kFlowsPerBlock;
+    if (f0 >= n) return;
     const uint32_t f = f0 + threadIdx.x;
 
     if (f < n) {
@@ -149,32 +151,32 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
 }
 
 template <int G>
-int launch_g(const sf_packets* pk, uint32_t N, float* feat, cudaStream_t st) {
+int launch_g(const sf_packets* pk, uint32_t N, float* feat, cudaStream_t st, const uint32_t* n_dev) {
     const uint32_t n = pk->n_flows;
     const bool vec = (pk->pitch_pkts % 8 == 0) && (((uintptr_t)pk->size & 15) == 0) && (((uintptr_t)pk->iat_us & 15) == 0);
     const size_t smem = (size_t)kFlowsPerBlock * (8 * G + 1) * sizeof(float);
     const uint32_t grid = (n + kFlowsPerBlock - 1) / kFlowsPerBlock;
     if (vec)
-        extract_kernel<G, true><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat);
+        extract_kernel<G, true><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev);
     else
-        extract_kernel<G, false><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat);
+        extract_kernel<G, false><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev);
     SF_LAUNCH_CHECK("extract_kernel");
     return SF_OK;
 }
 
 }  // namespace
 
-int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st) {
+int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st, const uint32_t* n_dev) {
     if (pk->n_flows == 0) return SF_OK;
     switch (F / 8) {
-    case 1: return launch_g<1>(pk, N, feat, st);
-    case 2: return launch_g<2>(pk, N, feat, st);
-    case 3: return launch_g<3>(pk, N, feat, st);
-    case 4: return launch_g<4>(pk, N, feat, st);
-    case 5: return launch_g<5>(pk, N, feat, st);
-    case 6: return launch_g<6>(pk, N, feat, st);
-    case 7: return launch_g<7>(pk, N, feat, st);
-    case 8: return launch_g<8>(pk, N, feat, st);
+    case 1: return launch_g<1>(pk, N, feat, st, n_dev);
+    case 2: return launch_g<2>(pk, N, feat, st, n_dev);
+    case 3: return launch_g<3>(pk, N, feat, st, n_dev);
+    case 4: return launch_g<4>(pk, N, feat, st, n_dev);
+    case 5: return launch_g<5>(pk, N, feat, st, n_dev);
+    case 6: return launch_g<6>(pk, N, feat, st, n_dev);
+    case 7: return launch_g<7>(pk, N, feat, st, n_dev);
+    case 8: return launch_g<8>(pk, N, feat, st, n_dev);
     }
     return SF_ERR_UNSUPPORTED;
 }

@@ -91,9 +91,11 @@ __global__ void __launch_bounds__(kB, 1)
 forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
               const unsigned char* __restrict__ image, const float* __restrict__ leaf,
               uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
-              float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st)
+              float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
+    if (blockIdx.x * kB >= n) return;
     const uint32_t sbuf0 = smem_u32(smem_raw);
     float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][kB]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * kB * 4);   // [2] + flag
@@ -221,52 +223,52 @@ Plan make_plan(const sf_forest* fo) {
 }
 
 template <int KIND, int C, int NCH>
-int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     auto k = forest_kernel<KIND, C, NCH>;
     SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
     const uint32_t grid = (n + kB - 1) / kB;
     k<<<grid, kB, p.smem, st>>>(feat, n, fo->F, fo->d_image, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
-                                p.chunk_bytes, out, leaf_idx, fo->ctx->d_state);
+                                p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
 }
 
 template <int C>
-int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     const Plan p = make_plan(fo);
-    if (p.nch == 2) return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st);
-    return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st);
+    if (p.nch == 2) return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
-int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     const Plan p = make_plan(fo);
-    if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st);
-    if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st);
-    return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st);
+    if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
 }  // namespace
 
-int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st) {
+int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     if (n == 0) return SF_OK;
-    if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st);
+    if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st, n_dev);
     switch (fo->C) {
-    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st);
-    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st);
-    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st);
-    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st);
-    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st);
-    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st);
-    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st);
-    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st);
-    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st);
-    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st);
-    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st);
-    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st);
-    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st);
-    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st);
-    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st);
-    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st);
+    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev);
     }
     return SF_ERR_UNSUPPORTED;
 }

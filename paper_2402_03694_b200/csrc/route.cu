@@ -18,9 +18,10 @@ template <int RULE>
 __global__ void __launch_bounds__(kScoreBlock)
 score_kernel(const float* __restrict__ fast_out, uint32_t n, uint32_t C, const float* __restrict__ tau,
              uint8_t* __restrict__ decision, uint8_t* __restrict__ label, float* __restrict__ score,
-             uint32_t* __restrict__ block_counts)
+             uint32_t* __restrict__ block_counts, const uint32_t* __restrict__ n_dev = nullptr)
 {
     __shared__ uint32_t warp_cnt[kScoreBlock / 32];
+    if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
     const uint32_t f = blockIdx.x * kScoreBlock + threadIdx.x;
     bool esc = false;
     if (f < n) {
@@ -201,6 +202,38 @@ __global__ void merge_slow_kernel(const uint32_t* __restrict__ esc_ids, const ui
 }
 
 }  // namespace
+
+// score / label / decision only (no compaction), for at most n flows with the actual count on the device
+int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C, uint8_t* decision,
+                    uint8_t* label, float* score, uint32_t* block_counts, const uint32_t* n_dev, cudaStream_t st)
+{
+    const uint32_t nb = (n + kScoreBlock - 1) / kScoreBlock;
+    if (nb == 0) return SF_OK;
+    if (cfg->rule == SF_ABSMARGIN_LT)
+        score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
+    else
+        score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
+    SF_LAUNCH_CHECK("score_kernel");
+    return SF_OK;
+}
+
+// wide rows of `capacity` flows at most (ids and count on the device) out of any planes
+int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wide, const uint32_t* ids,
+                     const uint32_t* n_ids_dev, uint32_t capacity, void* rows, cudaStream_t st)
+{
+    if (capacity == 0) return SF_OK;
+    const uint32_t P = cfg->P, P_real = cfg->P_real ? cfg->P_real : cfg->P;
+    uint32_t blocks = (capacity + 7) / 8;
+    uint32_t max_blocks = (uint32_t)ctx->num_sms * 32;
+    if (blocks > max_blocks) blocks = max_blocks;
+#define SF_GATHER2(Wv, BF) gather_kernel<Wv, BF><<<blocks, 256, 0, st>>>(ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, \
+        wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, P, P_real, rows)
+    if (cfg->wide_layout == SF_MLP16) { if (cfg->row_dtype == SF_BF16) SF_GATHER2(16, true); else SF_GATHER2(16, false); }
+    else                              { if (cfg->row_dtype == SF_BF16) SF_GATHER2(8, true);  else SF_GATHER2(8, false); }
+#undef SF_GATHER2
+    SF_LAUNCH_CHECK("gather_kernel");
+    return SF_OK;
+}
 
 size_t sf_route_scratch_bytes(uint32_t n) {
     size_t nb = ((size_t)n + kScoreBlock - 1) / kScoreBlock;

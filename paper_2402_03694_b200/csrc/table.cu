@@ -1,8 +1,507 @@
-// Streaming per-flow state table: placeholder translation unit.
+// S0: device-resident per-flow state for the streaming workload.
+//
+// The paper's server joins first-packet features, later packets and escalations by flow id
+// through message queues (Sec. 3.1, Sec. 4.1).  Here one open-addressing hash table in HBM,
+// keyed by the 5-tuple, holds every flow's state, and a batch of interleaved packets is
+// ingested by a short chain of kernels on one stream:
+//   probe     one thread per packet: 128-bit compare-and-swap on the 16-byte key slot
+//             (claims an empty slot or recognises its own key; bounded linear probing)
+//   sort      one block: stable LSD radix sort of (slot, arrival index) so that each flow's
+//             packets of this batch sit together in ARRIVAL order, then their rank in the flow
+//   apply1    packets that fall into a flow's first `fast_pkts` positions are written to its
+//             fast context; flows that just reached fast_pkts packets are listed
+//   fast path the listed flows' contexts are copied into dense planes and run through the
+//             same S1 / S2 / S3 kernels as the batch path (flow count read on the device)
+//   route     answered flows are marked; assigned flows get a slab for their slow context
+//   apply2    later packets go to the slab of an assigned flow (or are counted as arriving
+//             after the decision); flows that just reached slow_pkts packets are listed
+//   slow path wide rows of the listed slabs (zero-padded to the model's width) -> S4 -> labels
+// Every loop is bounded; a key that finds no slot within the probe limit is counted as missed
+// and SF_ERR_TABLE_FULL is recorded in the context's error word.
 #include "common.cuh"
+#include <new>
+#include <string.h>
 
-extern "C" int sf_table_create(sf_ctx*, uint32_t, uint32_t, uint32_t, uint32_t, sf_table**) { return SF_ERR_UNSUPPORTED; }
-extern "C" void sf_table_destroy(sf_table*) {}
-extern "C" int sf_table_ingest(sf_ctx*, sf_table*, const sf_pkt_batch*, const sf_forest*, uint32_t, const sf_slow*,
-                               const sf_route_cfg*, sf_batch_result*, void*) { return SF_ERR_UNSUPPORTED; }
-extern "C" int sf_table_lookup(sf_ctx*, const sf_table*, const sf_key*, uint32_t, sf_flow_result*, void*) { return SF_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr uint32_t kMaxBatch = 65536;
+constexpr uint32_t kProbeLimit = 64;
+constexpr uint32_t kHdr = 13;
+constexpr uint32_t kMiss = 0xFFFFFFFFu;
+
+struct TableDev {
+    // per slot
+    ulonglong2* keys; uint32_t* cnt; uint8_t* stage; uint8_t* label_fast; uint8_t* label_slow; float* score; uint32_t* slab;
+    uint16_t* f_size; uint32_t* f_iat; uint32_t* f_dir; uint8_t* f_hdr;
+    // per slab
+    uint16_t* s_size; uint32_t* s_iat; uint32_t* s_dir; uint8_t* s_hdr;
+    uint32_t* slab_next;
+    uint32_t mask, n_slots, fast_pkts, slow_pkts, slow_slabs;
+};
+
+}  // namespace
+
+struct sf_table {
+    sf_ctx* ctx;
+    TableDev d;
+    uint32_t log2_slots;
+    // per-batch scratch with fixed addresses
+    uint32_t* key_a; uint32_t* key_b; uint32_t* idx_a; uint32_t* idx_b; uint32_t* rank; uint32_t* pos;
+    uint32_t* fire1_slot; uint32_t* fire2_slab; uint32_t* fire2_slot;
+    uint32_t* counts;                 // [0] n_fire1, [1] n_fire2
+    uint16_t* c_size; uint32_t* c_iat; uint32_t* c_dir;      // dense fast planes of the fired flows
+    void* all;                        // one allocation behind everything above
+};
+
+namespace {
+
+__device__ __forceinline__ void cas128(void* p, uint64_t nlo, uint64_t nhi, uint64_t& olo, uint64_t& ohi) {
+    // compare with zero (empty slot), swap in the key; returns what was there
+    asm volatile(
+        "{\n"
+        ".reg .b128 c, s, d;\n"
+        "mov.b128 c, {%2, %3};\n"
+        "mov.b128 s, {%4, %5};\n"
+        "atom.global.cas.b128 d, [%6], c, s;\n"
+        "mov.b128 {%0, %1}, d;\n"
+        "}\n"
+        : "=l"(olo), "=l"(ohi) : "l"(0ull), "l"(0ull), "l"(nlo), "l"(nhi), "l"(p) : "memory");
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {
+    x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;
+    x ^= x >> 27; x *= 0x94d049bb133111ebull;
+    x ^= x >> 31;
+    return x;
+}
+__device__ __forceinline__ void make_key(uint32_t src, uint32_t dst, uint32_t sport, uint32_t dport, uint32_t proto,
+                                         uint64_t& lo, uint64_t& hi) {
+    lo = (uint64_t)src | ((uint64_t)dst << 32);
+    hi = (uint64_t)sport | ((uint64_t)dport << 16) | ((uint64_t)proto << 32) | (1ull << 63);     // never zero
+}
+__device__ __forceinline__ uint32_t hash_key(uint64_t lo, uint64_t hi, uint32_t mask) {
+    return (uint32_t)mix64(lo ^ mix64(hi)) & mask;
+}
+
+__global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ pkt_slot, uint32_t* __restrict__ idx,
+                             sf_batch_result* res, sf_dev_state* st)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= b.n) return;
+    uint64_t lo, hi;
+    make_key(b.src[i], b.dst[i], b.sport[i], b.dport[i], b.proto[i], lo, hi);
+    uint32_t h = hash_key(lo, hi, t.mask);
+    uint32_t slot = t.n_slots;                       // "missed" sorts after every real slot
+    for (uint32_t p = 0; p < kProbeLimit; p++) {
+        uint64_t olo, ohi;
+        const ulonglong2 cur = t.keys[h];            // cheap look before the atomic
+        if (cur.x == lo && cur.y == hi) { slot = h; break; }
+        if (cur.x == 0 && cur.y == 0) {
+            cas128(&t.keys[h], lo, hi, olo, ohi);
+            if (olo == 0 && ohi == 0) { slot = h; atomicAdd(&res->n_new_flows, 1u); break; }
+            if (olo == lo && ohi == hi) { slot = h; break; }
+        }
+        h = (h + 1) & t.mask;
+    }
+    if (slot == t.n_slots) {
+        atomicAdd(&res->n_missed, 1u);
+        atomicAdd((unsigned long long*)&st->counters.n_missed, 1ull);
+        sf_dev_set_error(st, SF_ERR_TABLE_FULL);
+    }
+    pkt_slot[i] = slot;
+    idx[i] = i;
+}
+
+// One block, 1024 threads.  Stable LSD radix sort (4-bit digits) of n <= 65536 (key, idx) pairs,
+// thread t owning the contiguous chunk [t*per, (t+1)*per) in every pass, then the rank of each
+// sorted item inside its run of equal keys.
+__global__ void __launch_bounds__(1024, 1)
+sort_rank_kernel(uint32_t* key_a, uint32_t* idx_a, uint32_t* key_b, uint32_t* idx_b, uint32_t n, uint32_t key_bits,
+                 uint32_t* __restrict__ rank)
+{
+    extern __shared__ uint32_t sm[];                 // [16][1024] counts / offsets, then [1024] scan scratch
+    uint32_t* cnts = sm;
+    uint32_t* tot = sm + 16 * 1024;
+    const uint32_t t = threadIdx.x;
+    const uint32_t per = (n + 1023) / 1024;
+    const uint32_t lo = min(n, t * per), hi = min(n, lo + per);
+    uint32_t* ks = key_a; uint32_t* is = idx_a; uint32_t* kd = key_b; uint32_t* id = idx_b;
+    const uint32_t passes = (key_bits + 3) / 4;      // the host makes this even so the result lands in (key_a, idx_a)
+    for (uint32_t pass = 0; pass < passes; pass++) {
+        const uint32_t shift = pass * 4;
+        uint32_t h[16];
+#pragma unroll
+        for (int d = 0; d < 16; d++) h[d] = 0;
+        for (uint32_t j = lo; j < hi; j++) {
+            const uint32_t dg = (ks[j] >> shift) & 15u;
+#pragma unroll
+            for (int d = 0; d < 16; d++) h[d] += (dg == (uint32_t)d) ? 1u : 0u;
+        }
+#pragma unroll
+        for (int d = 0; d < 16; d++) cnts[d * 1024 + t] = h[d];
+        __syncthreads();
+        // exclusive scan of the 16384 counters in (digit, thread) order: thread t scans entries [16t, 16t+16)
+        uint32_t loc[16], s = 0;
+#pragma unroll
+        for (int e = 0; e < 16; e++) { loc[e] = s; s += cnts[t * 16 + e]; }
+        uint32_t x = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
+        if ((t & 31) == 31) tot[t >> 5] = x;
+        __syncthreads();
+        if (t < 32) {
+            uint32_t w = tot[t], z = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (t >= (uint32_t)o) z += y; }
+            tot[t] = z - w;
+        }
+        __syncthreads();
+        const uint32_t base = tot[t >> 5] + x - s;
+#pragma unroll
+        for (int e = 0; e < 16; e++) cnts[t * 16 + e] = base + loc[e];
+        __syncthreads();
+#pragma unroll
+        for (int d = 0; d < 16; d++) h[d] = cnts[d * 1024 + t];
+        for (uint32_t j = lo; j < hi; j++) {
+            const uint32_t k = ks[j], dg = (k >> shift) & 15u;
+            uint32_t p = 0;
+#pragma unroll
+            for (int d = 0; d < 16; d++) if (dg == (uint32_t)d) { p = h[d]; h[d] = p + 1; }
+            kd[p] = k; id[p] = is[j];
+        }
+        __syncthreads();
+        uint32_t* tk = ks; ks = kd; kd = tk;
+        uint32_t* ti = is; is = id; id = ti;
+    }
+    // rank inside runs of equal keys: position minus the position of the run's first item
+    int last_head = -1;
+    for (uint32_t j = lo; j < hi; j++) if (j == 0 || ks[j] != ks[j - 1]) last_head = (int)j;
+    int x = last_head;                               // inclusive max-scan over threads
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x = max(x, y); }
+    int* itot = reinterpret_cast<int*>(tot);
+    if ((t & 31) == 31) itot[t >> 5] = x;
+    __syncthreads();
+    if (t < 32) {
+        int z = itot[t];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (t >= (uint32_t)o) z = max(z, y); }
+        itot[t] = z;
+    }
+    __syncthreads();
+    int carry = -1;                                  // last run head strictly before this thread's chunk
+    {
+        int prev_lane = __shfl_up_sync(0xFFFFFFFFu, x, 1);
+        if ((t & 31) != 0) carry = prev_lane;
+        if ((t >> 5) > 0) carry = max(carry, itot[(t >> 5) - 1]);
+    }
+    int head = carry;
+    for (uint32_t j = lo; j < hi; j++) {
+        if (j == 0 || ks[j] != ks[j - 1]) head = (int)j;
+        rank[j] = j - (uint32_t)head;
+    }
+}
+
+__device__ __forceinline__ void store_packet(uint16_t* sz, uint32_t* ia, uint32_t* dirw, uint8_t* hd, uint32_t row,
+                                             uint32_t pitch, uint32_t words, uint32_t pos, const sf_pkt_batch& b, uint32_t i)
+{
+    sz[(size_t)row * pitch + pos] = b.size[i];
+    ia[(size_t)row * pitch + pos] = b.iat_us[i];
+    if (b.dir[i] & 1u) atomicOr(&dirw[(size_t)row * words + (pos >> 5)], 1u << (pos & 31));
+    uint8_t* o = hd + ((size_t)row * pitch + pos) * kHdr;
+    const uint8_t* s = b.hdr + (size_t)i * kHdr;
+#pragma unroll
+    for (int k = 0; k < (int)kHdr; k++) o[k] = s[k];
+}
+
+__global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
+                              const uint32_t* __restrict__ rank, uint32_t* __restrict__ pos_out,
+                              uint32_t* __restrict__ fire1_slot, uint32_t* __restrict__ counts)
+{
+    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= b.n) return;
+    const uint32_t slot = s_key[j];
+    if (slot >= t.n_slots) { pos_out[j] = kMiss; return; }
+    const uint32_t pos = t.cnt[slot] + rank[j];
+    pos_out[j] = pos;
+    if (pos < t.fast_pkts) {
+        store_packet(t.f_size, t.f_iat, t.f_dir, t.f_hdr, slot, t.fast_pkts, 1, pos, b, s_idx[j]);
+        if (pos == t.fast_pkts - 1) fire1_slot[atomicAdd(&counts[0], 1u)] = slot;
+    }
+}
+
+__global__ void gather_fast_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const uint32_t* __restrict__ counts,
+                                   uint16_t* __restrict__ c_size, uint32_t* __restrict__ c_iat, uint32_t* __restrict__ c_dir)
+{
+    const uint32_t e = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t k = e / t.fast_pkts, p = e - k * t.fast_pkts;
+    if (k >= counts[0]) return;
+    const uint32_t slot = fire1_slot[k];
+    c_size[e] = t.f_size[(size_t)slot * t.fast_pkts + p];
+    c_iat[e] = t.f_iat[(size_t)slot * t.fast_pkts + p];
+    if (p == 0) c_dir[k] = t.f_dir[slot];
+}
+
+__global__ void apply_route_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const uint32_t* __restrict__ counts,
+                                   const uint8_t* __restrict__ decision, const uint8_t* __restrict__ label,
+                                   const float* __restrict__ score, sf_batch_result* res, sf_dev_state* st)
+{
+    const uint32_t k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= counts[0]) return;
+    const uint32_t slot = fire1_slot[k];
+    t.label_fast[slot] = label[k];
+    t.score[slot] = score[k];
+    atomicAdd(&res->n_fast_fired, 1u);
+    bool assigned = decision[k] != 0;
+    if (assigned) {
+        const uint32_t s = atomicAdd(t.slab_next, 1u);
+        if (s < t.slow_slabs) {
+            t.slab[slot] = s;
+            const uint32_t words = (t.slow_pkts + 31) / 32;
+            for (uint32_t p = 0; p < t.fast_pkts; p++) {
+                t.s_size[(size_t)s * t.slow_pkts + p] = t.f_size[(size_t)slot * t.fast_pkts + p];
+                t.s_iat[(size_t)s * t.slow_pkts + p] = t.f_iat[(size_t)slot * t.fast_pkts + p];
+                const uint8_t* src = t.f_hdr + ((size_t)slot * t.fast_pkts + p) * kHdr;
+                uint8_t* dst = t.s_hdr + ((size_t)s * t.slow_pkts + p) * kHdr;
+                for (uint32_t q = 0; q < kHdr; q++) dst[q] = src[q];
+            }
+            atomicOr(&t.s_dir[(size_t)s * words], t.f_dir[slot]);
+        } else {
+            // no slab left: the flow keeps its fast answer and is counted as missed by the slow path
+            assigned = false;
+            atomicAdd(&res->n_missed, 1u);
+            atomicAdd((unsigned long long*)&st->counters.n_missed, 1ull);
+            sf_dev_set_error(st, SF_ERR_TABLE_FULL);
+        }
+    }
+    t.stage[slot] = assigned ? 2 : 1;
+    if (assigned) { atomicAdd(&res->n_escalated, 1u); atomicAdd((unsigned long long*)&st->counters.n_escalated, 1ull); }
+    else          { atomicAdd(&res->n_fast_done, 1u); atomicAdd((unsigned long long*)&st->counters.n_fast_done, 1ull); }
+    atomicAdd((unsigned long long*)&st->counters.n_flows, 1ull);
+}
+
+__global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
+                              const uint32_t* __restrict__ rank, const uint32_t* __restrict__ pos_in,
+                              uint32_t* __restrict__ fire2_slab, uint32_t* __restrict__ fire2_slot,
+                              uint32_t* __restrict__ counts, sf_batch_result* res, sf_dev_state* st)
+{
+    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= b.n) return;
+    const uint32_t slot = s_key[j];
+    if (slot >= t.n_slots) return;
+    const uint32_t pos = pos_in[j];
+    if (pos >= t.fast_pkts) {
+        const uint32_t stg = t.stage[slot];
+        if (stg == 2 && pos < t.slow_pkts) {
+            const uint32_t s = t.slab[slot];
+            store_packet(t.s_size, t.s_iat, t.s_dir, t.s_hdr, s, t.slow_pkts, (t.slow_pkts + 31) / 32, pos, b, s_idx[j]);
+            if (pos == t.slow_pkts - 1) {
+                const uint32_t k = atomicAdd(&counts[1], 1u);
+                fire2_slab[k] = s; fire2_slot[k] = slot;
+            }
+        } else {
+            atomicAdd(&res->n_dropped_after_decision, 1u);
+            atomicAdd((unsigned long long*)&st->counters.n_dropped_after_decision, 1ull);
+        }
+    }
+    // the last packet of the flow's run in this batch advances the flow's packet counter
+    if (j + 1 == b.n || s_key[j + 1] != slot) t.cnt[slot] += rank[j] + 1;
+}
+
+__global__ void apply_slow_kernel(TableDev t, const uint32_t* __restrict__ fire2_slot, const uint32_t* __restrict__ counts,
+                                  const uint8_t* __restrict__ label_slow, sf_batch_result* res)
+{
+    const uint32_t k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= counts[1]) return;
+    const uint32_t slot = fire2_slot[k];
+    t.label_slow[slot] = label_slow[k];
+    t.stage[slot] = 3;
+    atomicAdd(&res->n_slow_fired, 1u);
+}
+
+__global__ void lookup_kernel(TableDev t, const sf_key* __restrict__ keys, uint32_t n, sf_flow_result* __restrict__ out)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint64_t lo, hi;
+    make_key(keys[i].src, keys[i].dst, keys[i].sport, keys[i].dport, keys[i].proto, lo, hi);
+    uint32_t h = hash_key(lo, hi, t.mask);
+    sf_flow_result r;
+    r.found = 0; r.stage = 0; r.label_fast = 0; r.label_slow = 0; r.n_pkts = 0; r.score = 0.0f;
+    for (uint32_t p = 0; p < kProbeLimit; p++) {
+        const ulonglong2 cur = t.keys[h];
+        if (cur.x == lo && cur.y == hi) {
+            r.found = 1; r.stage = t.stage[h]; r.label_fast = t.label_fast[h]; r.label_slow = t.label_slow[h];
+            r.n_pkts = t.cnt[h]; r.score = t.score[h];
+            break;
+        }
+        if (cur.x == 0 && cur.y == 0) break;
+        h = (h + 1) & t.mask;
+    }
+    out[i] = r;
+}
+
+template <typename T>
+T* carve(char*& p, size_t count) {
+    T* r = reinterpret_cast<T*>(p);
+    p += sf_align256(count * sizeof(T));
+    return r;
+}
+
+}  // namespace
+
+extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_pkts, uint32_t slow_pkts,
+                               uint32_t slow_slabs, sf_table** out)
+{
+    if (!ctx || !out) return SF_ERR_ARG;
+    if (log2_slots < 4 || log2_slots > 28) return SF_ERR_ARG;
+    if (fast_pkts < 1 || fast_pkts > 32 || slow_pkts < fast_pkts || slow_pkts > 128 || slow_slabs < 1) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    sf_table* t = new (std::nothrow) sf_table();
+    if (!t) return SF_ERR_ALLOC;
+    memset(t, 0, sizeof(*t));
+    t->ctx = ctx; t->log2_slots = log2_slots;
+    const size_t S = (size_t)1 << log2_slots, B = slow_slabs, W = (slow_pkts + 31) / 32;
+    size_t total = 0;
+    auto need = [&](size_t bytes) { total += sf_align256(bytes); };
+    need(S * 16); need(S * 4); need(S); need(S); need(S); need(S * 4); need(S * 4);
+    need(S * fast_pkts * 2); need(S * fast_pkts * 4); need(S * 4); need(S * fast_pkts * kHdr);
+    need(B * slow_pkts * 2); need(B * slow_pkts * 4); need(B * W * 4); need(B * slow_pkts * kHdr); need(4);
+    for (int k = 0; k < 9; k++) need((size_t)kMaxBatch * 4);
+    need(64);
+    need((size_t)kMaxBatch * fast_pkts * 2); need((size_t)kMaxBatch * fast_pkts * 4); need((size_t)kMaxBatch * 4);
+    cudaError_t e = cudaMalloc(&t->all, total);
+    if (e != cudaSuccess) { delete t; sf_set_cuda_error(e, "cudaMalloc(table)"); return SF_ERR_ALLOC; }
+    e = cudaMemset(t->all, 0, total);
+    if (e != cudaSuccess) { cudaFree(t->all); delete t; return sf_set_cuda_error(e, "cudaMemset(table)"); }
+    char* p = reinterpret_cast<char*>(t->all);
+    TableDev& d = t->d;
+    d.keys = carve<ulonglong2>(p, S); d.cnt = carve<uint32_t>(p, S); d.stage = carve<uint8_t>(p, S);
+    d.label_fast = carve<uint8_t>(p, S); d.label_slow = carve<uint8_t>(p, S); d.score = carve<float>(p, S);
+    d.slab = carve<uint32_t>(p, S);
+    d.f_size = carve<uint16_t>(p, S * fast_pkts); d.f_iat = carve<uint32_t>(p, S * fast_pkts);
+    d.f_dir = carve<uint32_t>(p, S); d.f_hdr = carve<uint8_t>(p, S * fast_pkts * kHdr);
+    d.s_size = carve<uint16_t>(p, B * slow_pkts); d.s_iat = carve<uint32_t>(p, B * slow_pkts);
+    d.s_dir = carve<uint32_t>(p, B * W); d.s_hdr = carve<uint8_t>(p, B * slow_pkts * kHdr);
+    d.slab_next = carve<uint32_t>(p, 1);
+    d.mask = (uint32_t)(S - 1); d.n_slots = (uint32_t)S; d.fast_pkts = fast_pkts; d.slow_pkts = slow_pkts; d.slow_slabs = slow_slabs;
+    t->key_a = carve<uint32_t>(p, kMaxBatch); t->key_b = carve<uint32_t>(p, kMaxBatch);
+    t->idx_a = carve<uint32_t>(p, kMaxBatch); t->idx_b = carve<uint32_t>(p, kMaxBatch);
+    t->rank = carve<uint32_t>(p, kMaxBatch); t->pos = carve<uint32_t>(p, kMaxBatch);
+    t->fire1_slot = carve<uint32_t>(p, kMaxBatch); t->fire2_slab = carve<uint32_t>(p, kMaxBatch);
+    t->fire2_slot = carve<uint32_t>(p, kMaxBatch);
+    t->counts = carve<uint32_t>(p, 16);
+    t->c_size = carve<uint16_t>(p, (size_t)kMaxBatch * fast_pkts); t->c_iat = carve<uint32_t>(p, (size_t)kMaxBatch * fast_pkts);
+    t->c_dir = carve<uint32_t>(p, kMaxBatch);
+    *out = t;
+    return SF_OK;
+}
+
+extern "C" void sf_table_destroy(sf_table* t) {
+    if (!t) return;
+    if (t->all) cudaFree(t->all);
+    delete t;
+}
+
+extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_forest* fo, uint32_t F,
+                               const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_dev, void* stream)
+{
+    if (!ctx || !t || !batch || !fo || !slow || !cfg || !result_dev || !cfg->tau) return SF_ERR_ARG;
+    if (batch->n > kMaxBatch) return SF_ERR_ARG;
+    if (!batch->src || !batch->dst || !batch->sport || !batch->dport || !batch->proto || !batch->dir || !batch->size ||
+        !batch->iat_us || !batch->hdr) return SF_ERR_ARG;
+    if (F != fo->F || fo->kind != SF_RF || cfg->rule != SF_LC_GT) return SF_ERR_UNSUPPORTED;
+    if (slow->arch != SF_SLOW_MLP || cfg->wide_layout != SF_MLP16 || cfg->row_dtype != slow->dtype) return SF_ERR_UNSUPPORTED;
+    if (cfg->P * 16 != slow->dims[0] || cfg->P < t->d.slow_pkts) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint32_t n = batch->n;
+    SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_batch_result), st));
+    if (n == 0) return SF_OK;
+    const TableDev& d = t->d;
+    // workspace: features, probabilities, decisions, wide rows and slow-model scratch for at most n flows
+    const size_t esz = slow->dtype == SF_BF16 ? 2 : 4;
+    const uint32_t Cs = slow->dims[slow->n_layers];
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += sf_align256(bytes); return o; };
+    const size_t o_feat = take((size_t)n * F * 4), o_prob = take((size_t)n * fo->C * 4), o_dec = take(n), o_lab = take(n),
+                 o_score = take((size_t)n * 4), o_bc = take((size_t)(n / 1024 + 2) * 4),
+                 o_rows = take((size_t)n * slow->dims[0] * esz), o_logits = take((size_t)n * Cs * 4), o_slab_lab = take(n),
+                 o_slow = take(sf_slow_scratch_bytes(slow, n));
+    int rc = sf_ws_reserve(ctx, off);
+    if (rc != SF_OK) return rc;
+    sf_ws_reset(ctx);
+    char* w = reinterpret_cast<char*>(sf_ws_alloc(ctx, off));
+    if (!w) return SF_ERR_ALLOC;
+    sf_time_new_record(ctx);
+    sf_time_begin(ctx, SF_T_TABLE, st);
+    SF_CUDA(cudaMemsetAsync(t->counts, 0, 64, st));
+    const uint32_t blocks = (n + 255) / 256;
+    probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, result_dev, ctx->d_state);
+    SF_LAUNCH_CHECK("probe_kernel");
+    // an even number of 4-bit passes over the slot bits (+1 bit for the "missed" key) ends in (key_a, idx_a)
+    uint32_t key_bits = t->log2_slots + 1;
+    key_bits = ((key_bits + 7) / 8) * 8;
+    const size_t sort_smem = (16 * 1024 + 1024) * sizeof(uint32_t);
+    SF_CUDA(cudaFuncSetAttribute(sort_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem));
+    sort_rank_kernel<<<1, 1024, sort_smem, st>>>(t->key_a, t->idx_a, t->key_b, t->idx_b, n, key_bits, t->rank);
+    SF_LAUNCH_CHECK("sort_rank_kernel");
+    apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->rank, t->pos, t->fire1_slot, t->counts);
+    SF_LAUNCH_CHECK("apply1_kernel");
+    gather_fast_kernel<<<(n * d.fast_pkts + 255) / 256, 256, 0, st>>>(d, t->fire1_slot, t->counts, t->c_size, t->c_iat, t->c_dir);
+    SF_LAUNCH_CHECK("gather_fast_kernel");
+    sf_time_end(ctx, SF_T_TABLE, st);
+    // S1..S3 on the flows that just completed their fast context (count stays on the device)
+    sf_packets fpk;
+    fpk.size = t->c_size; fpk.iat_us = t->c_iat; fpk.dir_bits = t->c_dir; fpk.hdr = nullptr; fpk.n_valid = nullptr;
+    fpk.n_flows = n; fpk.pitch_pkts = d.fast_pkts; fpk.hdr_bytes = 0;
+    float* feat = reinterpret_cast<float*>(w + o_feat);
+    float* prob = reinterpret_cast<float*>(w + o_prob);
+    sf_time_begin(ctx, SF_T_EXTRACT, st);
+    rc = sf_launch_extract(&fpk, d.fast_pkts, F, feat, st, &t->counts[0]);
+    sf_time_end(ctx, SF_T_EXTRACT, st);
+    if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_FOREST, st);
+    rc = sf_launch_forest(fo, feat, n, prob, nullptr, st, &t->counts[0]);
+    sf_time_end(ctx, SF_T_FOREST, st);
+    if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_SCORE, st);
+    rc = sf_launch_score(cfg, prob, n, fo->C, reinterpret_cast<uint8_t*>(w + o_dec), reinterpret_cast<uint8_t*>(w + o_lab),
+                         reinterpret_cast<float*>(w + o_score), reinterpret_cast<uint32_t*>(w + o_bc), &t->counts[0], st);
+    if (rc != SF_OK) return rc;
+    apply_route_kernel<<<blocks, 256, 0, st>>>(d, t->fire1_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_dec),
+                                               reinterpret_cast<uint8_t*>(w + o_lab), reinterpret_cast<float*>(w + o_score),
+                                               result_dev, ctx->d_state);
+    SF_LAUNCH_CHECK("apply_route_kernel");
+    apply2_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->rank, t->pos, t->fire2_slab, t->fire2_slot,
+                                          t->counts, result_dev, ctx->d_state);
+    SF_LAUNCH_CHECK("apply2_kernel");
+    sf_time_end(ctx, SF_T_SCORE, st);
+    // S4 on the flows that just completed their slow context
+    sf_packets spk;
+    spk.size = d.s_size; spk.iat_us = d.s_iat; spk.dir_bits = d.s_dir; spk.hdr = d.s_hdr; spk.n_valid = nullptr;
+    spk.n_flows = d.slow_slabs; spk.pitch_pkts = d.slow_pkts; spk.hdr_bytes = kHdr;
+    sf_route_cfg gcfg = *cfg;
+    gcfg.P_real = d.slow_pkts;
+    sf_time_begin(ctx, SF_T_GATHER, st);
+    rc = sf_launch_gather(ctx, &gcfg, &spk, t->fire2_slab, &t->counts[1], n, w + o_rows, st);
+    sf_time_end(ctx, SF_T_GATHER, st);
+    if (rc != SF_OK) return rc;
+    rc = sf_launch_slow(ctx, slow, w + o_rows, &t->counts[1], n, reinterpret_cast<float*>(w + o_logits),
+                        reinterpret_cast<uint8_t*>(w + o_slab_lab), w + o_slow, st);
+    if (rc != SF_OK) return rc;
+    apply_slow_kernel<<<blocks, 256, 0, st>>>(d, t->fire2_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_slab_lab), result_dev);
+    SF_LAUNCH_CHECK("apply_slow_kernel");
+    return SF_OK;
+}
+
+extern "C" int sf_table_lookup(sf_ctx* ctx, const sf_table* t, const sf_key* keys_dev, uint32_t n,
+                               sf_flow_result* out_dev, void* stream)
+{
+    if (!ctx || !t || (n && (!keys_dev || !out_dev))) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    if (n == 0) return SF_OK;
+    lookup_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(t->d, keys_dev, n, out_dev);
+    SF_LAUNCH_CHECK("lookup_kernel");
+    return SF_OK;
+}

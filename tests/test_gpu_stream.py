@@ -1,0 +1,123 @@
+"""GPU parity of the streaming path (device hash table + per-batch fast/slow firing)
+against the sequential reference, per key (the order of flows inside a batch is free)."""
+import numpy as np
+import pytest
+
+import flowgen
+import oracle
+from oracle.stream import simulate_stream
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2402_03694_b200 import build, binding as sf, harness as hz
+    build.build()
+    ctx = sf.sf_ctx_create(0, 0)
+    yield sf, hz, ctx
+    sf.sf_ctx_destroy(ctx)
+
+
+def _models(F, T, depth, C, dims, seed):
+    w = flowgen.gen_packets(seed, 4096, 8, 0)
+    feat = oracle.extract_features(w, 8, F, threads=4)
+    forest = flowgen.gen_forest(seed, "rf", T, depth, F, C, feat)
+    u = oracle.route_lc(oracle.forest_infer(forest, feat, threads=4), 2.0)["score"]
+    tau = np.full(C, oracle.universal_thresholds(u, [60])[0], np.float32)     # ~40 % assigned
+    return forest, tau, flowgen.gen_mlp(seed, dims)
+
+
+def _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg):
+    totals = np.zeros(8, np.int64)
+    res = torch.zeros(8, dtype=torch.int32, device="cuda")
+    for b in batches:
+        d = {k: hz.dev(b[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
+        pb = sf.make_pkt_batch(d["src"], d["dst"], d["sport"], d["dport"], d["proto"], d["dir"], d["size"], d["iat_us"], d["hdr"])
+        sf.sf_table_ingest(ctx, table, pb, forest_h, F, slow_h, rcfg, res)
+        torch.cuda.synchronize()
+        totals += res.cpu().numpy().astype(np.int64)
+    names = ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision", "missed")
+    return dict(zip(names, totals[:7].tolist()))
+
+
+def _lookup(sf, hz, ctx, table, keys):
+    arr = np.zeros(len(keys), sf.KEY_DTYPE)
+    for i, k in enumerate(keys):
+        arr[i]["src"], arr[i]["dst"], arr[i]["sport"], arr[i]["dport"], arr[i]["proto"] = k
+    kd = torch.from_numpy(arr.view(np.uint8).reshape(len(keys), 16).copy()).cuda()
+    out = torch.zeros((len(keys), 12), dtype=torch.uint8, device="cuda")
+    sf.sf_table_lookup(ctx, table, kd, len(keys), out)
+    torch.cuda.synchronize()
+    return out.cpu().numpy().reshape(-1).view(sf.FLOW_RESULT_DTYPE)
+
+
+@pytest.mark.parametrize("shape", ["config5_models", "small_models"])
+def test_stream_matches_sequential_reference(env, shape):
+    sf, hz, ctx = env
+    if shape == "config5_models":       # config 2's forest on 8 packets, config 2's MLP on 64 packets padded to 128
+        F, T, depth, C, dims, P_model = 48, 100, 12, 8, (2048, 1024, 1024, 1024, 8), 128
+        n_keys, n_batches, m = 1500, 24, 4096
+    else:
+        F, T, depth, C, dims, P_model = 24, 16, 8, 4, (1024, 256, 4), 64
+        n_keys, n_batches, m = 4000, 10, 8192 + 37
+    fast_pkts, slow_pkts = 8, 64
+    forest, tau, slow = _models(F, T, depth, C, dims, 91)
+    src = flowgen.StreamSource(92, n_keys, 1.1)
+    batches = [src.batch(b, m) for b in range(n_batches)]
+    per, cnt = simulate_stream(batches, fast_pkts, slow_pkts, F, forest, tau, slow, P_model, True, threads=8)
+    assert cnt["slow_fired"] > 5 and cnt["fast_done"] > 50 and cnt["dropped_after_decision"] > 0
+
+    forest_h = hz.make_forest(ctx, forest)
+    slow_h = sf.sf_mlp_create(ctx, sf.SF_BF16, slow["dims"], slow["W"], slow["b"])
+    table = sf.sf_table_create(ctx, 13, fast_pkts, slow_pkts, n_keys)
+    rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
+    sf.sf_ctx_poll(ctx, reset=True)
+    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg)
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert got["missed"] == 0 and c.device_error == 0
+    for k in ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision"):
+        assert got[k] == cnt[k], k
+    assert c.n_flows == cnt["fast_fired"] and c.n_escalated == cnt["escalated"] and c.n_slow_done == cnt["slow_fired"]
+    assert c.n_dropped_after_decision == cnt["dropped_after_decision"]
+
+    keys = list(per.keys())
+    res = _lookup(sf, hz, ctx, table, keys + [(1, 2, 3, 4, 5)])
+    assert res[-1]["found"] == 0
+    tol = 2e-2
+    for i, k in enumerate(keys):
+        r, g = per[k], res[i]
+        assert g["found"] == 1 and g["n_pkts"] == r["n_pkts"] and g["stage"] == r["stage"], k
+        if r["stage"] >= 1:
+            assert g["label_fast"] == r["label_fast"]
+            assert np.float32(g["score"]).view(np.uint32) == np.float32(r["score"]).view(np.uint32)
+        if r["stage"] == 3:
+            s = np.sort(r["logits"])
+            if s[-1] - s[-2] >= 2 * tol:
+                assert g["label_slow"] == r["label_slow"]
+    sf.sf_table_destroy(table)
+    sf.sf_slow_destroy(slow_h)
+    sf.sf_forest_destroy(forest_h)
+
+
+def test_full_table_is_reported_not_fatal(env):
+    sf, hz, ctx = env
+    forest, tau, slow = _models(24, 4, 4, 4, (1024, 64, 4), 93)
+    src = flowgen.StreamSource(94, 3000, 1.1)
+    batches = [src.batch(b, 4096) for b in range(3)]
+    forest_h = hz.make_forest(ctx, forest)
+    slow_h = sf.sf_mlp_create(ctx, sf.SF_BF16, slow["dims"], slow["W"], slow["b"])
+    table = sf.sf_table_create(ctx, 6, 8, 64, 16)           # 64 slots for ~2,000 distinct keys
+    rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, 64, 0, P_real=64)
+    sf.sf_ctx_poll(ctx, reset=True)
+    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, 24, slow_h, rcfg)
+    c = sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    assert got["missed"] > 0 and got["new_flows"] == 64
+    assert c.device_error == sf.SF_ERR_TABLE_FULL and c.n_missed == got["missed"]
+    assert sf.sf_ctx_poll(ctx).device_error == 0            # the context stays usable
+    sf.sf_table_destroy(table)
+    sf.sf_slow_destroy(slow_h)
+    sf.sf_forest_destroy(forest_h)
