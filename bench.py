@@ -32,12 +32,15 @@ METRIC = "flows/s end-to-end on 1 B200; fast-path HBM GB/s and slow-path TC % of
 UNIT = "flows/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 SM_COUNT, SM_MAX_MHZ = 148, 1965.0
-# thread-instructions a tree-node visit cannot do without: node load, feature address,
-# feature load, compare, child index, node address, loop counter/branch
-FOREST_INSTR_PER_VISIT = 7
-# DRAM bytes per launch measured with ncu for a kernel class, keyed by (class, config,
-# hash of the kernel's source) so that the figure turns null as soon as the kernel changes
-TRAFFIC_BY_SOURCE = {}
+# The tree walk is bound by the SM's load/store data pipe (one 128-byte wavefront per clock
+# per SM), not by HBM.  Wavefronts a warp cannot do without: per node visit one 64-bit node
+# load (32 lanes x 8 B = 2 wavefronts) and one feature load (1); per tree the leaf payload
+# (32 lanes x 4*C bytes, at 128 B per wavefront).
+FOREST_WAVEFRONTS_PER_VISIT = 3
+# DRAM bytes per launch measured with ncu for a kernel class (profiles/kernels_config2_262144_flows.md:
+# 766.5 MB over the three hidden-layer launches on 62,207 rows), keyed by (class, config, hash of the
+# kernel's source) so that the figure turns null as soon as the kernel changes
+TRAFFIC_BY_SOURCE = {("gemm", 2, "d10ca7bb842fcaa6"): {"bytes_per_row_per_launch": 766.5e6 / 3 / 62207}}
 
 
 def load_peaks():
@@ -155,7 +158,7 @@ def kernel_launches_per_step(cfg):
     if cfg.slow == "mlp":
         slow = (len(cfg.dims) - 1) + (1 if cfg.slow_dtype == "f32" else 0)    # layers (+ argmax for fp32)
     else:
-        slow = 2
+        slow = 1                                                              # the fused CNN kernel
     return 1 + 1 + 4 + slow + 1 + 2      # extract, forest, score/scan/scatter/gather, slow, count, merge x2
 
 
@@ -198,6 +201,85 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def run_stream(args, cfg):
+    """Config 5: interleaved packets of many concurrent flows in 64K-packet batches through the
+    device state table.  A step is `--batches-per-step` batches.  Reports first-seen flows/s,
+    packets/s, answered flows/s and the share of answered flows that ended at the fast stage."""
+    import torch
+    from paper_2402_03694_b200 import build as sfbuild
+    sfbuild.build()
+    from paper_2402_03694_b200 import binding as sf, harness as hz
+    torch.cuda.set_device(0)
+    ctx = sf.sf_ctx_create(0, 0)
+    n_keys = args.flows or cfg.n
+    m = 65536
+    bps = args.batches_per_step
+    n_batches = (args.warmup + args.steps) * bps
+    log2_slots = max(10, int(np.ceil(np.log2(n_keys / 0.3))))
+    src = flowgen.StreamSource(cfg.seed_data, n_keys, 1.1)
+    # models of config 2 (forest on 8 packets with the 48-feature definition, 2048-wide MLP on 64 packets + zero padding)
+    sample = flowgen.gen_packets(cfg.seed_data, 65536, cfg.N, 0)
+    sd = hz.upload_packets(sample, with_hdr=False)
+    feat = torch.empty((65536, cfg.F), dtype=torch.float32, device="cuda")
+    sf.sf_extract_features(ctx, sd["struct"], cfg.N, cfg.F, feat)
+    forest_np = flowgen.gen_forest(cfg.seed_model, "rf", cfg.T, cfg.depth, cfg.F, cfg.C, feat.cpu().numpy())
+    forest = hz.make_forest(ctx, forest_np)
+    pv = torch.empty((65536, cfg.C), dtype=torch.float32, device="cuda")
+    sc = torch.empty(65536, dtype=torch.float32, device="cuda")
+    ids = torch.empty(1, dtype=torch.uint32, device="cuda"); ne = torch.empty(1, dtype=torch.uint32, device="cuda")
+    sf.sf_fast_infer(ctx, forest, feat, 65536, pv)
+    never = hz.dev(np.full(cfg.C, 2.0, np.float32))
+    sf.sf_route(ctx, sf.make_route_cfg(sf.SF_LC_GT, never, sf.SF_MLP16, sf.SF_BF16, 128, 1), pv, 65536, cfg.C, None, ids, ne,
+                None, None, None, sc)
+    tau = np.full(cfg.C, sf.sf_universal_thresholds(sc.cpu().numpy(), [cfg.q_percent])[0], np.float32)
+    slow_np = flowgen.gen_mlp(cfg.seed_model, cfg.dims)
+    slow = sf.sf_mlp_create(ctx, sf.SF_BF16, slow_np["dims"], slow_np["W"], slow_np["b"])
+    sf.sf_ctx_poll(ctx, reset=True)
+    slabs = min(n_keys, max(1 << 16, (n_batches * m) // 16))
+    table = sf.sf_table_create(ctx, log2_slots, cfg.N, cfg.P, slabs)
+    rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, 128, 0, P_real=cfg.P)
+    dev_batches = []
+    for b in range(n_batches):
+        hb = src.batch(b, m)
+        d = {k: hz.dev(hb[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
+        dev_batches.append(sf.make_pkt_batch(d["src"], d["dst"], d["sport"], d["dport"], d["proto"], d["dir"], d["size"],
+                                             d["iat_us"], d["hdr"]))
+    res = torch.zeros((n_batches, 8), dtype=torch.int32, device="cuda")
+    for b in range(args.warmup * bps):
+        sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
+    torch.cuda.synchronize()
+    sampler = ClockSampler(os.environ.get("CUDA_VISIBLE_DEVICES", "0").split(",")[0])
+    sampler.start(); time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for b in range(args.warmup * bps, n_batches):
+        sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    c = sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    r = res[args.warmup * bps:].cpu().numpy().astype(np.int64).sum(0)
+    new_flows, fast_fired, fast_done, escalated, slow_fired, dropped, missed = [int(x) for x in r[:7]]
+    secs = ms * 1e-3
+    pk = (n_batches - args.warmup * bps) * m
+    answered = fast_done + slow_fired
+    line = {"metric": "sustained new flows/s through the device state table (config 5)", "value": new_flows / secs,
+            "unit": "new flows/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "keys": n_keys, "log2_slots": log2_slots, "batch_packets": m,
+                       "batches_per_step": bps, "zipf": 1.1, "l2": "state table larger than L2 (%.1f GB)" %
+                       ((1 << log2_slots) * (31 + cfg.N * 19 + 4) / 1e9)},
+            "packets_per_s": pk / secs, "answered_flows_per_s": answered / secs,
+            "fraction_answered_at_fast_stage": (fast_done / answered) if answered else None,
+            "counts": {"new_flows": new_flows, "fast_fired": fast_fired, "fast_done": fast_done, "escalated": escalated,
+                       "slow_fired": slow_fired, "dropped_after_decision": dropped, "missed": missed},
+            "us_per_batch": 1e3 * ms / (n_batches - args.warmup * bps), "gpu_launches": 16 * (n_batches - args.warmup * bps),
+            "clocks": clocks, "device_error": c.device_error}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -207,16 +289,20 @@ def main():
     ap.add_argument("--flows", type=int, default=0, help="override flows per batch (0 = the config's)")
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--ref-flows", type=int, default=4096)
-    ap.add_argument("--cpu-sample", type=int, default=32768)
+    ap.add_argument("--cpu-sample", type=int, default=262144)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batches-per-step", type=int, default=16)
     args = ap.parse_args()
     cfg = flowgen.get_config(args.config)
     if args.impl == "reference":
         run_reference(args, cfg)
         return
     args.warmup = max(args.warmup, 3)
+    if cfg.c == 5:
+        run_stream(args, cfg)
+        return
 
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -297,8 +383,10 @@ def main():
         "extract": ("hbm", n * (in_b + 4 * cfg.F) / 1e9, "GB/s", peaks["hbm_gbs"]),
         "gather": ("hbm", k_esc * (per_esc_in + cfg.D * esz) / 1e9, "GB/s", peaks["hbm_gbs"]),
         "gemm": ("tensor", k_esc * hidden_flops_per_row(cfg) / 1e12, "TFLOP/s", peaks["bf16_tflops_sustained"]),
-        "forest": ("alu", n * cfg.T * cfg.depth * FOREST_INSTR_PER_VISIT / 1e12, "Tinst/s",
-                   SM_COUNT * 128 * SM_MAX_MHZ * 1e6 / 1e12),
+        # "alu" here = the load/store unit's wavefront rate (148 SMs x 1 wavefront/clk x max SM clock)
+        "forest": ("alu", (n / 32.0) * cfg.T * (cfg.depth * FOREST_WAVEFRONTS_PER_VISIT +
+                                               (4 * (cfg.C if cfg.kind == "rf" else 1) * 32) / 128.0) / 1e9,
+                   "Gwavefront/s", SM_COUNT * SM_MAX_MHZ * 1e6 / 1e9),
     }
     roof_all = {}
     for k, (bound, work, unit, peak) in alg.items():
@@ -307,6 +395,8 @@ def main():
     dom = max(alg, key=lambda k: avg[k])
     src = {"gemm": "gemm_tc.cu", "forest": "forest.cu", "extract": "extract.cu", "gather": "route.cu"}[dom]
     traffic = TRAFFIC_BY_SOURCE.get((dom, cfg.c, src_hash(src)))
+    if traffic is not None:
+        traffic = traffic["bytes_per_row_per_launch"] * k_esc      # scaled by rows: traffic grows in proportion
     roofline = dict(roof_all[dom], kernel=dom, traffic=traffic, peak_source=peak_kind,
                     launches_per_step=(len(cfg.dims) - 2) if dom == "gemm" and cfg.slow == "mlp" else 1)
     roofline.pop("ms")
