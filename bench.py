@@ -248,6 +248,7 @@ def run_stream(args, cfg):
     for b in range(args.warmup * bps):
         sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
     torch.cuda.synchronize()
+    sf.sf_ctx_set_timing(ctx, True)
     sampler = ClockSampler(os.environ.get("CUDA_VISIBLE_DEVICES", "0").split(",")[0])
     sampler.start(); time.sleep(0.3)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -259,6 +260,9 @@ def run_stream(args, cfg):
     clocks = sampler.stop()
     ms = ev0.elapsed_time(ev1)
     c = sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    recs = [sf.sf_ctx_get_timing(ctx, back) for back in range(min(n_batches - args.warmup * bps, 64))]
+    sf.sf_ctx_set_timing(ctx, False)
+    stage_ms = {k: float(np.mean([x[k] for x in recs])) for k in recs[0]}
     r = res[args.warmup * bps:].cpu().numpy().astype(np.int64).sum(0)
     new_flows, fast_fired, fast_done, escalated, slow_fired, dropped, missed = [int(x) for x in r[:7]]
     secs = ms * 1e-3
@@ -275,7 +279,7 @@ def run_stream(args, cfg):
             "fraction_answered_at_fast_stage": (fast_done / answered) if answered else None,
             "counts": {"new_flows": new_flows, "fast_fired": fast_fired, "fast_done": fast_done, "escalated": escalated,
                        "slow_fired": slow_fired, "dropped_after_decision": dropped, "missed": missed},
-            "us_per_batch": 1e3 * ms / (n_batches - args.warmup * bps), "gpu_launches": 16 * (n_batches - args.warmup * bps),
+            "per_batch_stage_ms": stage_ms, "us_per_batch": 1e3 * ms / (n_batches - args.warmup * bps), "gpu_launches": 16 * (n_batches - args.warmup * bps),
             "clocks": clocks, "device_error": c.device_error}
     print(json.dumps(line))
 

@@ -6,8 +6,9 @@
 // ingested by a short chain of kernels on one stream:
 //   probe     one thread per packet: 128-bit compare-and-swap on the 16-byte key slot
 //             (claims an empty slot or recognises its own key; bounded linear probing)
-//   sort      one block: stable LSD radix sort of (slot, arrival index) so that each flow's
-//             packets of this batch sit together in ARRIVAL order, then their rank in the flow
+//   sort      key = arrival index of the flow's first packet in the batch (16 bits, unique per
+//             flow); stable LSD radix sort (4 passes of 4 bits, tiles of 1024) puts each flow's
+//             packets together in ARRIVAL order; rank = position minus start of the run
 //   apply1    packets that fall into a flow's first `fast_pkts` positions are written to its
 //             fast context; flows that just reached fast_pkts packets are listed
 //   fast path the listed flows' contexts are copied into dense planes and run through the
@@ -36,6 +37,7 @@ struct TableDev {
     // per slab
     uint16_t* s_size; uint32_t* s_iat; uint32_t* s_dir; uint8_t* s_hdr;
     uint32_t* slab_next;
+    uint32_t* first;              // per slot: arrival index of the flow's first packet in the current batch (else ~0)
     uint32_t mask, n_slots, fast_pkts, slow_pkts, slow_slabs;
 };
 
@@ -49,6 +51,7 @@ struct sf_table {
     uint32_t* key_a; uint32_t* key_b; uint32_t* idx_a; uint32_t* idx_b; uint32_t* rank; uint32_t* pos;
     uint32_t* fire1_slot; uint32_t* fire2_slab; uint32_t* fire2_slot;
     uint32_t* counts;                 // [0] n_fire1, [1] n_fire2
+    uint32_t* pkt_slot; uint32_t* hist;
     uint16_t* c_size; uint32_t* c_iat; uint32_t* c_dir;      // dense fast planes of the fired flows
     void* all;                        // one allocation behind everything above
 };
@@ -83,7 +86,7 @@ __device__ __forceinline__ uint32_t hash_key(uint64_t lo, uint64_t hi, uint32_t 
     return (uint32_t)mix64(lo ^ mix64(hi)) & mask;
 }
 
-__global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ pkt_slot, uint32_t* __restrict__ idx,
+__global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ pkt_slot,
                              sf_batch_result* res, sf_dev_state* st)
 {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -108,98 +111,118 @@ __global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ 
         atomicAdd((unsigned long long*)&st->counters.n_missed, 1ull);
         sf_dev_set_error(st, SF_ERR_TABLE_FULL);
     }
+    else atomicMin(&t.first[slot], i);
     pkt_slot[i] = slot;
+}
+
+// Sort key of a packet = arrival index of its flow's first packet in this batch: 16 bits,
+// unique per flow; a packet that found no slot is a run of its own.
+__global__ void key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
+                           uint32_t* __restrict__ key, uint32_t* __restrict__ idx)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const uint32_t slot = pkt_slot[i];
+    key[i] = (slot < t.n_slots) ? t.first[slot] : i;
     idx[i] = i;
 }
 
-// One block, 1024 threads.  Stable LSD radix sort (4-bit digits) of n <= 65536 (key, idx) pairs,
-// thread t owning the contiguous chunk [t*per, (t+1)*per) in every pass, then the rank of each
-// sorted item inside its run of equal keys.
-__global__ void __launch_bounds__(1024, 1)
-sort_rank_kernel(uint32_t* key_a, uint32_t* idx_a, uint32_t* key_b, uint32_t* idx_b, uint32_t n, uint32_t key_bits,
-                 uint32_t* __restrict__ rank)
+// Stable LSD radix sort, 4-bit digits, tiles of 1024 items (256 threads x 4 consecutive items).
+constexpr uint32_t kTile = 1024;
+__global__ void __launch_bounds__(256)
+radix_hist_kernel(const uint32_t* __restrict__ keys, uint32_t n, uint32_t shift, uint32_t* __restrict__ hist, uint32_t nblk)
 {
-    extern __shared__ uint32_t sm[];                 // [16][1024] counts / offsets, then [1024] scan scratch
-    uint32_t* cnts = sm;
-    uint32_t* tot = sm + 16 * 1024;
+    __shared__ uint32_t c[16];
+    if (threadIdx.x < 16) c[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t j0 = blockIdx.x * kTile + threadIdx.x * 4;
+#pragma unroll
+    for (uint32_t e = 0; e < 4; e++)
+        if (j0 + e < n) atomicAdd(&c[(keys[j0 + e] >> shift) & 15u], 1u);
+    __syncthreads();
+    if (threadIdx.x < 16) hist[threadIdx.x * nblk + blockIdx.x] = c[threadIdx.x];
+}
+
+__global__ void __launch_bounds__(1024)
+radix_scan_kernel(uint32_t* __restrict__ hist, uint32_t entries)        // exclusive scan of <= 1024 entries
+{
+    __shared__ uint32_t tot[32];
     const uint32_t t = threadIdx.x;
-    const uint32_t per = (n + 1023) / 1024;
-    const uint32_t lo = min(n, t * per), hi = min(n, lo + per);
-    uint32_t* ks = key_a; uint32_t* is = idx_a; uint32_t* kd = key_b; uint32_t* id = idx_b;
-    const uint32_t passes = (key_bits + 3) / 4;      // the host makes this even so the result lands in (key_a, idx_a)
-    for (uint32_t pass = 0; pass < passes; pass++) {
-        const uint32_t shift = pass * 4;
-        uint32_t h[16];
+    const uint32_t v = (t < entries) ? hist[t] : 0u;
+    uint32_t x = v;
 #pragma unroll
-        for (int d = 0; d < 16; d++) h[d] = 0;
-        for (uint32_t j = lo; j < hi; j++) {
-            const uint32_t dg = (ks[j] >> shift) & 15u;
-#pragma unroll
-            for (int d = 0; d < 16; d++) h[d] += (dg == (uint32_t)d) ? 1u : 0u;
-        }
-#pragma unroll
-        for (int d = 0; d < 16; d++) cnts[d * 1024 + t] = h[d];
-        __syncthreads();
-        // exclusive scan of the 16384 counters in (digit, thread) order: thread t scans entries [16t, 16t+16)
-        uint32_t loc[16], s = 0;
-#pragma unroll
-        for (int e = 0; e < 16; e++) { loc[e] = s; s += cnts[t * 16 + e]; }
-        uint32_t x = s;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
-        if ((t & 31) == 31) tot[t >> 5] = x;
-        __syncthreads();
-        if (t < 32) {
-            uint32_t w = tot[t], z = w;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (t >= (uint32_t)o) z += y; }
-            tot[t] = z - w;
-        }
-        __syncthreads();
-        const uint32_t base = tot[t >> 5] + x - s;
-#pragma unroll
-        for (int e = 0; e < 16; e++) cnts[t * 16 + e] = base + loc[e];
-        __syncthreads();
-#pragma unroll
-        for (int d = 0; d < 16; d++) h[d] = cnts[d * 1024 + t];
-        for (uint32_t j = lo; j < hi; j++) {
-            const uint32_t k = ks[j], dg = (k >> shift) & 15u;
-            uint32_t p = 0;
-#pragma unroll
-            for (int d = 0; d < 16; d++) if (dg == (uint32_t)d) { p = h[d]; h[d] = p + 1; }
-            kd[p] = k; id[p] = is[j];
-        }
-        __syncthreads();
-        uint32_t* tk = ks; ks = kd; kd = tk;
-        uint32_t* ti = is; is = id; id = ti;
-    }
-    // rank inside runs of equal keys: position minus the position of the run's first item
-    int last_head = -1;
-    for (uint32_t j = lo; j < hi; j++) if (j == 0 || ks[j] != ks[j - 1]) last_head = (int)j;
-    int x = last_head;                               // inclusive max-scan over threads
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x = max(x, y); }
-    int* itot = reinterpret_cast<int*>(tot);
-    if ((t & 31) == 31) itot[t >> 5] = x;
+    for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
+    if ((t & 31) == 31) tot[t >> 5] = x;
     __syncthreads();
     if (t < 32) {
-        int z = itot[t];
+        uint32_t w = tot[t], z = w;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (t >= (uint32_t)o) z = max(z, y); }
-        itot[t] = z;
+        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (t >= (uint32_t)o) z += y; }
+        tot[t] = z - w;
     }
     __syncthreads();
-    int carry = -1;                                  // last run head strictly before this thread's chunk
-    {
-        int prev_lane = __shfl_up_sync(0xFFFFFFFFu, x, 1);
-        if ((t & 31) != 0) carry = prev_lane;
-        if ((t >> 5) > 0) carry = max(carry, itot[(t >> 5) - 1]);
+    if (t < entries) hist[t] = tot[t >> 5] + x - v;
+}
+
+__global__ void __launch_bounds__(256)
+radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ iin, uint32_t* __restrict__ kout,
+                     uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk)
+{
+    __shared__ uint32_t cnt[16 * 256];
+    __shared__ uint32_t tot[8];
+    const uint32_t t = threadIdx.x;
+    const uint32_t j0 = blockIdx.x * kTile + t * 4;
+    uint32_t k[4], dg[4];
+    uint32_t h[16];
+#pragma unroll
+    for (int d = 0; d < 16; d++) h[d] = 0;
+#pragma unroll
+    for (uint32_t e = 0; e < 4; e++) {
+        k[e] = (j0 + e < n) ? kin[j0 + e] : 0u;
+        dg[e] = (k[e] >> shift) & 15u;
+        if (j0 + e < n) {
+#pragma unroll
+            for (int d = 0; d < 16; d++) h[d] += (dg[e] == (uint32_t)d) ? 1u : 0u;
+        }
     }
-    int head = carry;
-    for (uint32_t j = lo; j < hi; j++) {
-        if (j == 0 || ks[j] != ks[j - 1]) head = (int)j;
-        rank[j] = j - (uint32_t)head;
+#pragma unroll
+    for (int d = 0; d < 16; d++) cnt[d * 256 + t] = h[d];
+    __syncthreads();
+    // exclusive scan of the 4096 counters in (digit, thread) order; thread t owns entries [16t, 16t+16)
+    uint32_t loc[16], s = 0;
+#pragma unroll
+    for (int e = 0; e < 16; e++) { loc[e] = s; s += cnt[t * 16 + e]; }
+    uint32_t x = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
+    if ((t & 31) == 31) tot[t >> 5] = x;
+    __syncthreads();
+    uint32_t wbase = 0;
+    for (uint32_t w = 0; w < (t >> 5); w++) wbase += tot[w];
+    __syncthreads();
+    const uint32_t base = wbase + x - s;
+#pragma unroll
+    for (int e = 0; e < 16; e++) cnt[t * 16 + e] = base + loc[e];
+    __syncthreads();
+    // position = start of (digit, this block) in the output + rank among the block's items of that digit
+#pragma unroll
+    for (uint32_t e = 0; e < 4; e++) {
+        if (j0 + e < n) {
+            const uint32_t d = dg[e];
+            uint32_t before = 0;                         // earlier items of this thread with the same digit
+#pragma unroll
+            for (uint32_t q = 0; q < 4; q++) if (q < e && dg[q] == d) before++;
+            const uint32_t p = hist[d * nblk + blockIdx.x] + (cnt[d * 256 + t] - cnt[d * 256]) + before;
+            kout[p] = k[e];
+            iout[p] = iin[j0 + e];
+        }
     }
+}
+
+__device__ __forceinline__ uint32_t run_start(const uint32_t* __restrict__ s_key, uint32_t n, uint32_t key) {
+    uint32_t lo = 0, hi = n;                             // first position whose key is >= key
+    while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (s_key[mid] < key) lo = mid + 1; else hi = mid; }
+    return lo;
 }
 
 __device__ __forceinline__ void store_packet(uint16_t* sz, uint32_t* ia, uint32_t* dirw, uint8_t* hd, uint32_t row,
@@ -215,14 +238,16 @@ __device__ __forceinline__ void store_packet(uint16_t* sz, uint32_t* ia, uint32_
 }
 
 __global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
-                              const uint32_t* __restrict__ rank, uint32_t* __restrict__ pos_out,
+                              const uint32_t* __restrict__ pkt_slot, uint32_t* __restrict__ rank, uint32_t* __restrict__ pos_out,
                               uint32_t* __restrict__ fire1_slot, uint32_t* __restrict__ counts)
 {
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= b.n) return;
-    const uint32_t slot = s_key[j];
-    if (slot >= t.n_slots) { pos_out[j] = kMiss; return; }
-    const uint32_t pos = t.cnt[slot] + rank[j];
+    const uint32_t slot = pkt_slot[s_idx[j]];
+    if (slot >= t.n_slots) { pos_out[j] = kMiss; rank[j] = 0; return; }
+    const uint32_t rk = j - run_start(s_key, b.n, s_key[j]);     // arrival rank among the flow's packets of this batch
+    rank[j] = rk;
+    const uint32_t pos = t.cnt[slot] + rk;
     pos_out[j] = pos;
     if (pos < t.fast_pkts) {
         store_packet(t.f_size, t.f_iat, t.f_dir, t.f_hdr, slot, t.fast_pkts, 1, pos, b, s_idx[j]);
@@ -281,13 +306,13 @@ __global__ void apply_route_kernel(TableDev t, const uint32_t* __restrict__ fire
 }
 
 __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
-                              const uint32_t* __restrict__ rank, const uint32_t* __restrict__ pos_in,
+                              const uint32_t* __restrict__ pkt_slot, const uint32_t* __restrict__ rank, const uint32_t* __restrict__ pos_in,
                               uint32_t* __restrict__ fire2_slab, uint32_t* __restrict__ fire2_slot,
                               uint32_t* __restrict__ counts, sf_batch_result* res, sf_dev_state* st)
 {
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= b.n) return;
-    const uint32_t slot = s_key[j];
+    const uint32_t slot = pkt_slot[s_idx[j]];
     if (slot >= t.n_slots) return;
     const uint32_t pos = pos_in[j];
     if (pos >= t.fast_pkts) {
@@ -305,7 +330,7 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
         }
     }
     // the last packet of the flow's run in this batch advances the flow's packet counter
-    if (j + 1 == b.n || s_key[j + 1] != slot) t.cnt[slot] += rank[j] + 1;
+    if (j + 1 == b.n || s_key[j + 1] != s_key[j]) { t.cnt[slot] += rank[j] + 1; t.first[slot] = 0xFFFFFFFFu; }
 }
 
 __global__ void apply_slow_kernel(TableDev t, const uint32_t* __restrict__ fire2_slot, const uint32_t* __restrict__ counts,
@@ -368,7 +393,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     need(S * fast_pkts * 2); need(S * fast_pkts * 4); need(S * 4); need(S * fast_pkts * kHdr);
     need(B * slow_pkts * 2); need(B * slow_pkts * 4); need(B * W * 4); need(B * slow_pkts * kHdr); need(4);
     for (int k = 0; k < 9; k++) need((size_t)kMaxBatch * 4);
-    need(64);
+    need(64); need((size_t)kMaxBatch * 4); need(1024 * 4); need(S * 4);
     need((size_t)kMaxBatch * fast_pkts * 2); need((size_t)kMaxBatch * fast_pkts * 4); need((size_t)kMaxBatch * 4);
     cudaError_t e = cudaMalloc(&t->all, total);
     if (e != cudaSuccess) { delete t; sf_set_cuda_error(e, "cudaMalloc(table)"); return SF_ERR_ALLOC; }
@@ -391,6 +416,10 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     t->fire1_slot = carve<uint32_t>(p, kMaxBatch); t->fire2_slab = carve<uint32_t>(p, kMaxBatch);
     t->fire2_slot = carve<uint32_t>(p, kMaxBatch);
     t->counts = carve<uint32_t>(p, 16);
+    t->pkt_slot = carve<uint32_t>(p, kMaxBatch); t->hist = carve<uint32_t>(p, 1024);
+    d.first = carve<uint32_t>(p, S);
+    e = cudaMemset(d.first, 0xFF, S * 4);
+    if (e != cudaSuccess) { cudaFree(t->all); delete t; return sf_set_cuda_error(e, "cudaMemset(table)"); }
     t->c_size = carve<uint16_t>(p, (size_t)kMaxBatch * fast_pkts); t->c_iat = carve<uint32_t>(p, (size_t)kMaxBatch * fast_pkts);
     t->c_dir = carve<uint32_t>(p, kMaxBatch);
     *out = t;
@@ -437,16 +466,24 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     sf_time_begin(ctx, SF_T_TABLE, st);
     SF_CUDA(cudaMemsetAsync(t->counts, 0, 64, st));
     const uint32_t blocks = (n + 255) / 256;
-    probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, result_dev, ctx->d_state);
+    probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->pkt_slot, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("probe_kernel");
-    // an even number of 4-bit passes over the slot bits (+1 bit for the "missed" key) ends in (key_a, idx_a)
-    uint32_t key_bits = t->log2_slots + 1;
-    key_bits = ((key_bits + 7) / 8) * 8;
-    const size_t sort_smem = (16 * 1024 + 1024) * sizeof(uint32_t);
-    SF_CUDA(cudaFuncSetAttribute(sort_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem));
-    sort_rank_kernel<<<1, 1024, sort_smem, st>>>(t->key_a, t->idx_a, t->key_b, t->idx_b, n, key_bits, t->rank);
-    SF_LAUNCH_CHECK("sort_rank_kernel");
-    apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->rank, t->pos, t->fire1_slot, t->counts);
+    key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a);
+    SF_LAUNCH_CHECK("key_kernel");
+    {
+        // 16-bit keys: four 4-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
+        const uint32_t nblk = (n + kTile - 1) / kTile;
+        uint32_t* kin = t->key_a; uint32_t* iin = t->idx_a; uint32_t* kout = t->key_b; uint32_t* iout = t->idx_b;
+        for (uint32_t pass = 0; pass < 4; pass++) {
+            radix_hist_kernel<<<nblk, 256, 0, st>>>(kin, n, pass * 4, t->hist, nblk);
+            radix_scan_kernel<<<1, 1024, 0, st>>>(t->hist, 16 * nblk);
+            radix_scatter_kernel<<<nblk, 256, 0, st>>>(kin, iin, kout, iout, n, pass * 4, t->hist, nblk);
+            SF_LAUNCH_CHECK("radix pass");
+            uint32_t* tk = kin; kin = kout; kout = tk;
+            uint32_t* ti = iin; iin = iout; iout = ti;
+        }
+    }
+    apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts);
     SF_LAUNCH_CHECK("apply1_kernel");
     gather_fast_kernel<<<(n * d.fast_pkts + 255) / 256, 256, 0, st>>>(d, t->fire1_slot, t->counts, t->c_size, t->c_iat, t->c_dir);
     SF_LAUNCH_CHECK("gather_fast_kernel");
@@ -473,7 +510,7 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
                                                reinterpret_cast<uint8_t*>(w + o_lab), reinterpret_cast<float*>(w + o_score),
                                                result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("apply_route_kernel");
-    apply2_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->rank, t->pos, t->fire2_slab, t->fire2_slot,
+    apply2_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire2_slab, t->fire2_slot,
                                           t->counts, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("apply2_kernel");
     sf_time_end(ctx, SF_T_SCORE, st);
