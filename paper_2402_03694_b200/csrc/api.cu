@@ -6,6 +6,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <atomic>
+#include <thread>
 #include <vector>
 
 static thread_local char g_cuda_err[512] = "";
@@ -131,6 +133,8 @@ extern "C" void sf_ctx_destroy(sf_ctx* c) {
     cudaSetDevice(c->device);
     if (c->ws) cudaFree(c->ws);
     if (c->stage) cudaFree(c->stage);
+    if (c->stage2) cudaFree(c->stage2);
+    if (c->pin) cudaFreeHost(c->pin);
     if (c->d_state) cudaFree(c->d_state);
     if (c->t_ev[0][0][0])
         for (int r = 0; r < 64; r++)
@@ -172,7 +176,7 @@ extern "C" int sf_universal_thresholds(const float* scores, uint64_t n, const ui
 namespace {
 
 struct ServePlan {
-    size_t feat, fast_out, decision, label_fast, esc_ids, rows, logits, label_slow, route_scratch, slow_scratch, total;
+    size_t feat, fast_out, decision, label_fast, esc_ids, iota, rows, logits, label_slow, route_scratch, slow_scratch, total;
 };
 
 uint32_t slow_classes(const sf_slow* s) { return s->arch == SF_SLOW_CNN ? s->n_cls : s->dims[s->n_layers]; }
@@ -188,6 +192,7 @@ ServePlan plan_serve(const sf_forest* fo, const sf_slow* s, uint32_t n, uint32_t
     p.decision = take(n);
     p.label_fast = take(n);
     p.esc_ids = take((size_t)cfg->capacity * 4);
+    p.iota = take((size_t)cfg->capacity * 4);
     p.rows = take((size_t)cfg->capacity * slow_width(s) * esz);
     p.logits = take((size_t)cfg->capacity * slow_classes(s) * 4);
     p.label_slow = take(cfg->capacity);
@@ -219,16 +224,20 @@ int check_serve_args(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const s
     return SF_OK;
 }
 
+// phases: 1 = S1..S3 without the wide-row gather, 2 = gather (rows 0..n_esc-1 of `wide`, which then holds
+// only the assigned flows' planes in list order) + S4 + S5 on the state phase 1 left, 3 = everything.
+enum { SF_PHASE_FAST = 1, SF_PHASE_SLOW = 2, SF_PHASE_ALL = 3 };
+
 int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf_packets* fast, uint32_t N, uint32_t F,
                     const sf_packets* wide, const sf_route_cfg* cfg, uint8_t* label_out, uint8_t* stage_out,
-                    uint32_t* n_esc_out, cudaStream_t st)
+                    uint32_t* n_esc_out, cudaStream_t st, int phases = SF_PHASE_ALL)
 {
     const uint32_t n = fast->n_flows;
     const ServePlan p = plan_serve(fo, s, n, F, cfg);
     int rc = sf_ws_reserve(ctx, p.total);
     if (rc != SF_OK) return rc;
-    sf_ws_reset(ctx);
-    char* base = reinterpret_cast<char*>(sf_ws_alloc(ctx, p.total));
+    if (phases & SF_PHASE_FAST) sf_ws_reset(ctx);
+    char* base = (phases & SF_PHASE_FAST) ? reinterpret_cast<char*>(sf_ws_alloc(ctx, p.total)) : ctx->ws;
     if (!base) return SF_ERR_ALLOC;
     float* feat = reinterpret_cast<float*>(base + p.feat);
     float* fast_out = reinterpret_cast<float*>(base + p.fast_out);
@@ -240,18 +249,31 @@ int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf
     uint8_t* label_slow = reinterpret_cast<uint8_t*>(base + p.label_slow);
     uint32_t* n_esc_dev = &ctx->d_state->scan_total;
 
-    sf_time_new_record(ctx);
-    sf_time_begin(ctx, SF_T_EXTRACT, st);
-    rc = sf_launch_extract(fast, N, F, feat, st);
-    sf_time_end(ctx, SF_T_EXTRACT, st);
-    if (rc != SF_OK) return rc;
-    sf_time_begin(ctx, SF_T_FOREST, st);
-    rc = sf_launch_forest(fo, feat, n, fast_out, nullptr, st);
-    sf_time_end(ctx, SF_T_FOREST, st);
-    if (rc != SF_OK) return rc;
-    rc = sf_launch_route(ctx, cfg, fast_out, n, fo->C, wide, esc_ids, n_esc_out, rows, decision, label_fast, nullptr,
-                         base + p.route_scratch, st);
-    if (rc != SF_OK) return rc;
+    if (phases & SF_PHASE_FAST) {
+        sf_time_new_record(ctx);
+        sf_time_begin(ctx, SF_T_EXTRACT, st);
+        rc = sf_launch_extract(fast, N, F, feat, st);
+        sf_time_end(ctx, SF_T_EXTRACT, st);
+        if (rc != SF_OK) return rc;
+        sf_time_begin(ctx, SF_T_FOREST, st);
+        rc = sf_launch_forest(fo, feat, n, fast_out, nullptr, st);
+        sf_time_end(ctx, SF_T_FOREST, st);
+        if (rc != SF_OK) return rc;
+        rc = sf_launch_route(ctx, cfg, fast_out, n, fo->C, (phases & SF_PHASE_SLOW) ? wide : nullptr, esc_ids, n_esc_out,
+                             rows, decision, label_fast, nullptr, base + p.route_scratch, st);
+        if (rc != SF_OK) return rc;
+        ctx->last_feat = feat; ctx->last_fast_out = fast_out; ctx->last_esc_ids = esc_ids; ctx->last_rows = rows;
+        ctx->last_logits = logits; ctx->last_label_fast = label_fast; ctx->last_label_slow = label_slow;
+        if (!(phases & SF_PHASE_SLOW)) return SF_OK;
+    } else {
+        uint32_t* iota = reinterpret_cast<uint32_t*>(base + p.iota);
+        rc = sf_launch_iota(iota, cfg->capacity, st);
+        if (rc != SF_OK) return rc;
+        sf_time_begin(ctx, SF_T_GATHER, st);
+        rc = sf_launch_gather(ctx, cfg, wide, iota, n_esc_dev, cfg->capacity, rows, st);
+        sf_time_end(ctx, SF_T_GATHER, st);
+        if (rc != SF_OK) return rc;
+    }
     rc = sf_launch_slow(ctx, s, rows, n_esc_dev, cfg->capacity, logits, label_slow, base + p.slow_scratch, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_MERGE, st);
@@ -288,6 +310,112 @@ extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_sl
     const uint32_t n = fast_h->n_flows;
     const bool shared = fast_h->size == wide_h->size && fast_h->iat_us == wide_h->iat_us &&
                         fast_h->dir_bits == wide_h->dir_bits && fast_h->pitch_pkts == wide_h->pitch_pkts;
+    if (!shared) {
+        // Two-phase host path: only the fast planes of all flows cross the bus first; after S1..S3 the
+        // assigned ids come back, worker threads compact those flows' wide rows into pinned memory and
+        // copy them over chunk by chunk (the gather of one chunk overlaps the copy of the previous one),
+        // and only then S4/S5 run.  The slow model sees more packets only of the flows assigned to it.
+        const uint32_t Pw = wide_h->pitch_pkts, Hb = wide_h->hdr_bytes, words = (Pw + 31) / 32;
+        const size_t fsz = (size_t)n * fast_h->pitch_pkts * 2, fia = (size_t)n * fast_h->pitch_pkts * 4,
+                     fdr = (size_t)n * ((fast_h->pitch_pkts + 31) / 32) * 4, fnv = fast_h->n_valid ? (size_t)n : 0;
+        const uint32_t n_tau2 = cfg_h->rule == SF_LC_GT ? fo->C : 1;
+        size_t off2 = 0;
+        auto take2 = [&](size_t bytes) { size_t o = off2; off2 += sf_align256(bytes); return o; };
+        const size_t a_fs = take2(fsz), a_fi = take2(fia), a_fd = take2(fdr), a_fv = take2(fnv), a_tau = take2(n_tau2 * 4),
+                     a_lab = take2(n), a_stg = take2(n), a_ne = take2(4);
+        if (off2 > ctx->stage_bytes) {
+            SF_CUDA(cudaDeviceSynchronize());
+            if (ctx->stage) { cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
+            cudaError_t e = cudaMalloc(&ctx->stage, off2);
+            if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(staging)"); return SF_ERR_ALLOC; }
+            ctx->stage_bytes = off2;
+        }
+        char* sb2 = ctx->stage;
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_fs, fast_h->size, fsz, cudaMemcpyHostToDevice, st));
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_fi, fast_h->iat_us, fia, cudaMemcpyHostToDevice, st));
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_fd, fast_h->dir_bits, fdr, cudaMemcpyHostToDevice, st));
+        if (fnv) SF_CUDA(cudaMemcpyAsync(sb2 + a_fv, fast_h->n_valid, fnv, cudaMemcpyHostToDevice, st));
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_tau, cfg_h->tau, (size_t)n_tau2 * 4, cudaMemcpyHostToDevice, st));
+        sf_packets fd2 = *fast_h;
+        fd2.size = (const uint16_t*)(sb2 + a_fs); fd2.iat_us = (const uint32_t*)(sb2 + a_fi);
+        fd2.dir_bits = (const uint32_t*)(sb2 + a_fd); fd2.hdr = nullptr;
+        fd2.n_valid = fnv ? (const uint8_t*)(sb2 + a_fv) : nullptr;
+        sf_route_cfg cd2 = *cfg_h;
+        cd2.tau = (const float*)(sb2 + a_tau);
+        rc = serve_on_device(ctx, fo, s, &fd2, N, F, wide_h, &cd2, (uint8_t*)(sb2 + a_lab), (uint8_t*)(sb2 + a_stg),
+                             (uint32_t*)(sb2 + a_ne), st, SF_PHASE_FAST);
+        if (rc != SF_OK) return rc;
+        uint32_t k = 0;
+        SF_CUDA(cudaMemcpyAsync(&k, sb2 + a_ne, 4, cudaMemcpyDeviceToHost, st));
+        SF_CUDA(cudaStreamSynchronize(st));
+        std::vector<uint32_t> ids(k);
+        if (k) SF_CUDA(cudaMemcpy(ids.data(), ctx->last_esc_ids, (size_t)k * 4, cudaMemcpyDeviceToHost));
+        // compact planes of the k assigned flows: [k][Pw] sizes, [k][Pw] iats, [k][words] dir words, [k][Pw][Hb] header bytes, [k] n_valid
+        const size_t r_sz = (size_t)Pw * 2, r_ia = (size_t)Pw * 4, r_dr = (size_t)words * 4, r_hd = (size_t)Pw * Hb;
+        const size_t c_sz = 0, c_ia = sf_align256(c_sz + k * r_sz), c_dr = sf_align256(c_ia + k * r_ia),
+                     c_hd = sf_align256(c_dr + k * r_dr), c_nv = sf_align256(c_hd + k * r_hd),
+                     c_total = sf_align256(c_nv + (wide_h->n_valid ? k : 0)) + 256;
+        if (c_total > ctx->stage2_bytes) {
+            SF_CUDA(cudaDeviceSynchronize());
+            if (ctx->stage2) { cudaFree(ctx->stage2); ctx->stage2 = nullptr; }
+            if (ctx->pin) { cudaFreeHost(ctx->pin); ctx->pin = nullptr; }
+            ctx->stage2_bytes = 0;
+            const size_t want = c_total + c_total / 4;
+            cudaError_t e = cudaMalloc(&ctx->stage2, want);
+            if (e == cudaSuccess) e = cudaMallocHost(&ctx->pin, want);
+            if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(compact staging)"); return SF_ERR_ALLOC; }
+            ctx->stage2_bytes = want;
+        }
+        char* pin = ctx->pin; char* dv = ctx->stage2;
+        const uint32_t chunk = 4096, n_chunks = (k + chunk - 1) / chunk;
+        std::atomic<uint32_t> next(0);
+        std::atomic<int> failed(0);
+        auto worker = [&]() {
+            if (cudaSetDevice(ctx->device) != cudaSuccess) { failed = 1; return; }
+            for (;;) {
+                const uint32_t c = next.fetch_add(1);
+                if (c >= n_chunks) break;
+                const uint32_t r0 = c * chunk, r1 = std::min(k, r0 + chunk);
+                for (uint32_t r = r0; r < r1; r++) {
+                    const size_t f = ids[r];
+                    memcpy(pin + c_sz + r * r_sz, (const char*)wide_h->size + f * r_sz, r_sz);
+                    memcpy(pin + c_ia + r * r_ia, (const char*)wide_h->iat_us + f * r_ia, r_ia);
+                    memcpy(pin + c_dr + r * r_dr, (const char*)wide_h->dir_bits + f * r_dr, r_dr);
+                    memcpy(pin + c_hd + r * r_hd, (const char*)wide_h->hdr + f * r_hd, r_hd);
+                    if (wide_h->n_valid) pin[c_nv + r] = (char)wide_h->n_valid[f];
+                }
+                const size_t m = r1 - r0;
+                cudaError_t e = cudaMemcpyAsync(dv + c_sz + r0 * r_sz, pin + c_sz + r0 * r_sz, m * r_sz, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess) e = cudaMemcpyAsync(dv + c_ia + r0 * r_ia, pin + c_ia + r0 * r_ia, m * r_ia, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess) e = cudaMemcpyAsync(dv + c_dr + r0 * r_dr, pin + c_dr + r0 * r_dr, m * r_dr, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess) e = cudaMemcpyAsync(dv + c_hd + r0 * r_hd, pin + c_hd + r0 * r_hd, m * r_hd, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess && wide_h->n_valid) e = cudaMemcpyAsync(dv + c_nv + r0, pin + c_nv + r0, m, cudaMemcpyHostToDevice, st);
+                if (e != cudaSuccess) failed = 1;
+            }
+        };
+        {
+            uint32_t n_thr = std::thread::hardware_concurrency();
+            n_thr = std::max(1u, std::min(std::min(n_thr, 16u), n_chunks));
+            std::vector<std::thread> pool;
+            for (uint32_t i = 1; i < n_thr; i++) pool.emplace_back(worker);
+            worker();
+            for (auto& th : pool) th.join();
+        }
+        if (failed) return sf_set_cuda_error(cudaGetLastError(), "compact copy");
+        sf_packets wd2 = *wide_h;
+        wd2.size = (const uint16_t*)(dv + c_sz); wd2.iat_us = (const uint32_t*)(dv + c_ia);
+        wd2.dir_bits = (const uint32_t*)(dv + c_dr); wd2.hdr = (const uint8_t*)(dv + c_hd);
+        wd2.n_valid = wide_h->n_valid ? (const uint8_t*)(dv + c_nv) : nullptr;
+        wd2.n_flows = k;
+        rc = serve_on_device(ctx, fo, s, &fd2, N, F, &wd2, &cd2, (uint8_t*)(sb2 + a_lab), (uint8_t*)(sb2 + a_stg),
+                             (uint32_t*)(sb2 + a_ne), st, SF_PHASE_SLOW);
+        if (rc != SF_OK) return rc;
+        SF_CUDA(cudaMemcpyAsync(label_h, sb2 + a_lab, n, cudaMemcpyDeviceToHost, st));
+        SF_CUDA(cudaMemcpyAsync(stage_h, sb2 + a_stg, n, cudaMemcpyDeviceToHost, st));
+        if (n_esc_h) *n_esc_h = k;
+        SF_CUDA(cudaStreamSynchronize(st));
+        return SF_OK;
+    }
     auto plane_bytes = [](const sf_packets* p, size_t& s_sz, size_t& s_iat, size_t& s_dir, size_t& s_hdr, size_t& s_nv) {
         s_sz = (size_t)p->n_flows * p->pitch_pkts * 2;
         s_iat = (size_t)p->n_flows * p->pitch_pkts * 4;

@@ -27,6 +27,9 @@ struct sf_ctx {
     // staging for the host-pointer entry point
     char*  stage;
     size_t stage_bytes;
+    char*  stage2;               // compact wide planes of the assigned flows (device) and their pinned host mirror
+    char*  pin;
+    size_t stage2_bytes;
     // optional per-kernel-class timing: ring of event pairs
     int timing;
     uint32_t t_rec;                               // records started so far
@@ -94,6 +97,7 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
                     uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st);
 int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C, uint8_t* decision,
                     uint8_t* label, float* score, uint32_t* block_counts, const uint32_t* n_dev, cudaStream_t st);
+int sf_launch_iota(uint32_t* out, uint32_t n, cudaStream_t st);      // out[i] = i
 int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wide, const uint32_t* ids,
                      const uint32_t* n_ids_dev, uint32_t capacity, void* rows, cudaStream_t st);
 size_t sf_slow_scratch_bytes(const sf_slow* s, uint32_t capacity);

@@ -217,6 +217,14 @@ int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, 
     return SF_OK;
 }
 
+namespace { __global__ void iota_kernel(uint32_t* out, uint32_t n) { uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; if (i < n) out[i] = i; } }
+int sf_launch_iota(uint32_t* out, uint32_t n, cudaStream_t st) {
+    if (n == 0) return SF_OK;
+    iota_kernel<<<(n + 255) / 256, 256, 0, st>>>(out, n);
+    SF_LAUNCH_CHECK("iota_kernel");
+    return SF_OK;
+}
+
 // wide rows of `capacity` flows at most (ids and count on the device) out of any planes
 int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wide, const uint32_t* ids,
                      const uint32_t* n_ids_dev, uint32_t capacity, void* rows, cudaStream_t st)
