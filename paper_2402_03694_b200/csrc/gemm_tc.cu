@@ -6,8 +6,10 @@
 // swizzled row per matrix row).  Warp roles:
 //   warp 0      TMA producer: loads the A and W slices of a ring of stages
 //   warp 1      allocates TMEM; one lane issues tcgen05.mma (4 per stage, K = 16 each)
-//   warps 2..5  epilogue: tcgen05.ld the fp32 accumulators (one TMEM lane quarter per
-//               warp), add bias, ReLU, round to bf16, 16-byte stores
+//   warps 2..9  epilogue: tcgen05.ld the fp32 accumulators (TMEM lane quarter = warp % 4,
+//               column half = (warp - 2) / 4), add bias, ReLU, round to bf16, transpose each
+//               32 x 32 block through shared memory so that global stores are whole 64-byte
+//               row segments (8 rows per instruction)
 // Two accumulator buffers in TMEM (2 x BN columns) let the MMAs of tile i+1 overlap
 // the epilogue of tile i.  The row count lives in device memory, so routing and the
 // slow model need no host round trip; tiles past the count are never scheduled and
@@ -49,7 +51,8 @@ using namespace sftc;
 
 constexpr uint32_t BM = 128;
 constexpr uint32_t BK = 64;
-constexpr uint32_t kGemmThreads = 192;
+constexpr uint32_t kEpiWarps = 8;
+constexpr uint32_t kGemmThreads = 64 + kEpiWarps * 32;
 
 template <uint32_t BN> struct GemmCfg {
     static constexpr uint32_t kStageBytesA = BM * BK * 2;
@@ -57,7 +60,8 @@ template <uint32_t BN> struct GemmCfg {
     static constexpr uint32_t kStageBytes = kStageBytesA + kStageBytesB;
     static constexpr uint32_t kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : (BN == 64 ? 8 : 10));
     static constexpr uint32_t kTmemCols = 2 * BN;             // a power of two >= 32
-    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                           kEpiWarps * 2048 /*epilogue staging*/;
 };
 
 struct GemmBars {
@@ -95,7 +99,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < Cfg::kStages; s++) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        for (uint32_t b = 0; b < 2; b++) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], 4); }
+        for (uint32_t b = 0; b < 2; b++) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], kEpiWarps); }
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -154,7 +158,10 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             }
         }
     } else {
-        const uint32_t quarter = warp & 3u;                        // TMEM lanes [32q, 32q+32)
+        // 8 epilogue warps: TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
+        const uint32_t quarter = warp & 3u;
+        const uint32_t half = (warp - 2u) >> 2;
+        uint8_t* stg = tiles + Cfg::kStages * Cfg::kStageBytes + 256 + (warp - 2u) * 2048u;   // 32 rows x 64 B, XOR-swizzled
         uint32_t buf = 0, bphase = 0;
         bool ok = true;
         for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -163,47 +170,63 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->tmem_full[buf], bphase, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t row = tm * BM + quarter * 32u + lane;
+            const uint32_t row0 = tm * BM + quarter * 32u;
             const uint32_t col0 = tn * BN;
             const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BN;
             if constexpr (HEAD) {
-                uint32_t v[16];
-                tmem_ld16(taddr, v);
-                tmem_ld_wait();
-                if (row < n_rows) {
-                    uint32_t a = 0; float mx = 0.0f;
+                if (half == 0) {
+                    const uint32_t row = row0 + lane;
+                    uint32_t v[16];
+                    tmem_ld16(taddr, v);
+                    tmem_ld_wait();
+                    if (row < n_rows) {
+                        uint32_t a = 0; float mx = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < 16; c++) {
-                        if ((uint32_t)c < C) {
-                            float x = __uint_as_float(v[c]) + __ldg(bias + c);
-                            logits[(size_t)row * C + c] = x;
-                            if (c == 0 || x > mx) { mx = x; a = c; }
+                        for (int c = 0; c < 16; c++) {
+                            if ((uint32_t)c < C) {
+                                float x = __uint_as_float(v[c]) + __ldg(bias + c);
+                                logits[(size_t)row * C + c] = x;
+                                if (c == 0 || x > mx) { mx = x; a = c; }
+                            }
                         }
+                        if (label) label[row] = (uint8_t)a;
                     }
-                    if (label) label[row] = (uint8_t)a;
                 }
             } else {
-            __nv_bfloat16* orow = out + (size_t)row * N + col0;
+                constexpr uint32_t kHalfCols = BN / 2;
+                const uint32_t sw = (lane >> 1) & 3u;                       // swizzle of this lane's staging row
 #pragma unroll 1
-            for (uint32_t c = 0; c < BN; c += 32) {
-                uint32_t v[32];
-                tmem_ld32(taddr + c, v);
-                tmem_ld_wait();
-                if (row < n_rows) {
-                    uint32_t packed[16];
+                for (uint32_t c = half * kHalfCols; c < (half + 1) * kHalfCols; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    const float4* b4 = reinterpret_cast<const float4*>(bias + col0 + c);
+                    // bias + ReLU + bf16, staged as this lane's 64-byte row (16-byte pieces XOR-swizzled by row)
 #pragma unroll
-                    for (int j = 0; j < 16; j++) {
-                        float x0 = __uint_as_float(v[2 * j]) + __ldg(bias + col0 + c + 2 * j);
-                        float x1 = __uint_as_float(v[2 * j + 1]) + __ldg(bias + col0 + c + 2 * j + 1);
-                        __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(x0, 0.0f), fmaxf(x1, 0.0f));
-                        packed[j] = *reinterpret_cast<uint32_t*>(&h);
+                    for (int pc = 0; pc < 4; pc++) {
+                        const float4 ba = __ldg(b4 + 2 * pc), bb = __ldg(b4 + 2 * pc + 1);
+                        const float bv[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; e++) {
+                            float x0 = fmaxf(__uint_as_float(v[pc * 8 + 2 * e]) + bv[2 * e], 0.0f);
+                            float x1 = fmaxf(__uint_as_float(v[pc * 8 + 2 * e + 1]) + bv[2 * e + 1], 0.0f);
+                            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                            pk[e] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(stg + lane * 64u + (((uint32_t)pc ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
-                    uint4* dst = reinterpret_cast<uint4*>(orow + c);
+                    __syncwarp();
+                    // read back 8 rows x 64 B per instruction and store full 64-byte row segments
 #pragma unroll
-                    for (int q = 0; q < 4; q++)
-                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    for (uint32_t it = 0; it < 4; it++) {
+                        const uint32_t rr = it * 8u + (lane >> 2), pp = lane & 3u;
+                        const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 64u + ((pp ^ ((rr >> 1) & 3u)) << 4));
+                        if (row0 + rr < n_rows)
+                            *reinterpret_cast<uint4*>(out + (size_t)(row0 + rr) * N + col0 + c + pp * 8u) = val;
+                    }
+                    __syncwarp();
                 }
-            }
             }
             tc_fence_before();
             __syncwarp();
