@@ -3,7 +3,8 @@
 // One thread per flow.  A thread streams its packets in chunks of 8 (16-byte
 // vector loads of the uint16 sizes and uint32 inter-arrival times when the row
 // pitch allows it), keeps one integer accumulator set per feature group in
-// registers, converts once at the end, and the block hands its [flows][F] tile to
+// registers (subset membership, counts, first and last come from bit masks of the
+// direction word), converts once at the end, and the block hands its [flows][F] tile to
 // global memory through shared memory so that the stores are fully coalesced.
 // All statistics come from exact integer sums (128-bit for the variance numerator
 // of inter-arrival times); each fp32 value is produced by exactly one rounding
@@ -14,31 +15,41 @@ namespace {
 
 constexpr int kFlowsPerBlock = 128;
 
+// Integer accumulators of one (quantity, subset) group.  Counts, first and last come from
+// the subset's bit mask (popcount / lowest / highest set bit), so the per-packet work is
+// two selects, a min, a max and the exact sums.
 struct Acc {
-    uint32_t cnt, mn, mx, first, last;
+    uint32_t mn, mx;
     uint64_t s1;        // sum
     uint64_t s2lo;      // sum of squares, low 64 bits
     uint32_t s2hi;      // high part (only inter-arrival times can carry into it)
 };
 
-__device__ __forceinline__ void acc_init(Acc& a) {
-    a.cnt = 0; a.mn = 0xFFFFFFFFu; a.mx = 0; a.first = 0; a.last = 0; a.s1 = 0; a.s2lo = 0; a.s2hi = 0;
-}
+__device__ __forceinline__ void acc_init(Acc& a) { a.mn = 0xFFFFFFFFu; a.mx = 0; a.s1 = 0; a.s2lo = 0; a.s2hi = 0; }
 
-template <bool WIDE>
-__device__ __forceinline__ void acc_add(Acc& a, uint32_t x, bool take) {
-    if (take) {
-        if (a.cnt == 0) a.first = x;
-        a.mn = min(a.mn, x);
-        a.mx = max(a.mx, x);
-        a.last = x;
-        a.s1 += x;
-        uint64_t sq = (uint64_t)x * (uint64_t)x;
-        uint64_t lo = a.s2lo + sq;
-        if (WIDE) a.s2hi += (lo < sq) ? 1u : 0u;
-        a.s2lo = lo;
-        a.cnt += 1;
-    }
+// sizes (16 bit): the square fits 32 bits and the sums never carry out of 64 bits
+__device__ __forceinline__ void add_size(Acc& a, uint32_t x, bool take) {
+    const uint32_t x0 = take ? x : 0u, xm = take ? x : 0xFFFFFFFFu;
+    a.mn = min(a.mn, xm);
+    a.mx = max(a.mx, x0);
+    a.s1 += x0;
+    a.s2lo += (uint64_t)(x0 * x0);
+}
+// inter-arrival times (32 bit): 64-bit squares, 128-bit sum of squares
+__device__ __forceinline__ void add_iat(Acc& a, uint32_t x, bool take) {
+    const uint32_t x0 = take ? x : 0u, xm = take ? x : 0xFFFFFFFFu;
+    a.mn = min(a.mn, xm);
+    a.mx = max(a.mx, x0);
+    a.s1 += x0;
+    const uint64_t sq = (uint64_t)x0 * (uint64_t)x0;
+    const uint64_t lo = a.s2lo + sq;
+    a.s2hi += (lo < sq) ? 1u : 0u;
+    a.s2lo = lo;
+}
+// min / max only (the sums of the complementary subset come from a subtraction)
+__device__ __forceinline__ void add_minmax(Acc& a, uint32_t x, bool take) {
+    a.mn = min(a.mn, take ? x : 0xFFFFFFFFu);
+    a.mx = max(a.mx, take ? x : 0u);
 }
 
 // exact unsigned 128-bit value (hi:lo) -> fp32, round to nearest even.
@@ -55,44 +66,48 @@ __device__ __forceinline__ float u128_to_f32(uint64_t hi, uint64_t lo) {
     return __fmul_rn(f, __uint_as_float((uint32_t)(127 + s) << 23));   // * 2^s, exact
 }
 
-__device__ __forceinline__ void acc_finish(const Acc& a, float* o) {
-    if (a.cnt == 0) {
+// eight slots of one group: cnt, sum, min, max, mean, var, first, last
+__device__ __forceinline__ void finish(uint32_t cnt, uint32_t mn, uint32_t mx, uint64_t s1, uint64_t s2lo, uint64_t s2hi,
+                                       uint32_t first, uint32_t last, float* o) {
+    if (cnt == 0) {
 #pragma unroll
         for (int k = 0; k < 8; k++) o[k] = 0.0f;
         return;
     }
-    float fc = __uint2float_rn(a.cnt);
-    float fs = __ull2float_rn(a.s1);
+    const float fc = __uint2float_rn(cnt);
+    const float fs = __ull2float_rn(s1);
     // V = cnt * S2 - S1^2 as an exact 128-bit integer
-    uint64_t c = a.cnt;
-    uint64_t p_lo = c * a.s2lo;
-    uint64_t p_hi = __umul64hi(c, a.s2lo) + c * (uint64_t)a.s2hi;
-    uint64_t q_lo = a.s1 * a.s1;
-    uint64_t q_hi = __umul64hi(a.s1, a.s1);
-    uint64_t v_lo = p_lo - q_lo;
-    uint64_t v_hi = p_hi - q_hi - ((p_lo < q_lo) ? 1ull : 0ull);
+    const uint64_t c = cnt;
+    const uint64_t p_lo = c * s2lo;
+    const uint64_t p_hi = __umul64hi(c, s2lo) + c * s2hi;
+    const uint64_t q_lo = s1 * s1;
+    const uint64_t q_hi = __umul64hi(s1, s1);
+    const uint64_t v_lo = p_lo - q_lo;
+    const uint64_t v_hi = p_hi - q_hi - ((p_lo < q_lo) ? 1ull : 0ull);
     o[0] = fc;
     o[1] = fs;
-    o[2] = __uint2float_rn(a.mn);
-    o[3] = __uint2float_rn(a.mx);
+    o[2] = __uint2float_rn(mn);
+    o[3] = __uint2float_rn(mx);
     o[4] = __fdiv_rn(fs, fc);
-    o[5] = __fdiv_rn(u128_to_f32(v_hi, v_lo), __uint2float_rn(a.cnt * a.cnt));
-    o[6] = __uint2float_rn(a.first);
-    o[7] = __uint2float_rn(a.last);
+    o[5] = __fdiv_rn(u128_to_f32(v_hi, v_lo), __uint2float_rn(cnt * cnt));
+    o[6] = __uint2float_rn(first);
+    o[7] = __uint2float_rn(last);
 }
 
+// Groups: g0 size/all, g1 iat/all, g2 size/fwd, g3 size/bwd, g4 iat/fwd, g5 iat/bwd, g6 size/turn, g7 iat/turn.
+// Sums of the backward subsets are (all - forward): exact, because everything is an integer.
 template <int G>
-__device__ __forceinline__ void packet(Acc (&A)[G], uint32_t sz, uint32_t ia, uint32_t i, uint32_t dirw) {
-    bool d = (dirw >> i) & 1u;
-    bool turn = (i >= 1) && (((dirw >> (i - 1)) & 1u) != (uint32_t)d);
-    acc_add<false>(A[0], sz, true);
-    if (G > 1) acc_add<true>(A[1], ia, true);
-    if (G > 2) acc_add<false>(A[2], sz, !d);
-    if (G > 3) acc_add<false>(A[3], sz, d);
-    if (G > 4) acc_add<true>(A[4], ia, !d);
-    if (G > 5) acc_add<true>(A[5], ia, d);
-    if (G > 6) acc_add<false>(A[6], sz, turn);
-    if (G > 7) acc_add<true>(A[7], ia, turn);
+__device__ __forceinline__ void packet(Acc (&A)[8], uint32_t sz, uint32_t ia, uint32_t i, uint32_t fwd_mask, uint32_t turn_mask) {
+    const bool f = (fwd_mask >> i) & 1u;
+    const bool tn = (turn_mask >> i) & 1u;
+    add_size(A[0], sz, true);
+    if (G > 1) add_iat(A[1], ia, true);
+    if (G > 2) add_size(A[2], sz, f);
+    if (G > 3) add_minmax(A[3], sz, !f);
+    if (G > 4) add_iat(A[4], ia, f);
+    if (G > 5) add_minmax(A[5], ia, !f);
+    if (G > 6) add_size(A[6], sz, tn);
+    if (G > 7) add_iat(A[7], ia, tn);
 }
 
 // VEC: row pitch is a multiple of 8 packets, so size rows are 16-byte aligned
@@ -112,13 +127,17 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
     const uint32_t f = f0 + threadIdx.x;
 
     if (f < n) {
-        Acc A[G];
+        Acc A[8];
 #pragma unroll
-        for (int g = 0; g < G; g++) acc_init(A[g]);
+        for (int g = 0; g < 8; g++) acc_init(A[g]);
         uint32_t m = N;
         if (n_valid) m = min(m, (uint32_t)n_valid[f]);
         // N <= 32: all direction bits of the window are in the row's first word
         const uint32_t dirw = dir_bits[(size_t)f * ((pitch + 31) >> 5)];
+        const uint32_t all_mask = (m >= 32) ? 0xFFFFFFFFu : ((1u << m) - 1u);
+        const uint32_t fwd_mask = ~dirw & all_mask;
+        const uint32_t bwd_mask = dirw & all_mask;
+        const uint32_t turn_mask = (dirw ^ (dirw << 1)) & ~1u & all_mask;        // packet i >= 1 whose direction differs from i-1
         const uint16_t* srow = size + (size_t)f * pitch;
         const uint32_t* irow = iat + (size_t)f * pitch;
         if (VEC) {
@@ -131,14 +150,33 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
                 uint32_t ia[8] = {a4.x, a4.y, a4.z, a4.w, b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
                 for (int j = 0; j < 8; j++)
-                    if (base + j < m) packet<G>(A, sz[j], ia[j], base + j, dirw);
+                    if (base + j < m) packet<G>(A, sz[j], ia[j], base + j, fwd_mask, turn_mask);
             }
         } else {
-            for (uint32_t i = 0; i < m; i++) packet<G>(A, srow[i], irow[i], i, dirw);
+            for (uint32_t i = 0; i < m; i++) packet<G>(A, srow[i], irow[i], i, fwd_mask, turn_mask);
         }
         float* o = tile + threadIdx.x * STRIDE;
 #pragma unroll
-        for (int g = 0; g < G; g++) acc_finish(A[g], o + 8 * g);
+        for (int g = 0; g < G; g++) {
+            const uint32_t mask = (g < 2) ? all_mask : (g == 2 || g == 4) ? fwd_mask : (g == 3 || g == 5) ? bwd_mask : turn_mask;
+            const bool is_size = (g == 0 || g == 2 || g == 3 || g == 6);
+            const uint32_t cnt = __popc(mask);
+            uint32_t first = 0, last = 0;
+            if (cnt) {                               // the row was just read: these hit in L1
+                const uint32_t i0 = __ffs(mask) - 1, i1 = 31 - __clz(mask);
+                first = is_size ? (uint32_t)srow[i0] : irow[i0];
+                last = is_size ? (uint32_t)srow[i1] : irow[i1];
+            }
+            uint64_t s1 = A[g].s1, s2lo = A[g].s2lo, s2hi = A[g].s2hi;
+            if (g == 3 || g == 5) {                  // backward = all - forward
+                const Acc& all = A[g == 3 ? 0 : 1];
+                const Acc& fw = A[g == 3 ? 2 : 4];
+                s1 = all.s1 - fw.s1;
+                s2lo = all.s2lo - fw.s2lo;
+                s2hi = (uint64_t)all.s2hi - fw.s2hi - ((all.s2lo < fw.s2lo) ? 1u : 0u);
+            }
+            finish(cnt, A[g].mn, A[g].mx, s1, s2lo, s2hi, first, last, o + 8 * g);
+        }
     }
     __syncthreads();
     const uint32_t rows = min((uint32_t)kFlowsPerBlock, n - f0);
