@@ -69,9 +69,10 @@ __device__ __forceinline__ float u128_to_f32(uint64_t hi, uint64_t lo) {
 // eight slots of one group: cnt, sum, min, max, mean, var, first, last
 __device__ __forceinline__ void finish(uint32_t cnt, uint32_t mn, uint32_t mx, uint64_t s1, uint64_t s2lo, uint64_t s2hi,
                                        uint32_t first, uint32_t last, float* o) {
+    float4* o4 = reinterpret_cast<float4*>(o);       // 16-byte stores: conflict-free across a quarter warp
     if (cnt == 0) {
-#pragma unroll
-        for (int k = 0; k < 8; k++) o[k] = 0.0f;
+        o4[0] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        o4[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         return;
     }
     const float fc = __uint2float_rn(cnt);
@@ -84,14 +85,9 @@ __device__ __forceinline__ void finish(uint32_t cnt, uint32_t mn, uint32_t mx, u
     const uint64_t q_hi = __umul64hi(s1, s1);
     const uint64_t v_lo = p_lo - q_lo;
     const uint64_t v_hi = p_hi - q_hi - ((p_lo < q_lo) ? 1ull : 0ull);
-    o[0] = fc;
-    o[1] = fs;
-    o[2] = __uint2float_rn(mn);
-    o[3] = __uint2float_rn(mx);
-    o[4] = __fdiv_rn(fs, fc);
-    o[5] = __fdiv_rn(u128_to_f32(v_hi, v_lo), __uint2float_rn(cnt * cnt));
-    o[6] = __uint2float_rn(first);
-    o[7] = __uint2float_rn(last);
+    o4[0] = make_float4(fc, fs, __uint2float_rn(mn), __uint2float_rn(mx));
+    o4[1] = make_float4(__fdiv_rn(fs, fc), __fdiv_rn(u128_to_f32(v_hi, v_lo), __uint2float_rn(cnt * cnt)),
+                        __uint2float_rn(first), __uint2float_rn(last));
 }
 
 // Groups: g0 size/all, g1 iat/all, g2 size/fwd, g3 size/bwd, g4 iat/fwd, g5 iat/bwd, g6 size/turn, g7 iat/turn.
@@ -119,8 +115,8 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
                uint32_t n, uint32_t pitch, uint32_t N, float* __restrict__ feat, const uint32_t* __restrict__ n_dev)
 {
     constexpr int F = 8 * G;
-    constexpr int STRIDE = F + 1;                  // odd stride: conflict-free row writes
-    extern __shared__ float tile[];                // [kFlowsPerBlock][STRIDE]
+    constexpr int STRIDE = F + 4;                  // 16-byte aligned rows; 8 lanes x 16 B land in distinct bank groups
+    extern __shared__ __align__(16) float tile[];                // [kFlowsPerBlock][STRIDE]
     if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
     const uint32_t f0 = blockIdx.x * kFlowsPerBlock;
     if (f0 >= n) return;
@@ -141,16 +137,26 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
         const uint16_t* srow = size + (size_t)f * pitch;
         const uint32_t* irow = iat + (size_t)f * pitch;
         if (VEC) {
-            for (uint32_t base = 0; base < m; base += 8) {
-                uint4 s4 = __ldg(reinterpret_cast<const uint4*>(srow + base));
-                uint4 a4 = __ldg(reinterpret_cast<const uint4*>(irow + base));
-                uint4 b4 = __ldg(reinterpret_cast<const uint4*>(irow + base + 4));
-                uint32_t sz[8] = {s4.x & 0xFFFFu, s4.x >> 16, s4.y & 0xFFFFu, s4.y >> 16,
-                                  s4.z & 0xFFFFu, s4.z >> 16, s4.w & 0xFFFFu, s4.w >> 16};
-                uint32_t ia[8] = {a4.x, a4.y, a4.z, a4.w, b4.x, b4.y, b4.z, b4.w};
+            // issue every load of the window first (N <= 32: at most four chunks of eight packets), then reduce
+            uint4 s4[4], a4[4], b4[4];
 #pragma unroll
-                for (int j = 0; j < 8; j++)
-                    if (base + j < m) packet<G>(A, sz[j], ia[j], base + j, fwd_mask, turn_mask);
+            for (int ch = 0; ch < 4; ch++) {
+                if ((uint32_t)ch * 8 < m) {
+                    s4[ch] = __ldg(reinterpret_cast<const uint4*>(srow + ch * 8));
+                    a4[ch] = __ldg(reinterpret_cast<const uint4*>(irow + ch * 8));
+                    b4[ch] = __ldg(reinterpret_cast<const uint4*>(irow + ch * 8 + 4));
+                }
+            }
+#pragma unroll
+            for (int ch = 0; ch < 4; ch++) {
+                if ((uint32_t)ch * 8 < m) {
+                    const uint32_t sz[8] = {s4[ch].x & 0xFFFFu, s4[ch].x >> 16, s4[ch].y & 0xFFFFu, s4[ch].y >> 16,
+                                            s4[ch].z & 0xFFFFu, s4[ch].z >> 16, s4[ch].w & 0xFFFFu, s4[ch].w >> 16};
+                    const uint32_t ia[8] = {a4[ch].x, a4[ch].y, a4[ch].z, a4[ch].w, b4[ch].x, b4[ch].y, b4[ch].z, b4[ch].w};
+#pragma unroll
+                    for (int j = 0; j < 8; j++)
+                        if ((uint32_t)(ch * 8 + j) < m) packet<G>(A, sz[j], ia[j], ch * 8 + j, fwd_mask, turn_mask);
+                }
             }
         } else {
             for (uint32_t i = 0; i < m; i++) packet<G>(A, srow[i], irow[i], i, fwd_mask, turn_mask);
@@ -180,11 +186,11 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
     }
     __syncthreads();
     const uint32_t rows = min((uint32_t)kFlowsPerBlock, n - f0);
-    const uint32_t total = rows * F;
-    float* dst = feat + (size_t)f0 * F;
-    for (uint32_t e = threadIdx.x; e < total; e += kFlowsPerBlock) {
-        uint32_t r = e / F, c = e - r * F;
-        dst[e] = tile[r * STRIDE + c];
+    const uint32_t total4 = rows * (F / 4);
+    float4* dst = reinterpret_cast<float4*>(feat + (size_t)f0 * F);
+    for (uint32_t e = threadIdx.x; e < total4; e += kFlowsPerBlock) {
+        const uint32_t r = e / (F / 4), c = e - r * (F / 4);
+        dst[e] = *reinterpret_cast<const float4*>(tile + r * STRIDE + 4 * c);
     }
 }
 
@@ -192,7 +198,7 @@ template <int G>
 int launch_g(const sf_packets* pk, uint32_t N, float* feat, cudaStream_t st, const uint32_t* n_dev) {
     const uint32_t n = pk->n_flows;
     const bool vec = (pk->pitch_pkts % 8 == 0) && (((uintptr_t)pk->size & 15) == 0) && (((uintptr_t)pk->iat_us & 15) == 0);
-    const size_t smem = (size_t)kFlowsPerBlock * (8 * G + 1) * sizeof(float);
+    const size_t smem = (size_t)kFlowsPerBlock * (8 * G + 4) * sizeof(float);
     const uint32_t grid = (n + kFlowsPerBlock - 1) / kFlowsPerBlock;
     if (vec)
         extract_kernel<G, true><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev);
