@@ -111,7 +111,7 @@ def build_gpu_workload(cfg, n, rank, sf, hz, ctx, torch):
     method's arithmetic (feature sample for the split thresholds, validation scores
     for Algorithm 1)."""
     t0 = time.time()
-    wide = flowgen.gen_packets(cfg.seed_data + 7919 * rank, n, cfg.P, cfg.H)
+    wide = flowgen.gen_packets(rank_data_seed(cfg, rank), n, cfg.P, cfg.H)
     fast = flowgen.fast_view(wide, cfg.N)
     t_gen = time.time() - t0
     fast_d = hz.upload_packets(fast, with_hdr=False)
@@ -145,6 +145,25 @@ def build_gpu_workload(cfg, n, rank, sf, hz, ctx, torch):
     del feat
     return {"wide": wide, "fast": fast, "wide_d": wide_d, "fast_d": fast_d, "forest": forest, "slow": slow,
             "tau": tau, "forest_np": forest_np, "slow_np": slow_np, "t_gen": t_gen}
+
+
+def rank_data_seed(cfg, rank):
+    """Every rank serves its own batch: flows are independent units, so ranks share nothing but the models."""
+    return cfg.seed_data + 7919 * rank
+
+
+def max_over_ranks(ms_local, dist, device):
+    """The job's time is the slowest rank's (the only collective of the multi-GPU run)."""
+    if dist is None:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([float(ms_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_flows_per_s(world, flows_per_rank, steps, ms_total):
+    return world * flows_per_rank * steps / (ms_total * 1e-3)
 
 
 def hidden_flops_per_row(cfg):
@@ -360,11 +379,7 @@ def main():
     if dist is not None:
         dist.barrier()
     clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, torch.device("cuda", local))
     counters = sf.sf_ctx_poll(ctx, reset=True)
     k_esc = int(n_esc.cpu().numpy()[0])
     # per-kernel-class times of the timed steps (the ring keeps the last 64)
@@ -372,7 +387,7 @@ def main():
     sf.sf_ctx_set_timing(ctx, False)
     avg = {k: float(np.mean([r[k] for r in recs])) for k in recs[0]}
     ms_step = ms_total / args.steps
-    value = world * n * args.steps / (ms_total * 1e-3)
+    value = whole_job_flows_per_s(world, n, args.steps, ms_total)
 
     if rank != 0:
         if dist is not None:
