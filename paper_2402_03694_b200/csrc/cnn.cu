@@ -1,28 +1,31 @@
 // S4 (1-D CNN slow model), one fused kernel per batch of assigned flows:
 //   conv1 (k=5, 8 -> 64) + ReLU -> conv2 (k=5, 64 -> 128) + ReLU -> mean over the 128
 //   positions -> linear 128 -> n_cls -> argmax.
-// Both convolutions run on the tcgen05 tensor cores as implicit GEMMs with one flow's
-// 128 positions as the M = 128 rows of a tile; nothing but the 2 KB input row and the
-// logits ever touches global memory.
+// All three contractions run on the tcgen05 tensor cores with one flow's 128 positions as
+// the M = 128 rows of a tile; nothing but the 2 KB input row and the logits touches HBM.
 //
-// How the shifted ("same" padded) operands are expressed without im2col.  Activations
-// are kept in shared memory in the un-swizzled core-matrix layout: for every group of
-// 8 channels a column of 16-byte rows, one row per position, with two zero rows above
-// and below.  In that layout a matrix descriptor's start address may be moved by whole
-// rows, so tap t of a convolution is the same buffer started t rows further down; the
-// zero rows supply the padding.  For conv1 (8 input channels = one 16-byte row per
-// position) consecutive taps are consecutive rows, so a K = 16 step (two taps) uses a
-// K-direction stride of 16 bytes: the im2col matrix is never materialised.
+// Shifted ("same" padded) operands without im2col.  Activations are kept in shared memory
+// in the un-swizzled core-matrix layout: for every group of 8 channels a column of 16-byte
+// rows, one row per position, with zero rows above and below.  In that layout a matrix
+// descriptor's start address may be moved by whole rows, so tap t of a convolution is the
+// same buffer started t rows further down; the zero rows supply the padding.  For conv1
+// (8 input channels = one 16-byte row per position) consecutive taps are consecutive rows,
+// so a K = 16 step (two taps) uses a K-direction stride of 16 bytes.
 //
-// Persistent CTAs, one per SM, loop over flows.  Warp 0 streams input rows with bulk
-// copies into a ring; warp 1 issues the MMAs (3 for conv1, 20 for conv2 per flow) in the
-// order conv1(i+1), conv2(i) so that the first epilogue of the next flow overlaps the
-// second convolution of this one; warps 2..17 are the epilogues (lane quarter = warp % 4, four column groups each): E1 turns the conv1
-// accumulators (TMEM) into bf16 activations in shared memory (conv2's A operand), E2
-// applies bias + ReLU + bf16 rounding to the conv2 accumulators, reduces over positions
-// with a fixed shuffle tree (deterministic), and evaluates the linear head.
-// Accumulators, activations and input rows are all double (or more) buffered.
-// Every wait is bounded; on a timeout the block records SF_ERR_DEVICE_TIMEOUT and leaves.
+// Pooling and the linear head are one more MMA: mean_p(h2[p][:]) . W3^T = sum_p (h2[p][:] .
+// (W3/128)^T), i.e. a [128 positions] x [16 classes] product over the 128 channels followed
+// by a sum over positions (TMEM lanes), which a shuffle tree and four partial sums finish in a
+// fixed order (deterministic).
+//
+// Persistent CTAs, one per SM, loop over flows.  Warp roles:
+//   warp 0        streams input rows with bulk copies into a ring
+//   warp 1        issues the MMAs in the order conv1(i+1), conv2(i), head(i-1)
+//   warps 2..5    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's A operand (shared memory)
+//   warps 6..21   E2: conv2 accumulators -> bias + ReLU -> bf16 -> the head's A operand
+//   warps 22..25  E3: head accumulators -> sum over positions -> + bias -> logits, argmax
+// Every accumulator and activation buffer is double buffered, so the three epilogues and the
+// tensor pipe overlap.  Every wait is bounded; on a timeout the block records
+// SF_ERR_DEVICE_TIMEOUT and leaves.
 #include "tc_common.cuh"
 #include <stdlib.h>
 #include <string.h>
@@ -31,38 +34,45 @@ namespace {
 using namespace sftc;
 
 constexpr uint32_t L = 128, CIN = 8, C1 = 64, C2 = 128, KW = 5, NCLS_MAX = 16;
-constexpr uint32_t kEpiWarps = 16;                          // 4 TMEM lane quarters x 4 column groups
-constexpr uint32_t kEpiThreads = kEpiWarps * 32;
-constexpr uint32_t kThreads = 64 + kEpiThreads;
+constexpr uint32_t kE1Warps = 4, kE2Warps = 16, kE3Warps = 4;
+constexpr uint32_t kE1First = 2, kE2First = kE1First + kE1Warps, kE3First = kE2First + kE2Warps;
+constexpr uint32_t kThreads = (kE3First + kE3Warps) * 32;       // 832
 constexpr uint32_t XS = 4;                                  // input-row ring depth
 constexpr uint32_t X_STAGE = (2 + L + 3) * 16;              // 2 zero rows, 128 rows, 3 zero rows (tap 5 is a zero tap)
 constexpr uint32_t H1_COL = (2 + L + 2) * 16;               // one 8-channel column of conv1's output: 2112 bytes
 constexpr uint32_t H1_BYTES = (C1 / 8) * H1_COL;            // 16,896
+constexpr uint32_t H2_COL = L * 16;                         // one 8-channel column of conv2's output: 2048 bytes
+constexpr uint32_t H2_BYTES = (C2 / 8) * H2_COL;            // 32,768
 // weight blob (device and shared memory share this layout)
 constexpr uint32_t W2_OFF = 0;                              // [5 taps][8 k-chunks][128 n][8] bf16
 constexpr uint32_t W2_BYTES = KW * (C1 / 8) * C2 * 16;      // 81,920
 constexpr uint32_t W1_OFF = W2_OFF + W2_BYTES;              // [6 taps][64 n][8] bf16 (tap 5 = 0)
 constexpr uint32_t W1_BYTES = 6 * C1 * 16;                  // 6,144
-constexpr uint32_t W3_OFF = W1_OFF + W1_BYTES;              // fp32 [16][128]
-constexpr uint32_t W3_BYTES = NCLS_MAX * C2 * 4;            // 8,192
+constexpr uint32_t W3_OFF = W1_OFF + W1_BYTES;              // [16 k-chunks][16 classes][8] bf16, scaled by 1/128
+constexpr uint32_t W3_BYTES = (C2 / 8) * NCLS_MAX * 16;     // 4,096
 constexpr uint32_t B1_OFF = W3_OFF + W3_BYTES;              // fp32 [64]
 constexpr uint32_t B2_OFF = B1_OFF + C1 * 4;                // fp32 [128]
 constexpr uint32_t B3_OFF = B2_OFF + C2 * 4;                // fp32 [16]
-constexpr uint32_t BLOB_BYTES = B3_OFF + NCLS_MAX * 4;      // 97,088
+constexpr uint32_t BLOB_BYTES = B3_OFF + NCLS_MAX * 4;
 // shared memory map
 constexpr uint32_t SM_BLOB = 0;
 constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // 2 buffers
-constexpr uint32_t SM_X = SM_H1 + 2 * H1_BYTES;             // XS stages
-constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // fp32 [4 warps][128] column partial sums
-constexpr uint32_t SM_LOGIT = SM_PART + 4 * C2 * 4;         // fp32 [16]
-constexpr uint32_t SM_BARS = SM_LOGIT + 64;
+constexpr uint32_t SM_H2 = SM_H1 + 2 * H1_BYTES;            // 2 buffers
+constexpr uint32_t SM_X = SM_H2 + 2 * H2_BYTES;             // XS stages
+constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // fp32 [4 warps][16] partial logits
+constexpr uint32_t SM_BARS = SM_PART + 4 * NCLS_MAX * 4;
 constexpr uint32_t SM_TOTAL = SM_BARS + 256;
-static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_X % 16 == 0 && SM_BARS % 8 == 0, "alignment");
+static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_H2 % 16 == 0 && SM_X % 16 == 0 && SM_BARS % 8 == 0, "alignment");
+static_assert(SM_TOTAL <= 232448, "shared memory");
+// TMEM columns: conv1 accumulators [2][64], conv2 [2][128], head [2][16]
+constexpr uint32_t TM_D1 = 0, TM_D2 = 128, TM_D4 = 384;
 
 struct Bars {
     uint64_t w_full;
     uint64_t x_full[XS], x_empty[XS];
-    uint64_t d1_full[2], d1_empty[2], h1_full[2], h1_empty[2], d2_full[2], d2_empty[2];
+    uint64_t d1_full[2], d1_empty[2], h1_full[2], h1_empty[2];
+    uint64_t d2_full[2], d2_empty[2], h2_full[2], h2_empty[2];
+    uint64_t d4_full[2], d4_empty[2];
     uint32_t tmem_base, abort_flag;
 };
 static_assert(sizeof(Bars) <= 256, "barrier block");
@@ -71,11 +81,13 @@ __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t count) 
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-// sum over the 32 lanes of each of 32 per-lane values; lane l ends up with column l's total.
-// The order of additions is a fixed tree, so the result is reproducible run to run.
-__device__ __forceinline__ float transpose_reduce32(float (&v)[32], uint32_t lane) {
+// sum over the 32 lanes of each of 16 per-lane values; lanes l and l+16 end up with column (l & 15)'s
+// total.  The order of additions is a fixed tree, so the result is reproducible run to run.
+__device__ __forceinline__ float transpose_reduce16(float (&v)[16], uint32_t lane) {
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
+    for (int j = 0; j < 16; j++) v[j] += __shfl_xor_sync(0xFFFFFFFFu, v[j], 16);
+#pragma unroll
+    for (int off = 8; off >= 1; off >>= 1) {
         const bool up = (lane & off) != 0;
 #pragma unroll
         for (int j = 0; j < off; j++) {
@@ -85,6 +97,11 @@ __device__ __forceinline__ float transpose_reduce32(float (&v)[32], uint32_t lan
         }
     }
     return v[0];
+}
+
+__device__ __forceinline__ uint32_t pack_relu_bf16(uint32_t a, uint32_t b, float ba, float bb) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(__uint_as_float(a) + ba, 0.0f), fmaxf(__uint_as_float(b) + bb, 0.0f));
+    return *reinterpret_cast<uint32_t*>(&h);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -102,15 +119,17 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     const uint32_t n_mine = (n_rows > blockIdx.x) ? (n_rows - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
     // zero everything that acts as padding (and the rest of the activation buffers)
-    for (uint32_t i = threadIdx.x; i < (2 * H1_BYTES + XS * X_STAGE) / 16; i += kThreads)
+    for (uint32_t i = threadIdx.x; i < (2 * H1_BYTES + 2 * H2_BYTES + XS * X_STAGE) / 16; i += kThreads)
         reinterpret_cast<uint4*>(smem + SM_H1)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
         mbar_init(&bars->w_full, 1);
         for (uint32_t s = 0; s < XS; s++) { mbar_init(&bars->x_full[s], 1); mbar_init(&bars->x_empty[s], 1); }
         for (uint32_t b = 0; b < 2; b++) {
-            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kEpiWarps);
-            mbar_init(&bars->h1_full[b], kEpiWarps); mbar_init(&bars->h1_empty[b], 1);
-            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], kEpiWarps);
+            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kE1Warps);
+            mbar_init(&bars->h1_full[b], kE1Warps); mbar_init(&bars->h1_empty[b], 1);
+            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], kE2Warps);
+            mbar_init(&bars->h2_full[b], kE2Warps); mbar_init(&bars->h2_empty[b], 1);
+            mbar_init(&bars->d4_full[b], 1); mbar_init(&bars->d4_empty[b], kE3Warps);
         }
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -121,6 +140,8 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
+    const uint32_t q = warp & 3u;                    // TMEM lane quarter an epilogue warp may read
+    const uint32_t p = q * 32u + lane;               // position handled by an epilogue thread
 
     if (warp == 0) {
         if (lane == 0 && n_mine > 0) {
@@ -138,6 +159,7 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
         if (lane == 0 && n_mine > 0) {
             constexpr uint32_t idesc1 = make_idesc_bf16(128, C1);
             constexpr uint32_t idesc2 = make_idesc_bf16(128, C2);
+            constexpr uint32_t idesc4 = make_idesc_bf16(128, NCLS_MAX);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
             auto conv1 = [&](uint32_t i) -> bool {
                 const uint32_t s = i % XS, xph = (i / XS) & 1u, b = i & 1u, ph = (i >> 1) & 1u;
@@ -149,7 +171,7 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 for (uint32_t k = 0; k < 3; k++) {           // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
                     const uint64_t ad = make_smem_desc(xa + k * 32u, 16, 128, 0);
                     const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W1_OFF + k * 2u * (C1 * 16u), C1 * 16u, 128, 0);
-                    umma_bf16(tmem_base + b * C1, ad, bd, idesc1, k != 0 ? 1u : 0u);
+                    umma_bf16(tmem_base + TM_D1 + b * C1, ad, bd, idesc1, k != 0 ? 1u : 0u);
                 }
                 umma_commit(&bars->x_empty[s]);
                 umma_commit(&bars->d1_full[b]);
@@ -168,54 +190,61 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                         const uint64_t ad = make_smem_desc(ha + (2u * k) * H1_COL + t * 16u, H1_COL, 128, 0);
                         const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W2_OFF + t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u),
                                                            C2 * 16u, 128, 0);
-                        umma_bf16(tmem_base + 128u + b * C2, ad, bd, idesc2, (t | k) != 0 ? 1u : 0u);
+                        umma_bf16(tmem_base + TM_D2 + b * C2, ad, bd, idesc2, (t | k) != 0 ? 1u : 0u);
                     }
                 }
                 umma_commit(&bars->h1_empty[b]);
                 umma_commit(&bars->d2_full[b]);
                 return true;
             };
+            auto head = [&](uint32_t i) -> bool {
+                const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
+                if (!mbar_wait(&bars->h2_full[b], ph, abort_flag)) return false;
+                if (!mbar_wait(&bars->d4_empty[b], ph ^ 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t ha = sbase + SM_H2 + b * H2_BYTES;
+#pragma unroll
+                for (uint32_t k = 0; k < C2 / 16; k++) {
+                    const uint64_t ad = make_smem_desc(ha + (2u * k) * H2_COL, H2_COL, 128, 0);
+                    const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W3_OFF + (2u * k) * (NCLS_MAX * 16u), NCLS_MAX * 16u, 128, 0);
+                    umma_bf16(tmem_base + TM_D4 + b * NCLS_MAX, ad, bd, idesc4, k != 0 ? 1u : 0u);
+                }
+                umma_commit(&bars->h2_empty[b]);
+                umma_commit(&bars->d4_full[b]);
+                return true;
+            };
             if (ok) ok = conv1(0);
             for (uint32_t i = 0; i < n_mine && ok; i++) {
                 if (i + 1 < n_mine) ok = conv1(i + 1);
                 if (ok) ok = conv2(i);
+                if (ok && i >= 1) ok = head(i - 1);
             }
+            if (ok) ok = head(n_mine - 1);
         }
-    } else if (n_mine > 0) {
-        const uint32_t q = warp & 3u;                    // TMEM lane quarter of this warp
-        const uint32_t p = q * 32u + lane;               // position handled by this thread
-        const uint32_t g = (warp - 2u) >> 2;             // column group handled by this warp (0..3)
-        const uint32_t et = (warp - 2u) * 32u + lane;    // 0..511 among the epilogue threads
+    } else if (n_mine > 0 && warp < kE2First) {
+        // ---- E1: conv1 accumulators -> conv2's A operand -------------------------------
         const float* b1 = reinterpret_cast<const float*>(smem + SM_BLOB + B1_OFF);
-        const float* b2 = reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF);
-        const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
-        const float* w3 = reinterpret_cast<const float*>(smem + SM_BLOB + W3_OFF);
-        float* part = reinterpret_cast<float*>(smem + SM_PART);
-        float* slog = reinterpret_cast<float*>(smem + SM_LOGIT);
         bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
-
-        auto E1 = [&](uint32_t i) -> bool {
+        for (uint32_t i = 0; i < n_mine && ok; i++) {
             const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
             bool w = mbar_wait(&bars->d1_full[b], ph, abort_flag) && mbar_wait(&bars->h1_empty[b], ph ^ 1u, abort_flag);
-            if (!__all_sync(0xFFFFFFFFu, w)) return false;
+            ok = __all_sync(0xFFFFFFFFu, w);
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t c0 = g * 16u;                 // this warp's 16 of the 64 conv1 channels
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + b * C1 + c0;
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D1 + b * C1;
             uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (p + 2u) * 16u;
-            {
-                uint32_t v[16];
-                tmem_ld16(taddr, v);
+#pragma unroll
+            for (uint32_t c0 = 0; c0 < C1; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(taddr + c0, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 2; j++) {            // 2 columns of 8 channels
+                for (int j = 0; j < 4; j++) {            // 4 columns of 8 channels
                     uint32_t pk[4];
 #pragma unroll
                     for (int e = 0; e < 4; e++) {
                         const int c = j * 8 + e * 2;
-                        float x0 = fmaxf(__uint_as_float(v[c]) + b1[c0 + c], 0.0f);
-                        float x1 = fmaxf(__uint_as_float(v[c + 1]) + b1[c0 + c + 1], 0.0f);
-                        __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
-                        pk[e] = *reinterpret_cast<uint32_t*>(&h);
+                        pk[e] = pack_relu_bf16(v[c], v[c + 1], b1[c0 + c], b1[c0 + c + 1]);
                     }
                     *reinterpret_cast<uint4*>(hrow + ((c0 >> 3) + j) * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
@@ -224,58 +253,79 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             tc_fence_before();
             __syncwarp();
             if (lane == 0) { mbar_arrive(&bars->d1_empty[b]); mbar_arrive(&bars->h1_full[b]); }
-            return true;
-        };
-        auto E2 = [&](uint32_t i) -> bool {
+        }
+    } else if (n_mine > 0 && warp < kE3First) {
+        // ---- E2: conv2 accumulators -> the head's A operand ----------------------------
+        const uint32_t g = (warp - kE2First) >> 2;        // 32 of the 128 conv2 channels
+        const float* b2 = reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF);
+        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
+        for (uint32_t i = 0; i < n_mine && ok; i++) {
             const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&bars->d2_full[b], ph, abort_flag))) return false;
+            bool w = mbar_wait(&bars->d2_full[b], ph, abort_flag) && mbar_wait(&bars->h2_empty[b], ph ^ 1u, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, w);
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t c0 = g * 32u;                 // this warp's 32 of the 128 conv2 channels
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 128u + b * C2 + c0;
-            {
-                uint32_t v[32];
-                float x[32];
-                tmem_ld32(taddr, v);
-                tmem_ld_wait();
+            const uint32_t c0 = g * 32u;
+            uint32_t v[32];
+            tmem_ld32(tmem_base + ((q * 32u) << 16) + TM_D2 + b * C2 + c0, v);
+            tmem_ld_wait();
+            uint8_t* hrow = smem + SM_H2 + b * H2_BYTES + p * 16u;
 #pragma unroll
-                for (int c = 0; c < 32; c++)
-                    x[c] = __bfloat162float(__float2bfloat16_rn(fmaxf(__uint_as_float(v[c]) + b2[c0 + c], 0.0f)));
-                const float colsum = transpose_reduce32(x, lane);     // over this warp's 32 positions
-                part[q * C2 + c0 + lane] = colsum;
+            for (int j = 0; j < 4; j++) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const int c = j * 8 + e * 2;
+                    pk[e] = pack_relu_bf16(v[c], v[c + 1], b2[c0 + c], b2[c0 + c + 1]);
+                }
+                *reinterpret_cast<uint4*>(hrow + ((c0 >> 3) + j) * H2_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
+            fence_proxy_async();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->d2_empty[b]);
-            named_barrier_sync(1, kEpiThreads);
-            // linear head: epilogue warp w -> class w, lane -> channels 4*lane .. 4*lane+3
-            {
-                const uint32_t cls = et >> 5;
-                float acc = 0.0f;
-#pragma unroll
-                for (uint32_t k = 0; k < 4; k++) {
-                    const uint32_t ch = lane * 4u + k;
-                    const float pooled = (((part[ch] + part[C2 + ch]) + part[2 * C2 + ch]) + part[3 * C2 + ch]) * (1.0f / 128.0f);
-                    acc = fmaf(w3[cls * C2 + ch], pooled, acc);
-                }
-#pragma unroll
-                for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-                if (lane == 0) slog[cls] = acc + b3[cls];
-            }
-            named_barrier_sync(1, kEpiThreads);
-            const uint32_t r = blockIdx.x + i * gridDim.x;
-            if (et < n_cls) logits[(size_t)r * n_cls + et] = slog[et];
-            if (et == 32 && label) {
-                uint32_t a = 0; float mx = slog[0];
-                for (uint32_t c = 1; c < n_cls; c++) if (slog[c] > mx) { mx = slog[c]; a = c; }
-                label[r] = (uint8_t)a;
-            }
-            named_barrier_sync(1, kEpiThreads);          // slog / part are free again
-            return true;
-        };
-        if (ok) ok = E1(0);
+            if (lane == 0) { mbar_arrive(&bars->d2_empty[b]); mbar_arrive(&bars->h2_full[b]); }
+        }
+    } else if (n_mine > 0) {
+        // ---- E3: head accumulators [position][class] -> sum over positions -> logits ----
+        const uint32_t et = (warp - kE3First) * 32u + lane;           // 0..127
+        const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
+        float* part = reinterpret_cast<float*>(smem + SM_PART);
+        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
         for (uint32_t i = 0; i < n_mine && ok; i++) {
-            if (i + 1 < n_mine) ok = E1(i + 1);
-            if (ok) ok = E2(i);
+            const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->d4_full[b], ph, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t v[16];
+            tmem_ld16(tmem_base + ((q * 32u) << 16) + TM_D4 + b * NCLS_MAX, v);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->d4_empty[b]);
+            float x[16];
+#pragma unroll
+            for (int c = 0; c < 16; c++) x[c] = __uint_as_float(v[c]);
+            const float tot = transpose_reduce16(x, lane);            // this warp's 32 positions, class lane & 15
+            if (lane < 16) part[(warp - kE3First) * NCLS_MAX + lane] = tot;
+            named_barrier_sync(1, kE3Warps * 32);
+            const uint32_t r = blockIdx.x + i * gridDim.x;
+            if (et < 32) {                                            // first E3 warp: lane c < n_cls finishes class c
+                float lg = -3.0e38f;
+                if (lane < n_cls) {
+                    lg = ((part[lane] + part[NCLS_MAX + lane]) + part[2 * NCLS_MAX + lane]) + part[3 * NCLS_MAX + lane] + b3[lane];
+                    logits[(size_t)r * n_cls + lane] = lg;
+                }
+                // argmax, lowest index on ties
+                float best = lg; uint32_t arg = lane;
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) {
+                    const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+                    const uint32_t oa = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+                    if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+                }
+                if (lane == 0 && label) label[r] = (uint8_t)arg;
+            }
+            named_barrier_sync(1, kE3Warps * 32);                     // part is free again
         }
     }
 
@@ -295,7 +345,6 @@ uint16_t bf16_bits(float x) {
     if (low > 0x8000u || (low == 0x8000u && (up & 1u))) up++;
     return (uint16_t)up;
 }
-float bf16_value(float x) { uint32_t u = (uint32_t)bf16_bits(x) << 16; float f; memcpy(&f, &u, 4); return f; }
 
 }  // namespace
 
@@ -315,9 +364,14 @@ int sf_cnn_prepare(sf_slow* s, const float* w1, const float* b1, const float* w2
         for (uint32_t n = 0; n < C1; n++)
             for (uint32_t e = 0; e < CIN; e++)
                 W1[(t * C1 + n) * 8 + e] = bf16_bits(w1[((size_t)n * KW + t) * CIN + e]);
-    float* W3 = reinterpret_cast<float*>(h + W3_OFF);
+    // head weights rounded to bf16, then scaled by 2^-7 (exact) so that the MMA yields the mean's contribution
+    uint16_t* W3 = reinterpret_cast<uint16_t*>(h + W3_OFF);
     for (uint32_t c = 0; c < s->n_cls; c++)
-        for (uint32_t k = 0; k < C2; k++) W3[c * C2 + k] = bf16_value(w3[(size_t)c * C2 + k]);
+        for (uint32_t k = 0; k < C2; k++) {
+            uint32_t bits = (uint32_t)bf16_bits(w3[(size_t)c * C2 + k]) << 16;
+            float f; memcpy(&f, &bits, 4);
+            W3[((k / 8) * NCLS_MAX + c) * 8 + (k % 8)] = bf16_bits(f * (1.0f / 128.0f));
+        }
     memcpy(h + B1_OFF, b1, C1 * 4);
     memcpy(h + B2_OFF, b2, C2 * 4);
     memcpy(h + B3_OFF, b3, s->n_cls * 4);
