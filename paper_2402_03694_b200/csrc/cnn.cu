@@ -19,7 +19,7 @@
 //
 // Persistent CTAs, one per SM, loop over flows.  Warp roles:
 //   warp 0        streams input rows with bulk copies into a ring
-//   warp 1        issues the MMAs in the order conv1(i+1), conv2(i), head(i-1)
+//   warp 1        issues the MMAs in the order conv1(i+1), head(i-2), conv2(i)
 //   warps 2..5    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's A operand (shared memory)
 //   warps 6..21   E2: conv2 accumulators -> bias + ReLU -> bf16 -> the head's A operand
 //   warps 22..25  E3: head accumulators -> sum over positions -> + bias -> logits, argmax
@@ -213,12 +213,15 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 umma_commit(&bars->d4_full[b]);
                 return true;
             };
+            // head(i-2) goes BEFORE conv2(i): its input is ready by then (conv2(i) needs the same epilogue to have
+            // drained the accumulator), and it frees the activation buffer that E2(i) will write
             if (ok) ok = conv1(0);
             for (uint32_t i = 0; i < n_mine && ok; i++) {
                 if (i + 1 < n_mine) ok = conv1(i + 1);
+                if (ok && i >= 2) ok = head(i - 2);
                 if (ok) ok = conv2(i);
-                if (ok && i >= 1) ok = head(i - 1);
             }
+            if (ok && n_mine >= 2) ok = head(n_mine - 2);
             if (ok) ok = head(n_mine - 1);
         }
     } else if (n_mine > 0 && warp < kE2First) {
@@ -233,26 +236,27 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D1 + b * C1;
             uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (p + 2u) * 16u;
-#pragma unroll
-            for (uint32_t c0 = 0; c0 < C1; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(taddr + c0, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 4; j++) {            // 4 columns of 8 channels
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int e = 0; e < 4; e++) {
-                        const int c = j * 8 + e * 2;
-                        pk[e] = pack_relu_bf16(v[c], v[c + 1], b1[c0 + c], b1[c0 + c + 1]);
-                    }
-                    *reinterpret_cast<uint4*>(hrow + ((c0 >> 3) + j) * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
-            }
-            fence_proxy_async();                         // activations -> visible to the MMA's shared-memory reads
+            uint32_t v0[32], v1[32];
+            tmem_ld32(taddr, v0);
+            tmem_ld32(taddr + 32, v1);
+            tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(&bars->d1_empty[b]); mbar_arrive(&bars->h1_full[b]); }
+            if (lane == 0) mbar_arrive(&bars->d1_empty[b]);      // the accumulator is in registers: conv1 may reuse it
+#pragma unroll
+            for (int j = 0; j < 8; j++) {                // 8 columns of 8 channels
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const int c = (j & 3) * 8 + e * 2;
+                    const uint32_t a = (j < 4) ? v0[c] : v1[c], bq = (j < 4) ? v0[c + 1] : v1[c + 1];
+                    pk[e] = pack_relu_bf16(a, bq, b1[j * 8 + e * 2], b1[j * 8 + e * 2 + 1]);
+                }
+                *reinterpret_cast<uint4*>(hrow + j * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            fence_proxy_async();                         // activations -> visible to the MMA's shared-memory reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->h1_full[b]);
         }
     } else if (n_mine > 0 && warp < kE3First) {
         // ---- E2: conv2 accumulators -> the head's A operand ----------------------------
@@ -269,6 +273,9 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             uint32_t v[32];
             tmem_ld32(tmem_base + ((q * 32u) << 16) + TM_D2 + b * C2 + c0, v);
             tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->d2_empty[b]);      // the accumulator is in registers: conv2 may reuse it
             uint8_t* hrow = smem + SM_H2 + b * H2_BYTES + p * 16u;
 #pragma unroll
             for (int j = 0; j < 4; j++) {
@@ -281,9 +288,8 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 *reinterpret_cast<uint4*>(hrow + ((c0 >> 3) + j) * H2_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
             fence_proxy_async();
-            tc_fence_before();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(&bars->d2_empty[b]); mbar_arrive(&bars->h2_full[b]); }
+            if (lane == 0) mbar_arrive(&bars->h2_full[b]);
         }
     } else if (n_mine > 0) {
         // ---- E3: head accumulators [position][class] -> sum over positions -> logits ----
