@@ -19,11 +19,11 @@
 //
 // Persistent CTAs, one per SM, loop over flows.  Warp roles:
 //   warp 0        streams input rows with bulk copies into a ring
-//   warp 1        issues the MMAs in the order conv1(i+1), head(i-2), conv2(i)
+//   warp 1        issues the MMAs in the order conv1(i+2), conv2(i), head(i-2)
 //   warps 2..5    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's A operand (shared memory)
 //   warps 6..21   E2: conv2 accumulators -> bias + ReLU -> bf16 -> the head's A operand
 //   warps 22..25  E3: head accumulators -> sum over positions -> + bias -> logits, argmax
-// Every accumulator and activation buffer is double buffered, so the three epilogues and the
+// Every accumulator and activation buffer is double (conv1: triple) buffered, so the three epilogues and the
 // tensor pipe overlap.  Every wait is bounded; on a timeout the block records
 // SF_ERR_DEVICE_TIMEOUT and leaves.
 #include "tc_common.cuh"
@@ -56,26 +56,27 @@ constexpr uint32_t B3_OFF = B2_OFF + C2 * 4;                // fp32 [16]
 constexpr uint32_t BLOB_BYTES = B3_OFF + NCLS_MAX * 4;
 // shared memory map
 constexpr uint32_t SM_BLOB = 0;
-constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // 2 buffers
-constexpr uint32_t SM_H2 = SM_H1 + 2 * H1_BYTES;            // 2 buffers
+constexpr uint32_t NB1 = 3;                                 // conv1 accumulator / activation buffers (conv1 runs two flows ahead)
+constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // NB1 buffers
+constexpr uint32_t SM_H2 = SM_H1 + NB1 * H1_BYTES;          // 2 buffers
 constexpr uint32_t SM_X = SM_H2 + 2 * H2_BYTES;             // XS stages
 constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // fp32 [4 warps][16] partial logits
 constexpr uint32_t SM_BARS = SM_PART + 4 * NCLS_MAX * 4;
-constexpr uint32_t SM_TOTAL = SM_BARS + 256;
+constexpr uint32_t SM_TOTAL = SM_BARS + 320;
 static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_H2 % 16 == 0 && SM_X % 16 == 0 && SM_BARS % 8 == 0, "alignment");
 static_assert(SM_TOTAL <= 232448, "shared memory");
-// TMEM columns: conv1 accumulators [2][64], conv2 [2][128], head [2][16]
-constexpr uint32_t TM_D1 = 0, TM_D2 = 128, TM_D4 = 384;
+// TMEM columns: conv1 accumulators [3][64], conv2 [2][128], head [2][16]
+constexpr uint32_t TM_D1 = 0, TM_D2 = 192, TM_D4 = 448;
 
 struct Bars {
     uint64_t w_full;
     uint64_t x_full[XS], x_empty[XS];
-    uint64_t d1_full[2], d1_empty[2], h1_full[2], h1_empty[2];
+    uint64_t d1_full[NB1], d1_empty[NB1], h1_full[NB1], h1_empty[NB1];
     uint64_t d2_full[2], d2_empty[2], h2_full[2], h2_empty[2];
     uint64_t d4_full[2], d4_empty[2];
     uint32_t tmem_base, abort_flag;
 };
-static_assert(sizeof(Bars) <= 256, "barrier block");
+static_assert(sizeof(Bars) <= 320, "barrier block");
 
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -119,14 +120,16 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     const uint32_t n_mine = (n_rows > blockIdx.x) ? (n_rows - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
     // zero everything that acts as padding (and the rest of the activation buffers)
-    for (uint32_t i = threadIdx.x; i < (2 * H1_BYTES + 2 * H2_BYTES + XS * X_STAGE) / 16; i += kThreads)
+    for (uint32_t i = threadIdx.x; i < (NB1 * H1_BYTES + 2 * H2_BYTES + XS * X_STAGE) / 16; i += kThreads)
         reinterpret_cast<uint4*>(smem + SM_H1)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
         mbar_init(&bars->w_full, 1);
         for (uint32_t s = 0; s < XS; s++) { mbar_init(&bars->x_full[s], 1); mbar_init(&bars->x_empty[s], 1); }
-        for (uint32_t b = 0; b < 2; b++) {
+        for (uint32_t b = 0; b < NB1; b++) {
             mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kE1Warps);
             mbar_init(&bars->h1_full[b], kE1Warps); mbar_init(&bars->h1_empty[b], 1);
+        }
+        for (uint32_t b = 0; b < 2; b++) {
             mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], kE2Warps);
             mbar_init(&bars->h2_full[b], kE2Warps); mbar_init(&bars->h2_empty[b], 1);
             mbar_init(&bars->d4_full[b], 1); mbar_init(&bars->d4_empty[b], kE3Warps);
@@ -149,7 +152,7 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             bulk_load(smem + SM_BLOB, blob, BLOB_BYTES, &bars->w_full);
             for (uint32_t i = 0; i < n_mine; i++) {
                 const uint32_t s = i % XS, ph = (i / XS) & 1u;
-                if (!mbar_wait(&bars->x_empty[s], ph ^ 1u, abort_flag)) break;
+                if (!mbar_wait_relaxed(&bars->x_empty[s], ph ^ 1u, abort_flag)) break;
                 const uint32_t r = blockIdx.x + i * gridDim.x;
                 mbar_expect_tx(&bars->x_full[s], L * CIN * 2);
                 bulk_load(smem + SM_X + s * X_STAGE + 32, rows + (size_t)r * L * CIN, L * CIN * 2, &bars->x_full[s]);
@@ -160,40 +163,42 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             constexpr uint32_t idesc1 = make_idesc_bf16(128, C1);
             constexpr uint32_t idesc2 = make_idesc_bf16(128, C2);
             constexpr uint32_t idesc4 = make_idesc_bf16(128, NCLS_MAX);
+            // descriptor = constant fields + (address >> 4) in the low bits: build the bases once, add offsets per MMA
+            const uint64_t dX = make_smem_desc(sbase + SM_X, 16, 128, 0);
+            const uint64_t dW1 = make_smem_desc(sbase + SM_BLOB + W1_OFF, C1 * 16u, 128, 0);
+            const uint64_t dH1 = make_smem_desc(sbase + SM_H1, H1_COL, 128, 0);
+            const uint64_t dW2 = make_smem_desc(sbase + SM_BLOB + W2_OFF, C2 * 16u, 128, 0);
+            const uint64_t dH2 = make_smem_desc(sbase + SM_H2, H2_COL, 128, 0);
+            const uint64_t dW3 = make_smem_desc(sbase + SM_BLOB + W3_OFF, NCLS_MAX * 16u, 128, 0);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
             auto conv1 = [&](uint32_t i) -> bool {
-                const uint32_t s = i % XS, xph = (i / XS) & 1u, b = i & 1u, ph = (i >> 1) & 1u;
+                const uint32_t s = i % XS, xph = (i / XS) & 1u, b = i % NB1, ph = (i / NB1) & 1u;
                 if (!mbar_wait(&bars->x_full[s], xph, abort_flag)) return false;
                 if (!mbar_wait(&bars->d1_empty[b], ph ^ 1u, abort_flag)) return false;
                 tc_fence_after();
-                const uint32_t xa = sbase + SM_X + s * X_STAGE;
+                const uint64_t ax = dX + (uint64_t)((s * X_STAGE) >> 4);
 #pragma unroll
-                for (uint32_t k = 0; k < 3; k++) {           // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
-                    const uint64_t ad = make_smem_desc(xa + k * 32u, 16, 128, 0);
-                    const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W1_OFF + k * 2u * (C1 * 16u), C1 * 16u, 128, 0);
-                    umma_bf16(tmem_base + TM_D1 + b * C1, ad, bd, idesc1, k != 0 ? 1u : 0u);
-                }
+                for (uint32_t k = 0; k < 3; k++)             // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
+                    umma_bf16(tmem_base + TM_D1 + b * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4), idesc1,
+                              k != 0 ? 1u : 0u);
                 umma_commit(&bars->x_empty[s]);
                 umma_commit(&bars->d1_full[b]);
                 return true;
             };
             auto conv2 = [&](uint32_t i) -> bool {
-                const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-                if (!mbar_wait(&bars->h1_full[b], ph, abort_flag)) return false;
+                const uint32_t b = i & 1u, ph = (i >> 1) & 1u, b1i = i % NB1, ph1 = (i / NB1) & 1u;
+                if (!mbar_wait(&bars->h1_full[b1i], ph1, abort_flag)) return false;
                 if (!mbar_wait(&bars->d2_empty[b], ph ^ 1u, abort_flag)) return false;
                 tc_fence_after();
-                const uint32_t ha = sbase + SM_H1 + b * H1_BYTES;
+                const uint64_t ah = dH1 + (uint64_t)((b1i * H1_BYTES) >> 4);
 #pragma unroll
                 for (uint32_t t = 0; t < KW; t++) {
 #pragma unroll
-                    for (uint32_t k = 0; k < C1 / 16; k++) {
-                        const uint64_t ad = make_smem_desc(ha + (2u * k) * H1_COL + t * 16u, H1_COL, 128, 0);
-                        const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W2_OFF + t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u),
-                                                           C2 * 16u, 128, 0);
-                        umma_bf16(tmem_base + TM_D2 + b * C2, ad, bd, idesc2, (t | k) != 0 ? 1u : 0u);
-                    }
+                    for (uint32_t k = 0; k < C1 / 16; k++)
+                        umma_bf16(tmem_base + TM_D2 + b * C2, ah + (((2u * k) * H1_COL + t * 16u) >> 4),
+                                  dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
                 }
-                umma_commit(&bars->h1_empty[b]);
+                umma_commit(&bars->h1_empty[b1i]);
                 umma_commit(&bars->d2_full[b]);
                 return true;
             };
@@ -202,24 +207,23 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 if (!mbar_wait(&bars->h2_full[b], ph, abort_flag)) return false;
                 if (!mbar_wait(&bars->d4_empty[b], ph ^ 1u, abort_flag)) return false;
                 tc_fence_after();
-                const uint32_t ha = sbase + SM_H2 + b * H2_BYTES;
+                const uint64_t ah = dH2 + (uint64_t)((b * H2_BYTES) >> 4);
 #pragma unroll
-                for (uint32_t k = 0; k < C2 / 16; k++) {
-                    const uint64_t ad = make_smem_desc(ha + (2u * k) * H2_COL, H2_COL, 128, 0);
-                    const uint64_t bd = make_smem_desc(sbase + SM_BLOB + W3_OFF + (2u * k) * (NCLS_MAX * 16u), NCLS_MAX * 16u, 128, 0);
-                    umma_bf16(tmem_base + TM_D4 + b * NCLS_MAX, ad, bd, idesc4, k != 0 ? 1u : 0u);
-                }
+                for (uint32_t k = 0; k < C2 / 16; k++)
+                    umma_bf16(tmem_base + TM_D4 + b * NCLS_MAX, ah + (((2u * k) * H2_COL) >> 4),
+                              dW3 + (((2u * k) * (NCLS_MAX * 16u)) >> 4), idesc4, k != 0 ? 1u : 0u);
                 umma_commit(&bars->h2_empty[b]);
                 umma_commit(&bars->d4_full[b]);
                 return true;
             };
-            // head(i-2) goes BEFORE conv2(i): its input is ready by then (conv2(i) needs the same epilogue to have
-            // drained the accumulator), and it frees the activation buffer that E2(i) will write
+            // conv1 runs two flows ahead and the head two flows behind conv2, so that each epilogue has two
+            // conv2 periods to turn its accumulator into the next operand
             if (ok) ok = conv1(0);
+            if (ok && n_mine > 1) ok = conv1(1);
             for (uint32_t i = 0; i < n_mine && ok; i++) {
-                if (i + 1 < n_mine) ok = conv1(i + 1);
-                if (ok && i >= 2) ok = head(i - 2);
+                if (i + 2 < n_mine) ok = conv1(i + 2);
                 if (ok) ok = conv2(i);
+                if (ok && i >= 2) ok = head(i - 2);
             }
             if (ok && n_mine >= 2) ok = head(n_mine - 2);
             if (ok) ok = head(n_mine - 1);
@@ -227,10 +231,10 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     } else if (n_mine > 0 && warp < kE2First) {
         // ---- E1: conv1 accumulators -> conv2's A operand -------------------------------
         const float* b1 = reinterpret_cast<const float*>(smem + SM_BLOB + B1_OFF);
-        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
+        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
         for (uint32_t i = 0; i < n_mine && ok; i++) {
-            const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-            bool w = mbar_wait(&bars->d1_full[b], ph, abort_flag) && mbar_wait(&bars->h1_empty[b], ph ^ 1u, abort_flag);
+            const uint32_t b = i % NB1, ph = (i / NB1) & 1u;
+            bool w = mbar_wait_relaxed(&bars->d1_full[b], ph, abort_flag) && mbar_wait_relaxed(&bars->h1_empty[b], ph ^ 1u, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, w);
             if (!ok) break;
             tc_fence_after();
@@ -262,10 +266,10 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
         // ---- E2: conv2 accumulators -> the head's A operand ----------------------------
         const uint32_t g = (warp - kE2First) >> 2;        // 32 of the 128 conv2 channels
         const float* b2 = reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF);
-        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
+        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
         for (uint32_t i = 0; i < n_mine && ok; i++) {
             const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-            bool w = mbar_wait(&bars->d2_full[b], ph, abort_flag) && mbar_wait(&bars->h2_empty[b], ph ^ 1u, abort_flag);
+            bool w = mbar_wait_relaxed(&bars->d2_full[b], ph, abort_flag) && mbar_wait_relaxed(&bars->h2_empty[b], ph ^ 1u, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, w);
             if (!ok) break;
             tc_fence_after();
@@ -296,10 +300,10 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
         const uint32_t et = (warp - kE3First) * 32u + lane;           // 0..127
         const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
         float* part = reinterpret_cast<float*>(smem + SM_PART);
-        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->w_full, 0, abort_flag));
+        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
         for (uint32_t i = 0; i < n_mine && ok; i++) {
             const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->d4_full[b], ph, abort_flag));
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->d4_full[b], ph, abort_flag));
             if (!ok) break;
             tc_fence_after();
             uint32_t v[16];
