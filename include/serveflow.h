@@ -264,6 +264,18 @@ int  sf_serve_batch(sf_ctx* ctx, const sf_forest* forest, const sf_slow* slow, c
 int  sf_serve_batch_host(sf_ctx* ctx, const sf_forest* forest, const sf_slow* slow, const sf_packets* fast_ctx_host,
                          uint32_t N, uint32_t F, const sf_packets* slow_ctx_host, const sf_route_cfg* cfg_host_tau,
                          uint8_t* label_host_out, uint8_t* stage_host_out, uint32_t* n_esc_host_out, void* stream);
+/* Three-tier cascade (Sec. 3.1: the fastest model answers what it is sure of, the fast model
+ * looks at the rest using the SAME features, the slow model at what is still uncertain, with
+ * more packets; Sec. 3.2: thresholds per predicted class).  Both tree models are SF_RF
+ * ensembles over the same F features (the fastest one is typically a single tree).
+ * cfg_fastest: only rule (SF_LC_GT) and tau (fp32[C of fastest]) are used; cfg_fast: as in
+ * sf_serve_batch.  stage_out: 1, 2 or 3.  n_esc_out (device, nullable): uint32[2] = flows
+ * passed on by the fastest model, flows assigned to the slow model.  The context counters
+ * count routing decisions: n_flows grows by n plus the first count. */
+int  sf_serve_batch3(sf_ctx* ctx, const sf_forest* fastest, const sf_forest* fast, const sf_slow* slow,
+                     const sf_packets* fast_ctx, uint32_t N, uint32_t F, const sf_packets* slow_ctx,
+                     const sf_route_cfg* cfg_fastest, const sf_route_cfg* cfg_fast, uint8_t* label_out,
+                     uint8_t* stage_out, uint32_t* n_esc_out, void* stream);
 /* Pointers into the workspace to the intermediates of the last sf_serve_batch on
  * this context (for inspection and tests): any out pointer may be NULL. */
 int  sf_serve_batch_intermediates(sf_ctx* ctx, const float** feat, const float** fast_out, const uint32_t** esc_ids,

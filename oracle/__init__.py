@@ -268,3 +268,30 @@ def serve_batch(cfg, fast_pk, wide_pk, forest, slow_model, tau, threads=1):
     label, stage = merge(r["label"], r["esc_ids"], label_slow)
     return {"feat": feat, "fast_out": fo, **r, "rows": rows, "logits": logits, "label_slow": label_slow,
             "label_final": label, "stage": stage}
+
+
+def serve_batch3(cfg, fast_pk, wide_pk, fastest, fast, slow_model, tau1, tau2, threads=1):
+    """Three-tier cascade (Sec. 3.1): the fastest model answers what it is sure of; the rest goes to the
+    fast model on the SAME features; what that is still unsure of goes to the slow model, which sees more
+    packets.  tau1 / tau2 are per-class thresholds (Sec. 3.2).  stage = 1, 2 or 3."""
+    feat = extract_features(fast_pk, cfg.N, cfg.F, threads=threads)
+    p1 = forest_infer(fastest, feat, threads=threads)
+    r1 = route_lc(p1, tau1)
+    ids1 = r1["esc_ids"]
+    p2 = forest_infer(fast, feat[ids1], threads=threads) if len(ids1) else np.zeros((0, fast["C"]), np.float32)
+    r2 = route_lc(p2, tau2) if len(ids1) else {"esc_ids": np.zeros(0, np.uint32), "label": np.zeros(0, np.uint8),
+                                               "n_esc": 0, "score": np.zeros(0, np.float32)}
+    ids2 = ids1[r2["esc_ids"]]
+    bf16 = cfg.slow_dtype == "bf16"
+    rows = wide_rows(0 if cfg.slow == "mlp" else 1, ids2, wide_pk, cfg.P, bf16, threads=threads)
+    if cfg.slow == "mlp":
+        logits, label_slow = mlp(slow_model, rows, bf16, threads=threads)
+    else:
+        logits, label_slow = cnn(slow_model, rows, bf16, threads=threads)
+    n = feat.shape[0]
+    label = r1["label"].copy()
+    stage = np.ones(n, np.uint8)
+    label[ids1] = r2["label"]; stage[ids1] = 2
+    label[ids2] = label_slow; stage[ids2] = 3
+    return {"feat": feat, "prob1": p1, "ids1": ids1, "prob2": p2, "ids2": ids2, "rows": rows, "logits": logits,
+            "label_slow": label_slow, "label_final": label, "stage": stage, "label1": r1["label"], "label2": r2["label"]}

@@ -84,7 +84,7 @@ EXPORTS = [
     "sf_extract_features", "sf_forest_create", "sf_forest_destroy", "sf_fast_infer", "sf_route",
     "sf_route_noalloc",
     "sf_universal_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
-    "sf_serve_batch", "sf_serve_batch_host", "sf_serve_batch_intermediates",
+    "sf_serve_batch", "sf_serve_batch3", "sf_serve_batch_host", "sf_serve_batch_intermediates",
     "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_lookup",
 ]
 
@@ -123,6 +123,8 @@ def _lib():
         L.sf_serve_batch.argtypes = [V, V, V, C.POINTER(sf_packets), U32, U32, C.POINTER(sf_packets),
                                      C.POINTER(sf_route_cfg), V, V, V, V]
         L.sf_serve_batch_host.argtypes = L.sf_serve_batch.argtypes
+        L.sf_serve_batch3.argtypes = [V, V, V, V, C.POINTER(sf_packets), U32, U32, C.POINTER(sf_packets),
+                                      C.POINTER(sf_route_cfg), C.POINTER(sf_route_cfg), V, V, V, V]
         L.sf_serve_batch_intermediates.argtypes = [V] + [C.POINTER(V)] * 7
         L.sf_table_create.argtypes = [V, U32, U32, U32, U32, C.POINTER(V)]
         L.sf_table_ingest.argtypes = [V, V, C.POINTER(sf_pkt_batch), V, U32, V, C.POINTER(sf_route_cfg), V, V]
@@ -294,6 +296,13 @@ def sf_serve_batch(ctx, forest, slow, fast_ctx, N, F, slow_ctx, cfg, label_out, 
                    stream=None):
     _check(_lib().sf_serve_batch(ctx, forest, slow, C.byref(fast_ctx), N, F, C.byref(slow_ctx), C.byref(cfg),
                                  _dp(label_out), _dp(stage_out), _dp(n_esc_out), _stream(stream)), "sf_serve_batch")
+
+
+def sf_serve_batch3(ctx, fastest, fast, slow, fast_ctx, N, F, slow_ctx, cfg_fastest, cfg_fast, label_out, stage_out,
+                    n_esc_out=None, stream=None):
+    _check(_lib().sf_serve_batch3(ctx, fastest, fast, slow, C.byref(fast_ctx), N, F, C.byref(slow_ctx), C.byref(cfg_fastest),
+                                  C.byref(cfg_fast), _dp(label_out), _dp(stage_out), _dp(n_esc_out), _stream(stream)),
+           "sf_serve_batch3")
 
 
 def sf_serve_batch_host(ctx, forest, slow, fast_ctx_host, N, F, slow_ctx_host, cfg_host_tau, label_host_out,

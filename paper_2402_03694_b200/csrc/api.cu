@@ -298,6 +298,79 @@ extern "C" int sf_serve_batch(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s
     return serve_on_device(ctx, fo, s, fast, N, F, wide, cfg, label_out, stage_out, n_esc_out, (cudaStream_t)stream);
 }
 
+extern "C" int sf_serve_batch3(sf_ctx* ctx, const sf_forest* f1, const sf_forest* f2, const sf_slow* s, const sf_packets* fast,
+                               uint32_t N, uint32_t F, const sf_packets* wide, const sf_route_cfg* cfg1,
+                               const sf_route_cfg* cfg2, uint8_t* label_out, uint8_t* stage_out, uint32_t* n_esc_out,
+                               void* stream)
+{
+    if (!f1 || !cfg1 || !cfg1->tau) return SF_ERR_ARG;
+    int rc = check_serve_args(ctx, f2, s, fast, N, F, wide, cfg2);
+    if (rc != SF_OK) return rc;
+    if (!label_out || !stage_out) return SF_ERR_ARG;
+    if (f1->kind != SF_RF || f1->F != F || cfg1->rule != SF_LC_GT || cfg2->rule != SF_LC_GT) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint32_t n = fast->n_flows, cap = cfg2->capacity;
+    const size_t esz = cfg2->row_dtype == SF_BF16 ? 2 : 4;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += sf_align256(bytes); return o; };
+    const size_t o_feat = take((size_t)n * F * 4), o_p1 = take((size_t)n * f1->C * 4), o_dec1 = take(n), o_lab1 = take(n),
+                 o_ids1 = take((size_t)n * 4), o_feat2 = take((size_t)n * F * 4), o_p2 = take((size_t)n * f2->C * 4),
+                 o_dec2 = take(n), o_lab2 = take(n), o_ids2l = take((size_t)cap * 4), o_ids2 = take((size_t)cap * 4),
+                 o_rows = take((size_t)cap * slow_width(s) * esz), o_logits = take((size_t)cap * slow_classes(s) * 4),
+                 o_labs = take(cap), o_rs1 = take(sf_route_scratch_bytes(n)), o_rs2 = take(sf_route_scratch_bytes(n)),
+                 o_slow = take(sf_slow_scratch_bytes(s, cap)), o_cnt = take(64);
+    rc = sf_ws_reserve(ctx, off);
+    if (rc != SF_OK) return rc;
+    sf_ws_reset(ctx);
+    char* w = reinterpret_cast<char*>(sf_ws_alloc(ctx, off));
+    if (!w) return SF_ERR_ALLOC;
+    float* feat = (float*)(w + o_feat); float* feat2 = (float*)(w + o_feat2);
+    float* p1 = (float*)(w + o_p1); float* p2 = (float*)(w + o_p2);
+    uint32_t* ids1 = (uint32_t*)(w + o_ids1); uint32_t* ids2l = (uint32_t*)(w + o_ids2l); uint32_t* ids2 = (uint32_t*)(w + o_ids2);
+    uint32_t* cnt = n_esc_out ? n_esc_out : (uint32_t*)(w + o_cnt);          // [0] after the fastest model, [1] after the fast one
+    sf_time_new_record(ctx);
+    sf_time_begin(ctx, SF_T_EXTRACT, st);
+    rc = sf_launch_extract(fast, N, F, feat, st);
+    sf_time_end(ctx, SF_T_EXTRACT, st);
+    if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_FOREST, st);
+    rc = sf_launch_forest(f1, feat, n, p1, nullptr, st);
+    if (rc != SF_OK) return rc;
+    // tier 1 -> 2: every flow the fastest model is unsure of (capacity n: the list cannot overflow)
+    sf_route_cfg c1 = *cfg1;
+    c1.capacity = n;
+    rc = sf_launch_route(ctx, &c1, p1, n, f1->C, nullptr, ids1, &cnt[0], nullptr, (uint8_t*)(w + o_dec1), (uint8_t*)(w + o_lab1),
+                         nullptr, w + o_rs1, st);
+    if (rc != SF_OK) return rc;
+    rc = sf_launch_gather_feat(feat, ids1, &cnt[0], n, F, feat2, st);
+    if (rc != SF_OK) return rc;
+    rc = sf_launch_forest(f2, feat2, n, p2, nullptr, st, &cnt[0]);
+    sf_time_end(ctx, SF_T_FOREST, st);
+    if (rc != SF_OK) return rc;
+    // tier 2 -> 3: positions in the first list, then the flow ids themselves
+    rc = sf_launch_route(ctx, cfg2, p2, n, f2->C, nullptr, ids2l, &cnt[1], nullptr, (uint8_t*)(w + o_dec2), (uint8_t*)(w + o_lab2),
+                         nullptr, w + o_rs2, st, &cnt[0]);
+    if (rc != SF_OK) return rc;
+    rc = sf_launch_compose_ids(ids1, ids2l, &cnt[1], cap, ids2, st);
+    if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_GATHER, st);
+    rc = sf_launch_gather(ctx, cfg2, wide, ids2, &cnt[1], cap, w + o_rows, st);
+    sf_time_end(ctx, SF_T_GATHER, st);
+    if (rc != SF_OK) return rc;
+    rc = sf_launch_slow(ctx, s, w + o_rows, &cnt[1], cap, (float*)(w + o_logits), (uint8_t*)(w + o_labs), w + o_slow, st);
+    if (rc != SF_OK) return rc;
+    sf_time_begin(ctx, SF_T_MERGE, st);
+    rc = sf_launch_merge((uint8_t*)(w + o_lab1), nullptr, n, ids1, &cnt[0], n, (uint8_t*)(w + o_lab2), label_out, stage_out, st, 2, true);
+    if (rc == SF_OK)
+        rc = sf_launch_merge(nullptr, nullptr, n, ids2, &cnt[1], cap, (uint8_t*)(w + o_labs), label_out, stage_out, st, 3, false);
+    sf_time_end(ctx, SF_T_MERGE, st);
+    if (rc != SF_OK) return rc;
+    ctx->last_feat = feat; ctx->last_fast_out = p2; ctx->last_esc_ids = ids2; ctx->last_rows = w + o_rows;
+    ctx->last_logits = (float*)(w + o_logits); ctx->last_label_fast = (uint8_t*)(w + o_lab1); ctx->last_label_slow = (uint8_t*)(w + o_labs);
+    return SF_OK;
+}
+
 extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf_packets* fast_h,
                                    uint32_t N, uint32_t F, const sf_packets* wide_h, const sf_route_cfg* cfg_h,
                                    uint8_t* label_h, uint8_t* stage_h, uint32_t* n_esc_h, void* stream)

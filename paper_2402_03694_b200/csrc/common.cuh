@@ -94,7 +94,8 @@ int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* 
 size_t sf_route_scratch_bytes(uint32_t n);
 int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,
                     const sf_packets* wide, uint32_t* esc_ids, uint32_t* n_esc, void* rows,
-                    uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st);
+                    uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st,
+                    const uint32_t* n_dev = nullptr);       // n_dev: optional device-side count of scored flows (<= n)
 int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C, uint8_t* decision,
                     uint8_t* label, float* score, uint32_t* block_counts, const uint32_t* n_dev, cudaStream_t st);
 int sf_launch_iota(uint32_t* out, uint32_t n, cudaStream_t st);      // out[i] = i
@@ -105,7 +106,11 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
                    float* logits, uint8_t* label, void* scratch, cudaStream_t st);
 int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t n, const uint32_t* esc_ids,
                     const uint32_t* n_esc, uint32_t capacity, const uint8_t* label_slow,
-                    uint8_t* label, uint8_t* stage, cudaStream_t st);
+                    uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value = 2, bool write_fast = true);
+int sf_launch_gather_feat(const float* feat, const uint32_t* ids, const uint32_t* n_dev, uint32_t n_max, uint32_t F,
+                          float* out, cudaStream_t st);
+int sf_launch_compose_ids(const uint32_t* ids1, const uint32_t* ids2_local, const uint32_t* n_dev, uint32_t n_max,
+                          uint32_t* out, cudaStream_t st);
 
 // bf16 tensor-core layers (gemm_tc.cu)
 int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,

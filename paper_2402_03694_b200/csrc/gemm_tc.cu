@@ -1,5 +1,5 @@
 // S4 (bf16 MLP): hidden layers as tcgen05 GEMMs with TMEM accumulators fed by
-// TMA, and the narrow last layer (<= 16 classes) as a CUDA-core dot-product head.
+// TMA; the narrow last layer (<= 16 classes) runs through the same kernel as a 128 x 16 tile.
 //
 // Hidden layer: out[r][o] = bf16( ReLU( sum_k A[r][k] * W[o][k] + b[o] ) ), r < *n_rows.
 // Persistent kernel, one CTA per SM, tile 128 x BN, K slices of 64 bf16 (one 128-byte
@@ -246,72 +246,6 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     if (warp == 1) { __syncwarp(); tmem_dealloc(tmem_base, Cfg::kTmemCols); }
 }
 
-// Last layer: logits[r][c] = sum_k h[r][k] * W[c][k] + b[c], c < C <= 16; one warp per row,
-// weights staged in shared memory, 16-byte loads, fp32 accumulation, warp-shuffle reduce.
-__global__ void __launch_bounds__(256)
-head_bf16_kernel(const __nv_bfloat16* __restrict__ h, const __nv_bfloat16* __restrict__ W, const float* __restrict__ b,
-                 const uint32_t* __restrict__ n_rows_dev, uint32_t K, uint32_t C,
-                 float* __restrict__ logits, uint8_t* __restrict__ label)
-{
-    extern __shared__ __align__(16) uint8_t smem_w[];
-    __nv_bfloat16* sW = reinterpret_cast<__nv_bfloat16*>(smem_w);
-    const uint32_t n_rows = *n_rows_dev;
-    {
-        const uint4* src = reinterpret_cast<const uint4*>(W);
-        uint4* dst = reinterpret_cast<uint4*>(sW);
-        const uint32_t vecs = C * K / 8;
-        for (uint32_t v = threadIdx.x; v < vecs; v += blockDim.x) dst[v] = __ldg(src + v);
-    }
-    __syncthreads();
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
-    for (uint32_t r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_rows; r += warps) {
-        float acc[16];
-#pragma unroll
-        for (int c = 0; c < 16; c++) acc[c] = 0.0f;
-        const __nv_bfloat16* hr = h + (size_t)r * K;
-        for (uint32_t k = lane * 8; k < K; k += 256) {
-            uint4 hv = __ldg(reinterpret_cast<const uint4*>(hr + k));
-            const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
-            float2 x[4];
-#pragma unroll
-            for (int j = 0; j < 4; j++) x[j] = __bfloat1622float2(hp[j]);
-#pragma unroll
-            for (int c = 0; c < 16; c++) {
-                if ((uint32_t)c < C) {
-                    uint4 wv = *reinterpret_cast<const uint4*>(sW + (size_t)c * K + k);
-                    const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
-#pragma unroll
-                    for (int j = 0; j < 4; j++) {
-                        float2 w = __bfloat1622float2(wp[j]);
-                        acc[c] = fmaf(x[j].x, w.x, acc[c]);
-                        acc[c] = fmaf(x[j].y, w.y, acc[c]);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int c = 0; c < 16; c++) {
-            if ((uint32_t)c < C) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xFFFFFFFFu, acc[c], o);
-            }
-        }
-        if (lane == 0) {
-            uint32_t a = 0; float mx = 0.0f;
-#pragma unroll
-            for (int c = 0; c < 16; c++) {
-                if ((uint32_t)c < C) {
-                    float v = acc[c] + b[c];
-                    logits[(size_t)r * C + c] = v;
-                    if (c == 0 || v > mx) { mx = v; a = c; }
-                }
-            }
-            if (label) label[r] = (uint8_t)a;
-        }
-    }
-}
-
 template <uint32_t BN>
 int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, const uint32_t* n_rows_dev,
                 uint32_t capacity, uint32_t N, uint32_t K, void* out, cudaStream_t st)
@@ -352,20 +286,6 @@ int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bia
 }
 
 }  // namespace
-
-int sf_launch_head_bf16(sf_ctx* ctx, const void* h, const void* W, const float* b, const uint32_t* n_rows_dev,
-                        uint32_t capacity, uint32_t K, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
-{
-    size_t smem = (size_t)C * K * 2;
-    SF_CUDA(cudaFuncSetAttribute(head_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    uint32_t blocks = (capacity + 7) / 8;
-    uint32_t maxb = (uint32_t)ctx->num_sms * 4;
-    if (blocks > maxb) blocks = maxb;
-    head_bf16_kernel<<<blocks, 256, smem, st>>>(reinterpret_cast<const __nv_bfloat16*>(h),
-                                                reinterpret_cast<const __nv_bfloat16*>(W), b, n_rows_dev, K, C, logits, label);
-    SF_LAUNCH_CHECK("head_bf16_kernel");
-    return SF_OK;
-}
 
 int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
                         float* logits, uint8_t* label, void* scratch, cudaStream_t st)

@@ -56,8 +56,9 @@ score_kernel(const float* __restrict__ fast_out, uint32_t n, uint32_t C, const f
 // exclusive scan of nb block counts in place; total (clamped) -> *n_esc and the state block
 __global__ void __launch_bounds__(1024)
 scan_kernel(uint32_t* __restrict__ block_counts, uint32_t nb, uint32_t n, uint32_t capacity,
-            uint32_t* __restrict__ n_esc, sf_dev_state* __restrict__ st)
+            uint32_t* __restrict__ n_esc, sf_dev_state* __restrict__ st, const uint32_t* __restrict__ n_dev = nullptr)
 {
+    if (n_dev) n = min(n, *n_dev);               // flows actually scored (blocks past the count contributed zeros)
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry_s;
     if (threadIdx.x == 0) carry_s = 0;
@@ -97,8 +98,9 @@ scan_kernel(uint32_t* __restrict__ block_counts, uint32_t nb, uint32_t n, uint32
 
 __global__ void __launch_bounds__(kScoreBlock)
 scatter_kernel(const uint8_t* __restrict__ decision, uint32_t n, const uint32_t* __restrict__ block_offsets,
-               uint32_t capacity, uint32_t* __restrict__ esc_ids)
+               uint32_t capacity, uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__ n_dev = nullptr)
 {
+    if (n_dev) n = min(n, *n_dev);
     __shared__ uint32_t warp_off[kScoreBlock / 32];
     const uint32_t f = blockIdx.x * kScoreBlock + threadIdx.x;
     const bool esc = (f < n) && decision[f] != 0;
@@ -191,14 +193,32 @@ __global__ void merge_fast_kernel(const uint8_t* __restrict__ label_fast, const 
 
 __global__ void merge_slow_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__ n_esc_dev,
                                   const uint8_t* __restrict__ label_slow, uint8_t* __restrict__ label,
-                                  uint8_t* __restrict__ stage, sf_dev_state* st)
+                                  uint8_t* __restrict__ stage, uint8_t stage_value)
 {
     const uint32_t n_esc = *n_esc_dev;
     for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < n_esc; r += gridDim.x * blockDim.x) {
         uint32_t f = esc_ids[r];
         if (label) label[f] = label_slow[r];
-        if (stage) stage[f] = 2;
+        if (stage) stage[f] = stage_value;
     }
+}
+
+// rows of feat picked by an id list (count on the device): out[r][:] = feat[ids[r]][:]
+__global__ void gather_feat_kernel(const float* __restrict__ feat, const uint32_t* __restrict__ ids,
+                                   const uint32_t* __restrict__ n_dev, uint32_t F4, float4* __restrict__ out)
+{
+    const uint32_t e = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t r = e / F4, c = e - r * F4;
+    if (r >= *n_dev) return;
+    out[e] = reinterpret_cast<const float4*>(feat)[(size_t)ids[r] * F4 + c];
+}
+
+// ids of the second list are positions in the first: out[r] = ids1[ids2_local[r]]
+__global__ void compose_ids_kernel(const uint32_t* __restrict__ ids1, const uint32_t* __restrict__ ids2_local,
+                                   const uint32_t* __restrict__ n_dev, uint32_t* __restrict__ out)
+{
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < *n_dev) out[r] = ids1[ids2_local[r]];
 }
 
 }  // namespace
@@ -222,6 +242,25 @@ int sf_launch_iota(uint32_t* out, uint32_t n, cudaStream_t st) {
     if (n == 0) return SF_OK;
     iota_kernel<<<(n + 255) / 256, 256, 0, st>>>(out, n);
     SF_LAUNCH_CHECK("iota_kernel");
+    return SF_OK;
+}
+
+int sf_launch_gather_feat(const float* feat, const uint32_t* ids, const uint32_t* n_dev, uint32_t n_max, uint32_t F,
+                          float* out, cudaStream_t st)
+{
+    if (n_max == 0) return SF_OK;
+    const uint32_t F4 = F / 4;
+    const size_t total = (size_t)n_max * F4;
+    gather_feat_kernel<<<(uint32_t)((total + 255) / 256), 256, 0, st>>>(feat, ids, n_dev, F4, reinterpret_cast<float4*>(out));
+    SF_LAUNCH_CHECK("gather_feat_kernel");
+    return SF_OK;
+}
+int sf_launch_compose_ids(const uint32_t* ids1, const uint32_t* ids2_local, const uint32_t* n_dev, uint32_t n_max,
+                          uint32_t* out, cudaStream_t st)
+{
+    if (n_max == 0) return SF_OK;
+    compose_ids_kernel<<<(n_max + 255) / 256, 256, 0, st>>>(ids1, ids2_local, n_dev, out);
+    SF_LAUNCH_CHECK("compose_ids_kernel");
     return SF_OK;
 }
 
@@ -250,7 +289,8 @@ size_t sf_route_scratch_bytes(uint32_t n) {
 
 int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,
                     const sf_packets* wide, uint32_t* esc_ids, uint32_t* n_esc, void* rows,
-                    uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st)
+                    uint8_t* decision, uint8_t* label_fast, float* score, void* scratch, cudaStream_t st,
+                    const uint32_t* n_dev)
 {
     const uint32_t nb = (n + kScoreBlock - 1) / kScoreBlock;
     uint32_t* block_counts = reinterpret_cast<uint32_t*>(scratch);
@@ -259,15 +299,15 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
     sf_time_begin(ctx, SF_T_SCORE, st);
     if (n > 0) {
         if (cfg->rule == SF_ABSMARGIN_LT)
-            score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts);
+            score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         else
-            score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts);
+            score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         SF_LAUNCH_CHECK("score_kernel");
     }
-    scan_kernel<<<1, 1024, 0, st>>>(block_counts, nb, n, cfg->capacity, n_esc, ctx->d_state);
+    scan_kernel<<<1, 1024, 0, st>>>(block_counts, nb, n, cfg->capacity, n_esc, ctx->d_state, n_dev);
     SF_LAUNCH_CHECK("scan_kernel");
     if (n > 0) {
-        scatter_kernel<<<nb, kScoreBlock, 0, st>>>(dec, n, block_counts, cfg->capacity, esc_ids);
+        scatter_kernel<<<nb, kScoreBlock, 0, st>>>(dec, n, block_counts, cfg->capacity, esc_ids, n_dev);
         SF_LAUNCH_CHECK("scatter_kernel");
     }
     sf_time_end(ctx, SF_T_SCORE, st);
@@ -292,15 +332,16 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
 
 int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t n, const uint32_t* esc_ids,
                     const uint32_t* n_esc, uint32_t capacity, const uint8_t* label_slow,
-                    uint8_t* label, uint8_t* stage, cudaStream_t st)
+                    uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value, bool write_fast)
 {
     if (n == 0) return SF_OK;
+    if (write_fast)
     merge_fast_kernel<<<(n + 255) / 256, 256, 0, st>>>(label_fast, decision, n, label, stage);
-    SF_LAUNCH_CHECK("merge_fast_kernel");
+    if (write_fast) SF_LAUNCH_CHECK("merge_fast_kernel");
     uint32_t blocks = (capacity + 255) / 256;
     if (blocks > 1184) blocks = 1184;
     if (blocks > 0) {
-        merge_slow_kernel<<<blocks, 256, 0, st>>>(esc_ids, n_esc, label_slow, label, stage, nullptr);
+        merge_slow_kernel<<<blocks, 256, 0, st>>>(esc_ids, n_esc, label_slow, label, stage, stage_value);
         SF_LAUNCH_CHECK("merge_slow_kernel");
     }
     return SF_OK;

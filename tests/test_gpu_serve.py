@@ -117,3 +117,49 @@ def test_c4_shapes_reduced_flow_count(env):
     sf, hz, ctx = env
     wl = make_workload(flowgen.get_config(4), n=5000)
     run_and_check(sf, hz, ctx, wl)
+
+
+@pytest.mark.parametrize("c,n", [(1, 3000), (2, 5000)])
+def test_three_tier_cascade(env, c, n):
+    """fastest (one decision tree) -> fast (forest) -> slow, per-class thresholds at both tiers."""
+    sf, hz, ctx = env
+    cfg = dataclasses.replace(flowgen.get_config(c), n=n)
+    wl = make_workload(cfg, n=n)
+    feat = oracle.extract_features(wl["fast"], cfg.N, cfg.F, threads=8)
+    fastest = flowgen.gen_forest(4242, "rf", 1, 7, cfg.F, cfg.C, feat)
+    rng = np.random.default_rng(c)
+    tau1 = rng.uniform(0.2, 0.7, cfg.C).astype(np.float32)
+    tau2 = (wl["tau"] + rng.uniform(-0.05, 0.05, cfg.C)).astype(np.float32)
+    ref = oracle.serve_batch3(cfg, wl["fast"], wl["wide"], fastest, wl["forest"], wl["slow"], tau1, tau2, threads=8)
+    tol = 2e-2 if cfg.slow_dtype == "bf16" else 1e-4
+    h1 = hz.make_forest(ctx, fastest); h2 = hz.make_forest(ctx, wl["forest"]); hs = hz.make_slow(ctx, cfg, wl["slow"])
+    fast_d = hz.upload_packets(wl["fast"], with_hdr=False); wide_d = hz.upload_packets(wl["wide"])
+    cfg1 = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau1), sf.SF_MLP16, sf.SF_BF16, cfg.P, n)
+    cfg2 = hz.route_cfg_for(cfg, hz.dev(tau2), n)
+    label = torch.full((n,), 255, dtype=torch.uint8, device="cuda")
+    stage = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.uint32, device="cuda")
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_serve_batch3(ctx, h1, h2, hs, fast_d["struct"], cfg.N, cfg.F, wide_d["struct"], cfg1, cfg2, label, stage, cnt)
+    torch.cuda.synchronize()
+    c_ = sf.sf_ctx_poll(ctx, reset=True)
+    k1, k2 = [int(x) for x in cnt.cpu().numpy()]
+    assert (k1, k2) == (len(ref["ids1"]), len(ref["ids2"])) and 0 < k2 < k1 < n
+    assert c_.device_error == 0 and c_.n_flows == n + k1 and c_.n_escalated == k1 + k2 and c_.n_slow_done == k2
+    st = stage.cpu().numpy(); lab = label.cpu().numpy()
+    assert np.array_equal(st, ref["stage"])
+    assert np.array_equal(lab[st < 3], ref["label_final"][st < 3])
+    p = sf.sf_serve_batch_intermediates(ctx)
+    assert np.array_equal(hz.ptr_tensor(p["esc_ids"], (k2,), torch.uint32).cpu().numpy(), ref["ids2"])
+    logits = hz.ptr_tensor(p["logits"], (k2, cfg.n_slow_classes), torch.float32).cpu().numpy()
+    assert np.max(np.abs(logits - ref["logits"])) <= tol
+    s = np.sort(ref["logits"], axis=1)
+    clear = (s[:, -1] - s[:, -2]) >= 2 * tol
+    assert np.array_equal(lab[ref["ids2"]][clear], ref["label_slow"][clear])
+    # with a cfg_fastest that lets nothing through the fastest model, every flow is stage 1
+    never = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(np.full(cfg.C, 2.0, np.float32)), sf.SF_MLP16, sf.SF_BF16, cfg.P, n)
+    sf.sf_serve_batch3(ctx, h1, h2, hs, fast_d["struct"], cfg.N, cfg.F, wide_d["struct"], never, cfg2, label, stage, cnt)
+    torch.cuda.synchronize()
+    assert cnt.cpu().numpy().tolist() == [0, 0] and bool((stage == 1).all())
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_slow_destroy(hs); sf.sf_forest_destroy(h2); sf.sf_forest_destroy(h1)
