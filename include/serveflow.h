@@ -48,6 +48,8 @@ extern "C" {
 #define SF_GBDT         1          /* boosted trees, binary logistic: sum of leaf scalars (margin) */
 #define SF_LC_GT        0          /* assign iff 1 - max_c prob[c] > tau[argmax]  (Sec. 3.2, least confidence) */
 #define SF_ABSMARGIN_LT 1          /* assign iff |margin| < tau[0]  (|p-0.5| < 0.2  <=>  |margin| < ln(7/3)) */
+#define SF_ENTROPY_GT   2          /* assign iff -sum_c prob[c] ln prob[c] > tau[argmax]  (Sec. 3.2, entropy; fp32 logf:
+                                      scores agree with a double-precision evaluation to about 1e-6, not bit for bit) */
 #define SF_MLP16        0          /* wide row = P packets x 16 fields */
 #define SF_CNN8         1          /* wide row = P positions x 8 channels (channels last) */
 #define SF_F32          0
@@ -157,7 +159,7 @@ int  sf_fast_infer(sf_ctx* ctx, const sf_forest* forest, const float* feat, uint
 
 /* ---- S3: uncertainty score, threshold, compaction, wide rows --------------- */
 typedef struct {
-    int rule;               /* SF_LC_GT | SF_ABSMARGIN_LT */
+    int rule;               /* SF_LC_GT | SF_ABSMARGIN_LT | SF_ENTROPY_GT */
     const float* tau;       /* device: fp32[C] per predicted class (all equal = universal threshold) for
                                SF_LC_GT; fp32[1] for SF_ABSMARGIN_LT */
     int wide_layout;        /* SF_MLP16 | SF_CNN8 */

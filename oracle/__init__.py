@@ -43,6 +43,7 @@ def lib():
         _lib.sfo_sigmoid.argtypes = [C.c_double]
         _lib.sfo_route_lc.restype = C.c_uint64
         _lib.sfo_route_absmargin.restype = C.c_uint64
+        _lib.sfo_route_entropy.restype = C.c_uint64
         _lib.sfo_ilog.restype = C.c_uint32
         _lib.sfo_ilog.argtypes = [C.c_uint32]
     return _lib
@@ -156,6 +157,19 @@ def route_lc(prob, tau):
     ids = np.empty(n, np.uint32)
     k = lib().sfo_route_lc(_p(prob), C.c_uint64(n), C.c_uint32(Cc), _p(tau), _p(score), _p(label),
                            _p(dec), _p(ids), C.c_uint64(n))
+    return {"score": score, "label": label, "decision": dec, "esc_ids": ids[:k].copy(), "n_esc": int(k)}
+
+
+def route_entropy(prob, tau):
+    prob = _c(prob, np.float32)
+    n, Cc = prob.shape
+    tau = _c(np.broadcast_to(np.asarray(tau, dtype=np.float32), (Cc,)), np.float32)
+    score = np.empty(n, np.float32)
+    label = np.empty(n, np.uint8)
+    dec = np.empty(n, np.uint8)
+    ids = np.empty(n, np.uint32)
+    k = lib().sfo_route_entropy(_p(prob), C.c_uint64(n), C.c_uint32(Cc), _p(tau), _p(score), _p(label),
+                                _p(dec), _p(ids), C.c_uint64(n))
     return {"score": score, "label": label, "decision": dec, "esc_ids": ids[:k].copy(), "n_esc": int(k)}
 
 

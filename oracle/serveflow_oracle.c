@@ -243,6 +243,27 @@ uint64_t sfo_route_lc(const float* prob, uint64_t n, uint32_t C, const float* ta
     return k;
 }
 
+/* Entropy rule (Sec. 3.2): score H(x) = -sum_i P(y_i|x) log P(y_i|x), evaluated in double and
+ * stored as fp32; label = argmax; assigned iff H > tau[label] (strict). */
+uint64_t sfo_route_entropy(const float* prob, uint64_t n, uint32_t C, const float* tau,
+                           float* score, uint8_t* label, uint8_t* decision,
+                           uint32_t* esc_ids, uint64_t capacity)
+{
+    uint64_t k = 0;
+    for (uint64_t f = 0; f < n; f++) {
+        const float* p = prob + f * C;
+        uint32_t a = 0;
+        for (uint32_t c = 1; c < C; c++) if (p[c] > p[a]) a = c;
+        float h = (float)sfo_entropy(p, C);
+        int esc = h > tau[a];
+        if (score) score[f] = h;
+        if (label) label[f] = (uint8_t)a;
+        if (decision) decision[f] = (uint8_t)esc;
+        if (esc) { if (esc_ids && k < capacity) esc_ids[k] = (uint32_t)f; k++; }
+    }
+    return k;
+}
+
 /* Binary boosted rule, taken in margin space: |p - 0.5| < 0.2 with p =
  * sigmoid(margin) is the same set as |margin| < ln(0.7/0.3) because the sigmoid
  * is monotone and odd about (0, 0.5).  score = |margin|, label = margin > 0,

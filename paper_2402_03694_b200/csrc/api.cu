@@ -211,7 +211,8 @@ int check_serve_args(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const s
     if (N < 1 || N > 32 || N > fast->pitch_pkts) return SF_ERR_ARG;
     if (F != fo->F || F < 8 || F > 64 || F % 8) return SF_ERR_ARG;
     if (wide->n_flows < fast->n_flows) return SF_ERR_ARG;
-    if (cfg->rule == SF_LC_GT && fo->kind != SF_RF) return SF_ERR_ARG;
+    if ((cfg->rule == SF_LC_GT || cfg->rule == SF_ENTROPY_GT) && fo->kind != SF_RF) return SF_ERR_ARG;
+    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ENTROPY_GT && cfg->rule != SF_ABSMARGIN_LT) return SF_ERR_ARG;
     if (cfg->rule == SF_ABSMARGIN_LT && fo->kind != SF_GBDT) return SF_ERR_ARG;
     const uint32_t W = cfg->wide_layout == SF_MLP16 ? 16u : 8u;
     if (cfg->wide_layout != SF_MLP16 && cfg->wide_layout != SF_CNN8) return SF_ERR_ARG;

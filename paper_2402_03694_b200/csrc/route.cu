@@ -35,7 +35,14 @@ score_kernel(const float* __restrict__ fast_out, uint32_t n, uint32_t C, const f
             const float* p = fast_out + (size_t)f * C;
             float mx = p[0]; a = 0;
             for (uint32_t c = 1; c < C; c++) { float v = p[c]; if (v > mx) { mx = v; a = c; } }
-            u = __fsub_rn(1.0f, mx);
+            if (RULE == SF_ENTROPY_GT) {
+                // H = -sum p ln p (Sec. 3.2); fp32 logf, so this score is compared by tolerance, not bit for bit
+                float h = 0.0f;
+                for (uint32_t c = 0; c < C; c++) { float v = p[c]; if (v > 0.0f) h -= v * logf(v); }
+                u = h;
+            } else {
+                u = __fsub_rn(1.0f, mx);
+            }
             esc = u > __ldg(tau + a);
         }
         if (decision) decision[f] = esc ? 1 : 0;
@@ -231,6 +238,8 @@ int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, 
     if (nb == 0) return SF_OK;
     if (cfg->rule == SF_ABSMARGIN_LT)
         score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
+    else if (cfg->rule == SF_ENTROPY_GT)
+        score_kernel<SF_ENTROPY_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
     else
         score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
     SF_LAUNCH_CHECK("score_kernel");
@@ -300,6 +309,8 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
     if (n > 0) {
         if (cfg->rule == SF_ABSMARGIN_LT)
             score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
+        else if (cfg->rule == SF_ENTROPY_GT)
+            score_kernel<SF_ENTROPY_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         else
             score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         SF_LAUNCH_CHECK("score_kernel");
@@ -352,8 +363,8 @@ extern "C" int sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_
                         uint8_t* decision_out, uint8_t* label_fast_out, float* score_out, void* stream)
 {
     if (!ctx || !cfg || !fast_out || !esc_ids_out || !n_esc_out || !cfg->tau) return SF_ERR_ARG;
-    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT) return SF_ERR_ARG;
-    if (cfg->rule == SF_LC_GT && (C < 1 || C > 256)) return SF_ERR_ARG;
+    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT && cfg->rule != SF_ENTROPY_GT) return SF_ERR_ARG;
+    if (cfg->rule != SF_ABSMARGIN_LT && (C < 1 || C > 256)) return SF_ERR_ARG;
     if (rows_out) {
         if (!wide || !wide->size || !wide->iat_us || !wide->dir_bits || !wide->hdr) return SF_ERR_ARG;
         if (cfg->wide_layout != SF_MLP16 && cfg->wide_layout != SF_CNN8) return SF_ERR_ARG;

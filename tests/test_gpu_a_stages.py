@@ -367,3 +367,29 @@ def test_cnn_within_tolerance(env, n_rows, cap, n_cls):
     logits2, label2 = _run_slow(sf, hz, ctx, h, rt, n_rows, cap, n_cls)      # run-to-run identical bits
     assert np.array_equal(logits[:n_rows], logits2[:n_rows]) and np.array_equal(label[:n_rows], label2[:n_rows])
     sf.sf_slow_destroy(h)
+
+
+def test_route_entropy_within_tolerance(env):
+    """Entropy score (Sec. 3.2): fp32 logf on the device against the double-precision oracle."""
+    sf, hz, ctx = env
+    n, C = 20011, 8
+    rng = np.random.default_rng(23)
+    prob = rng.dirichlet([0.5] * C, size=n).astype(np.float32)
+    prob[3] = 0; prob[3, 1] = 1.0
+    tau = rng.uniform(0.6, 1.4, C).astype(np.float32)
+    ref = oracle.route_entropy(prob, tau)
+    cfg = sf.make_route_cfg(sf.SF_ENTROPY_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, 64, n)
+    ids = torch.zeros(n, dtype=torch.uint32, device="cuda"); n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    dec = torch.empty(n, dtype=torch.uint8, device="cuda"); lab = torch.empty(n, dtype=torch.uint8, device="cuda")
+    sc = torch.empty(n, dtype=torch.float32, device="cuda")
+    sf.sf_route(ctx, cfg, hz.dev(prob), n, C, None, ids, n_esc, None, dec, lab, sc)
+    torch.cuda.synchronize()
+    sf.sf_ctx_poll(ctx, reset=True)
+    score = sc.cpu().numpy(); d = dec.cpu().numpy()
+    assert np.max(np.abs(score - ref["score"])) <= 2e-6 and score[3] == 0.0
+    assert np.array_equal(lab.cpu().numpy(), ref["label"])
+    away = np.abs(ref["score"] - tau[ref["label"]]) > 1e-5
+    assert np.array_equal(d[away], ref["decision"][away])
+    k = int(n_esc.cpu().numpy()[0])
+    assert k == int(d.sum()) and np.array_equal(ids.cpu().numpy()[:k], np.nonzero(d)[0])      # the list is consistent with its own decisions
+    assert abs(k - ref["n_esc"]) <= int((~away).sum())

@@ -229,3 +229,24 @@ def test_merge():
     lf = np.array([1, 2, 3, 0, 1], np.uint8)
     label, stage = oracle.merge(lf, np.array([1, 4], np.uint32), np.array([7, 9], np.uint8))
     assert label.tolist() == [1, 7, 3, 0, 9] and stage.tolist() == [1, 2, 1, 1, 2]
+
+
+def test_entropy_rule_matches_direct_evaluation():
+    rng = np.random.default_rng(21)
+    p = rng.dirichlet([0.5] * 6, size=3000).astype(np.float32)
+    p[0] = 0; p[0, 2] = 1.0                                   # a certain prediction: H = 0
+    tau = rng.uniform(0.4, 1.2, 6).astype(np.float32)
+    r = oracle.route_entropy(p, tau)
+    pd = p.astype(np.float64)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        h = -np.where(pd > 0, pd * np.log(pd), 0.0).sum(1)     # Sec. 3.2
+    assert np.allclose(r["score"], h, atol=1e-6) and r["score"][0] == 0.0
+    lab = p.argmax(1)
+    assert np.array_equal(r["label"], lab)
+    away = np.abs(h - tau[lab]) > 1e-5
+    assert np.array_equal(r["decision"].astype(bool)[away], (h > tau[lab])[away])
+    assert r["n_esc"] == int(r["decision"].sum()) and np.array_equal(r["esc_ids"], np.nonzero(r["decision"])[0])
+    # entropy and least confidence order two-class predictions the same way
+    q = np.stack([np.linspace(0.5, 0.99, 50), 1 - np.linspace(0.5, 0.99, 50)], 1).astype(np.float32)
+    he = oracle.route_entropy(q, 9.0)["score"]; lc = oracle.route_lc(q, 9.0)["score"]
+    assert np.all(np.diff(he) < 0) and np.all(np.diff(lc) < 0)
