@@ -396,7 +396,9 @@ int sf_cnn_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
                         float* logits, uint8_t* label, void* scratch, cudaStream_t st)
 {
     (void)scratch;
-    SF_CUDA(cudaFuncSetAttribute(cnn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL));
+    static bool attr_set_dev[64] = {};                 // the opt-in is per device
+    bool& attr_set = attr_set_dev[ctx->device & 63];
+    if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(cnn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL)); attr_set = true; }
     uint32_t grid = (uint32_t)ctx->num_sms < capacity ? (uint32_t)ctx->num_sms : capacity;
     sf_time_begin(ctx, SF_T_GEMM, st);
     cnn_fused_kernel<<<grid, kThreads, SM_TOTAL, st>>>(reinterpret_cast<const __nv_bfloat16*>(rows), n_rows_dev,

@@ -214,8 +214,10 @@ struct Plan { uint32_t chunk_bytes, tpc, nch; size_t smem; };
 Plan make_plan(const sf_forest* fo) {
     Plan p;
     const size_t feat_bytes = (size_t)fo->F * kB * sizeof(float);
-    p.chunk_bytes = (feat_bytes + 2 * 65536 + 32 <= kMaxSmem) ? 65536u : 32768u;
-    p.tpc = p.chunk_bytes / fo->tree_stride;          // >= 1: a depth-12 tree is 32 KB
+    // two chunk buffers share what the feature tile leaves of the 227 KB: up to 64 KB each
+    const uint32_t avail = (uint32_t)(((kMaxSmem - feat_bytes - 32) / 2) & ~(size_t)15);
+    p.chunk_bytes = avail < 65536u ? avail : 65536u;
+    p.tpc = p.chunk_bytes / fo->tree_stride;          // 0 if one tree does not fit (checked by the callers)
     if (p.tpc > fo->T) p.tpc = fo->T;
     p.nch = (fo->kind == SF_GBDT) ? (p.tpc >= 4 ? 4u : (p.tpc >= 2 ? 2u : 1u)) : (p.tpc >= 2 ? 2u : 1u);
     p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes + 32;       // + two mbarriers and the abort flag
@@ -225,7 +227,12 @@ Plan make_plan(const sf_forest* fo) {
 template <int KIND, int C, int NCH>
 int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     auto k = forest_kernel<KIND, C, NCH>;
-    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
+    static size_t smem_set_dev[64] = {};               // per kernel instance and device: raise the opt-in limit only when it grows
+    size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
+    if (p.smem > smem_set) {
+        SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
+        smem_set = p.smem;
+    }
     const uint32_t grid = (n + kB - 1) / kB;
     k<<<grid, kB, p.smem, st>>>(feat, n, fo->F, fo->d_image, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
                                 p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev);
@@ -236,12 +243,14 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
 template <int C>
 int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     const Plan p = make_plan(fo);
+    if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
     if (p.nch == 2) return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
     return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
 int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     const Plan p = make_plan(fo);
+    if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
     if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st, n_dev);
     if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
     return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);

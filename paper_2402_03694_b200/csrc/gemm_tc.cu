@@ -257,7 +257,9 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
     if (rc != SF_OK) return rc;
     auto k = gemm_bias_relu_bf16_kernel<BN, false>;
-    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes));
+    static bool attr_set_dev[64] = {};                 // the opt-in is per device
+    bool& attr_set = attr_set_dev[ctx->device & 63];
+    if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
     uint32_t max_tiles = ((capacity + BM - 1) / BM) * (N / BN);
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
@@ -277,7 +279,9 @@ int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bia
     rc = encode_tmap_bf16_2d(&tmW, W16, 16, K, 16, BK);
     if (rc != SF_OK) return rc;
     auto k = gemm_bias_relu_bf16_kernel<16, true>;
-    SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes));
+    static bool attr_set_dev[64] = {};                 // the opt-in is per device
+    bool& attr_set = attr_set_dev[ctx->device & 63];
+    if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
     uint32_t max_tiles = (capacity + BM - 1) / BM;
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C);

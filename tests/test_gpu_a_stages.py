@@ -89,6 +89,9 @@ def _features(n, N, F, seed):
     ("rf", 5, 3, 8, 3, 600),         # class count that is not a multiple of 4
     ("gbdt", 70, 6, 32, 2, 5001),    # 64 trees per chunk + a ragged second chunk
     ("gbdt", 3, 1, 8, 2, 33),
+    ("rf", 5, 12, 64, 16, 700),      # largest shapes: 128 KB feature tile, one 32 KB tree per chunk
+    ("gbdt", 4, 12, 64, 2, 900),     # 48 KB tree images (nodes + leaves) next to the 128 KB tile
+    ("rf", 33, 2, 24, 4, 513),       # many trees per chunk, odd count (ragged group), one flow past a block
 ])
 def test_forest_bit_exact(env, kind, T, d, F, C, n):
     sf, hz, ctx = env

@@ -163,3 +163,30 @@ def test_three_tier_cascade(env, c, n):
     assert cnt.cpu().numpy().tolist() == [0, 0] and bool((stage == 1).all())
     sf.sf_ctx_poll(ctx, reset=True)
     sf.sf_slow_destroy(hs); sf.sf_forest_destroy(h2); sf.sf_forest_destroy(h1)
+
+
+def test_empty_batch_and_nothing_assigned(env):
+    sf, hz, ctx = env
+    cfg = dataclasses.replace(flowgen.get_config(1), n=700)
+    wl = make_workload(cfg, n=700)
+    forest = hz.make_forest(ctx, wl["forest"]); slow = hz.make_slow(ctx, cfg, wl["slow"])
+    fast_d = hz.upload_packets(wl["fast"], with_hdr=False); wide_d = hz.upload_packets(wl["wide"])
+    label = torch.full((700,), 255, dtype=torch.uint8, device="cuda"); stage = torch.zeros(700, dtype=torch.uint8, device="cuda")
+    n_esc = torch.full((1,), 7, dtype=torch.uint32, device="cuda")
+    # thresholds nobody exceeds: the slow model sees zero rows and every flow keeps its fast answer
+    never = hz.route_cfg_for(cfg, hz.dev(np.full(cfg.C, 2.0, np.float32)), 700)
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_serve_batch(ctx, forest, slow, fast_d["struct"], cfg.N, cfg.F, wide_d["struct"], never, label, stage, n_esc)
+    torch.cuda.synchronize()
+    ref = oracle.route_lc(oracle.forest_infer(wl["forest"], oracle.extract_features(wl["fast"], cfg.N, cfg.F)), 2.0)
+    assert int(n_esc.cpu().numpy()[0]) == 0 and bool((stage == 1).all()) and np.array_equal(label.cpu().numpy(), ref["label"])
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert c.device_error == 0 and c.n_slow_done == 0 and c.n_fast_done == 700
+    # an empty batch is accepted and touches nothing
+    fast0 = sf.make_packets(fast_d["size"], fast_d["iat_us"], fast_d["dir_bits"], None, None, n_flows=0)
+    wide0 = sf.make_packets(wide_d["size"], wide_d["iat_us"], wide_d["dir_bits"], wide_d["hdr"], None, n_flows=0)
+    zero_cap = hz.route_cfg_for(cfg, hz.dev(wl["tau"]), 0)
+    sf.sf_serve_batch(ctx, forest, slow, fast0, cfg.N, cfg.F, wide0, zero_cap, label, stage, n_esc)
+    torch.cuda.synchronize()
+    assert int(n_esc.cpu().numpy()[0]) == 0 and sf.sf_ctx_poll(ctx, reset=True).device_error == 0
+    sf.sf_slow_destroy(slow); sf.sf_forest_destroy(forest)
