@@ -72,3 +72,17 @@ def fast_view(wide, N):
         "dir_bits": d,
         "hdr": np.ascontiguousarray(wide["hdr"][:, :N]),
     }
+
+
+def gen_first_packet_headers(seed, n):
+    """Synthetic first-packet header bytes: [n][128] = IPv4 (60) | TCP (60) | UDP (8), and the number
+    of bytes present in each section: IPv4 20..60 in steps of 4; 70 % TCP (20..60 in steps of 4, no UDP),
+    30 % UDP (8 bytes, no TCP).  Bytes beyond a section's length are filled with noise on purpose
+    (a reader must mask them by the lengths)."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence(int(seed) + 80_000)))
+    b = rng.integers(0, 256, size=(n, 128), dtype=np.uint8)
+    ip_len = (20 + 4 * rng.integers(0, 11, size=n)).astype(np.uint8)
+    is_tcp = rng.random(n) < 0.7
+    tcp_len = np.where(is_tcp, 20 + 4 * rng.integers(0, 11, size=n), 0).astype(np.uint8)
+    udp_len = np.where(is_tcp, 0, 8).astype(np.uint8)
+    return b, np.stack([ip_len, tcp_len, udp_len], axis=1).astype(np.uint8)

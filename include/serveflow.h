@@ -140,6 +140,16 @@ typedef struct {
 int  sf_extract_features(sf_ctx* ctx, const sf_packets* pk, uint32_t N, uint32_t F,
                          float* feat_out, void* stream);
 
+/* First-packet header-bit features (Sec. 4.1 and 4.4: 1024 header bits per packet from the
+ * IPv4, TCP and UDP headers, with a subscription to a subset of the columns).  bytes:
+ * uint8[n][128] = IPv4 header bytes 0..59 | TCP header bytes 0..59 | UDP header bytes 0..7
+ * (16-byte aligned); sec_len: uint8[n][3] = bytes present in each section; sub: uint16[m]
+ * (device), column indices 0..1023, m <= 1024.  Column i is bit (7 - i%8) of byte i/8;
+ * out fp32[n][m]: -1 if that byte is not present, else 0 or 1.  With m <= 64 the rows can go
+ * straight into sf_fast_infer as the features of a first-packet model. */
+int  sf_header_bits(sf_ctx* ctx, const uint8_t* bytes, const uint8_t* sec_len, uint32_t n,
+                    const uint16_t* sub, uint32_t m, float* out, void* stream);
+
 /* ---- S2: fast model (tree ensemble) ---------------------------------------- */
 /* Builds an ensemble of T complete binary trees of depth `depth` (heap order:
  * children of node i are 2i+1, 2i+2) from HOST arrays fid uint16[T][2^d-1],

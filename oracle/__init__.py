@@ -120,6 +120,16 @@ def extract_features(pk, N, F, n_valid=None, threads=1):
     return feat
 
 
+def header_bits(bytes128, sec_len, sub):
+    """Subscribed columns of the 1024 first-packet header bits as -1 / 0 / 1."""
+    b = _c(bytes128, np.uint8); sl = _c(sec_len, np.uint8); sub = _c(sub, np.uint16)
+    n = b.shape[0]
+    assert b.shape[1] == 128 and sl.shape == (n, 3)
+    out = np.empty((n, sub.shape[0]), np.float32)
+    lib().sfo_header_bits(_p(b), _p(sl), C.c_uint64(n), _p(sub), C.c_uint32(sub.shape[0]), _p(out))
+    return out
+
+
 def forest_infer(forest, feat, want_leaf_idx=False, threads=1):
     feat = _c(feat, np.float32)
     n, F = feat.shape

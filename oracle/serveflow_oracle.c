@@ -142,6 +142,27 @@ void sfo_extract_features(const uint16_t* size, const uint32_t* iat_us, const ui
     }
 }
 
+/* First-packet header-bit features (Sec. 4.1, Sec. 4.4: 1024 header bits per packet from the
+ * IPv4, TCP and UDP headers, with a subscription to a subset of the columns).
+ * Reading (the bit layout is re-derived from the header sizes, not taken from any tool): a
+ * packet row holds 128 bytes = IPv4 header bytes 0..59, TCP header bytes 0..59, UDP header
+ * bytes 0..7; column i of the 1024 is bit (7 - i%8) of byte i/8 (network bit order).  A column
+ * whose byte lies at or beyond the number of bytes present in its section (sec_len[3]: a
+ * 20-byte IPv4 header has no option bytes, a UDP packet has no TCP section) is -1; otherwise
+ * it is 0 or 1.  Only the subscribed columns are written: out[f][j] = column sub[j]. */
+void sfo_header_bits(const uint8_t* bytes, const uint8_t* sec_len, uint64_t n, const uint16_t* sub, uint32_t m,
+                     float* out)
+{
+    static const uint32_t sec_start[3] = {0, 60, 120};
+    for (uint64_t f = 0; f < n; f++)
+        for (uint32_t j = 0; j < m; j++) {
+            uint32_t col = sub[j], byte = col / 8, bit = 7 - col % 8;
+            uint32_t sec = byte < 60 ? 0 : (byte < 120 ? 1 : 2);
+            if (byte - sec_start[sec] >= sec_len[f * 3 + sec]) out[f * m + j] = -1.0f;
+            else out[f * m + j] = (float)((bytes[f * 128 + byte] >> bit) & 1u);
+        }
+}
+
 /* ------------------------------------------------------------------------- */
 /* S2: tree ensembles                                                        */
 /* ------------------------------------------------------------------------- */

@@ -81,7 +81,7 @@ FLOW_RESULT_DTYPE = np.dtype([("found", "u1"), ("stage", "u1"), ("label_fast", "
 EXPORTS = [
     "sf_strerror", "sf_last_cuda_error", "sf_version", "sf_ctx_create", "sf_ctx_destroy", "sf_ctx_poll",
     "sf_ctx_set_timing", "sf_ctx_get_timing",
-    "sf_extract_features", "sf_forest_create", "sf_forest_destroy", "sf_fast_infer", "sf_route",
+    "sf_extract_features", "sf_header_bits", "sf_forest_create", "sf_forest_destroy", "sf_fast_infer", "sf_route",
     "sf_route_noalloc",
     "sf_universal_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
     "sf_serve_batch", "sf_serve_batch3", "sf_serve_batch_host", "sf_serve_batch_intermediates",
@@ -112,6 +112,7 @@ def _lib():
         L.sf_ctx_set_timing.argtypes = [V, I]
         L.sf_ctx_get_timing.argtypes = [V, U32, V, V]
         L.sf_extract_features.argtypes = [V, C.POINTER(sf_packets), U32, U32, V, V]
+        L.sf_header_bits.argtypes = [V, V, V, U32, V, U32, V, V]
         L.sf_forest_create.argtypes = [V, I, U32, U32, U32, U32, V, V, V, C.POINTER(V)]
         L.sf_fast_infer.argtypes = [V, V, V, U32, V, V, V]
         L.sf_route.argtypes = [V, C.POINTER(sf_route_cfg), V, U32, U32, C.POINTER(sf_packets), V, V, V, V, V, V, V]
@@ -217,6 +218,11 @@ def sf_ctx_get_timing(ctx, back=0, stream=None):
 
 def sf_extract_features(ctx, pk, N, F, feat_out, stream=None):
     _check(_lib().sf_extract_features(ctx, C.byref(pk), N, F, _dp(feat_out), _stream(stream)), "sf_extract_features")
+
+
+def sf_header_bits(ctx, bytes128, sec_len, n, sub, m, out, stream=None):
+    _check(_lib().sf_header_bits(ctx, _dp(bytes128), _dp(sec_len), n, _dp(sub), m, _dp(out), _stream(stream)),
+           "sf_header_bits")
 
 
 def sf_forest_create(ctx, kind, T, depth, F, Cn, fid, thr, leaf):

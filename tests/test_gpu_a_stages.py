@@ -396,3 +396,24 @@ def test_route_entropy_within_tolerance(env):
     k = int(n_esc.cpu().numpy()[0])
     assert k == int(d.sum()) and np.array_equal(ids.cpu().numpy()[:k], np.nonzero(d)[0])      # the list is consistent with its own decisions
     assert abs(k - ref["n_esc"]) <= int((~away).sum())
+
+
+# ------------------------------------------------------- first-packet header bits ---
+@pytest.mark.parametrize("n,m", [(5000, 64), (77, 1024), (1, 1), (130, 37)])
+def test_header_bits_bit_exact_and_feed_a_first_packet_tree(env, n, m):
+    sf, hz, ctx = env
+    b, sl = flowgen.gen_first_packet_headers(31 + n, n)
+    rng = np.random.default_rng(m)
+    sub = np.sort(rng.choice(1024, size=m, replace=False)).astype(np.uint16)
+    ref = oracle.header_bits(b, sl, sub)
+    out = torch.full((n, m), 9.0, dtype=torch.float32, device="cuda")
+    sf.sf_header_bits(ctx, hz.dev(b), hz.dev(sl), n, hz.dev(sub), m, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), ref)
+    if m == 64:        # the paper's fastest model: one decision tree on first-packet bits
+        fo = flowgen.gen_forest(55, "rf", 1, 8, 64, 4, ref)
+        h = hz.make_forest(ctx, fo)
+        p = torch.empty((n, 4), dtype=torch.float32, device="cuda")
+        sf.sf_fast_infer(ctx, h, out, n, p)
+        assert np.array_equal(bits(p.cpu().numpy()), bits(oracle.forest_infer(fo, ref)))
+        sf.sf_forest_destroy(h)

@@ -181,3 +181,26 @@ def test_pitch_larger_than_window():
     a = oracle.extract_features(w, 8, 24)                       # pitch 64, window 8
     b = oracle.extract_features(flowgen.fast_view(w, 8), 8, 24)  # pitch 8
     assert np.array_equal(a, b)
+
+
+def test_header_bits_hand_example_and_masks():
+    """First-packet header bits (Sec. 4.1): hand-built rows."""
+    b = np.zeros((3, 128), np.uint8)
+    sl = np.array([[20, 20, 0], [24, 0, 8], [60, 60, 8]], np.uint8)
+    b[0, 0] = 0x45                      # version 4, IHL 5: bits 0100 0101
+    b[0, 9] = 6                         # protocol TCP: 0000 0110 -> columns 72..79
+    b[0, 60 + 13] = 0x12                # TCP flags SYN+ACK at TCP byte 13: 0001 0010
+    b[1, 120 + 2] = 0x80                # first bit of UDP byte 2
+    b[1, 30] = 0xFF                     # noise beyond the 24-byte IPv4 header: must be masked
+    sub = np.array([0, 1, 2, 3, 4, 5, 6, 7, 77, 78, 79, 480 + 13 * 8 + 3, 480 + 13 * 8 + 6, 960 + 16, 240, 20 * 8 - 1, 20 * 8, 1023], np.uint16)
+    o = oracle.header_bits(b, sl, sub)
+    assert o[0].tolist() == [0, 1, 0, 0, 0, 1, 0, 1,  1, 1, 0,  1, 1,  -1,  -1, 0, -1, -1]
+    assert o[1, 13] == 1 and o[1, 14] == -1 and o[1, 11] == -1       # UDP present, byte 30 masked, no TCP section
+    assert o[1, 15] == 0 and o[1, 16] == 0                           # bytes 19 and 20 are inside a 24-byte header
+    assert not np.any(o[2] == -1)                                    # everything present
+    # all 1024 columns: the count of -1 columns follows from the lengths; present bits reproduce the bytes
+    bb, ll = flowgen.gen_first_packet_headers(5, 200)
+    full = oracle.header_bits(bb, ll, np.arange(1024, dtype=np.uint16))
+    assert np.array_equal((full == -1).sum(1), 8 * (128 - ll.astype(np.int64).sum(1)))
+    bits = np.unpackbits(bb, axis=1).astype(np.float32)              # numpy unpacks MSB first
+    assert np.array_equal(full[full >= 0], bits[full >= 0])
