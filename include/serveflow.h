@@ -234,6 +234,32 @@ int  sf_route_noalloc(int device, const sf_route_cfg* cfg, const float* prob_or_
 int  sf_universal_thresholds(const float* scores_host, uint64_t n, const uint32_t* q_num_host,
                              uint32_t q_den, uint32_t n_q, float* thresholds_host_out);
 
+/* Algorithm 1 on DEVICE scores (float32[n], no NaNs): a stable radix sort of the scores on the
+ * device, then the same 1-based pick ceil(q*n) per quantile; tau_out is a DEVICE float32[n_q]
+ * (n_q <= 64), so it can be handed to sf_route_cfg.tau without a host round trip.  q_num is a
+ * host array.  Uses the context's workspace (may grow it, synchronising); asynchronous on
+ * `stream` otherwise.  Scores compare as IEEE values with -0 before +0. */
+int  sf_universal_thresholds_dev(sf_ctx* ctx, const float* scores, uint32_t n, const uint32_t* q_num_host,
+                                 uint32_t q_den, uint32_t n_q, float* tau_out, void* stream);
+
+/* Algorithm 2 (slope-based per-class uncertainty thresholds, Sec. 3.2) on a validation batch
+ * that lives on the device: scores float32[n], label uint8[n] = the fast model's predicted
+ * class (< C <= 256), correct uint8[n] = 1 where that prediction was right.  Reading of the
+ * outline the paper gives: per predicted class the candidate thresholds are the quantiles
+ * (Q-k)/Q, k = 1..Q (Q <= 1000), of that class's scores by Algorithm 1's pick; a step's slope
+ * is (newly assigned incorrect flows) / (newly assigned flows), steps that assign nothing
+ * new are dropped; thresholds start at each class's maximum and, while fewer than
+ * floor(a_num/a_den * n) validation flows are assigned, the steepest next step over all
+ * classes is taken (fractions compared exactly; ties: the larger step, then the lower
+ * class).  A class with no validation flow gets the global maximum score.
+ * The device sorts (class, score) keys, picks the thresholds and counts the flows between
+ * them; the selection over the <= C*Q steps runs on the host.  tau_host_out: float32[C];
+ * assigned_host_out (nullable): validation flows with score > tau[label].  Synchronises
+ * `stream`. */
+int  sf_per_class_thresholds(sf_ctx* ctx, const float* scores, const uint8_t* label, const uint8_t* correct,
+                             uint32_t n, uint32_t C, uint32_t Q, uint32_t a_num, uint32_t a_den,
+                             float* tau_host_out, uint64_t* assigned_host_out, void* stream);
+
 /* ---- S4: slow model -------------------------------------------------------- */
 /* MLP h_{k+1} = ReLU(W_k h_k + b_k), logits = W_L h_L + b_L.  dims_host has
  * n_layers+1 entries; W_host[k] is fp32 [dims[k+1]][dims[k]] (HOST), b_host[k]

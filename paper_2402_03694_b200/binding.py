@@ -83,7 +83,7 @@ EXPORTS = [
     "sf_ctx_set_timing", "sf_ctx_get_timing",
     "sf_extract_features", "sf_header_bits", "sf_forest_create", "sf_forest_destroy", "sf_fast_infer", "sf_route",
     "sf_route_noalloc",
-    "sf_universal_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
+    "sf_universal_thresholds", "sf_universal_thresholds_dev", "sf_per_class_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
     "sf_serve_batch", "sf_serve_batch3", "sf_serve_batch_host", "sf_serve_batch_intermediates",
     "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_lookup",
 ]
@@ -118,6 +118,8 @@ def _lib():
         L.sf_route.argtypes = [V, C.POINTER(sf_route_cfg), V, U32, U32, C.POINTER(sf_packets), V, V, V, V, V, V, V]
         L.sf_route_noalloc.argtypes = [I, C.POINTER(sf_route_cfg), V, U32, U32, V, V, V, V, V, V, V]
         L.sf_universal_thresholds.argtypes = [V, C.c_uint64, V, U32, U32, V]
+        L.sf_universal_thresholds_dev.argtypes = [V, V, U32, V, U32, U32, V, V]
+        L.sf_per_class_thresholds.argtypes = [V, V, V, V, U32, U32, U32, U32, U32, V, V, V]
         L.sf_mlp_create.argtypes = [V, I, U32, V, C.POINTER(V), C.POINTER(V), C.POINTER(V)]
         L.sf_cnn_create.argtypes = [V, I, U32, U32, U32, U32, U32, U32, V, V, V, V, V, V, C.POINTER(V)]
         L.sf_slow_infer.argtypes = [V, V, V, V, U32, V, V, V]
@@ -267,6 +269,20 @@ def sf_universal_thresholds(scores, q_num, q_den=100):
     _check(_lib().sf_universal_thresholds(scores.ctypes.data, scores.shape[0], q.ctypes.data, q_den, q.shape[0],
                                           out.ctypes.data), "sf_universal_thresholds")
     return out
+
+
+def sf_universal_thresholds_dev(ctx, scores, n, q_num, q_den, tau_out, stream=None):
+    q = np.ascontiguousarray(np.atleast_1d(q_num), np.uint32)
+    _check(_lib().sf_universal_thresholds_dev(ctx, _dp(scores), n, q.ctypes.data, q_den, q.shape[0], _dp(tau_out),
+                                              _stream(stream)), "sf_universal_thresholds_dev")
+
+
+def sf_per_class_thresholds(ctx, scores, label, correct, n, n_classes, Q, a_num, a_den, stream=None):
+    tau = np.empty(n_classes, np.float32)
+    assigned = C.c_uint64(0)
+    _check(_lib().sf_per_class_thresholds(ctx, _dp(scores), _dp(label), _dp(correct), n, n_classes, Q, a_num, a_den,
+                                          tau.ctypes.data, C.addressof(assigned), _stream(stream)), "sf_per_class_thresholds")
+    return tau, int(assigned.value)
 
 
 def sf_mlp_create(ctx, dtype, dims, W, b):

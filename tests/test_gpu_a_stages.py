@@ -417,3 +417,48 @@ def test_header_bits_bit_exact_and_feed_a_first_packet_tree(env, n, m):
         sf.sf_fast_infer(ctx, h, out, n, p)
         assert np.array_equal(bits(p.cpu().numpy()), bits(oracle.forest_infer(fo, ref)))
         sf.sf_forest_destroy(h)
+
+
+# ------------------------------------------------------- threshold calibration on the device ---
+@pytest.mark.parametrize("n", [1, 255, 4096, 4097, 300007])
+def test_algorithm_1_on_device_scores(env, n):
+    sf, hz, ctx = env
+    rng = np.random.default_rng(n)
+    u = rng.random(n).astype(np.float32)
+    u[rng.integers(0, n, n // 3)] = np.float32(0.25)            # many ties
+    if n > 10:
+        u[:5] = [0.0, 1.0, 3e38, 1e-40, 0.5]                    # zero, a huge value, a subnormal
+    q = [0, 1, 50, 75, 76, 99, 100]
+    ref = oracle.universal_thresholds(u, q)
+    tau = torch.zeros(len(q), dtype=torch.float32, device="cuda")
+    sf.sf_universal_thresholds_dev(ctx, hz.dev(u), n, q, 100, tau)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(tau.cpu().numpy()), bits(ref))
+    assert np.array_equal(bits(sf.sf_universal_thresholds(u, q)), bits(ref))
+
+
+def test_algorithm_1_on_device_orders_negative_scores(env):
+    sf, hz, ctx = env
+    u = np.random.default_rng(5).normal(size=20000).astype(np.float32)
+    ref = oracle.universal_thresholds(u, [10, 50, 90])
+    tau = torch.zeros(3, dtype=torch.float32, device="cuda")
+    sf.sf_universal_thresholds_dev(ctx, hz.dev(u), 20000, [10, 50, 90], 100, tau)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(tau.cpu().numpy()), bits(ref))
+
+
+@pytest.mark.parametrize("n,C,Q", [(50000, 8, 100), (3000, 16, 1000), (9, 2, 4), (120000, 3, 20)])
+def test_algorithm_2_per_class_thresholds(env, n, C, Q):
+    from oracle.calibrate import per_class_thresholds
+    sf, hz, ctx = env
+    rng = np.random.default_rng(n + C)
+    u = rng.random(n).astype(np.float32)
+    u[rng.integers(0, n, n // 4)] = np.float32(0.5)
+    pred = rng.integers(0, max(C - 1, 1), n).astype(np.uint8)   # the last class is never predicted (when C > 1)
+    slope = rng.uniform(0.2, 1.0, C)
+    correct = (rng.random(n) > u * slope[pred]).astype(np.uint8)
+    for a in (0, 24, 70, 100):
+        ref_tau, ref_assigned, _ = per_class_thresholds(u, pred, correct, C, Q, a, 100)
+        tau, assigned = sf.sf_per_class_thresholds(ctx, hz.dev(u), hz.dev(pred), hz.dev(correct), n, C, Q, a, 100)
+        assert np.array_equal(bits(tau), bits(ref_tau)) and assigned == ref_assigned
+        assert assigned == int(np.count_nonzero(u > tau[pred]))
