@@ -369,6 +369,29 @@ int  sf_table_ingest(sf_ctx* ctx, sf_table* table, const sf_pkt_batch* batch, co
 int  sf_table_lookup(sf_ctx* ctx, const sf_table* table, const sf_key* keys_dev, uint32_t n,
                      sf_flow_result* out_dev, void* stream);
 
+/* Table lifecycle.  Sec. 3.1 and 4.1: data that waits without a match is discarded after a
+ * timeout; the QoE task of Sec. 5.1 needs a monitored flow to be inferred again and again.
+ * sf_table_set_time: the time stamp (caller's unit, 32 bits, may wrap) that the packets of
+ * the following sf_table_ingest calls carry; a flow remembers the stamp of its last batch.
+ * sf_table_sweep: one pass over all slots on `stream`: a flow with now - last_seen >
+ * idle_timeout (unsigned 32-bit difference) is discarded whatever its stage - its slot can be
+ * claimed by a later flow, its slow-context slab returns to the pool, its key, if it comes
+ * back, is a new flow; with rearm != 0 every remaining flow that has its answer (stage 1 or
+ * 3) starts a new window (packet count 0, stage 0; the old labels stay readable until the
+ * next answer).  result_dev (device) is overwritten with the counts.  Slabs are also returned
+ * when the slow model has answered.  Do not overlap a sweep with an ingest on another stream. */
+typedef struct {
+    uint32_t n_expired_pending;    /* discarded before the fast model ran */
+    uint32_t n_expired_assigned;   /* discarded while waiting for their slow context */
+    uint32_t n_expired_done;       /* discarded after their answer */
+    uint32_t n_rearmed;
+    uint32_t n_live;               /* flows in the table after the sweep */
+    uint32_t pad[3];
+} sf_sweep_result;
+int  sf_table_set_time(sf_table* table, uint32_t now);
+int  sf_table_sweep(sf_ctx* ctx, sf_table* table, uint32_t now, uint32_t idle_timeout, int rearm,
+                    sf_sweep_result* result_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

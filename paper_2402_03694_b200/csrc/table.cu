@@ -17,6 +17,11 @@
 //   apply2    later packets go to the slab of an assigned flow (or are counted as arriving
 //             after the decision); flows that just reached slow_pkts packets are listed
 //   slow path wide rows of the listed slabs (zero-padded to the model's width) -> S4 -> labels
+//   sweep     (on request) one thread per slot: a flow idle for longer than the timeout is discarded
+//             (Sec. 3.1 / 4.1: unmatched data is purged after a timeout): its slot becomes a tombstone
+//             that a later insertion may claim, its slab goes back to the free list; optionally every
+//             answered flow is re-armed for a new window (continuous inference on long-lived flows)
+// Slabs are also returned when the slow model has answered.
 // Every loop is bounded; a key that finds no slot within the probe limit is counted as missed
 // and SF_ERR_TABLE_FULL is recorded in the context's error word.
 #include "common.cuh"
@@ -36,7 +41,10 @@ struct TableDev {
     uint16_t* f_size; uint32_t* f_iat; uint32_t* f_dir; uint8_t* f_hdr;
     // per slab
     uint16_t* s_size; uint32_t* s_iat; uint32_t* s_dir; uint8_t* s_hdr;
-    uint32_t* slab_next;
+    uint32_t* slab_next;          // bump allocator for slabs never used before
+    uint32_t* slab_free; int* slab_free_n;      // stack of returned slabs
+    uint32_t* last_seen;          // per slot: time stamp of the last batch that held a packet of the flow
+    uint32_t now;                 // time stamp of the batch being ingested
     uint32_t* first;              // per slot: arrival index of the flow's first packet in the current batch (else ~0)
     uint32_t mask, n_slots, fast_pkts, slow_pkts, slow_slabs;
 };
@@ -58,8 +66,10 @@ struct sf_table {
 
 namespace {
 
-__device__ __forceinline__ void cas128(void* p, uint64_t nlo, uint64_t nhi, uint64_t& olo, uint64_t& ohi) {
-    // compare with zero (empty slot), swap in the key; returns what was there
+constexpr uint64_t kTomb = ~0ull;      // both halves all ones: no real key (bits 40..62 of the high half are zero)
+
+__device__ __forceinline__ void cas128(void* p, uint64_t clo, uint64_t chi, uint64_t nlo, uint64_t nhi, uint64_t& olo, uint64_t& ohi) {
+    // compare with (clo, chi), swap in the key; returns what was there
     asm volatile(
         "{\n"
         ".reg .b128 c, s, d;\n"
@@ -68,7 +78,7 @@ __device__ __forceinline__ void cas128(void* p, uint64_t nlo, uint64_t nhi, uint
         "atom.global.cas.b128 d, [%6], c, s;\n"
         "mov.b128 {%0, %1}, d;\n"
         "}\n"
-        : "=l"(olo), "=l"(ohi) : "l"(0ull), "l"(0ull), "l"(nlo), "l"(nhi), "l"(p) : "memory");
+        : "=l"(olo), "=l"(ohi) : "l"(clo), "l"(chi), "l"(nlo), "l"(nhi), "l"(p) : "memory");
 }
 
 __device__ __forceinline__ uint64_t mix64(uint64_t x) {
@@ -93,18 +103,28 @@ __global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ 
     if (i >= b.n) return;
     uint64_t lo, hi;
     make_key(b.src[i], b.dst[i], b.sport[i], b.dport[i], b.proto[i], lo, hi);
-    uint32_t h = hash_key(lo, hi, t.mask);
     uint32_t slot = t.n_slots;                       // "missed" sorts after every real slot
-    for (uint32_t p = 0; p < kProbeLimit; p++) {
-        uint64_t olo, ohi;
-        const ulonglong2 cur = t.keys[h];            // cheap look before the atomic
-        if (cur.x == lo && cur.y == hi) { slot = h; break; }
-        if (cur.x == 0 && cur.y == 0) {
-            cas128(&t.keys[h], lo, hi, olo, ohi);
-            if (olo == 0 && ohi == 0) { slot = h; atomicAdd(&res->n_new_flows, 1u); break; }
-            if (olo == lo && ohi == hi) { slot = h; break; }
+    // Walk the whole probe chain: the key may sit behind a tombstone.  If it is absent, claim the
+    // first tombstone seen, else the empty slot that ends the chain.  Every thread with this key
+    // walks the same chain and slots only ever change from free to taken during a batch, so all
+    // of them end at one slot.  A lost race against another key restarts the walk (bounded).
+    for (uint32_t attempt = 0; attempt < 16 && slot == t.n_slots; attempt++) {
+        uint32_t h = hash_key(lo, hi, t.mask), cand = t.n_slots;
+        bool cand_tomb = false;
+        for (uint32_t p = 0; p < kProbeLimit; p++) {
+            const ulonglong2 cur = __ldcg(&t.keys[h]);       // from L2: another SM may just have claimed it
+            if (cur.x == lo && cur.y == hi) { slot = h; break; }
+            if (cur.x == kTomb && cur.y == kTomb) { if (cand == t.n_slots) { cand = h; cand_tomb = true; } }
+            else if (cur.x == 0 && cur.y == 0) { if (cand == t.n_slots) cand = h; break; }
+            h = (h + 1) & t.mask;
         }
-        h = (h + 1) & t.mask;
+        if (slot != t.n_slots) break;
+        if (cand == t.n_slots) break;                // no free slot within the probe limit
+        uint64_t olo, ohi;
+        const uint64_t c = cand_tomb ? kTomb : 0ull;
+        cas128(&t.keys[cand], c, c, lo, hi, olo, ohi);
+        if (olo == c && ohi == c) { slot = cand; atomicAdd(&res->n_new_flows, 1u); }
+        else if (olo == lo && ohi == hi) slot = cand;
     }
     if (slot == t.n_slots) {
         atomicAdd(&res->n_missed, 1u);
@@ -237,6 +257,13 @@ __device__ __forceinline__ void store_packet(uint16_t* sz, uint32_t* ia, uint32_
     for (int k = 0; k < (int)kHdr; k++) o[k] = s[k];
 }
 
+// Returns a slab to the free stack with its direction words cleared (they are filled by atomicOr).
+__device__ __forceinline__ void release_slab(const TableDev& t, uint32_t s) {
+    const uint32_t words = (t.slow_pkts + 31) / 32;
+    for (uint32_t w = 0; w < words; w++) t.s_dir[(size_t)s * words + w] = 0;
+    t.slab_free[atomicAdd(t.slab_free_n, 1)] = s;
+}
+
 __global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
                               const uint32_t* __restrict__ pkt_slot, uint32_t* __restrict__ rank, uint32_t* __restrict__ pos_out,
                               uint32_t* __restrict__ fire1_slot, uint32_t* __restrict__ counts)
@@ -279,7 +306,10 @@ __global__ void apply_route_kernel(TableDev t, const uint32_t* __restrict__ fire
     atomicAdd(&res->n_fast_fired, 1u);
     bool assigned = decision[k] != 0;
     if (assigned) {
-        const uint32_t s = atomicAdd(t.slab_next, 1u);
+        uint32_t s;
+        const int k_free = atomicSub(t.slab_free_n, 1);              // returned slabs first, then never-used ones
+        if (k_free >= 1) s = t.slab_free[k_free - 1];
+        else { atomicAdd(t.slab_free_n, 1); s = atomicAdd(t.slab_next, 1u); if (s >= t.slow_slabs) atomicSub(t.slab_next, 1u); }
         if (s < t.slow_slabs) {
             t.slab[slot] = s;
             const uint32_t words = (t.slow_pkts + 31) / 32;
@@ -330,7 +360,7 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
         }
     }
     // the last packet of the flow's run in this batch advances the flow's packet counter
-    if (j + 1 == b.n || s_key[j + 1] != s_key[j]) { t.cnt[slot] += rank[j] + 1; t.first[slot] = 0xFFFFFFFFu; }
+    if (j + 1 == b.n || s_key[j + 1] != s_key[j]) { t.cnt[slot] += rank[j] + 1; t.first[slot] = 0xFFFFFFFFu; t.last_seen[slot] = t.now; }
 }
 
 __global__ void apply_slow_kernel(TableDev t, const uint32_t* __restrict__ fire2_slot, const uint32_t* __restrict__ counts,
@@ -342,6 +372,42 @@ __global__ void apply_slow_kernel(TableDev t, const uint32_t* __restrict__ fire2
     t.label_slow[slot] = label_slow[k];
     t.stage[slot] = 3;
     atomicAdd(&res->n_slow_fired, 1u);
+    release_slab(t, t.slab[slot]);                                   // the slow context has been used
+}
+
+__global__ void sweep_kernel(TableDev t, uint32_t now, uint32_t timeout, int rearm, sf_sweep_result* res)
+{
+    const uint32_t slot = blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t what = 0;                     // 1 pending, 2 assigned, 3 done expired; 4 re-armed; 5 live
+    if (slot < t.n_slots) {
+        const ulonglong2 key = t.keys[slot];
+        if (!(key.x == 0 && key.y == 0) && !(key.x == kTomb && key.y == kTomb)) {
+            const uint32_t stg = t.stage[slot];
+            if (now - t.last_seen[slot] > timeout) {
+                what = stg == 0 ? 1 : (stg == 2 ? 2 : 3);
+                if (stg == 2) release_slab(t, t.slab[slot]);
+                t.cnt[slot] = 0; t.stage[slot] = 0; t.label_fast[slot] = 0; t.label_slow[slot] = 0; t.score[slot] = 0.0f;
+                t.f_dir[slot] = 0;
+                t.keys[slot] = make_ulonglong2(kTomb, kTomb);
+            } else if (rearm && (stg == 1 || stg == 3)) {
+                t.cnt[slot] = 0; t.stage[slot] = 0; t.f_dir[slot] = 0;
+                what = 4;
+            } else what = 5;
+        }
+    }
+    // block-level counts, one atomic per counter and block
+    __shared__ uint32_t c[6];
+    if (threadIdx.x < 6) c[threadIdx.x] = 0;
+    __syncthreads();
+    if (what) atomicAdd(&c[what], 1u);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (c[1]) atomicAdd(&res->n_expired_pending, c[1]);
+        if (c[2]) atomicAdd(&res->n_expired_assigned, c[2]);
+        if (c[3]) atomicAdd(&res->n_expired_done, c[3]);
+        if (c[4]) atomicAdd(&res->n_rearmed, c[4]);
+        if (c[4] + c[5]) atomicAdd(&res->n_live, c[4] + c[5]);
+    }
 }
 
 __global__ void lookup_kernel(TableDev t, const sf_key* __restrict__ keys, uint32_t n, sf_flow_result* __restrict__ out)
@@ -392,6 +458,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     need(S * 16); need(S * 4); need(S); need(S); need(S); need(S * 4); need(S * 4);
     need(S * fast_pkts * 2); need(S * fast_pkts * 4); need(S * 4); need(S * fast_pkts * kHdr);
     need(B * slow_pkts * 2); need(B * slow_pkts * 4); need(B * W * 4); need(B * slow_pkts * kHdr); need(4);
+    need(B * 4); need(4); need(S * 4);
     for (int k = 0; k < 9; k++) need((size_t)kMaxBatch * 4);
     need(64); need((size_t)kMaxBatch * 4); need(1024 * 4); need(S * 4);
     need((size_t)kMaxBatch * fast_pkts * 2); need((size_t)kMaxBatch * fast_pkts * 4); need((size_t)kMaxBatch * 4);
@@ -409,6 +476,8 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     d.s_size = carve<uint16_t>(p, B * slow_pkts); d.s_iat = carve<uint32_t>(p, B * slow_pkts);
     d.s_dir = carve<uint32_t>(p, B * W); d.s_hdr = carve<uint8_t>(p, B * slow_pkts * kHdr);
     d.slab_next = carve<uint32_t>(p, 1);
+    d.slab_free = carve<uint32_t>(p, B); d.slab_free_n = carve<int>(p, 1); d.last_seen = carve<uint32_t>(p, S);
+    d.now = 0;
     d.mask = (uint32_t)(S - 1); d.n_slots = (uint32_t)S; d.fast_pkts = fast_pkts; d.slow_pkts = slow_pkts; d.slow_slabs = slow_slabs;
     t->key_a = carve<uint32_t>(p, kMaxBatch); t->key_b = carve<uint32_t>(p, kMaxBatch);
     t->idx_a = carve<uint32_t>(p, kMaxBatch); t->idx_b = carve<uint32_t>(p, kMaxBatch);
@@ -529,6 +598,25 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     if (rc != SF_OK) return rc;
     apply_slow_kernel<<<blocks, 256, 0, st>>>(d, t->fire2_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_slab_lab), result_dev);
     SF_LAUNCH_CHECK("apply_slow_kernel");
+    return SF_OK;
+}
+
+extern "C" int sf_table_set_time(sf_table* t, uint32_t now)
+{
+    if (!t) return SF_ERR_ARG;
+    t->d.now = now;
+    return SF_OK;
+}
+
+extern "C" int sf_table_sweep(sf_ctx* ctx, sf_table* t, uint32_t now, uint32_t idle_timeout, int rearm,
+                              sf_sweep_result* result_dev, void* stream)
+{
+    if (!ctx || !t || !result_dev) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_sweep_result), st));
+    sweep_kernel<<<(t->d.n_slots + 255) / 256, 256, 0, st>>>(t->d, now, idle_timeout, rearm, result_dev);
+    SF_LAUNCH_CHECK("sweep_kernel");
     return SF_OK;
 }
 

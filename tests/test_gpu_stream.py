@@ -121,3 +121,78 @@ def test_full_table_is_reported_not_fatal(env):
     sf.sf_table_destroy(table)
     sf.sf_slow_destroy(slow_h)
     sf.sf_forest_destroy(forest_h)
+
+
+# ---- table lifecycle: idle timeout, slot and slab reuse, re-arming ----
+def _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg):
+    names = ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision", "missed")
+    totals = np.zeros(8, np.int64)
+    sweeps = []
+    res = torch.zeros(8, dtype=torch.int32, device="cuda")
+    sw = torch.zeros(8, dtype=torch.int32, device="cuda")
+    for ev in events:
+        if ev[0] == "batch":
+            b = ev[1]
+            sf.sf_table_set_time(table, ev[2])
+            d = {k: hz.dev(b[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
+            pb = sf.make_pkt_batch(d["src"], d["dst"], d["sport"], d["dport"], d["proto"], d["dir"], d["size"], d["iat_us"], d["hdr"])
+            sf.sf_table_ingest(ctx, table, pb, forest_h, F, slow_h, rcfg, res)
+            torch.cuda.synchronize()
+            totals += res.cpu().numpy().astype(np.int64)
+        else:
+            sf.sf_table_sweep(ctx, table, ev[1], ev[2], ev[3], sw)
+            torch.cuda.synchronize()
+            sweeps.append(dict(zip(sf.SWEEP_FIELDS, sw.cpu().numpy()[:5].tolist())))
+    return dict(zip(names, totals[:7].tolist())), sweeps
+
+
+@pytest.mark.parametrize("rearm", [False, True])
+def test_lifecycle_matches_sequential_reference(env, rearm):
+    from oracle.lifecycle import simulate_lifecycle
+    sf, hz, ctx = env
+    F, T, depth, C, dims, P_model, fast_pkts, slow_pkts = 24, 16, 8, 4, (1024, 256, 4), 64, 8, 64
+    forest, tau, slow = _models(F, T, depth, C, dims, 95)
+    # two key populations that alternate, so that the first one idles out and comes back; a small table
+    # (2^11 slots for ~1,300 live keys, 600 slabs) makes tombstone and slab reuse necessary
+    srcA, srcB = flowgen.StreamSource(96, 700, 0.9), flowgen.StreamSource(97, 700, 0.9)
+    events, now = [], 0
+    for phase in range(6):
+        s = srcA if phase % 2 == 0 else srcB
+        for j in range(3):
+            now += 10
+            events.append(("batch", s.batch(phase * 3 + j, 6000 + 13 * j), now))
+            if j == 1:
+                events.append(("sweep", now + 1, 25, rearm))
+        events.append(("sweep", now + 2, 25, rearm))
+    per, tot, sweeps = simulate_lifecycle(events, fast_pkts, slow_pkts, F, forest, tau, slow, P_model, True)
+    assert sum(s["expired_assigned"] for s in sweeps) > 500 and sum(s["expired_pending"] for s in sweeps) > 1000
+    assert tot["slow_fired"] > 50 and tot["new_flows"] > 4000        # 1,400 keys: most of them came back as new flows
+    assert sum(s["rearmed"] for s in sweeps) > 1000 if rearm else sum(s["expired_done"] for s in sweeps) > 1000
+
+    forest_h = hz.make_forest(ctx, forest)
+    slow_h = sf.sf_mlp_create(ctx, sf.SF_BF16, slow["dims"], slow["W"], slow["b"])
+    table = sf.sf_table_create(ctx, 11, fast_pkts, slow_pkts, 600)
+    rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
+    sf.sf_ctx_poll(ctx, reset=True)
+    got, got_sweeps = _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg)
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert got["missed"] == 0 and c.device_error == 0
+    assert tot["escalated"] > 600                      # more assignments than slabs: returned slabs were used again
+    for k in tot:
+        assert got[k] == tot[k], k
+    assert got_sweeps == sweeps
+    keys = list(per.keys())
+    res = _lookup(sf, hz, ctx, table, keys)
+    for i, k in enumerate(keys):
+        r, g = per[k], res[i]
+        assert g["found"] == 1 and g["n_pkts"] == r["n_pkts"] and g["stage"] == r["stage"], k
+        if r["stage"] >= 1:
+            assert g["label_fast"] == r["label_fast"]
+            assert np.float32(g["score"]).view(np.uint32) == np.float32(r["score"]).view(np.uint32)
+    gone = [k for k in zip(srcA.keys["src"][:50].tolist(), srcA.keys["dst"][:50].tolist(), srcA.keys["sport"][:50].tolist(),
+                           srcA.keys["dport"][:50].tolist(), srcA.keys["proto"][:50].tolist()) if k not in per]
+    if gone:
+        assert not _lookup(sf, hz, ctx, table, gone)["found"].any()
+    sf.sf_table_destroy(table)
+    sf.sf_slow_destroy(slow_h)
+    sf.sf_forest_destroy(forest_h)
