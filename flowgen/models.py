@@ -27,7 +27,8 @@ def gen_forest(seed, kind, T, depth, F, C, feat_sample, sigma=0.1):
         g = rng.standard_gamma(0.5, size=(T, n_leaf, C))
         g = np.maximum(g, 1e-300)
         leaf = (g / g.sum(axis=2, keepdims=True)).astype(np.float32)
-    elif kind == "gbdt":
+    elif kind in ("gbdt", "gbdt_mc"):       # gbdt_mc: tree t belongs to class t mod C (T a multiple of C)
+        assert kind == "gbdt" or T % C == 0
         leaf = rng.normal(0.0, sigma, size=(T, n_leaf)).astype(np.float32)
     else:
         raise ValueError(kind)

@@ -44,6 +44,8 @@ def lib():
         _lib.sfo_route_lc.restype = C.c_uint64
         _lib.sfo_route_absmargin.restype = C.c_uint64
         _lib.sfo_route_entropy.restype = C.c_uint64
+        _lib.sfo_route_softmax_lc.restype = C.c_uint64
+        _lib.sfo_softmax_lc.restype = C.c_double
         _lib.sfo_ilog.restype = C.c_uint32
         _lib.sfo_ilog.argtypes = [C.c_uint32]
     return _lib
@@ -146,6 +148,13 @@ def forest_infer(forest, feat, want_leaf_idx=False, threads=1):
             L.sfo_forest_rf(_p(feat[lo:hi]), C.c_uint64(hi - lo), C.c_uint32(F), C.c_uint32(T), C.c_uint32(d),
                             C.c_uint32(Cc), _p(fid), _p(thr), _p(leaf), _p(out[lo:hi]),
                             None if li is None else _p(li[lo:hi]))
+    elif forest["kind"] == "gbdt_mc":
+        out = np.empty((n, Cc), dtype=np.float32)
+
+        def work(lo, hi):
+            L.sfo_forest_gbdt_mc(_p(feat[lo:hi]), C.c_uint64(hi - lo), C.c_uint32(F), C.c_uint32(T), C.c_uint32(d),
+                                 C.c_uint32(Cc), _p(fid), _p(thr), _p(leaf), _p(out[lo:hi]),
+                                 None if li is None else _p(li[lo:hi]))
     else:
         out = np.empty((n,), dtype=np.float32)
 
@@ -180,6 +189,19 @@ def route_entropy(prob, tau):
     ids = np.empty(n, np.uint32)
     k = lib().sfo_route_entropy(_p(prob), C.c_uint64(n), C.c_uint32(Cc), _p(tau), _p(score), _p(label),
                                 _p(dec), _p(ids), C.c_uint64(n))
+    return {"score": score, "label": label, "decision": dec, "esc_ids": ids[:k].copy(), "n_esc": int(k)}
+
+
+def route_softmax_lc(margin, tau):
+    margin = _c(margin, np.float32)
+    n, Cc = margin.shape
+    tau = _c(np.broadcast_to(np.asarray(tau, dtype=np.float32), (Cc,)), np.float32)
+    score = np.empty(n, np.float32)
+    label = np.empty(n, np.uint8)
+    dec = np.empty(n, np.uint8)
+    ids = np.empty(n, np.uint32)
+    k = lib().sfo_route_softmax_lc(_p(margin), C.c_uint64(n), C.c_uint32(Cc), _p(tau), _p(score), _p(label),
+                                   _p(dec), _p(ids), C.c_uint64(n))
     return {"score": score, "label": label, "decision": dec, "esc_ids": ids[:k].copy(), "n_esc": int(k)}
 
 

@@ -221,6 +221,27 @@ void sfo_forest_gbdt(const float* feat, uint64_t n, uint32_t F, uint32_t T, uint
 
 double sfo_sigmoid(double margin) { return 1.0 / (1.0 + exp(-margin)); }
 
+/* Boosted trees, multi-class (the layout of the gradient-boosting libraries the paper names in
+ * Sec. 4.4): one tree per class and boosting round, tree t belongs to class t mod C;
+ * margin[c] = 0 + sum of the leaf scalars of class c's trees in tree order (fp32).  The class
+ * probabilities are softmax(margin); the label is the largest margin (lowest index on ties). */
+void sfo_forest_gbdt_mc(const float* feat, uint64_t n, uint32_t F, uint32_t T, uint32_t depth, uint32_t C,
+                        const uint16_t* fid, const float* thr, const float* leaf,
+                        float* margin, uint16_t* leaf_idx)
+{
+    uint32_t n_int = (1u << depth) - 1u, n_leaf = 1u << depth;
+    for (uint64_t f = 0; f < n; f++) {
+        const float* x = feat + f * F;
+        float* m = margin + f * C;
+        for (uint32_t c = 0; c < C; c++) m[c] = 0.0f;
+        for (uint32_t t = 0; t < T; t++) {
+            uint32_t l = walk(x, fid + (uint64_t)t * n_int, thr + (uint64_t)t * n_int, depth);
+            if (leaf_idx) leaf_idx[f * T + t] = (uint16_t)l;
+            m[t % C] = m[t % C] + leaf[(uint64_t)t * n_leaf + l];
+        }
+    }
+}
+
 /* ------------------------------------------------------------------------- */
 /* S3: uncertainty, threshold, assignment                                    */
 /* ------------------------------------------------------------------------- */
@@ -278,6 +299,36 @@ uint64_t sfo_route_entropy(const float* prob, uint64_t n, uint32_t C, const floa
         float h = (float)sfo_entropy(p, C);
         int esc = h > tau[a];
         if (score) score[f] = h;
+        if (label) label[f] = (uint8_t)a;
+        if (decision) decision[f] = (uint8_t)esc;
+        if (esc) { if (esc_ids && k < capacity) esc_ids[k] = (uint32_t)f; k++; }
+    }
+    return k;
+}
+
+/* Least confidence of a softmax over margins (Sec. 3.2 applied to a multi-class boosted model):
+ * LC = 1 - max_c softmax(m)_c = 1 - 1 / sum_j exp(m_j - m_max), in double precision. */
+double sfo_softmax_lc(const float* m, uint32_t C)
+{
+    float mx = m[0];
+    for (uint32_t c = 1; c < C; c++) if (m[c] > mx) mx = m[c];
+    double s = 0.0;
+    for (uint32_t c = 0; c < C; c++) s += exp((double)m[c] - (double)mx);
+    return 1.0 - 1.0 / s;
+}
+
+uint64_t sfo_route_softmax_lc(const float* margin, uint64_t n, uint32_t C, const float* tau,
+                              float* score, uint8_t* label, uint8_t* decision,
+                              uint32_t* esc_ids, uint64_t capacity)
+{
+    uint64_t k = 0;
+    for (uint64_t f = 0; f < n; f++) {
+        const float* m = margin + f * C;
+        uint32_t a = 0;
+        for (uint32_t c = 1; c < C; c++) if (m[c] > m[a]) a = c;
+        float u = (float)sfo_softmax_lc(m, C);
+        int esc = u > tau[a];
+        if (score) score[f] = u;
         if (label) label[f] = (uint8_t)a;
         if (decision) decision[f] = (uint8_t)esc;
         if (esc) { if (esc_ids && k < capacity) esc_ids[k] = (uint32_t)f; k++; }

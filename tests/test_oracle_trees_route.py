@@ -1,4 +1,5 @@
 """Pins for the oracle's tree-ensemble, scoring, threshold and wide-row stages."""
+import ctypes as C
 import math
 from fractions import Fraction
 
@@ -250,3 +251,38 @@ def test_entropy_rule_matches_direct_evaluation():
     q = np.stack([np.linspace(0.5, 0.99, 50), 1 - np.linspace(0.5, 0.99, 50)], 1).astype(np.float32)
     he = oracle.route_entropy(q, 9.0)["score"]; lc = oracle.route_lc(q, 9.0)["score"]
     assert np.all(np.diff(he) < 0) and np.all(np.diff(lc) < 0)
+
+
+# ---- multi-class boosted trees and the softmax least-confidence rule ----
+def test_gbdt_mc_equals_the_scalar_model_on_each_class_subensemble():
+    rng = np.random.default_rng(41)
+    F, C, rounds, depth, n = 12, 5, 7, 4, 300
+    feat = rng.normal(size=(n, F)).astype(np.float32)
+    fo = flowgen.gen_forest(42, "gbdt_mc", rounds * C, depth, F, C, feat, sigma=0.3)
+    m, li = oracle.forest_infer(fo, feat, want_leaf_idx=True)
+    assert m.shape == (n, C)
+    for c in range(C):
+        sub = {"kind": "gbdt", "T": rounds, "depth": depth, "F": F, "C": 1, "fid": fo["fid"][c::C].copy(),
+               "thr": fo["thr"][c::C].copy(), "leaf": fo["leaf"][c::C].copy()}
+        mc, lic = oracle.forest_infer(sub, feat, want_leaf_idx=True)
+        assert np.array_equal(m[:, c].view(np.uint32), mc.view(np.uint32)) and np.array_equal(li[:, c::C], lic)
+    one = dict(fo, C=1, kind="gbdt_mc")
+    assert np.array_equal(oracle.forest_infer(one, feat)[:, 0].view(np.uint32),
+                          oracle.forest_infer(dict(fo, kind="gbdt", C=1), feat).view(np.uint32))
+
+
+def test_softmax_least_confidence_closed_forms():
+    L = oracle.lib()
+    def lc(m):
+        a = np.asarray(m, np.float32)
+        return L.sfo_softmax_lc(a.ctypes.data_as(C.c_void_p), C.c_uint32(len(a)))
+    assert abs(lc([0.3] * 7) - (1 - 1 / 7)) < 1e-15                   # equal margins: uniform
+    assert lc([50.0, -50.0, -50.0]) < 1e-40 and lc([50.0, -50.0, -50.0]) >= 0
+    assert abs(lc([1.0, 2.0, 3.0]) - lc([-9.0, -8.0, -7.0])) < 1e-15   # shift invariance
+    assert abs(lc([0.0, np.log(3.0)]) - 0.25) < 1e-7                   # two classes: 1 - sigmoid(gap) = 1 - 3/4
+    m = np.array([[0.2, 1.5, -0.3]], np.float32)
+    p = np.exp(m[0].astype(np.float64)); p /= p.sum()
+    r = oracle.route_softmax_lc(m, [0.0, 0.9, 0.0])
+    assert abs(float(r["score"][0]) - (1 - p.max())) < 1e-7 and r["label"][0] == 1 and r["decision"][0] == 0
+    r = oracle.route_softmax_lc(np.array([[1.0, 1.0, 0.0]], np.float32), 0.5)
+    assert r["label"][0] == 0 and r["decision"][0] == 1                # tie -> lowest index; LC = 1 - e/(2e+1) > 0.5
