@@ -46,10 +46,14 @@ extern "C" {
 /* enums passed as int */
 #define SF_RF           0          /* random forest: mean of leaf class-probability vectors */
 #define SF_GBDT         1          /* boosted trees, binary logistic: sum of leaf scalars (margin) */
+#define SF_GBDT_MC      2          /* boosted trees, multi-class: tree t belongs to class t mod C (one tree per class and
+                                      boosting round, the layout of the libraries Sec. 4.4 names); C margins per flow */
 #define SF_LC_GT        0          /* assign iff 1 - max_c prob[c] > tau[argmax]  (Sec. 3.2, least confidence) */
 #define SF_ABSMARGIN_LT 1          /* assign iff |margin| < tau[0]  (|p-0.5| < 0.2  <=>  |margin| < ln(7/3)) */
 #define SF_ENTROPY_GT   2          /* assign iff -sum_c prob[c] ln prob[c] > tau[argmax]  (Sec. 3.2, entropy; fp32 logf:
                                       scores agree with a double-precision evaluation to about 1e-6, not bit for bit) */
+#define SF_SOFTMAX_LC_GT 3         /* input = C margins (SF_GBDT_MC): assign iff 1 - max softmax(margin) > tau[argmax], i.e.
+                                      1 - 1/sum_j exp(m_j - m_max) (Sec. 3.2's least confidence; fp32 expf, tolerance as above) */
 #define SF_MLP16        0          /* wide row = P packets x 16 fields */
 #define SF_CNN8         1          /* wide row = P positions x 8 channels (channels last) */
 #define SF_F32          0
@@ -154,7 +158,9 @@ int  sf_header_bits(sf_ctx* ctx, const uint8_t* bytes, const uint8_t* sec_len, u
 /* Builds an ensemble of T complete binary trees of depth `depth` (heap order:
  * children of node i are 2i+1, 2i+2) from HOST arrays fid uint16[T][2^d-1],
  * thr fp32[T][2^d-1], leaf fp32[T][2^d][C] (SF_RF) or fp32[T][2^d] (SF_GBDT, C
- * ignored and treated as 2 classes).  depth 1..12, F <= 64, C <= 16. */
+ * ignored and treated as 2 classes; SF_GBDT_MC, T a multiple of C).  depth 1..12,
+ * F <= 64, C <= 16.  SF_GBDT_MC needs a whole boosting round (C trees of 12*2^d bytes)
+ * within one shared-memory chunk, else sf_fast_infer returns SF_ERR_UNSUPPORTED. */
 int  sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t depth, uint32_t F, uint32_t C,
                       const uint16_t* fid_host, const float* thr_host, const float* leaf_host,
                       sf_forest** out);
@@ -163,13 +169,14 @@ void sf_forest_destroy(sf_forest* forest);
  * node a flow goes LEFT iff x[fid] <= thr.  SF_RF: prob[c] = (sum over trees
  * t = 0..T-1, in that order, fp32) of leaf[t][l_t][c], divided by fp32(T) ->
  * out fp32[n][C].  SF_GBDT: margin = sum of leaf[t][l_t] in tree order ->
- * out fp32[n].  leaf_idx_out (nullable): uint16[n][T]. */
+ * out fp32[n].  SF_GBDT_MC: margin[c] = sum over the trees t = c, c+C, c+2C, ... in that
+ * order -> out fp32[n][C].  leaf_idx_out (nullable): uint16[n][T]. */
 int  sf_fast_infer(sf_ctx* ctx, const sf_forest* forest, const float* feat, uint32_t n,
                    float* prob_or_margin_out, uint16_t* leaf_idx_out, void* stream);
 
 /* ---- S3: uncertainty score, threshold, compaction, wide rows --------------- */
 typedef struct {
-    int rule;               /* SF_LC_GT | SF_ABSMARGIN_LT | SF_ENTROPY_GT */
+    int rule;               /* SF_LC_GT | SF_ABSMARGIN_LT | SF_ENTROPY_GT | SF_SOFTMAX_LC_GT */
     const float* tau;       /* device: fp32[C] per predicted class (all equal = universal threshold) for
                                SF_LC_GT; fp32[1] for SF_ABSMARGIN_LT */
     int wide_layout;        /* SF_MLP16 | SF_CNN8 */
@@ -304,8 +311,9 @@ int  sf_serve_batch_host(sf_ctx* ctx, const sf_forest* forest, const sf_slow* sl
                          uint8_t* label_host_out, uint8_t* stage_host_out, uint32_t* n_esc_host_out, void* stream);
 /* Three-tier cascade (Sec. 3.1: the fastest model answers what it is sure of, the fast model
  * looks at the rest using the SAME features, the slow model at what is still uncertain, with
- * more packets; Sec. 3.2: thresholds per predicted class).  Both tree models are SF_RF
- * ensembles over the same F features (the fastest one is typically a single tree).
+ * more packets; Sec. 3.2: thresholds per predicted class).  The fastest model is an SF_RF
+ * ensemble (typically a single tree), the fast model SF_RF with SF_LC_GT or SF_GBDT_MC with
+ * SF_SOFTMAX_LC_GT, both over the same F features.
  * cfg_fastest: only rule (SF_LC_GT) and tau (fp32[C of fastest]) are used; cfg_fast: as in
  * sf_serve_batch.  stage_out: 1, 2 or 3.  n_esc_out (device, nullable): uint32[2] = flows
  * passed on by the fastest model, flows assigned to the slow model.  The context counters

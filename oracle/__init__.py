@@ -325,7 +325,8 @@ def serve_batch3(cfg, fast_pk, wide_pk, fastest, fast, slow_model, tau1, tau2, t
     r1 = route_lc(p1, tau1)
     ids1 = r1["esc_ids"]
     p2 = forest_infer(fast, feat[ids1], threads=threads) if len(ids1) else np.zeros((0, fast["C"]), np.float32)
-    r2 = route_lc(p2, tau2) if len(ids1) else {"esc_ids": np.zeros(0, np.uint32), "label": np.zeros(0, np.uint8),
+    route2 = route_softmax_lc if fast["kind"] == "gbdt_mc" else route_lc      # boosted fast model: softmax of its margins
+    r2 = route2(p2, tau2) if len(ids1) else {"esc_ids": np.zeros(0, np.uint32), "label": np.zeros(0, np.uint8),
                                                "n_esc": 0, "score": np.zeros(0, np.float32)}
     ids2 = ids1[r2["esc_ids"]]
     bf16 = cfg.slow_dtype == "bf16"
@@ -340,4 +341,5 @@ def serve_batch3(cfg, fast_pk, wide_pk, fastest, fast, slow_model, tau1, tau2, t
     label[ids1] = r2["label"]; stage[ids1] = 2
     label[ids2] = label_slow; stage[ids2] = 3
     return {"feat": feat, "prob1": p1, "ids1": ids1, "prob2": p2, "ids2": ids2, "rows": rows, "logits": logits,
-            "label_slow": label_slow, "label_final": label, "stage": stage, "label1": r1["label"], "label2": r2["label"]}
+            "label_slow": label_slow, "label_final": label, "stage": stage, "label1": r1["label"], "label2": r2["label"],
+            "score2": r2["score"]}

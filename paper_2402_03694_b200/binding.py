@@ -18,8 +18,8 @@ SF_ERR_ARG, SF_ERR_ALLOC, SF_ERR_CUDA, SF_ERR_CAPACITY = -1, -2, -3, -4
 SF_ERR_TABLE_FULL, SF_ERR_UNSUPPORTED, SF_ERR_DEVICE_TIMEOUT = -5, -6, -7
 SF_ERR_STATIC_LIMIT = -8
 SF_NOALLOC_MAX_FLOWS = 4194304
-SF_RF, SF_GBDT = 0, 1
-SF_LC_GT, SF_ABSMARGIN_LT, SF_ENTROPY_GT = 0, 1, 2
+SF_RF, SF_GBDT, SF_GBDT_MC = 0, 1, 2
+SF_LC_GT, SF_ABSMARGIN_LT, SF_ENTROPY_GT, SF_SOFTMAX_LC_GT = 0, 1, 2, 3
 SF_MLP16, SF_CNN8 = 0, 1
 SF_F32, SF_BF16 = 0, 1
 SF_TAU_MARGIN_DEFAULT = float.fromhex("0x1.b1d106p-1")

@@ -212,8 +212,9 @@ int check_serve_args(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const s
     if (F != fo->F || F < 8 || F > 64 || F % 8) return SF_ERR_ARG;
     if (wide->n_flows < fast->n_flows) return SF_ERR_ARG;
     if ((cfg->rule == SF_LC_GT || cfg->rule == SF_ENTROPY_GT) && fo->kind != SF_RF) return SF_ERR_ARG;
-    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ENTROPY_GT && cfg->rule != SF_ABSMARGIN_LT) return SF_ERR_ARG;
+    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ENTROPY_GT && cfg->rule != SF_ABSMARGIN_LT && cfg->rule != SF_SOFTMAX_LC_GT) return SF_ERR_ARG;
     if (cfg->rule == SF_ABSMARGIN_LT && fo->kind != SF_GBDT) return SF_ERR_ARG;
+    if (cfg->rule == SF_SOFTMAX_LC_GT && fo->kind != SF_GBDT_MC) return SF_ERR_ARG;
     const uint32_t W = cfg->wide_layout == SF_MLP16 ? 16u : 8u;
     if (cfg->wide_layout != SF_MLP16 && cfg->wide_layout != SF_CNN8) return SF_ERR_ARG;
     if ((cfg->wide_layout == SF_CNN8) != (s->arch == SF_SLOW_CNN)) return SF_ERR_ARG;
@@ -308,7 +309,8 @@ extern "C" int sf_serve_batch3(sf_ctx* ctx, const sf_forest* f1, const sf_forest
     int rc = check_serve_args(ctx, f2, s, fast, N, F, wide, cfg2);
     if (rc != SF_OK) return rc;
     if (!label_out || !stage_out) return SF_ERR_ARG;
-    if (f1->kind != SF_RF || f1->F != F || cfg1->rule != SF_LC_GT || cfg2->rule != SF_LC_GT) return SF_ERR_ARG;
+    if (f1->kind != SF_RF || f1->F != F || cfg1->rule != SF_LC_GT) return SF_ERR_ARG;
+    if (cfg2->rule != SF_LC_GT && cfg2->rule != SF_SOFTMAX_LC_GT) return SF_ERR_ARG;      // fast model: forest or multi-class boosted trees
     SF_CUDA(cudaSetDevice(ctx->device));
     cudaStream_t st = (cudaStream_t)stream;
     const uint32_t n = fast->n_flows, cap = cfg2->capacity;
@@ -392,7 +394,7 @@ extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_sl
         const uint32_t Pw = wide_h->pitch_pkts, Hb = wide_h->hdr_bytes, words = (Pw + 31) / 32;
         const size_t fsz = (size_t)n * fast_h->pitch_pkts * 2, fia = (size_t)n * fast_h->pitch_pkts * 4,
                      fdr = (size_t)n * ((fast_h->pitch_pkts + 31) / 32) * 4, fnv = fast_h->n_valid ? (size_t)n : 0;
-        const uint32_t n_tau2 = cfg_h->rule == SF_LC_GT ? fo->C : 1;
+        const uint32_t n_tau2 = cfg_h->rule == SF_ABSMARGIN_LT ? 1 : fo->C;
         size_t off2 = 0;
         auto take2 = [&](size_t bytes) { size_t o = off2; off2 += sf_align256(bytes); return o; };
         const size_t a_fs = take2(fsz), a_fi = take2(fia), a_fd = take2(fdr), a_fv = take2(fnv), a_tau = take2(n_tau2 * 4),
@@ -506,7 +508,7 @@ extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_sl
     if (!shared) { o_fs = take(fs); o_fi = take(fi); o_fd = take(fd); }
     o_fv = take(fv);
     size_t o_ws = take(ws_), o_wi = take(wi), o_wd = take(wd), o_wh = take(wh), o_wv = take(wv);
-    const uint32_t n_tau = cfg_h->rule == SF_LC_GT ? fo->C : 1;
+    const uint32_t n_tau = cfg_h->rule == SF_ABSMARGIN_LT ? 1 : fo->C;
     size_t o_tau = take(n_tau * 4), o_label = take(n), o_stage = take(n), o_nesc = take(4);
     if (off > ctx->stage_bytes) {
         SF_CUDA(cudaDeviceSynchronize());

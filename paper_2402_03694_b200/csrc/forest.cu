@@ -84,8 +84,10 @@ __device__ __forceinline__ void load_leaf_vec(const float* __restrict__ lv, floa
     }
 }
 
-// KIND: SF_RF (leaf = C-vector of class probabilities in global memory) or SF_GBDT (leaf =
-// scalar stored behind the tree's nodes in the image, C = 1).  NCH: trees walked at once.
+// KIND: SF_RF (leaf = C-vector of class probabilities in global memory), SF_GBDT (leaf =
+// scalar stored behind the tree's nodes in the image, C = 1) or SF_GBDT_MC (scalar leaves, tree t
+// adds to class t mod C; a chunk holds whole boosting rounds, so the class of every tree in the
+// unrolled round loop is a compile-time register index).  NCH: trees walked at once.
 template <int KIND, int C, int NCH>
 __global__ void __launch_bounds__(kB, 1)
 forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
@@ -162,6 +164,32 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         const uint32_t t0 = ck * trees_per_chunk;
         const uint32_t nt = min(trees_per_chunk, T - t0);
         uint32_t tt = 0;
+        if (KIND == SF_GBDT_MC) {
+            for (uint32_t r0 = 0; r0 < nt; r0 += C) {             // one boosting round: classes 0..C-1 in order
+#pragma unroll
+                for (int c0 = 0; c0 + NCH <= C; c0 += NCH) {
+                    uint32_t l[NCH];
+                    float v[NCH];
+                    walk<NCH>(cur + (r0 + c0) * tree_stride, tree_stride, xbase, depth, l);
+                    if (leaf_idx && live) {
+#pragma unroll
+                        for (int k = 0; k < NCH; k++) leaf_idx[(size_t)f * T + t0 + r0 + c0 + k] = (uint16_t)l[k];
+                    }
+#pragma unroll
+                    for (int k = 0; k < NCH; k++) v[k] = lds32f(cur + (r0 + c0 + k) * tree_stride + n_leaf * 8u + l[k] * 4u);
+#pragma unroll
+                    for (int k = 0; k < NCH; k++) acc[c0 + k] = __fadd_rn(acc[c0 + k], v[k]);
+                }
+#pragma unroll
+                for (int c1 = (C / NCH) * NCH; c1 < C; c1++) {
+                    uint32_t l[1];
+                    walk<1>(cur + (r0 + c1) * tree_stride, tree_stride, xbase, depth, l);
+                    if (leaf_idx && live) leaf_idx[(size_t)f * T + t0 + r0 + c1] = (uint16_t)l[0];
+                    acc[c1] = __fadd_rn(acc[c1], lds32f(cur + (r0 + c1) * tree_stride + n_leaf * 8u + l[0] * 4u));
+                }
+            }
+            tt = nt;
+        }
         for (; tt + NCH <= nt; tt += NCH) {
             uint32_t l[NCH];
             walk<NCH>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
@@ -202,6 +230,9 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
     if (!live) return;
     if (KIND == SF_GBDT) {
         out[f] = acc[0];
+    } else if (KIND == SF_GBDT_MC) {
+#pragma unroll
+        for (int c = 0; c < C; c++) out[(size_t)f * C + c] = acc[c];
     } else {
         const float fT = __uint2float_rn(T);
 #pragma unroll
@@ -219,7 +250,8 @@ Plan make_plan(const sf_forest* fo) {
     p.chunk_bytes = avail < 65536u ? avail : 65536u;
     p.tpc = p.chunk_bytes / fo->tree_stride;          // 0 if one tree does not fit (checked by the callers)
     if (p.tpc > fo->T) p.tpc = fo->T;
-    p.nch = (fo->kind == SF_GBDT) ? (p.tpc >= 4 ? 4u : (p.tpc >= 2 ? 2u : 1u)) : (p.tpc >= 2 ? 2u : 1u);
+    if (fo->kind == SF_GBDT_MC) p.tpc -= p.tpc % fo->C;          // whole boosting rounds per chunk
+    p.nch = (fo->kind == SF_GBDT_MC) ? (fo->C >= 4 ? 4u : (fo->C >= 2 ? 2u : 1u)) : (fo->kind == SF_GBDT) ? (p.tpc >= 4 ? 4u : (p.tpc >= 2 ? 2u : 1u)) : (p.tpc >= 2 ? 2u : 1u);
     p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes + 32;       // + two mbarriers and the abort flag
     return p;
 }
@@ -256,11 +288,39 @@ int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, 
     return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
+template <int C>
+int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+    const Plan p = make_plan(fo);
+    if (p.tpc == 0) return SF_ERR_UNSUPPORTED;           // one boosting round does not fit in a chunk
+    return launch3<SF_GBDT_MC, C, (C >= 4 ? 4 : (C >= 2 ? 2 : 1))>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+}
+
 }  // namespace
 
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     if (n == 0) return SF_OK;
     if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st, n_dev);
+    if (fo->kind == SF_GBDT_MC) {
+        switch (fo->C) {
+        case 1:  return launch_mc<1>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 2:  return launch_mc<2>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 3:  return launch_mc<3>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 4:  return launch_mc<4>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 5:  return launch_mc<5>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 6:  return launch_mc<6>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 7:  return launch_mc<7>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 8:  return launch_mc<8>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 9:  return launch_mc<9>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 10: return launch_mc<10>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 11: return launch_mc<11>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 12: return launch_mc<12>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 13: return launch_mc<13>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 14: return launch_mc<14>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 15: return launch_mc<15>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 16: return launch_mc<16>(fo, feat, n, out, leaf_idx, st, n_dev);
+        }
+        return SF_ERR_UNSUPPORTED;
+    }
     switch (fo->C) {
     case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev);
     case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev);
@@ -286,9 +346,10 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
                                 const uint16_t* fid, const float* thr, const float* leaf, sf_forest** out)
 {
     if (!ctx || !fid || !thr || !leaf || !out) return SF_ERR_ARG;
-    if (kind != SF_RF && kind != SF_GBDT) return SF_ERR_ARG;
+    if (kind != SF_RF && kind != SF_GBDT && kind != SF_GBDT_MC) return SF_ERR_ARG;
     if (T < 1 || depth < 1 || depth > 12 || F < 1 || F > 64) return SF_ERR_ARG;
-    if (kind == SF_RF && (C < 1 || C > 16)) return SF_ERR_ARG;
+    if (kind != SF_GBDT && (C < 1 || C > 16)) return SF_ERR_ARG;
+    if (kind == SF_GBDT_MC && T % C != 0) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
     const uint32_t n_int = (1u << depth) - 1u, n_ent = 1u << depth;
     for (size_t i = 0; i < (size_t)T * n_int; i++) if (fid[i] >= F) return SF_ERR_ARG;
@@ -299,7 +360,7 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     // Image of one tree: 2^d node entries of 8 bytes in a 1-based heap (host node i, children
     // 2i+1 / 2i+2, becomes entry i+1, children 2j / 2j+1; entry 0 unused), then for boosted
     // trees the 2^d leaf scalars; padded to a multiple of 16 bytes for the 16-byte copies.
-    uint32_t stride = n_ent * 8u + (kind == SF_GBDT ? n_ent * 4u : 0u);
+    uint32_t stride = n_ent * 8u + (kind != SF_RF ? n_ent * 4u : 0u);
     stride = (stride + 15u) & ~15u;
     fo->tree_stride = stride;
     unsigned char* h = (unsigned char*)calloc((size_t)T, stride);
@@ -312,9 +373,9 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
             ent[2 * (i + 1)] = bits;
             ent[2 * (i + 1) + 1] = (uint32_t)fid[(size_t)t * n_int + i] * kB * 4u;     // byte offset of the feature's row
         }
-        if (kind == SF_GBDT) memcpy(h + (size_t)t * stride + n_ent * 8u, leaf + (size_t)t * n_ent, n_ent * 4u);
+        if (kind != SF_RF) memcpy(h + (size_t)t * stride + n_ent * 8u, leaf + (size_t)t * n_ent, n_ent * 4u);
     }
-    const size_t leaf_count = (size_t)T * n_ent * fo->C;
+    const size_t leaf_count = (size_t)T * n_ent * (kind == SF_RF ? fo->C : 1u);
     cudaError_t e = cudaMalloc(&fo->d_image, (size_t)T * stride);
     if (e == cudaSuccess) e = cudaMalloc(&fo->d_leaf, sizeof(float) * leaf_count);
     if (e == cudaSuccess) e = cudaMemcpy(fo->d_image, h, (size_t)T * stride, cudaMemcpyHostToDevice);

@@ -40,6 +40,11 @@ score_kernel(const float* __restrict__ fast_out, uint32_t n, uint32_t C, const f
                 float h = 0.0f;
                 for (uint32_t c = 0; c < C; c++) { float v = p[c]; if (v > 0.0f) h -= v * logf(v); }
                 u = h;
+            } else if (RULE == SF_SOFTMAX_LC_GT) {
+                // least confidence of softmax(margins): 1 - 1 / sum_j exp(m_j - m_max); fp32 expf, compared by tolerance
+                float sum = 0.0f;
+                for (uint32_t c = 0; c < C; c++) sum += expf(p[c] - mx);
+                u = 1.0f - 1.0f / sum;
             } else {
                 u = __fsub_rn(1.0f, mx);
             }
@@ -240,6 +245,8 @@ int sf_launch_score(const sf_route_cfg* cfg, const float* fast_out, uint32_t n, 
         score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
     else if (cfg->rule == SF_ENTROPY_GT)
         score_kernel<SF_ENTROPY_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
+    else if (cfg->rule == SF_SOFTMAX_LC_GT)
+        score_kernel<SF_SOFTMAX_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
     else
         score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, decision, label, score, block_counts, n_dev);
     SF_LAUNCH_CHECK("score_kernel");
@@ -311,6 +318,8 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
             score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         else if (cfg->rule == SF_ENTROPY_GT)
             score_kernel<SF_ENTROPY_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
+        else if (cfg->rule == SF_SOFTMAX_LC_GT)
+            score_kernel<SF_SOFTMAX_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         else
             score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast, score, block_counts, n_dev);
         SF_LAUNCH_CHECK("score_kernel");
@@ -363,7 +372,7 @@ extern "C" int sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_
                         uint8_t* decision_out, uint8_t* label_fast_out, float* score_out, void* stream)
 {
     if (!ctx || !cfg || !fast_out || !esc_ids_out || !n_esc_out || !cfg->tau) return SF_ERR_ARG;
-    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT && cfg->rule != SF_ENTROPY_GT) return SF_ERR_ARG;
+    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT && cfg->rule != SF_ENTROPY_GT && cfg->rule != SF_SOFTMAX_LC_GT) return SF_ERR_ARG;
     if (cfg->rule != SF_ABSMARGIN_LT && (C < 1 || C > 256)) return SF_ERR_ARG;
     if (rows_out) {
         if (!wide || !wide->size || !wide->iat_us || !wide->dir_bits || !wide->hdr) return SF_ERR_ARG;

@@ -30,7 +30,7 @@ def pinned_packets(pk, with_hdr=True):
 
 
 def make_forest(ctx, fo):
-    kind = sf.SF_RF if fo["kind"] == "rf" else sf.SF_GBDT
+    kind = {"rf": sf.SF_RF, "gbdt": sf.SF_GBDT, "gbdt_mc": sf.SF_GBDT_MC}[fo["kind"]]
     return sf.sf_forest_create(ctx, kind, fo["T"], fo["depth"], fo["F"], fo["C"], fo["fid"], fo["thr"], fo["leaf"])
 
 

@@ -462,3 +462,61 @@ def test_algorithm_2_per_class_thresholds(env, n, C, Q):
         tau, assigned = sf.sf_per_class_thresholds(ctx, hz.dev(u), hz.dev(pred), hz.dev(correct), n, C, Q, a, 100)
         assert np.array_equal(bits(tau), bits(ref_tau)) and assigned == ref_assigned
         assert assigned == int(np.count_nonzero(u > tau[pred]))
+
+
+# ------------------------------------------------------- multi-class boosted trees ---
+@pytest.mark.parametrize("C,rounds,depth,F,n", [(1, 9, 5, 24, 700), (2, 30, 6, 32, 5000), (3, 11, 4, 24, 1537),
+                                                 (5, 40, 6, 48, 4099), (8, 25, 8, 48, 3000), (11, 20, 6, 64, 2500),
+                                                 (16, 12, 7, 64, 1111), (7, 3, 9, 16, 513)])
+def test_gbdt_multiclass_margins_bit_exact(env, C, rounds, depth, F, n):
+    sf, hz, ctx = env
+    rng = np.random.default_rng(C * 100 + depth)
+    feat = rng.normal(size=(n, F)).astype(np.float32)
+    fo = flowgen.gen_forest(7 + C, "gbdt_mc", rounds * C, depth, F, C, feat, sigma=0.3)
+    ref, ref_li = oracle.forest_infer(fo, feat, want_leaf_idx=True, threads=4)
+    h = hz.make_forest(ctx, fo)
+    out = torch.full((n, C), 7.0, dtype=torch.float32, device="cuda")
+    li = torch.zeros((n, rounds * C), dtype=torch.uint16, device="cuda")
+    sf.sf_fast_infer(ctx, h, hz.dev(feat), n, out, li)
+    torch.cuda.synchronize()
+    assert sf.sf_ctx_poll(ctx, reset=True).device_error == 0
+    assert np.array_equal(li.cpu().numpy(), ref_li)
+    assert np.array_equal(bits(out.cpu().numpy()), bits(ref))
+    sf.sf_forest_destroy(h)
+
+
+def test_gbdt_multiclass_round_too_large_for_a_chunk_is_refused(env):
+    sf, hz, ctx = env
+    feat = np.random.default_rng(1).normal(size=(64, 16)).astype(np.float32)
+    fo = flowgen.gen_forest(3, "gbdt_mc", 4, 12, 16, 4, feat)          # 4 trees x 48 KB per round > 64 KB chunk
+    h = hz.make_forest(ctx, fo)
+    out = torch.zeros((64, 4), dtype=torch.float32, device="cuda")
+    with pytest.raises(Exception) as e:
+        sf.sf_fast_infer(ctx, h, hz.dev(feat), 64, out)
+    assert "unsupported" in str(e.value).lower() or "-6" in str(e.value)
+    sf.sf_forest_destroy(h)
+
+
+def test_route_softmax_least_confidence_within_tolerance(env):
+    sf, hz, ctx = env
+    n, C = 30011, 11
+    rng = np.random.default_rng(29)
+    m = (rng.normal(size=(n, C)) * rng.uniform(0.2, 3.0, (n, 1))).astype(np.float32)
+    m[5] = 0.25                                                  # all equal: LC = 1 - 1/C, label 0
+    tau = rng.uniform(0.3, 0.7, C).astype(np.float32)
+    ref = oracle.route_softmax_lc(m, tau)
+    cfg = sf.make_route_cfg(sf.SF_SOFTMAX_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, 64, n)
+    ids = torch.zeros(n, dtype=torch.uint32, device="cuda"); n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    dec = torch.empty(n, dtype=torch.uint8, device="cuda"); lab = torch.empty(n, dtype=torch.uint8, device="cuda")
+    sc = torch.empty(n, dtype=torch.float32, device="cuda")
+    sf.sf_route(ctx, cfg, hz.dev(m), n, C, None, ids, n_esc, None, dec, lab, sc)
+    torch.cuda.synchronize()
+    sf.sf_ctx_poll(ctx, reset=True)
+    score = sc.cpu().numpy(); d = dec.cpu().numpy()
+    assert np.max(np.abs(score - ref["score"])) <= 2e-6 and abs(score[5] - (1 - 1 / C)) <= 2e-6
+    assert np.array_equal(lab.cpu().numpy(), ref["label"]) and lab.cpu().numpy()[5] == 0
+    away = np.abs(ref["score"] - tau[ref["label"]]) > 1e-5
+    assert np.array_equal(d[away], ref["decision"][away])
+    k = int(n_esc.cpu().numpy()[0])
+    assert k == int(d.sum()) and np.array_equal(ids.cpu().numpy()[:k], np.nonzero(d)[0])
+    assert abs(k - ref["n_esc"]) <= int((~away).sum())

@@ -190,3 +190,45 @@ def test_empty_batch_and_nothing_assigned(env):
     torch.cuda.synchronize()
     assert int(n_esc.cpu().numpy()[0]) == 0 and sf.sf_ctx_poll(ctx, reset=True).device_error == 0
     sf.sf_slow_destroy(slow); sf.sf_forest_destroy(forest)
+
+
+def test_three_tier_with_boosted_fast_model(env):
+    """fastest (one decision tree, least confidence) -> fast (multi-class boosted trees, least confidence of the
+    softmax of their margins) -> slow.  The softmax is fp32 on the device, so flows whose tier-2 score lies within
+    1e-5 of its threshold may legitimately differ; everything else must match."""
+    sf, hz, ctx = env
+    n = 6000
+    cfg = dataclasses.replace(flowgen.get_config(2), n=n)
+    wl = make_workload(cfg, n=n)
+    feat = oracle.extract_features(wl["fast"], cfg.N, cfg.F, threads=8)
+    fastest = flowgen.gen_forest(4243, "rf", 1, 7, cfg.F, cfg.C, feat)
+    fast = flowgen.gen_forest(4244, "gbdt_mc", 30 * cfg.C, 6, cfg.F, cfg.C, feat, sigma=0.25)
+    rng = np.random.default_rng(9)
+    tau1 = rng.uniform(0.2, 0.6, cfg.C).astype(np.float32)
+    tau2 = rng.uniform(0.55, 0.7, cfg.C).astype(np.float32)
+    ref = oracle.serve_batch3(cfg, wl["fast"], wl["wide"], fastest, fast, wl["slow"], tau1, tau2, threads=8)
+    band = np.zeros(n, bool)
+    band[ref["ids1"]] = np.abs(ref["score2"] - tau2[ref["label2"]]) <= 1e-5
+    h1 = hz.make_forest(ctx, fastest); h2 = hz.make_forest(ctx, fast); hs = hz.make_slow(ctx, cfg, wl["slow"])
+    fast_d = hz.upload_packets(wl["fast"], with_hdr=False); wide_d = hz.upload_packets(wl["wide"])
+    cfg1 = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau1), sf.SF_MLP16, sf.SF_BF16, cfg.P, n)
+    cfg2 = sf.make_route_cfg(sf.SF_SOFTMAX_LC_GT, hz.dev(tau2), sf.SF_MLP16, sf.SF_BF16, cfg.P, n)
+    label = torch.full((n,), 255, dtype=torch.uint8, device="cuda")
+    stage = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.uint32, device="cuda")
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_serve_batch3(ctx, h1, h2, hs, fast_d["struct"], cfg.N, cfg.F, wide_d["struct"], cfg1, cfg2, label, stage, cnt)
+    torch.cuda.synchronize()
+    assert sf.sf_ctx_poll(ctx, reset=True).device_error == 0
+    k1, k2 = [int(x) for x in cnt.cpu().numpy()]
+    assert k1 == len(ref["ids1"]) and abs(k2 - len(ref["ids2"])) <= int(band.sum()) and 0 < k2 < k1 < n
+    assert len(ref["ids2"]) > 200 and band.sum() < 20
+    st = stage.cpu().numpy(); lab = label.cpu().numpy()
+    ok = ~band
+    assert np.array_equal(st[ok], ref["stage"][ok])
+    sel = ok & (st < 3)
+    assert np.array_equal(lab[sel], ref["label_final"][sel])
+    s = np.sort(ref["logits"], axis=1)
+    clear = ((s[:, -1] - s[:, -2]) >= 4e-2) & ok[ref["ids2"]]
+    assert np.array_equal(lab[ref["ids2"]][clear], ref["label_slow"][clear])
+    sf.sf_slow_destroy(hs); sf.sf_forest_destroy(h2); sf.sf_forest_destroy(h1)
