@@ -108,7 +108,8 @@ int  sf_ctx_poll(sf_ctx* ctx, sf_counters* host_out, int reset, void* stream);
 #define SF_T_HEAD    5   /* S4 last layer + argmax */
 #define SF_T_MERGE   6   /* S5 merge kernels */
 #define SF_T_TABLE   7   /* streaming table kernels */
-#define SF_N_TIMERS  8
+#define SF_T_PULL    8   /* host entry point: kernel that fetches the assigned flows' rows from pinned host memory */
+#define SF_N_TIMERS  9
 int  sf_ctx_set_timing(sf_ctx* ctx, int enable);
 int  sf_ctx_get_timing(sf_ctx* ctx, uint32_t back, float* ms_host_out, void* stream);
 
@@ -302,10 +303,15 @@ int  sf_serve_batch(sf_ctx* ctx, const sf_forest* forest, const sf_slow* slow, c
                     uint32_t N, uint32_t F, const sf_packets* slow_ctx, const sf_route_cfg* cfg,
                     uint8_t* label_out, uint8_t* stage_out, uint32_t* n_esc_out, void* stream);
 /* Same, but every plane pointer of fast_ctx / slow_ctx, cfg->tau, label_out,
- * stage_out and n_esc_out are HOST pointers (pinned memory recommended): the
- * planes are copied to device staging buffers owned by the context, the cascade
- * runs, the three outputs are copied back, and the call returns after
- * synchronising the stream. */
+ * stage_out and n_esc_out are HOST pointers, and the call returns after
+ * synchronising the stream.  With separate fast and slow planes only what the
+ * method needs crosses the bus: the fast planes of all flows go up, S1..S3 run,
+ * and then only the ASSIGNED flows' slow-context rows follow.  If the slow planes
+ * are pinned host memory that the device can address (cudaHostAlloc /
+ * cudaHostRegister), a kernel reads those rows straight out of them with no work on
+ * the host; otherwise the id list comes back, host threads compact the rows into the
+ * context's pinned buffer and they are copied up in chunks.  With shared planes
+ * everything is copied to device staging buffers first. */
 int  sf_serve_batch_host(sf_ctx* ctx, const sf_forest* forest, const sf_slow* slow, const sf_packets* fast_ctx_host,
                          uint32_t N, uint32_t F, const sf_packets* slow_ctx_host, const sf_route_cfg* cfg_host_tau,
                          uint8_t* label_host_out, uint8_t* stage_host_out, uint32_t* n_esc_host_out, void* stream);

@@ -206,7 +206,7 @@ def sf_ctx_poll(ctx, reset=False, stream=None, raise_on_error=True):
     return c
 
 
-SF_TIMER_NAMES = ("extract", "forest", "score", "gather", "gemm", "head", "merge", "table")
+SF_TIMER_NAMES = ("extract", "forest", "score", "gather", "gemm", "head", "merge", "table", "pull")
 
 
 def sf_ctx_set_timing(ctx, enable):

@@ -226,6 +226,47 @@ int check_serve_args(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const s
     return SF_OK;
 }
 
+// Pull path of the host entry point: when the caller's wide planes are pinned host memory that the
+// device can address, the assigned flows' rows are read straight out of it by this kernel (a warp per
+// flow, 16-byte loads, every byte crosses the bus once) into compact device planes in list order -
+// no host-side compaction, no round trip for the id list.
+struct PullPlanes {
+    const unsigned char* src[5]; unsigned char* dst[5]; uint32_t row_bytes[5];     // size, iat, dir words, header bytes, n_valid
+};
+
+__global__ void __launch_bounds__(256)
+pull_rows_kernel(PullPlanes pl, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ n_ids, uint32_t capacity)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t n = min(*n_ids, capacity);
+    for (uint32_t r = blockIdx.x * 8 + (threadIdx.x >> 5); r < n; r += gridDim.x * 8) {
+        const size_t f = ids[r];
+#pragma unroll
+        for (int p = 0; p < 5; p++) {
+            const uint32_t rb = pl.row_bytes[p];
+            if (rb == 0) continue;
+            const unsigned char* s = pl.src[p] + f * rb;
+            unsigned char* d = pl.dst[p] + (size_t)r * rb;
+            if ((rb & 15u) == 0 && ((uintptr_t)pl.src[p] & 15u) == 0) {
+                for (uint32_t o = lane * 16; o < rb; o += 512) *reinterpret_cast<uint4*>(d + o) = *reinterpret_cast<const uint4*>(s + o);
+            } else if ((rb & 3u) == 0 && ((uintptr_t)pl.src[p] & 3u) == 0) {
+                for (uint32_t o = lane * 4; o < rb; o += 128) *reinterpret_cast<uint32_t*>(d + o) = *reinterpret_cast<const uint32_t*>(s + o);
+            } else {
+                for (uint32_t o = lane; o < rb; o += 32) d[o] = s[o];
+            }
+        }
+    }
+}
+
+// device-side alias of a host pointer if it is pinned and mapped, else nullptr
+const void* mapped_alias(const void* host_ptr) {
+    if (!host_ptr) return nullptr;
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (a.type != cudaMemoryTypeHost || !a.devicePointer) return nullptr;
+    return a.devicePointer;
+}
+
 // phases: 1 = S1..S3 without the wide-row gather, 2 = gather (rows 0..n_esc-1 of `wide`, which then holds
 // only the assigned flows' planes in list order) + S4 + S5 on the state phase 1 left, 3 = everything.
 enum { SF_PHASE_FAST = 1, SF_PHASE_SLOW = 2, SF_PHASE_ALL = 3 };
@@ -421,26 +462,82 @@ extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_sl
         rc = serve_on_device(ctx, fo, s, &fd2, N, F, wide_h, &cd2, (uint8_t*)(sb2 + a_lab), (uint8_t*)(sb2 + a_stg),
                              (uint32_t*)(sb2 + a_ne), st, SF_PHASE_FAST);
         if (rc != SF_OK) return rc;
+        const size_t r_sz = (size_t)Pw * 2, r_ia = (size_t)Pw * 4, r_dr = (size_t)words * 4, r_hd = (size_t)Pw * Hb;
+        {
+            // Pull path: all wide planes pinned and device-addressable -> the device fetches the assigned rows itself.
+            const void* m_sz = mapped_alias(wide_h->size); const void* m_ia = mapped_alias(wide_h->iat_us);
+            const void* m_dr = mapped_alias(wide_h->dir_bits); const void* m_hd = mapped_alias(wide_h->hdr);
+            const void* m_nv = wide_h->n_valid ? mapped_alias(wide_h->n_valid) : nullptr;
+            if (m_sz && m_ia && m_dr && m_hd && (!wide_h->n_valid || m_nv)) {
+                const size_t kc = std::min<size_t>(cfg_h->capacity, n);
+                const size_t c_sz = 0, c_ia = sf_align256(c_sz + kc * r_sz), c_dr = sf_align256(c_ia + kc * r_ia),
+                             c_hd = sf_align256(c_dr + kc * r_dr), c_nv = sf_align256(c_hd + kc * r_hd),
+                             c_total = sf_align256(c_nv + (wide_h->n_valid ? kc : 0)) + 256;
+                if (c_total > ctx->stage2_bytes) {
+                    SF_CUDA(cudaDeviceSynchronize());
+                    if (ctx->stage2) { cudaFree(ctx->stage2); ctx->stage2 = nullptr; }
+                    ctx->stage2_bytes = 0;
+                    cudaError_t e = cudaMalloc(&ctx->stage2, c_total);
+                    if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(pulled rows)"); return SF_ERR_ALLOC; }
+                    ctx->stage2_bytes = c_total;
+                }
+                char* dv = ctx->stage2;
+                PullPlanes pl;
+                pl.src[0] = (const unsigned char*)m_sz; pl.dst[0] = (unsigned char*)dv + c_sz; pl.row_bytes[0] = (uint32_t)r_sz;
+                pl.src[1] = (const unsigned char*)m_ia; pl.dst[1] = (unsigned char*)dv + c_ia; pl.row_bytes[1] = (uint32_t)r_ia;
+                pl.src[2] = (const unsigned char*)m_dr; pl.dst[2] = (unsigned char*)dv + c_dr; pl.row_bytes[2] = (uint32_t)r_dr;
+                pl.src[3] = (const unsigned char*)m_hd; pl.dst[3] = (unsigned char*)dv + c_hd; pl.row_bytes[3] = (uint32_t)r_hd;
+                pl.src[4] = (const unsigned char*)m_nv; pl.dst[4] = (unsigned char*)dv + c_nv; pl.row_bytes[4] = m_nv ? 1u : 0u;
+                if (kc) {
+                    const uint32_t grid = (uint32_t)std::min<size_t>((kc + 7) / 8, (size_t)ctx->num_sms * 8);
+                    sf_time_begin(ctx, SF_T_PULL, st);
+                    pull_rows_kernel<<<grid, 256, 0, st>>>(pl, ctx->last_esc_ids, (const uint32_t*)(sb2 + a_ne), (uint32_t)kc);
+                    sf_time_end(ctx, SF_T_PULL, st);
+                    SF_LAUNCH_CHECK("pull_rows_kernel");
+                }
+                sf_packets wd2 = *wide_h;
+                wd2.size = (const uint16_t*)(dv + c_sz); wd2.iat_us = (const uint32_t*)(dv + c_ia);
+                wd2.dir_bits = (const uint32_t*)(dv + c_dr); wd2.hdr = (const uint8_t*)(dv + c_hd);
+                wd2.n_valid = wide_h->n_valid ? (const uint8_t*)(dv + c_nv) : nullptr;
+                wd2.n_flows = (uint32_t)kc;
+                rc = serve_on_device(ctx, fo, s, &fd2, N, F, &wd2, &cd2, (uint8_t*)(sb2 + a_lab), (uint8_t*)(sb2 + a_stg),
+                                     (uint32_t*)(sb2 + a_ne), st, SF_PHASE_SLOW);
+                if (rc != SF_OK) return rc;
+                uint32_t k_host = 0;
+                SF_CUDA(cudaMemcpyAsync(label_h, sb2 + a_lab, n, cudaMemcpyDeviceToHost, st));
+                SF_CUDA(cudaMemcpyAsync(stage_h, sb2 + a_stg, n, cudaMemcpyDeviceToHost, st));
+                SF_CUDA(cudaMemcpyAsync(&k_host, sb2 + a_ne, 4, cudaMemcpyDeviceToHost, st));
+                SF_CUDA(cudaStreamSynchronize(st));
+                if (n_esc_h) *n_esc_h = k_host;
+                return SF_OK;
+            }
+        }
         uint32_t k = 0;
         SF_CUDA(cudaMemcpyAsync(&k, sb2 + a_ne, 4, cudaMemcpyDeviceToHost, st));
         SF_CUDA(cudaStreamSynchronize(st));
         std::vector<uint32_t> ids(k);
         if (k) SF_CUDA(cudaMemcpy(ids.data(), ctx->last_esc_ids, (size_t)k * 4, cudaMemcpyDeviceToHost));
         // compact planes of the k assigned flows: [k][Pw] sizes, [k][Pw] iats, [k][words] dir words, [k][Pw][Hb] header bytes, [k] n_valid
-        const size_t r_sz = (size_t)Pw * 2, r_ia = (size_t)Pw * 4, r_dr = (size_t)words * 4, r_hd = (size_t)Pw * Hb;
         const size_t c_sz = 0, c_ia = sf_align256(c_sz + k * r_sz), c_dr = sf_align256(c_ia + k * r_ia),
                      c_hd = sf_align256(c_dr + k * r_dr), c_nv = sf_align256(c_hd + k * r_hd),
                      c_total = sf_align256(c_nv + (wide_h->n_valid ? k : 0)) + 256;
-        if (c_total > ctx->stage2_bytes) {
+        if (c_total > ctx->stage2_bytes || c_total > ctx->pin_bytes) {
             SF_CUDA(cudaDeviceSynchronize());
-            if (ctx->stage2) { cudaFree(ctx->stage2); ctx->stage2 = nullptr; }
-            if (ctx->pin) { cudaFreeHost(ctx->pin); ctx->pin = nullptr; }
-            ctx->stage2_bytes = 0;
             const size_t want = c_total + c_total / 4;
-            cudaError_t e = cudaMalloc(&ctx->stage2, want);
-            if (e == cudaSuccess) e = cudaMallocHost(&ctx->pin, want);
+            cudaError_t e = cudaSuccess;
+            if (c_total > ctx->stage2_bytes) {
+                if (ctx->stage2) { cudaFree(ctx->stage2); ctx->stage2 = nullptr; }
+                ctx->stage2_bytes = 0;
+                e = cudaMalloc(&ctx->stage2, want);
+                if (e == cudaSuccess) ctx->stage2_bytes = want;
+            }
+            if (e == cudaSuccess && c_total > ctx->pin_bytes) {
+                if (ctx->pin) { cudaFreeHost(ctx->pin); ctx->pin = nullptr; }
+                ctx->pin_bytes = 0;
+                e = cudaMallocHost(&ctx->pin, want);
+                if (e == cudaSuccess) ctx->pin_bytes = want;
+            }
             if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(compact staging)"); return SF_ERR_ALLOC; }
-            ctx->stage2_bytes = want;
         }
         char* pin = ctx->pin; char* dv = ctx->stage2;
         const uint32_t chunk = 4096, n_chunks = (k + chunk - 1) / chunk;

@@ -30,6 +30,7 @@ struct sf_ctx {
     char*  stage2;               // compact wide planes of the assigned flows (device) and their pinned host mirror
     char*  pin;
     size_t stage2_bytes;
+    size_t pin_bytes;
     // optional per-kernel-class timing: ring of event pairs
     int timing;
     uint32_t t_rec;                               // records started so far

@@ -19,11 +19,14 @@ def upload_packets(pk, n_valid=None, device="cuda:0", with_hdr=True):
     return t
 
 
-def pinned_packets(pk, with_hdr=True):
-    """Pinned host copies (for the host-pointer entry point)."""
+def pinned_packets(pk, with_hdr=True, pinned=True):
+    """Host copies for the host-pointer entry point: pinned (the device can address them: the assigned
+    rows are pulled straight out of them) or pageable (staged through the library's own pinned buffer)."""
     t = {}
     for k in ("size", "iat_us", "dir_bits") + (("hdr",) if with_hdr else ()):
-        t[k] = torch.from_numpy(np.ascontiguousarray(pk[k])).pin_memory()
+        t[k] = torch.from_numpy(np.ascontiguousarray(pk[k]).copy())
+        if pinned:
+            t[k] = t[k].pin_memory()
     hdr = t.get("hdr")
     t["struct"] = sf.make_packets(t["size"], t["iat_us"], t["dir_bits"], hdr, None)
     return t

@@ -76,6 +76,14 @@ def run_and_check(sf, hz, ctx, wl, capacity=None):
     lab_h = np.zeros(n, np.uint8); st_h = np.zeros(n, np.uint8); ne_h = np.zeros(1, np.uint32)
     sf.sf_serve_batch_host(ctx, forest, slow, fast_h["struct"], cfg.N, cfg.F, wide_h["struct"], rcfg_h, lab_h, st_h, ne_h)
     assert int(ne_h[0]) == k and np.array_equal(lab_h, lab) and np.array_equal(st_h, st)
+    # pageable host planes take the staged route (host-side compaction into the library's pinned buffer)
+    fast_p = hz.pinned_packets(wl["fast"], with_hdr=False, pinned=False)
+    wide_p = hz.pinned_packets(wl["wide"], pinned=False)
+    lab_p = np.zeros(n, np.uint8); st_p = np.zeros(n, np.uint8); ne_p = np.zeros(1, np.uint32)
+    sf.sf_serve_batch_host(ctx, forest, slow, fast_p["struct"], cfg.N, cfg.F, wide_p["struct"], rcfg_h, lab_p, st_p, ne_p)
+    assert int(ne_p[0]) == k and np.array_equal(lab_p, lab) and np.array_equal(st_p, st)
+    sf.sf_serve_batch_host(ctx, forest, slow, fast_h["struct"], cfg.N, cfg.F, wide_h["struct"], rcfg_h, lab_h, st_h, ne_h)   # and back
+    assert int(ne_h[0]) == k and np.array_equal(lab_h, lab) and np.array_equal(st_h, st)
     sf.sf_ctx_poll(ctx, reset=True)
     sf.sf_slow_destroy(slow)
     sf.sf_forest_destroy(forest)
