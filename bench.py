@@ -439,12 +439,17 @@ def main():
             step_host()
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+        sf.sf_ctx_set_timing(ctx, True)                    # one more call, untimed, for where the time goes
+        step_host()
+        e2e_stages = {k: round(v, 4) for k, v in sf.sf_ctx_get_timing(ctx, 0).items() if v > 0}
+        sf.sf_ctx_set_timing(ctx, False)
         # the library copies the fast planes of all flows, then only the assigned flows' wide rows
         h2d = sum(int(fast_h[k].numel() * fast_h[k].element_size()) for k in ("size", "iat_us", "dir_bits")) + \
             k_esc * (cfg.P * (6 + cfg.H) + 4 * ((cfg.P + 31) // 32)) + 4 * len(wl["tau"])
         e2e = {"value": world * n / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 2 * n + 4,
-               "ms_per_step": e2e_s * 1e3,
-               "note": "sf_serve_batch_host: pinned host planes in (fast planes copied up, the assigned flows' slow-context rows "
+               "ms_per_step": e2e_s * 1e3, "span_ms": e2e_stages,
+               "note": "span_ms = first start to last end of each kernel class inside one call (classes overlap); "
+                       "sf_serve_batch_host: pinned host planes in (fast planes copied up, the assigned flows' slow-context rows "
                        "read out of pinned memory by a kernel), labels out, synchronous; measured on rank 0"}
         assert np.array_equal(lab_h.numpy(), label.cpu().numpy())
 

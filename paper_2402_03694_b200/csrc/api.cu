@@ -134,6 +134,7 @@ extern "C" void sf_ctx_destroy(sf_ctx* c) {
     if (c->ws) cudaFree(c->ws);
     if (c->stage) cudaFree(c->stage);
     if (c->stage2) cudaFree(c->stage2);
+    if (c->aux) { cudaStreamDestroy(c->aux); cudaEventDestroy(c->ev_aux); cudaEventDestroy(c->ev_main); }
     if (c->pin) cudaFreeHost(c->pin);
     if (c->d_state) cudaFree(c->d_state);
     if (c->t_ev[0][0][0])
@@ -235,11 +236,11 @@ struct PullPlanes {
 };
 
 __global__ void __launch_bounds__(256)
-pull_rows_kernel(PullPlanes pl, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ n_ids, uint32_t capacity)
+pull_rows_kernel(PullPlanes pl, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ n_ids, uint32_t r_begin, uint32_t r_end)
 {
     const uint32_t lane = threadIdx.x & 31;
-    const uint32_t n = min(*n_ids, capacity);
-    for (uint32_t r = blockIdx.x * 8 + (threadIdx.x >> 5); r < n; r += gridDim.x * 8) {
+    const uint32_t n = min(*n_ids, r_end);
+    for (uint32_t r = r_begin + blockIdx.x * 8 + (threadIdx.x >> 5); r < n; r += gridDim.x * 8) {
         const size_t f = ids[r];
 #pragma unroll
         for (int p = 0; p < 5; p++) {
@@ -256,6 +257,16 @@ pull_rows_kernel(PullPlanes pl, const uint32_t* __restrict__ ids, const uint32_t
             }
         }
     }
+}
+
+// rows of the list that fall into each chunk of R rows
+__global__ void chunk_counts_kernel(const uint32_t* __restrict__ n_total, uint32_t cap, uint32_t R, uint32_t n_chunks,
+                                    uint32_t* __restrict__ cnt)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_chunks) return;
+    const uint32_t k = min(*n_total, cap), c0 = i * R;
+    cnt[i] = k > c0 ? min(k - c0, R) : 0u;
 }
 
 // device-side alias of a host pointer if it is pinned and mapped, else nullptr
@@ -325,6 +336,145 @@ int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf
     if (rc != SF_OK) return rc;
     ctx->last_feat = feat; ctx->last_fast_out = fast_out; ctx->last_esc_ids = esc_ids; ctx->last_rows = rows;
     ctx->last_logits = logits; ctx->last_label_fast = label_fast; ctx->last_label_slow = label_slow;
+    return SF_OK;
+}
+
+// Host entry point, pull route (separate fast and slow planes, slow planes pinned and device-addressable).
+// Two streams: transfers run on the context's second stream, kernels on the caller's.
+//   A  the fast planes go up in chunks of whole forest waves; extract + forest of a chunk start as soon
+//      as it has landed, so only the first chunk's copy and the last chunk's kernels are exposed;
+//   B  route over all flows; the count comes back (4 bytes) so that only chunks with rows are launched;
+//   C  the assigned flows' slow-context rows are pulled out of the pinned planes in chunks of 32,768 rows;
+//      gather + slow model of a chunk run while the next chunk crosses the bus;
+//   D  merge, labels back.
+int serve_host_pull(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf_packets* fast_h, uint32_t N, uint32_t F,
+                    const sf_packets* wide_h, const void* const m_wide[5], const sf_route_cfg* cfg_h, char* sb2,
+                    const size_t a_fast[4], size_t a_tau, size_t a_lab, size_t a_stg, size_t a_ne, uint32_t n_tau,
+                    uint8_t* label_h, uint8_t* stage_h, uint32_t* n_esc_h, cudaStream_t st)
+{
+    const uint32_t n = fast_h->n_flows, Pf = fast_h->pitch_pkts, wf = (Pf + 31) / 32;
+    const uint32_t Pw = wide_h->pitch_pkts, Hb = wide_h->hdr_bytes, words = (Pw + 31) / 32;
+    if (!ctx->aux) {
+        SF_CUDA(cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking));
+        SF_CUDA(cudaEventCreateWithFlags(&ctx->ev_aux, cudaEventDisableTiming));
+        SF_CUDA(cudaEventCreateWithFlags(&ctx->ev_main, cudaEventDisableTiming));
+    }
+    cudaStream_t sx = ctx->aux;
+    sf_route_cfg cd = *cfg_h;
+    cd.tau = (const float*)(sb2 + a_tau);
+    const ServePlan p = plan_serve(fo, s, n, F, &cd);
+    int rc = sf_ws_reserve(ctx, p.total);
+    if (rc != SF_OK) return rc;
+    sf_ws_reset(ctx);
+    char* base = reinterpret_cast<char*>(sf_ws_alloc(ctx, p.total));
+    if (!base) return SF_ERR_ALLOC;
+    float* feat = (float*)(base + p.feat); float* fast_out = (float*)(base + p.fast_out);
+    uint8_t* decision = (uint8_t*)(base + p.decision); uint8_t* label_fast = (uint8_t*)(base + p.label_fast);
+    uint32_t* esc_ids = (uint32_t*)(base + p.esc_ids); uint32_t* iota = (uint32_t*)(base + p.iota);
+    char* rows = base + p.rows; float* logits = (float*)(base + p.logits); uint8_t* label_slow = (uint8_t*)(base + p.label_slow);
+    uint32_t* n_esc_dev = &ctx->d_state->scan_total;
+    const uint32_t Cf = fo->kind == SF_GBDT ? 1 : fo->C;
+    sf_time_new_record(ctx);
+
+    // A: uploads on sx, kernels on st
+    SF_CUDA(cudaMemcpyAsync(sb2 + a_tau, cfg_h->tau, (size_t)n_tau * 4, cudaMemcpyHostToDevice, st));
+    SF_CUDA(cudaEventRecord(ctx->ev_main, st));
+    SF_CUDA(cudaStreamWaitEvent(sx, ctx->ev_main, 0));            // the staging buffers are free once earlier work on st is done
+    const uint32_t FC = (uint32_t)ctx->num_sms * 512u * 2u;       // two full waves of the forest kernel
+    for (uint32_t f0 = 0; f0 < n; f0 += FC) {
+        const uint32_t m = std::min(FC, n - f0);
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_fast[0] + (size_t)f0 * Pf * 2, (const char*)fast_h->size + (size_t)f0 * Pf * 2, (size_t)m * Pf * 2, cudaMemcpyHostToDevice, sx));
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_fast[1] + (size_t)f0 * Pf * 4, (const char*)fast_h->iat_us + (size_t)f0 * Pf * 4, (size_t)m * Pf * 4, cudaMemcpyHostToDevice, sx));
+        SF_CUDA(cudaMemcpyAsync(sb2 + a_fast[2] + (size_t)f0 * wf * 4, (const char*)fast_h->dir_bits + (size_t)f0 * wf * 4, (size_t)m * wf * 4, cudaMemcpyHostToDevice, sx));
+        if (fast_h->n_valid)
+            SF_CUDA(cudaMemcpyAsync(sb2 + a_fast[3] + f0, fast_h->n_valid + f0, m, cudaMemcpyHostToDevice, sx));
+        SF_CUDA(cudaEventRecord(ctx->ev_aux, sx));
+        SF_CUDA(cudaStreamWaitEvent(st, ctx->ev_aux, 0));
+        sf_packets fc = *fast_h;
+        fc.size = (const uint16_t*)(sb2 + a_fast[0]) + (size_t)f0 * Pf; fc.iat_us = (const uint32_t*)(sb2 + a_fast[1]) + (size_t)f0 * Pf;
+        fc.dir_bits = (const uint32_t*)(sb2 + a_fast[2]) + (size_t)f0 * wf; fc.hdr = nullptr;
+        fc.n_valid = fast_h->n_valid ? (const uint8_t*)(sb2 + a_fast[3]) + f0 : nullptr;
+        fc.n_flows = m;
+        sf_time_begin(ctx, SF_T_EXTRACT, st);
+        rc = sf_launch_extract(&fc, N, F, feat + (size_t)f0 * F, st);
+        sf_time_end(ctx, SF_T_EXTRACT, st);
+        if (rc != SF_OK) return rc;
+        sf_time_begin(ctx, SF_T_FOREST, st);
+        rc = sf_launch_forest(fo, feat + (size_t)f0 * F, m, fast_out + (size_t)f0 * Cf, nullptr, st);
+        sf_time_end(ctx, SF_T_FOREST, st);
+        if (rc != SF_OK) return rc;
+    }
+    // B: assignment over all flows; the count comes back
+    rc = sf_launch_route(ctx, &cd, fast_out, n, fo->C, nullptr, esc_ids, (uint32_t*)(sb2 + a_ne), nullptr, decision, label_fast,
+                         nullptr, base + p.route_scratch, st);
+    if (rc != SF_OK) return rc;
+    uint32_t k = 0;
+    SF_CUDA(cudaMemcpyAsync(&k, sb2 + a_ne, 4, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaStreamSynchronize(st));
+    // C: pull, gather and slow model chunk by chunk
+    const size_t r_sz = (size_t)Pw * 2, r_ia = (size_t)Pw * 4, r_dr = (size_t)words * 4, r_hd = (size_t)Pw * Hb;
+    const size_t esz = cd.row_dtype == SF_BF16 ? 2 : 4, D = slow_width(s), Cs = slow_classes(s);
+    if (k) {
+        const uint32_t R = std::min<uint32_t>(32768u, cd.capacity), n_chunks = (k + R - 1) / R;
+        const size_t c_sz = 0, c_ia = sf_align256(c_sz + k * r_sz), c_dr = sf_align256(c_ia + k * r_ia),
+                     c_hd = sf_align256(c_dr + k * r_dr), c_nv = sf_align256(c_hd + k * r_hd),
+                     c_cnt = sf_align256(c_nv + (wide_h->n_valid ? k : 0)), c_total = c_cnt + sf_align256((size_t)n_chunks * 4) + 256;
+        if (c_total > ctx->stage2_bytes) {
+            SF_CUDA(cudaDeviceSynchronize());
+            if (ctx->stage2) { cudaFree(ctx->stage2); ctx->stage2 = nullptr; }
+            ctx->stage2_bytes = 0;
+            const size_t want = c_total + c_total / 4;
+            cudaError_t e = cudaMalloc(&ctx->stage2, want);
+            if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(pulled rows)"); return SF_ERR_ALLOC; }
+            ctx->stage2_bytes = want;
+        }
+        char* dv = ctx->stage2;
+        uint32_t* cnt = (uint32_t*)(dv + c_cnt);
+        PullPlanes pl;
+        const size_t c_off[5] = {c_sz, c_ia, c_dr, c_hd, c_nv};
+        const uint32_t rb[5] = {(uint32_t)r_sz, (uint32_t)r_ia, (uint32_t)r_dr, (uint32_t)r_hd, wide_h->n_valid ? 1u : 0u};
+        for (int q = 0; q < 5; q++) { pl.src[q] = (const unsigned char*)m_wide[q]; pl.dst[q] = (unsigned char*)dv + c_off[q]; pl.row_bytes[q] = rb[q]; }
+        chunk_counts_kernel<<<(n_chunks + 255) / 256, 256, 0, st>>>(n_esc_dev, cd.capacity, R, n_chunks, cnt);
+        SF_LAUNCH_CHECK("chunk_counts_kernel");
+        rc = sf_launch_iota(iota, R, st);
+        if (rc != SF_OK) return rc;
+        SF_CUDA(cudaEventRecord(ctx->ev_main, st));
+        SF_CUDA(cudaStreamWaitEvent(sx, ctx->ev_main, 0));
+        sf_time_begin(ctx, SF_T_PULL, sx);
+        for (uint32_t c = 0; c < n_chunks; c++) {
+            const uint32_t r0 = c * R, r1 = std::min(k, r0 + R);
+            const uint32_t grid = std::min<uint32_t>((r1 - r0 + 7) / 8, (uint32_t)ctx->num_sms * 4u);
+            pull_rows_kernel<<<grid, 256, 0, sx>>>(pl, esc_ids, n_esc_dev, r0, r1);
+            SF_LAUNCH_CHECK("pull_rows_kernel");
+            if (c + 1 == n_chunks) sf_time_end(ctx, SF_T_PULL, sx);
+            SF_CUDA(cudaEventRecord(ctx->ev_aux, sx));
+            SF_CUDA(cudaStreamWaitEvent(st, ctx->ev_aux, 0));
+            sf_packets wc = *wide_h;
+            wc.size = (const uint16_t*)(dv + c_sz + r0 * r_sz); wc.iat_us = (const uint32_t*)(dv + c_ia + r0 * r_ia);
+            wc.dir_bits = (const uint32_t*)(dv + c_dr + r0 * r_dr); wc.hdr = (const uint8_t*)(dv + c_hd + r0 * r_hd);
+            wc.n_valid = wide_h->n_valid ? (const uint8_t*)(dv + c_nv + r0) : nullptr;
+            wc.n_flows = r1 - r0;
+            sf_time_begin(ctx, SF_T_GATHER, st);
+            rc = sf_launch_gather(ctx, &cd, &wc, iota, cnt + c, R, rows + (size_t)r0 * D * esz, st);
+            sf_time_end(ctx, SF_T_GATHER, st);
+            if (rc != SF_OK) return rc;
+            rc = sf_launch_slow(ctx, s, rows + (size_t)r0 * D * esz, cnt + c, R, logits + (size_t)r0 * Cs, label_slow + r0,
+                                base + p.slow_scratch, st);
+            if (rc != SF_OK) return rc;
+        }
+    }
+    // D: merge and results
+    sf_time_begin(ctx, SF_T_MERGE, st);
+    rc = sf_launch_merge(label_fast, decision, n, esc_ids, n_esc_dev, cd.capacity, label_slow, (uint8_t*)(sb2 + a_lab),
+                         (uint8_t*)(sb2 + a_stg), st);
+    sf_time_end(ctx, SF_T_MERGE, st);
+    if (rc != SF_OK) return rc;
+    ctx->last_feat = feat; ctx->last_fast_out = fast_out; ctx->last_esc_ids = esc_ids; ctx->last_rows = rows;
+    ctx->last_logits = logits; ctx->last_label_fast = label_fast; ctx->last_label_slow = label_slow;
+    SF_CUDA(cudaMemcpyAsync(label_h, sb2 + a_lab, n, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaMemcpyAsync(stage_h, sb2 + a_stg, n, cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaStreamSynchronize(st));
+    if (n_esc_h) *n_esc_h = k;
     return SF_OK;
 }
 
@@ -448,6 +598,15 @@ extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_sl
             ctx->stage_bytes = off2;
         }
         char* sb2 = ctx->stage;
+        {
+            const void* m_wide[5] = {mapped_alias(wide_h->size), mapped_alias(wide_h->iat_us), mapped_alias(wide_h->dir_bits),
+                                     mapped_alias(wide_h->hdr), wide_h->n_valid ? mapped_alias(wide_h->n_valid) : nullptr};
+            if (m_wide[0] && m_wide[1] && m_wide[2] && m_wide[3] && (!wide_h->n_valid || m_wide[4])) {
+                const size_t a_fast[4] = {a_fs, a_fi, a_fd, a_fv};
+                return serve_host_pull(ctx, fo, s, fast_h, N, F, wide_h, m_wide, cfg_h, sb2, a_fast, a_tau, a_lab, a_stg, a_ne,
+                                       n_tau2, label_h, stage_h, n_esc_h, st);
+            }
+        }
         SF_CUDA(cudaMemcpyAsync(sb2 + a_fs, fast_h->size, fsz, cudaMemcpyHostToDevice, st));
         SF_CUDA(cudaMemcpyAsync(sb2 + a_fi, fast_h->iat_us, fia, cudaMemcpyHostToDevice, st));
         SF_CUDA(cudaMemcpyAsync(sb2 + a_fd, fast_h->dir_bits, fdr, cudaMemcpyHostToDevice, st));
@@ -459,59 +618,10 @@ extern "C" int sf_serve_batch_host(sf_ctx* ctx, const sf_forest* fo, const sf_sl
         fd2.n_valid = fnv ? (const uint8_t*)(sb2 + a_fv) : nullptr;
         sf_route_cfg cd2 = *cfg_h;
         cd2.tau = (const float*)(sb2 + a_tau);
+        const size_t r_sz = (size_t)Pw * 2, r_ia = (size_t)Pw * 4, r_dr = (size_t)words * 4, r_hd = (size_t)Pw * Hb;
         rc = serve_on_device(ctx, fo, s, &fd2, N, F, wide_h, &cd2, (uint8_t*)(sb2 + a_lab), (uint8_t*)(sb2 + a_stg),
                              (uint32_t*)(sb2 + a_ne), st, SF_PHASE_FAST);
         if (rc != SF_OK) return rc;
-        const size_t r_sz = (size_t)Pw * 2, r_ia = (size_t)Pw * 4, r_dr = (size_t)words * 4, r_hd = (size_t)Pw * Hb;
-        {
-            // Pull path: all wide planes pinned and device-addressable -> the device fetches the assigned rows itself.
-            const void* m_sz = mapped_alias(wide_h->size); const void* m_ia = mapped_alias(wide_h->iat_us);
-            const void* m_dr = mapped_alias(wide_h->dir_bits); const void* m_hd = mapped_alias(wide_h->hdr);
-            const void* m_nv = wide_h->n_valid ? mapped_alias(wide_h->n_valid) : nullptr;
-            if (m_sz && m_ia && m_dr && m_hd && (!wide_h->n_valid || m_nv)) {
-                const size_t kc = std::min<size_t>(cfg_h->capacity, n);
-                const size_t c_sz = 0, c_ia = sf_align256(c_sz + kc * r_sz), c_dr = sf_align256(c_ia + kc * r_ia),
-                             c_hd = sf_align256(c_dr + kc * r_dr), c_nv = sf_align256(c_hd + kc * r_hd),
-                             c_total = sf_align256(c_nv + (wide_h->n_valid ? kc : 0)) + 256;
-                if (c_total > ctx->stage2_bytes) {
-                    SF_CUDA(cudaDeviceSynchronize());
-                    if (ctx->stage2) { cudaFree(ctx->stage2); ctx->stage2 = nullptr; }
-                    ctx->stage2_bytes = 0;
-                    cudaError_t e = cudaMalloc(&ctx->stage2, c_total);
-                    if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(pulled rows)"); return SF_ERR_ALLOC; }
-                    ctx->stage2_bytes = c_total;
-                }
-                char* dv = ctx->stage2;
-                PullPlanes pl;
-                pl.src[0] = (const unsigned char*)m_sz; pl.dst[0] = (unsigned char*)dv + c_sz; pl.row_bytes[0] = (uint32_t)r_sz;
-                pl.src[1] = (const unsigned char*)m_ia; pl.dst[1] = (unsigned char*)dv + c_ia; pl.row_bytes[1] = (uint32_t)r_ia;
-                pl.src[2] = (const unsigned char*)m_dr; pl.dst[2] = (unsigned char*)dv + c_dr; pl.row_bytes[2] = (uint32_t)r_dr;
-                pl.src[3] = (const unsigned char*)m_hd; pl.dst[3] = (unsigned char*)dv + c_hd; pl.row_bytes[3] = (uint32_t)r_hd;
-                pl.src[4] = (const unsigned char*)m_nv; pl.dst[4] = (unsigned char*)dv + c_nv; pl.row_bytes[4] = m_nv ? 1u : 0u;
-                if (kc) {
-                    const uint32_t grid = (uint32_t)std::min<size_t>((kc + 7) / 8, (size_t)ctx->num_sms * 8);
-                    sf_time_begin(ctx, SF_T_PULL, st);
-                    pull_rows_kernel<<<grid, 256, 0, st>>>(pl, ctx->last_esc_ids, (const uint32_t*)(sb2 + a_ne), (uint32_t)kc);
-                    sf_time_end(ctx, SF_T_PULL, st);
-                    SF_LAUNCH_CHECK("pull_rows_kernel");
-                }
-                sf_packets wd2 = *wide_h;
-                wd2.size = (const uint16_t*)(dv + c_sz); wd2.iat_us = (const uint32_t*)(dv + c_ia);
-                wd2.dir_bits = (const uint32_t*)(dv + c_dr); wd2.hdr = (const uint8_t*)(dv + c_hd);
-                wd2.n_valid = wide_h->n_valid ? (const uint8_t*)(dv + c_nv) : nullptr;
-                wd2.n_flows = (uint32_t)kc;
-                rc = serve_on_device(ctx, fo, s, &fd2, N, F, &wd2, &cd2, (uint8_t*)(sb2 + a_lab), (uint8_t*)(sb2 + a_stg),
-                                     (uint32_t*)(sb2 + a_ne), st, SF_PHASE_SLOW);
-                if (rc != SF_OK) return rc;
-                uint32_t k_host = 0;
-                SF_CUDA(cudaMemcpyAsync(label_h, sb2 + a_lab, n, cudaMemcpyDeviceToHost, st));
-                SF_CUDA(cudaMemcpyAsync(stage_h, sb2 + a_stg, n, cudaMemcpyDeviceToHost, st));
-                SF_CUDA(cudaMemcpyAsync(&k_host, sb2 + a_ne, 4, cudaMemcpyDeviceToHost, st));
-                SF_CUDA(cudaStreamSynchronize(st));
-                if (n_esc_h) *n_esc_h = k_host;
-                return SF_OK;
-            }
-        }
         uint32_t k = 0;
         SF_CUDA(cudaMemcpyAsync(&k, sb2 + a_ne, 4, cudaMemcpyDeviceToHost, st));
         SF_CUDA(cudaStreamSynchronize(st));

@@ -31,6 +31,8 @@ struct sf_ctx {
     char*  pin;
     size_t stage2_bytes;
     size_t pin_bytes;
+    cudaStream_t aux;            // second stream of the host entry point (transfers that overlap the kernels)
+    cudaEvent_t ev_aux, ev_main;
     // optional per-kernel-class timing: ring of event pairs
     int timing;
     uint32_t t_rec;                               // records started so far
