@@ -520,3 +520,33 @@ def test_route_softmax_least_confidence_within_tolerance(env):
     k = int(n_esc.cpu().numpy()[0])
     assert k == int(d.sum()) and np.array_equal(ids.cpu().numpy()[:k], np.nonzero(d)[0])
     assert abs(k - ref["n_esc"]) <= int((~away).sum())
+
+
+@pytest.mark.parametrize("kind", ["rf", "gbdt", "gbdt_mc"])
+def test_forest_threshold_edge_cases_bit_exact(env, kind):
+    """Values equal to thresholds, one float apart from them, signed zeros, infinities and negative values:
+    the kernel compares through integer keys with a 26-bit fast path, so these are the cases that matter."""
+    sf, hz, ctx = env
+    rng = np.random.default_rng(77)
+    base = np.concatenate([rng.normal(size=40) * 10.0 ** rng.integers(-3, 9, 40), [0.0, -0.0, 1.0, -1.0, 40.0, 1500.0, 3e38, -3e38,
+                                                                                    1e-40, -1e-40, 2.0 ** 32, 16777216.0]]).astype(np.float32)
+    up = np.nextafter(base, np.float32(np.inf)); dn = np.nextafter(base, np.float32(-np.inf))
+    far_up = (base.view(np.uint32) + np.uint32(63)).view(np.float32)      # same 64-key cell or the next one
+    pool_x = np.concatenate([base, up, dn, far_up]).astype(np.float32)
+    pool_x = pool_x[np.isfinite(pool_x)]
+    pool_t = np.concatenate([pool_x, [np.inf, -np.inf]]).astype(np.float32)
+    n, F, C, depth, T = 3000, 8, 4, 7, 24
+    feat = pool_x[rng.integers(0, len(pool_x), (n, F))]
+    fo = flowgen.gen_forest(5, kind, T, depth, F, C, feat, sigma=0.5)
+    fo["thr"] = np.ascontiguousarray(pool_t[rng.integers(0, len(pool_t), fo["thr"].shape)])
+    ref, ref_li = oracle.forest_infer(fo, feat, want_leaf_idx=True, threads=4)
+    assert len(np.unique(ref_li)) > 20
+    h = hz.make_forest(ctx, fo)
+    out = torch.zeros(ref.shape, dtype=torch.float32, device="cuda")
+    li = torch.zeros((n, T), dtype=torch.uint16, device="cuda")
+    sf.sf_fast_infer(ctx, h, hz.dev(feat), n, out, li)
+    torch.cuda.synchronize()
+    assert sf.sf_ctx_poll(ctx, reset=True).device_error == 0
+    assert np.array_equal(li.cpu().numpy(), ref_li)
+    assert np.array_equal(bits(out.cpu().numpy()), bits(ref))
+    sf.sf_forest_destroy(h)
