@@ -51,6 +51,7 @@ struct sf_forest {
     // per-tree image of tree_stride bytes: 2^depth node entries of 8 bytes {thr bits, byte offset of the
     // feature's row in the kernel's shared-memory tile}, 1-based heap (entry 0 unused), then (GBDT) 2^depth leaf scalars
     unsigned char* d_image;
+    unsigned char* d_image_small;      // same trees with feature offsets for the 128-flow tile (random forests only)
     uint32_t tree_stride;
     // leaves: RF fp32[T][2^d][C]; GBDT fp32[T][2^d]
     float* d_leaf;
@@ -92,7 +93,7 @@ static inline size_t sf_align256(size_t b) { return (b + 255) & ~(size_t)255; }
 int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st,
                       const uint32_t* n_dev = nullptr);   // n_dev: optional device-side flow count (<= pk->n_flows)
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st,
-                     const uint32_t* n_dev = nullptr);
+                     const uint32_t* n_dev = nullptr, bool small_tiles = false);   // small_tiles: 128 flows per block (few flows per launch)
 // route scratch: block_counts uint32[ceil(n/1024)+1], decision bytes if the caller gave none
 size_t sf_route_scratch_bytes(uint32_t n);
 int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,

@@ -14,6 +14,8 @@
 // t = 0..T-1, which fixes the fp32 summation order.  Random-forest leaf vectors are
 // gathered from L2 one group ahead of their use; boosted-tree leaf scalars travel
 // with their tree's nodes in the shared-memory image.
+// A second instantiation with 128 flows per block serves the streaming path, where a launch
+// carries a few thousand flows: more blocks, and a block's walk is latency-bound either way.
 #include "tc_common.cuh"
 #include <new>
 #include <stdlib.h>
@@ -22,6 +24,7 @@
 namespace {
 
 constexpr uint32_t kB = 512;                       // flows (= threads) per block
+constexpr uint32_t kBSmall = 128;                  // ... of the small-batch variant (streaming: a few thousand flows per launch)
 constexpr uint32_t kMaxSmem = 232448;              // 227 KB
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -88,8 +91,8 @@ __device__ __forceinline__ void load_leaf_vec(const float* __restrict__ lv, floa
 // scalar stored behind the tree's nodes in the image, C = 1) or SF_GBDT_MC (scalar leaves, tree t
 // adds to class t mod C; a chunk holds whole boosting rounds, so the class of every tree in the
 // unrolled round loop is a compile-time register index).  NCH: trees walked at once.
-template <int KIND, int C, int NCH>
-__global__ void __launch_bounds__(kB, 1)
+template <int KIND, int C, int NCH, uint32_t KB>
+__global__ void __launch_bounds__(KB, 1)
 forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
               const unsigned char* __restrict__ image, const float* __restrict__ leaf,
               uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
@@ -97,13 +100,13 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
-    if (blockIdx.x * kB >= n) return;
+    if (blockIdx.x * KB >= n) return;
     const uint32_t sbuf0 = smem_u32(smem_raw);
-    float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][kB]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * kB * 4);   // [2] + flag
+    float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][KB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * KB * 4);   // [2] + flag
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2);
     const uint32_t xbase = smem_u32(xs) + threadIdx.x * 4u;
-    const uint32_t f = blockIdx.x * kB + threadIdx.x;
+    const uint32_t f = blockIdx.x * KB + threadIdx.x;
     const bool live = f < n;
     const uint32_t n_leaf = 1u << depth;
     const uint32_t n_chunks = (T + trees_per_chunk - 1) / trees_per_chunk;
@@ -129,14 +132,14 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         if ((F & 3) == 0) {
             for (uint32_t j = 0; j < F; j += 4) {
                 float4 v = __ldg(reinterpret_cast<const float4*>(row + j));
-                xs[(j + 0) * kB + threadIdx.x] = v.x; xs[(j + 1) * kB + threadIdx.x] = v.y;
-                xs[(j + 2) * kB + threadIdx.x] = v.z; xs[(j + 3) * kB + threadIdx.x] = v.w;
+                xs[(j + 0) * KB + threadIdx.x] = v.x; xs[(j + 1) * KB + threadIdx.x] = v.y;
+                xs[(j + 2) * KB + threadIdx.x] = v.z; xs[(j + 3) * KB + threadIdx.x] = v.w;
             }
         } else {
-            for (uint32_t j = 0; j < F; j++) xs[j * kB + threadIdx.x] = row[j];
+            for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = row[j];
         }
     } else {
-        for (uint32_t j = 0; j < F; j++) xs[j * kB + threadIdx.x] = 0.0f;
+        for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = 0.0f;
     }
 
     float acc[C];
@@ -242,9 +245,9 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
 
 struct Plan { uint32_t chunk_bytes, tpc, nch; size_t smem; };
 
-Plan make_plan(const sf_forest* fo) {
+Plan make_plan(const sf_forest* fo, uint32_t kb = kB) {
     Plan p;
-    const size_t feat_bytes = (size_t)fo->F * kB * sizeof(float);
+    const size_t feat_bytes = (size_t)fo->F * kb * sizeof(float);
     // two chunk buffers share what the feature tile leaves of the 227 KB: up to 64 KB each
     const uint32_t avail = (uint32_t)(((kMaxSmem - feat_bytes - 32) / 2) & ~(size_t)15);
     p.chunk_bytes = avail < 65536u ? avail : 65536u;
@@ -256,24 +259,29 @@ Plan make_plan(const sf_forest* fo) {
     return p;
 }
 
-template <int KIND, int C, int NCH>
+template <int KIND, int C, int NCH, uint32_t KB = kB>
 int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
-    auto k = forest_kernel<KIND, C, NCH>;
+    auto k = forest_kernel<KIND, C, NCH, KB>;
     static size_t smem_set_dev[64] = {};               // per kernel instance and device: raise the opt-in limit only when it grows
     size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
     if (p.smem > smem_set) {
         SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem));
         smem_set = p.smem;
     }
-    const uint32_t grid = (n + kB - 1) / kB;
-    k<<<grid, kB, p.smem, st>>>(feat, n, fo->F, fo->d_image, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
+    const uint32_t grid = (n + KB - 1) / KB;
+    k<<<grid, KB, p.smem, st>>>(feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
                                 p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
 }
 
 template <int C>
-int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
+              bool small_tiles) {
+    if (small_tiles && fo->d_image_small) {
+        const Plan ps = make_plan(fo, kBSmall);
+        if (ps.tpc >= 2) return launch3<SF_RF, C, 2, kBSmall>(fo, ps, feat, n, out, leaf_idx, st, n_dev);
+    }
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
     if (p.nch == 2) return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
@@ -297,7 +305,8 @@ int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, ui
 
 }  // namespace
 
-int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
+                     bool small_tiles) {
     if (n == 0) return SF_OK;
     if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st, n_dev);
     if (fo->kind == SF_GBDT_MC) {
@@ -322,22 +331,22 @@ int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* 
         return SF_ERR_UNSUPPORTED;
     }
     switch (fo->C) {
-    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
     }
     return SF_ERR_UNSUPPORTED;
 }
@@ -356,7 +365,7 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     sf_forest* fo = new (std::nothrow) sf_forest();
     if (!fo) return SF_ERR_ALLOC;
     fo->ctx = ctx; fo->kind = kind; fo->T = T; fo->depth = depth; fo->F = F; fo->C = (kind == SF_GBDT) ? 1 : C;
-    fo->d_image = nullptr; fo->d_leaf = nullptr;
+    fo->d_image = nullptr; fo->d_leaf = nullptr; fo->d_image_small = nullptr;
     // Image of one tree: 2^d node entries of 8 bytes in a 1-based heap (host node i, children
     // 2i+1 / 2i+2, becomes entry i+1, children 2j / 2j+1; entry 0 unused), then for boosted
     // trees the 2^d leaf scalars; padded to a multiple of 16 bytes for the 16-byte copies.
@@ -375,12 +384,25 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
         }
         if (kind != SF_RF) memcpy(h + (size_t)t * stride + n_ent * 8u, leaf + (size_t)t * n_ent, n_ent * 4u);
     }
+    // the small-batch variant of the kernel has a narrower feature tile, so its feature offsets differ
+    unsigned char* h_small = nullptr;
+    if (kind == SF_RF) {
+        h_small = (unsigned char*)malloc((size_t)T * stride);
+        if (!h_small) { free(h); delete fo; return SF_ERR_ALLOC; }
+        memcpy(h_small, h, (size_t)T * stride);
+        for (uint32_t t = 0; t < T; t++) {
+            uint32_t* ent = reinterpret_cast<uint32_t*>(h_small + (size_t)t * stride);
+            for (uint32_t i = 0; i < n_int; i++) ent[2 * (i + 1) + 1] = (uint32_t)fid[(size_t)t * n_int + i] * kBSmall * 4u;
+        }
+    }
     const size_t leaf_count = (size_t)T * n_ent * (kind == SF_RF ? fo->C : 1u);
     cudaError_t e = cudaMalloc(&fo->d_image, (size_t)T * stride);
     if (e == cudaSuccess) e = cudaMalloc(&fo->d_leaf, sizeof(float) * leaf_count);
     if (e == cudaSuccess) e = cudaMemcpy(fo->d_image, h, (size_t)T * stride, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && h_small) e = cudaMalloc(&fo->d_image_small, (size_t)T * stride);
+    if (e == cudaSuccess && h_small) e = cudaMemcpy(fo->d_image_small, h_small, (size_t)T * stride, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(fo->d_leaf, leaf, sizeof(float) * leaf_count, cudaMemcpyHostToDevice);
-    free(h);
+    free(h); free(h_small);
     if (e != cudaSuccess) { sf_forest_destroy(fo); return sf_set_cuda_error(e, "sf_forest_create"); }
     *out = fo;
     return SF_OK;
@@ -389,6 +411,7 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
 extern "C" void sf_forest_destroy(sf_forest* fo) {
     if (!fo) return;
     if (fo->d_image) cudaFree(fo->d_image);
+    if (fo->d_image_small) cudaFree(fo->d_image_small);
     if (fo->d_leaf) cudaFree(fo->d_leaf);
     delete fo;
 }

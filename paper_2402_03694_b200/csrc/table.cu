@@ -568,7 +568,7 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     sf_time_end(ctx, SF_T_EXTRACT, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_FOREST, st);
-    rc = sf_launch_forest(fo, feat, n, prob, nullptr, st, &t->counts[0]);
+    rc = sf_launch_forest(fo, feat, n, prob, nullptr, st, &t->counts[0], true);      // a few thousand flows fire per batch
     sf_time_end(ctx, SF_T_FOREST, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_SCORE, st);
