@@ -40,7 +40,7 @@ FOREST_WAVEFRONTS_PER_VISIT = 3
 # DRAM bytes per launch measured with ncu for a kernel class (profiles/kernels_config2_262144_flows.md:
 # 788.7 MB over the three hidden-layer launches on 62,207 rows), keyed by (class, config, hash of the
 # kernel's source) so that the figure turns null as soon as the kernel changes
-TRAFFIC_BY_SOURCE = {("gemm", 2, "cfbb353860eac582"): {"bytes_per_row_per_launch": 788.7e6 / 3 / 62207}}
+TRAFFIC_BY_SOURCE = {("gemm", 2, "9bb65be47ecd2edb"): {"bytes_per_row_per_launch": 788.76e6 / 3 / 62207}}
 
 
 def load_peaks():
