@@ -1,31 +1,41 @@
 // S4 (1-D CNN slow model), one fused kernel per batch of assigned flows:
 //   conv1 (k=5, 8 -> 64) + ReLU -> conv2 (k=5, 64 -> 128) + ReLU -> mean over the 128
 //   positions -> linear 128 -> n_cls -> argmax.
-// All three contractions run on the tcgen05 tensor cores with one flow's 128 positions as
-// the M = 128 rows of a tile; nothing but the 2 KB input row and the logits touches HBM.
+// Both convolutions run on the tcgen05 tensor cores; nothing but the 2 KB input row and the
+// logits touches HBM.
 //
 // Shifted ("same" padded) operands without im2col.  Activations are kept in shared memory
 // in the un-swizzled core-matrix layout: for every group of 8 channels a column of 16-byte
 // rows, one row per position, with zero rows above and below.  In that layout a matrix
 // descriptor's start address may be moved by whole rows, so tap t of a convolution is the
-// same buffer started t rows further down; the zero rows supply the padding.  For conv1
-// (8 input channels = one 16-byte row per position) consecutive taps are consecutive rows,
-// so a K = 16 step (two taps) uses a K-direction stride of 16 bytes.
+// same buffer started t positions further down; the zero rows supply the padding.
 //
-// Pooling and the linear head are one more MMA: mean_p(h2[p][:]) . W3^T = sum_p (h2[p][:] .
-// (W3/128)^T), i.e. a [128 positions] x [16 classes] product over the 128 channels followed
-// by a sum over positions (TMEM lanes), which a shuffle tree and four partial sums finish in a
-// fixed order (deterministic).
+// conv1 takes one flow's 128 positions as the M = 128 rows of a tile (N = 64 output channels;
+// 8 input channels = one 16-byte row per position, so consecutive taps are consecutive rows and a
+// K = 16 step covers two taps with a K-direction stride of 16 bytes).
 //
-// Persistent CTAs, one per SM, loop over flows.  Warp roles:
+// conv2 is issued the other way round, for TWO flows at once: the weights of a tap are the A
+// operand (M = 128 output channels), the activations of a pair of flows are the B operand with
+// N = 256 = 128 positions x 2 flows, rows interleaved (row 2p + s = position p of flow s, so a tap
+// is a shift by two rows and the two flows share the zero padding rows).  On this part an
+// M = 128 tcgen05.mma of K = 16 holds the tensor pipe for max(N/2, ~98) cycles, so only N = 256
+// runs at the full rate; with a single flow per instruction (N = 128) a third of the pipe idles.
+// The accumulator then has the output channel as its TMEM lane and (position, flow) as its
+// column, so the mean over positions is a plain sum inside one thread: bias, ReLU and the bf16
+// rounding of the activation are applied per element, the rounded values are added in
+// position order, and no pooling pass or third contraction is needed.  The linear head
+// (128 -> n_cls, 2 Kflop per flow) runs on CUDA cores from the pooled values, with every cross-thread
+// sum a fixed shuffle tree (deterministic).
+//
+// Persistent CTAs, one per SM, loop over pairs of flows.  Warp roles:
 //   warp 0        streams input rows with bulk copies into a ring
-//   warp 1        issues the MMAs in the order conv1(i+2), conv2(i), head(i-2)
-//   warps 2..5    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's A operand (shared memory)
-//   warps 6..21   E2: conv2 accumulators -> bias + ReLU -> bf16 -> the head's A operand
-//   warps 22..25  E3: head accumulators -> sum over positions -> + bias -> logits, argmax
-// Every accumulator and activation buffer is double (conv1: triple) buffered, so the three epilogues and the
-// tensor pipe overlap.  Every wait is bounded; on a timeout the block records
-// SF_ERR_DEVICE_TIMEOUT and leaves.
+//   warp 1        issues the MMAs in the order conv2(pair i), conv1(pair i+2)
+//   warps 2..5    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's B operand (shared memory)
+//   warps 6..21   E2: conv2 accumulators -> bias + ReLU -> bf16 -> partial sums over 32 positions
+//   warps 22..25  E3: partial sums -> mean -> linear head -> logits, argmax
+// conv2's accumulator (256 TMEM columns) is single: the E2 warps pull it into registers first
+// thing and release it, and conv1 of a later pair keeps the pipe busy meanwhile.  Every wait is
+// bounded; on a timeout the block records SF_ERR_DEVICE_TIMEOUT and leaves.
 #include "tc_common.cuh"
 #include <stdlib.h>
 #include <string.h>
@@ -39,41 +49,40 @@ constexpr uint32_t kE1First = 2, kE2First = kE1First + kE1Warps, kE3First = kE2F
 constexpr uint32_t kThreads = (kE3First + kE3Warps) * 32;       // 832
 constexpr uint32_t XS = 4;                                  // input-row ring depth
 constexpr uint32_t X_STAGE = (2 + L + 3) * 16;              // 2 zero rows, 128 rows, 3 zero rows (tap 5 is a zero tap)
-constexpr uint32_t H1_COL = (2 + L + 2) * 16;               // one 8-channel column of conv1's output: 2112 bytes
-constexpr uint32_t H1_BYTES = (C1 / 8) * H1_COL;            // 16,896
-constexpr uint32_t H2_COL = L * 16;                         // one 8-channel column of conv2's output: 2048 bytes
-constexpr uint32_t H2_BYTES = (C2 / 8) * H2_COL;            // 32,768
+constexpr uint32_t H1_COL = 2 * (2 + L + 2) * 16;           // one 8-channel column of a PAIR's conv1 output: 264 rows, 4,224 bytes
+constexpr uint32_t H1_BYTES = (C1 / 8) * H1_COL;            // 33,792
 // weight blob (device and shared memory share this layout)
-constexpr uint32_t W2_OFF = 0;                              // [5 taps][8 k-chunks][128 n][8] bf16
+constexpr uint32_t W2_OFF = 0;                              // [5 taps][8 k-chunks][128 out][8] bf16
 constexpr uint32_t W2_BYTES = KW * (C1 / 8) * C2 * 16;      // 81,920
-constexpr uint32_t W1_OFF = W2_OFF + W2_BYTES;              // [6 taps][64 n][8] bf16 (tap 5 = 0)
+constexpr uint32_t W1_OFF = W2_OFF + W2_BYTES;              // [6 taps][64 out][8] bf16 (tap 5 = 0)
 constexpr uint32_t W1_BYTES = 6 * C1 * 16;                  // 6,144
-constexpr uint32_t W3_OFF = W1_OFF + W1_BYTES;              // [16 k-chunks][16 classes][8] bf16, scaled by 1/128
-constexpr uint32_t W3_BYTES = (C2 / 8) * NCLS_MAX * 16;     // 4,096
+constexpr uint32_t W3_OFF = W1_OFF + W1_BYTES;              // fp32 [16 classes][128], values rounded to bf16, zero beyond n_cls
+constexpr uint32_t W3_BYTES = NCLS_MAX * C2 * 4;            // 8,192
 constexpr uint32_t B1_OFF = W3_OFF + W3_BYTES;              // fp32 [64]
 constexpr uint32_t B2_OFF = B1_OFF + C1 * 4;                // fp32 [128]
 constexpr uint32_t B3_OFF = B2_OFF + C2 * 4;                // fp32 [16]
 constexpr uint32_t BLOB_BYTES = B3_OFF + NCLS_MAX * 4;
 // shared memory map
 constexpr uint32_t SM_BLOB = 0;
-constexpr uint32_t NB1 = 3;                                 // conv1 accumulator / activation buffers (conv1 runs two flows ahead)
-constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // NB1 buffers
-constexpr uint32_t SM_H2 = SM_H1 + NB1 * H1_BYTES;          // 2 buffers
-constexpr uint32_t SM_X = SM_H2 + 2 * H2_BYTES;             // XS stages
-constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // fp32 [4 warps][16] partial logits
-constexpr uint32_t SM_BARS = SM_PART + 4 * NCLS_MAX * 4;
+constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // 2 pair buffers
+constexpr uint32_t SM_X = SM_H1 + 2 * H1_BYTES;             // XS stages
+constexpr uint32_t PART_BYTES = 4 * 2 * C2 * 4;             // fp32 [4 position groups][2 flows][128 channels]
+constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // 2 buffers
+constexpr uint32_t SM_PART2 = SM_PART + 2 * PART_BYTES;     // fp32 [4 warps][32] partial logits
+constexpr uint32_t SM_BARS = SM_PART2 + kE3Warps * 32 * 4;
 constexpr uint32_t SM_TOTAL = SM_BARS + 320;
-static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_H2 % 16 == 0 && SM_X % 16 == 0 && SM_BARS % 8 == 0, "alignment");
+static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_X % 16 == 0 && SM_PART % 16 == 0 && SM_BARS % 8 == 0, "alignment");
 static_assert(SM_TOTAL <= 232448, "shared memory");
-// TMEM columns: conv1 accumulators [3][64], conv2 [2][128], head [2][16]
-constexpr uint32_t TM_D1 = 0, TM_D2 = 192, TM_D4 = 448;
+// TMEM columns: conv1 accumulators [2 flows of a pair][64], conv2 [256]
+constexpr uint32_t TM_D1 = 0, TM_D2 = 256;
 
 struct Bars {
     uint64_t w_full;
     uint64_t x_full[XS], x_empty[XS];
-    uint64_t d1_full[NB1], d1_empty[NB1], h1_full[NB1], h1_empty[NB1];
-    uint64_t d2_full[2], d2_empty[2], h2_full[2], h2_empty[2];
-    uint64_t d4_full[2], d4_empty[2];
+    uint64_t d1_full[2], d1_empty[2];          // per flow slot of a pair
+    uint64_t h1_full[2], h1_empty[2];          // per pair buffer
+    uint64_t d2_full, d2_empty;
+    uint64_t part_full[2], part_empty[2];
     uint32_t tmem_base, abort_flag;
 };
 static_assert(sizeof(Bars) <= 320, "barrier block");
@@ -82,13 +91,11 @@ __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t count) 
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-// sum over the 32 lanes of each of 16 per-lane values; lanes l and l+16 end up with column (l & 15)'s
-// total.  The order of additions is a fixed tree, so the result is reproducible run to run.
-__device__ __forceinline__ float transpose_reduce16(float (&v)[16], uint32_t lane) {
+// Sum over the 32 lanes of each of 32 per-lane values; lane l ends up with value l's total.
+// The order of additions is a fixed tree, so the result is reproducible run to run.
+__device__ __forceinline__ float transpose_reduce32(float (&v)[32], uint32_t lane) {
 #pragma unroll
-    for (int j = 0; j < 16; j++) v[j] += __shfl_xor_sync(0xFFFFFFFFu, v[j], 16);
-#pragma unroll
-    for (int off = 8; off >= 1; off >>= 1) {
+    for (int off = 16; off >= 1; off >>= 1) {
         const bool up = (lane & off) != 0;
 #pragma unroll
         for (int j = 0; j < off; j++) {
@@ -104,6 +111,12 @@ __device__ __forceinline__ uint32_t pack_relu_bf16(uint32_t a, uint32_t b, float
     __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(__uint_as_float(a) + ba, 0.0f), fmaxf(__uint_as_float(b) + bb, 0.0f));
     return *reinterpret_cast<uint32_t*>(&h);
 }
+// {high half: bf16(max(hi, 0)), low half: bf16(max(lo, 0))}, round to nearest even
+__device__ __forceinline__ uint32_t relu_bf16x2(float hi, float lo) {
+    uint32_t d;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restrict__ n_rows_dev,
@@ -116,24 +129,23 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     const uint32_t sbase = smem_u32(smem);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t n_rows = *n_rows_dev;
-    // flows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+    // flows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; flow m of the CTA is slot (m & 1) of pair (m >> 1)
     const uint32_t n_mine = (n_rows > blockIdx.x) ? (n_rows - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t n_pairs = (n_mine + 1) >> 1;
 
-    // zero everything that acts as padding (and the rest of the activation buffers)
-    for (uint32_t i = threadIdx.x; i < (NB1 * H1_BYTES + 2 * H2_BYTES + XS * X_STAGE) / 16; i += kThreads)
+    // zero everything that acts as padding (and the rest of the activation buffers: the unused
+    // slot of an odd last pair is multiplied like any other and must hold finite numbers)
+    for (uint32_t i = threadIdx.x; i < (2 * H1_BYTES + XS * X_STAGE) / 16; i += kThreads)
         reinterpret_cast<uint4*>(smem + SM_H1)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
         mbar_init(&bars->w_full, 1);
         for (uint32_t s = 0; s < XS; s++) { mbar_init(&bars->x_full[s], 1); mbar_init(&bars->x_empty[s], 1); }
-        for (uint32_t b = 0; b < NB1; b++) {
+        for (uint32_t b = 0; b < 2; b++) {
             mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kE1Warps);
             mbar_init(&bars->h1_full[b], kE1Warps); mbar_init(&bars->h1_empty[b], 1);
+            mbar_init(&bars->part_full[b], kE2Warps); mbar_init(&bars->part_empty[b], kE3Warps);
         }
-        for (uint32_t b = 0; b < 2; b++) {
-            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], kE2Warps);
-            mbar_init(&bars->h2_full[b], kE2Warps); mbar_init(&bars->h2_empty[b], 1);
-            mbar_init(&bars->d4_full[b], 1); mbar_init(&bars->d4_empty[b], kE3Warps);
-        }
+        mbar_init(&bars->d2_full, 1); mbar_init(&bars->d2_empty, kE2Warps);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -144,16 +156,15 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
     const uint32_t q = warp & 3u;                    // TMEM lane quarter an epilogue warp may read
-    const uint32_t p = q * 32u + lane;               // position handled by an epilogue thread
 
     if (warp == 0) {
         if (lane == 0 && n_mine > 0) {
             mbar_expect_tx(&bars->w_full, BLOB_BYTES);
             bulk_load(smem + SM_BLOB, blob, BLOB_BYTES, &bars->w_full);
-            for (uint32_t i = 0; i < n_mine; i++) {
-                const uint32_t s = i % XS, ph = (i / XS) & 1u;
+            for (uint32_t m = 0; m < n_mine; m++) {
+                const uint32_t s = m % XS, ph = (m / XS) & 1u;
                 if (!mbar_wait_relaxed(&bars->x_empty[s], ph ^ 1u, abort_flag)) break;
-                const uint32_t r = blockIdx.x + i * gridDim.x;
+                const uint32_t r = blockIdx.x + m * gridDim.x;
                 mbar_expect_tx(&bars->x_full[s], L * CIN * 2);
                 bulk_load(smem + SM_X + s * X_STAGE + 32, rows + (size_t)r * L * CIN, L * CIN * 2, &bars->x_full[s]);
             }
@@ -161,92 +172,79 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
     } else if (warp == 1) {
         if (lane == 0 && n_mine > 0) {
             constexpr uint32_t idesc1 = make_idesc_bf16(128, C1);
-            constexpr uint32_t idesc2 = make_idesc_bf16(128, C2);
-            constexpr uint32_t idesc4 = make_idesc_bf16(128, NCLS_MAX);
+            constexpr uint32_t idesc2 = make_idesc_bf16(C2, 2 * L);
             // descriptor = constant fields + (address >> 4) in the low bits: build the bases once, add offsets per MMA
             const uint64_t dX = make_smem_desc(sbase + SM_X, 16, 128, 0);
             const uint64_t dW1 = make_smem_desc(sbase + SM_BLOB + W1_OFF, C1 * 16u, 128, 0);
             const uint64_t dH1 = make_smem_desc(sbase + SM_H1, H1_COL, 128, 0);
             const uint64_t dW2 = make_smem_desc(sbase + SM_BLOB + W2_OFF, C2 * 16u, 128, 0);
-            const uint64_t dH2 = make_smem_desc(sbase + SM_H2, H2_COL, 128, 0);
-            const uint64_t dW3 = make_smem_desc(sbase + SM_BLOB + W3_OFF, NCLS_MAX * 16u, 128, 0);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
-            auto conv1 = [&](uint32_t i) -> bool {
-                const uint32_t s = i % XS, xph = (i / XS) & 1u, b = i % NB1, ph = (i / NB1) & 1u;
-                if (!mbar_wait(&bars->x_full[s], xph, abort_flag)) return false;
-                if (!mbar_wait(&bars->d1_empty[b], ph ^ 1u, abort_flag)) return false;
+            auto conv1_flow = [&](uint32_t m) -> bool {
+                const uint32_t xs = m % XS, xph = (m / XS) & 1u, s = m & 1u, i = m >> 1;
+                if (!mbar_wait(&bars->x_full[xs], xph, abort_flag)) return false;
+                if (!mbar_wait(&bars->d1_empty[s], (i & 1u) ^ 1u, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t ax = dX + (uint64_t)((s * X_STAGE) >> 4);
+                const uint64_t ax = dX + (uint64_t)((xs * X_STAGE) >> 4);
 #pragma unroll
                 for (uint32_t k = 0; k < 3; k++)             // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
-                    umma_bf16(tmem_base + TM_D1 + b * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4), idesc1,
+                    umma_bf16(tmem_base + TM_D1 + s * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4), idesc1,
                               k != 0 ? 1u : 0u);
-                umma_commit(&bars->x_empty[s]);
-                umma_commit(&bars->d1_full[b]);
+                umma_commit(&bars->x_empty[xs]);
+                umma_commit(&bars->d1_full[s]);
+                return true;
+            };
+            auto conv1_pair = [&](uint32_t i) -> bool {
+                if (!conv1_flow(2u * i)) return false;
+                if (2u * i + 1u < n_mine) return conv1_flow(2u * i + 1u);
                 return true;
             };
             auto conv2 = [&](uint32_t i) -> bool {
-                const uint32_t b = i & 1u, ph = (i >> 1) & 1u, b1i = i % NB1, ph1 = (i / NB1) & 1u;
-                if (!mbar_wait(&bars->h1_full[b1i], ph1, abort_flag)) return false;
-                if (!mbar_wait(&bars->d2_empty[b], ph ^ 1u, abort_flag)) return false;
+                const uint32_t b = i & 1u;
+                if (!mbar_wait(&bars->h1_full[b], (i >> 1) & 1u, abort_flag)) return false;
+                if (!mbar_wait(&bars->d2_empty, (i & 1u) ^ 1u, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t ah = dH1 + (uint64_t)((b1i * H1_BYTES) >> 4);
+                const uint64_t bh = dH1 + (uint64_t)((b * H1_BYTES) >> 4);
 #pragma unroll
                 for (uint32_t t = 0; t < KW; t++) {
 #pragma unroll
-                    for (uint32_t k = 0; k < C1 / 16; k++)
-                        umma_bf16(tmem_base + TM_D2 + b * C2, ah + (((2u * k) * H1_COL + t * 16u) >> 4),
-                                  dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
+                    for (uint32_t k = 0; k < C1 / 16; k++)      // A = weights of tap t, B = the pair's activations two rows per tap further down
+                        umma_bf16(tmem_base + TM_D2, dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4),
+                                  bh + (((2u * k) * H1_COL + t * 32u) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
                 }
-                umma_commit(&bars->h1_empty[b1i]);
-                umma_commit(&bars->d2_full[b]);
+                umma_commit(&bars->h1_empty[b]);
+                umma_commit(&bars->d2_full);
                 return true;
             };
-            auto head = [&](uint32_t i) -> bool {
-                const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-                if (!mbar_wait(&bars->h2_full[b], ph, abort_flag)) return false;
-                if (!mbar_wait(&bars->d4_empty[b], ph ^ 1u, abort_flag)) return false;
-                tc_fence_after();
-                const uint64_t ah = dH2 + (uint64_t)((b * H2_BYTES) >> 4);
-#pragma unroll
-                for (uint32_t k = 0; k < C2 / 16; k++)
-                    umma_bf16(tmem_base + TM_D4 + b * NCLS_MAX, ah + (((2u * k) * H2_COL) >> 4),
-                              dW3 + (((2u * k) * (NCLS_MAX * 16u)) >> 4), idesc4, k != 0 ? 1u : 0u);
-                umma_commit(&bars->h2_empty[b]);
-                umma_commit(&bars->d4_full[b]);
-                return true;
-            };
-            // conv1 runs two flows ahead and the head two flows behind conv2, so that each epilogue has two
-            // conv2 periods to turn its accumulator into the next operand
-            if (ok) ok = conv1(0);
-            if (ok && n_mine > 1) ok = conv1(1);
-            for (uint32_t i = 0; i < n_mine && ok; i++) {
-                if (i + 2 < n_mine) ok = conv1(i + 2);
-                if (ok) ok = conv2(i);
-                if (ok && i >= 2) ok = head(i - 2);
+            // conv1 runs two pairs ahead of conv2: its MMAs keep the pipe busy while the E2 warps pull conv2's
+            // accumulator out of TMEM, and E1 has a whole conv2 period to write the next operand
+            if (ok) ok = conv1_pair(0);
+            if (ok && n_pairs > 1) ok = conv1_pair(1);
+            for (uint32_t i = 0; i < n_pairs && ok; i++) {
+                ok = conv2(i);
+                if (ok && i + 2 < n_pairs) ok = conv1_pair(i + 2);
             }
-            if (ok && n_mine >= 2) ok = head(n_mine - 2);
-            if (ok) ok = head(n_mine - 1);
         }
     } else if (n_mine > 0 && warp < kE2First) {
-        // ---- E1: conv1 accumulators -> conv2's A operand -------------------------------
+        // ---- E1: conv1 accumulators -> conv2's B operand -------------------------------
+        const uint32_t p = q * 32u + lane;               // position handled by this thread
         const float* b1 = reinterpret_cast<const float*>(smem + SM_BLOB + B1_OFF);
         bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
-        for (uint32_t i = 0; i < n_mine && ok; i++) {
-            const uint32_t b = i % NB1, ph = (i / NB1) & 1u;
-            bool w = mbar_wait_relaxed(&bars->d1_full[b], ph, abort_flag) && mbar_wait_relaxed(&bars->h1_empty[b], ph ^ 1u, abort_flag);
+        for (uint32_t m = 0; m < n_mine && ok; m++) {
+            const uint32_t s = m & 1u, i = m >> 1, b = i & 1u;
+            bool w = mbar_wait_relaxed(&bars->d1_full[s], i & 1u, abort_flag);
+            if (s == 0) w = w && mbar_wait_relaxed(&bars->h1_empty[b], ((i >> 1) & 1u) ^ 1u, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, w);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D1 + b * C1;
-            uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (p + 2u) * 16u;
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D1 + s * C1;
+            uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (2u * (p + 2u) + s) * 16u;
             uint32_t v0[32], v1[32];
             tmem_ld32(taddr, v0);
             tmem_ld32(taddr + 32, v1);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->d1_empty[b]);      // the accumulator is in registers: conv1 may reuse it
+            if (lane == 0) mbar_arrive(&bars->d1_empty[s]);      // the accumulator is in registers: conv1 may reuse it
 #pragma unroll
             for (int j = 0; j < 8; j++) {                // 8 columns of 8 channels
                 uint32_t pk[4];
@@ -258,84 +256,103 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 }
                 *reinterpret_cast<uint4*>(hrow + j * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
-            fence_proxy_async();                         // activations -> visible to the MMA's shared-memory reads
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->h1_full[b]);
+            if (s == 1u || m + 1 == n_mine) {            // the pair is complete
+                fence_proxy_async();                     // activations -> visible to the MMA's shared-memory reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->h1_full[b]);
+            }
         }
     } else if (n_mine > 0 && warp < kE3First) {
-        // ---- E2: conv2 accumulators -> the head's A operand ----------------------------
-        const uint32_t g = (warp - kE2First) >> 2;        // 32 of the 128 conv2 channels
-        const float* b2 = reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF);
+        // ---- E2: conv2 accumulators [channel][position, flow] -> sums over 32 positions ----
+        const uint32_t g = (warp - kE2First) >> 2;        // positions 32g .. 32g+31 = columns 64g .. 64g+63
+        const uint32_t ch = q * 32u + lane;
         bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
-        for (uint32_t i = 0; i < n_mine && ok; i++) {
-            const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-            bool w = mbar_wait_relaxed(&bars->d2_full[b], ph, abort_flag) && mbar_wait_relaxed(&bars->h2_empty[b], ph ^ 1u, abort_flag);
-            ok = __all_sync(0xFFFFFFFFu, w);
+        const float bias = ok ? reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF)[ch] : 0.0f;
+        for (uint32_t i = 0; i < n_pairs && ok; i++) {
+            const uint32_t b = i & 1u;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->d2_full, i & 1u, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t c0 = g * 32u;
-            uint32_t v[32];
-            tmem_ld32(tmem_base + ((q * 32u) << 16) + TM_D2 + b * C2 + c0, v);
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D2 + g * 64u;
+            uint32_t v[32], pk[16];
+            tmem_ld32(taddr, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; j++)                  // columns 2j, 2j+1 = position 32g+j of flows 0, 1
+                pk[j] = relu_bf16x2(__uint_as_float(v[2 * j + 1]) + bias, __uint_as_float(v[2 * j]) + bias);
+            tmem_ld32(taddr + 32, v);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->d2_empty[b]);      // the accumulator is in registers: conv2 may reuse it
-            uint8_t* hrow = smem + SM_H2 + b * H2_BYTES + p * 16u;
+            if (lane == 0) mbar_arrive(&bars->d2_empty);         // the accumulator is in registers: conv2 may reuse it
+            float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int e = 0; e < 4; e++) {
-                    const int c = j * 8 + e * 2;
-                    pk[e] = pack_relu_bf16(v[c], v[c + 1], b2[c0 + c], b2[c0 + c + 1]);
-                }
-                *reinterpret_cast<uint4*>(hrow + ((c0 >> 3) + j) * H2_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            for (int j = 0; j < 16; j++) {
+                s0 += __uint_as_float(pk[j] << 16);
+                s1 += __uint_as_float(pk[j] & 0xFFFF0000u);
             }
-            fence_proxy_async();
+#pragma unroll
+            for (int j = 0; j < 16; j++) {
+                const uint32_t h = relu_bf16x2(__uint_as_float(v[2 * j + 1]) + bias, __uint_as_float(v[2 * j]) + bias);
+                s0 += __uint_as_float(h << 16);
+                s1 += __uint_as_float(h & 0xFFFF0000u);
+            }
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->part_empty[b], ((i >> 1) & 1u) ^ 1u, abort_flag));
+            if (!ok) break;
+            float* part = reinterpret_cast<float*>(smem + SM_PART + b * PART_BYTES) + g * 2u * C2;
+            part[ch] = s0;
+            part[C2 + ch] = s1;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->h2_full[b]);
+            if (lane == 0) mbar_arrive(&bars->part_full[b]);
         }
     } else if (n_mine > 0) {
-        // ---- E3: head accumulators [position][class] -> sum over positions -> logits ----
-        const uint32_t et = (warp - kE3First) * 32u + lane;           // 0..127
-        const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
-        float* part = reinterpret_cast<float*>(smem + SM_PART);
+        // ---- E3: partial sums -> mean -> linear head -> logits, argmax -----------------
+        const uint32_t ew = warp - kE3First;
+        const uint32_t ch = ew * 32u + lane;                              // 0..127
+        float* part2 = reinterpret_cast<float*>(smem + SM_PART2);
         bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
-        for (uint32_t i = 0; i < n_mine && ok; i++) {
-            const uint32_t b = i & 1u, ph = (i >> 1) & 1u;
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->d4_full[b], ph, abort_flag));
+        float w3r[NCLS_MAX];
+#pragma unroll
+        for (int c = 0; c < (int)NCLS_MAX; c++) w3r[c] = ok ? reinterpret_cast<const float*>(smem + SM_BLOB + W3_OFF)[c * C2 + ch] : 0.0f;
+        const float* b3 = reinterpret_cast<const float*>(smem + SM_BLOB + B3_OFF);
+        for (uint32_t i = 0; i < n_pairs && ok; i++) {
+            const uint32_t b = i & 1u;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->part_full[b], (i >> 1) & 1u, abort_flag));
             if (!ok) break;
-            tc_fence_after();
-            uint32_t v[16];
-            tmem_ld16(tmem_base + ((q * 32u) << 16) + TM_D4 + b * NCLS_MAX, v);
-            tmem_ld_wait();
-            tc_fence_before();
+            const float* part = reinterpret_cast<const float*>(smem + SM_PART + b * PART_BYTES);
+            float pooled[2];
+#pragma unroll
+            for (int s = 0; s < 2; s++)                                   // position groups in order, then the mean (an exact scaling)
+                pooled[s] = (((part[s * C2 + ch] + part[(2 + s) * C2 + ch]) + part[(4 + s) * C2 + ch]) + part[(6 + s) * C2 + ch]) * (1.0f / 128.0f);
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->d4_empty[b]);
-            float x[16];
+            if (lane == 0) mbar_arrive(&bars->part_empty[b]);
+            float x[32];
 #pragma unroll
-            for (int c = 0; c < 16; c++) x[c] = __uint_as_float(v[c]);
-            const float tot = transpose_reduce16(x, lane);            // this warp's 32 positions, class lane & 15
-            if (lane < 16) part[(warp - kE3First) * NCLS_MAX + lane] = tot;
+            for (int s = 0; s < 2; s++)
+#pragma unroll
+                for (int c = 0; c < (int)NCLS_MAX; c++) x[s * 16 + c] = pooled[s] * w3r[c];
+            const float tot = transpose_reduce32(x, lane);                // this warp's 32 channels; lane = flow slot * 16 + class
+            part2[ew * 32u + lane] = tot;
             named_barrier_sync(1, kE3Warps * 32);
-            const uint32_t r = blockIdx.x + i * gridDim.x;
-            if (et < 32) {                                            // first E3 warp: lane c < n_cls finishes class c
+            if (ew == 0) {
+                const uint32_t s = lane >> 4, c = lane & 15u, m = 2u * i + s;
+                const uint32_t r = blockIdx.x + m * gridDim.x;
                 float lg = -3.0e38f;
-                if (lane < n_cls) {
-                    lg = ((part[lane] + part[NCLS_MAX + lane]) + part[2 * NCLS_MAX + lane]) + part[3 * NCLS_MAX + lane] + b3[lane];
-                    logits[(size_t)r * n_cls + lane] = lg;
+                if (c < n_cls && m < n_mine) {
+                    lg = ((part2[lane] + part2[32 + lane]) + part2[64 + lane]) + part2[96 + lane] + b3[c];
+                    logits[(size_t)r * n_cls + c] = lg;
                 }
-                // argmax, lowest index on ties
-                float best = lg; uint32_t arg = lane;
+                // argmax over the 16 lanes of a flow slot, lowest index on ties
+                float best = lg; uint32_t arg = c;
 #pragma unroll
-                for (int o = 16; o >= 1; o >>= 1) {
+                for (int o = 8; o >= 1; o >>= 1) {
                     const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
                     const uint32_t oa = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
                     if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
                 }
-                if (lane == 0 && label) label[r] = (uint8_t)arg;
+                if (c == 0 && m < n_mine && label) label[r] = (uint8_t)arg;
             }
-            named_barrier_sync(1, kE3Warps * 32);                     // part is free again
+            named_barrier_sync(1, kE3Warps * 32);                     // part2 is free again
         }
     }
 
@@ -374,13 +391,12 @@ int sf_cnn_prepare(sf_slow* s, const float* w1, const float* b1, const float* w2
         for (uint32_t n = 0; n < C1; n++)
             for (uint32_t e = 0; e < CIN; e++)
                 W1[(t * C1 + n) * 8 + e] = bf16_bits(w1[((size_t)n * KW + t) * CIN + e]);
-    // head weights rounded to bf16, then scaled by 2^-7 (exact) so that the MMA yields the mean's contribution
-    uint16_t* W3 = reinterpret_cast<uint16_t*>(h + W3_OFF);
+    // head weights rounded to bf16 (the model's precision), kept as fp32 for the CUDA-core head
+    float* W3 = reinterpret_cast<float*>(h + W3_OFF);
     for (uint32_t c = 0; c < s->n_cls; c++)
         for (uint32_t k = 0; k < C2; k++) {
             uint32_t bits = (uint32_t)bf16_bits(w3[(size_t)c * C2 + k]) << 16;
-            float f; memcpy(&f, &bits, 4);
-            W3[((k / 8) * NCLS_MAX + c) * 8 + (k % 8)] = bf16_bits(f * (1.0f / 128.0f));
+            memcpy(&W3[c * C2 + k], &bits, 4);
         }
     memcpy(h + B1_OFF, b1, C1 * 4);
     memcpy(h + B2_OFF, b2, C2 * 4);
