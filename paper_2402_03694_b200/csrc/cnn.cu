@@ -29,12 +29,17 @@
 //
 // Persistent CTAs, one per SM, loop over pairs of flows.  Warp roles:
 //   warp 0        streams input rows with bulk copies into a ring
-//   warp 1        issues the MMAs in the order conv2(pair i), conv1(pair i+2)
-//   warps 2..5    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's B operand (shared memory)
-//   warps 6..21   E2: conv2 accumulators -> bias + ReLU -> bf16 -> partial sums over 32 positions
-//   warps 22..25  E3: partial sums -> mean -> linear head -> logits, argmax
+//   warp 1        issues conv2's MMAs, pair after pair
+//   warp 2        issues conv1's MMAs: those of pair i+2 right behind conv2 of pair i
+//   warps 3..6    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's B operand (shared memory)
+//   warps 7..22   E2: conv2 accumulators -> bias + ReLU -> bf16 -> partial sums over 32 positions
+//   warps 23..26  E3: partial sums -> mean -> linear head -> logits, argmax
+// The tensor pipe queues only two or three instructions, so a thread that issues MMAs must not do
+// anything else for long: with one issuing thread the barrier waits of conv1 left the pipe idle for a
+// third of the time.  Hence two issuing threads: while one sits in its waits the other keeps the queue full.
 // conv2's accumulator (256 TMEM columns) is single: the E2 warps pull it into registers first
-// thing and release it, and conv1 of a later pair keeps the pipe busy meanwhile.  Every wait is
+// thing and release it, and conv1 of a later pair keeps the pipe busy meanwhile.  conv1's bias reaches the
+// E1 threads as a kernel parameter (constant bank operands: no loads, no registers).  Every wait is
 // bounded; on a timeout the block records SF_ERR_DEVICE_TIMEOUT and leaves.
 #include "tc_common.cuh"
 #include <stdlib.h>
@@ -45,8 +50,8 @@ using namespace sftc;
 
 constexpr uint32_t L = 128, CIN = 8, C1 = 64, C2 = 128, KW = 5, NCLS_MAX = 16;
 constexpr uint32_t kE1Warps = 4, kE2Warps = 16, kE3Warps = 4;
-constexpr uint32_t kE1First = 2, kE2First = kE1First + kE1Warps, kE3First = kE2First + kE2Warps;
-constexpr uint32_t kThreads = (kE3First + kE3Warps) * 32;       // 832
+constexpr uint32_t kE1First = 3, kE2First = kE1First + kE1Warps, kE3First = kE2First + kE2Warps;
+constexpr uint32_t kThreads = (kE3First + kE3Warps) * 32;       // 864
 constexpr uint32_t XS = 4;                                  // input-row ring depth
 constexpr uint32_t X_STAGE = (2 + L + 3) * 16;              // 2 zero rows, 128 rows, 3 zero rows (tap 5 is a zero tap)
 constexpr uint32_t H1_COL = 2 * (2 + L + 2) * 16;           // one 8-channel column of a PAIR's conv1 output: 264 rows, 4,224 bytes
@@ -82,6 +87,7 @@ struct Bars {
     uint64_t d1_full[2], d1_empty[2];          // per flow slot of a pair
     uint64_t h1_full[2], h1_empty[2];          // per pair buffer
     uint64_t d2_full, d2_empty;
+    uint64_t c2_issued;                        // conv2 of a pair has been handed to the tensor pipe
     uint64_t part_full[2], part_empty[2];
     uint32_t tmem_base, abort_flag;
 };
@@ -118,9 +124,11 @@ __device__ __forceinline__ uint32_t relu_bf16x2(float hi, float lo) {
     return d;
 }
 
+struct Bias1 { float v[C1]; };
+
 __global__ void __launch_bounds__(kThreads, 1)
 cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restrict__ n_rows_dev,
-                 const unsigned char* __restrict__ blob, uint32_t n_cls,
+                 const unsigned char* __restrict__ blob, const __grid_constant__ Bias1 b1, uint32_t n_cls,
                  float* __restrict__ logits, uint8_t* __restrict__ label, sf_dev_state* st)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -146,6 +154,7 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             mbar_init(&bars->part_full[b], kE2Warps); mbar_init(&bars->part_empty[b], kE3Warps);
         }
         mbar_init(&bars->d2_full, 1); mbar_init(&bars->d2_empty, kE2Warps);
+        mbar_init(&bars->c2_issued, 1);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -170,19 +179,45 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             }
         }
     } else if (warp == 1) {
+        // ---- conv2: weights of tap t (A, M = 128 output channels) x the pair's activations (B, N = 256) ----
         if (lane == 0 && n_mine > 0) {
-            constexpr uint32_t idesc1 = make_idesc_bf16(128, C1);
             constexpr uint32_t idesc2 = make_idesc_bf16(C2, 2 * L);
             // descriptor = constant fields + (address >> 4) in the low bits: build the bases once, add offsets per MMA
-            const uint64_t dX = make_smem_desc(sbase + SM_X, 16, 128, 0);
-            const uint64_t dW1 = make_smem_desc(sbase + SM_BLOB + W1_OFF, C1 * 16u, 128, 0);
             const uint64_t dH1 = make_smem_desc(sbase + SM_H1, H1_COL, 128, 0);
             const uint64_t dW2 = make_smem_desc(sbase + SM_BLOB + W2_OFF, C2 * 16u, 128, 0);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
-            auto conv1_flow = [&](uint32_t m) -> bool {
+            for (uint32_t i = 0; i < n_pairs && ok; i++) {
+                const uint32_t b = i & 1u;
+                if (!mbar_wait(&bars->h1_full[b], (i >> 1) & 1u, abort_flag)) break;
+                if (!mbar_wait(&bars->d2_empty, (i & 1u) ^ 1u, abort_flag)) break;
+                tc_fence_after();
+                const uint64_t bh = dH1 + (uint64_t)((b * H1_BYTES) >> 4);
+#pragma unroll
+                for (uint32_t t = 0; t < KW; t++) {
+#pragma unroll
+                    for (uint32_t k = 0; k < C1 / 16; k++)      // the activations two rows per tap further down
+                        umma_bf16(tmem_base + TM_D2, dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4),
+                                  bh + (((2u * k) * H1_COL + t * 32u) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
+                }
+                umma_commit(&bars->h1_empty[b]);
+                umma_commit(&bars->d2_full);
+                mbar_arrive(&bars->c2_issued);
+            }
+        }
+    } else if (warp == 2) {
+        // ---- conv1: one flow's positions (A, M = 128) x the weights of two taps (B, N = 64) ----
+        if (lane == 0 && n_mine > 0) {
+            constexpr uint32_t idesc1 = make_idesc_bf16(128, C1);
+            const uint64_t dX = make_smem_desc(sbase + SM_X, 16, 128, 0);
+            const uint64_t dW1 = make_smem_desc(sbase + SM_BLOB + W1_OFF, C1 * 16u, 128, 0);
+            bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
+            for (uint32_t m = 0; m < n_mine && ok; m++) {
                 const uint32_t xs = m % XS, xph = (m / XS) & 1u, s = m & 1u, i = m >> 1;
-                if (!mbar_wait(&bars->x_full[xs], xph, abort_flag)) return false;
-                if (!mbar_wait(&bars->d1_empty[s], (i & 1u) ^ 1u, abort_flag)) return false;
+                // pairs 0 and 1 go ahead; pair i + 2 waits until conv2 of pair i is in the pipe's queue, so that it
+                // runs while the E2 warps empty conv2's accumulator
+                if (s == 0 && i >= 2 && !mbar_wait(&bars->c2_issued, i & 1u, abort_flag)) break;
+                if (!mbar_wait(&bars->x_full[xs], xph, abort_flag)) break;
+                if (!mbar_wait(&bars->d1_empty[s], (i & 1u) ^ 1u, abort_flag)) break;
                 tc_fence_after();
                 const uint64_t ax = dX + (uint64_t)((xs * X_STAGE) >> 4);
 #pragma unroll
@@ -191,43 +226,11 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                               k != 0 ? 1u : 0u);
                 umma_commit(&bars->x_empty[xs]);
                 umma_commit(&bars->d1_full[s]);
-                return true;
-            };
-            auto conv1_pair = [&](uint32_t i) -> bool {
-                if (!conv1_flow(2u * i)) return false;
-                if (2u * i + 1u < n_mine) return conv1_flow(2u * i + 1u);
-                return true;
-            };
-            auto conv2 = [&](uint32_t i) -> bool {
-                const uint32_t b = i & 1u;
-                if (!mbar_wait(&bars->h1_full[b], (i >> 1) & 1u, abort_flag)) return false;
-                if (!mbar_wait(&bars->d2_empty, (i & 1u) ^ 1u, abort_flag)) return false;
-                tc_fence_after();
-                const uint64_t bh = dH1 + (uint64_t)((b * H1_BYTES) >> 4);
-#pragma unroll
-                for (uint32_t t = 0; t < KW; t++) {
-#pragma unroll
-                    for (uint32_t k = 0; k < C1 / 16; k++)      // A = weights of tap t, B = the pair's activations two rows per tap further down
-                        umma_bf16(tmem_base + TM_D2, dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4),
-                                  bh + (((2u * k) * H1_COL + t * 32u) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
-                }
-                umma_commit(&bars->h1_empty[b]);
-                umma_commit(&bars->d2_full);
-                return true;
-            };
-            // conv1 runs two pairs ahead of conv2: its MMAs keep the pipe busy while the E2 warps pull conv2's
-            // accumulator out of TMEM, and E1 has a whole conv2 period to write the next operand
-            if (ok) ok = conv1_pair(0);
-            if (ok && n_pairs > 1) ok = conv1_pair(1);
-            for (uint32_t i = 0; i < n_pairs && ok; i++) {
-                ok = conv2(i);
-                if (ok && i + 2 < n_pairs) ok = conv1_pair(i + 2);
             }
         }
     } else if (n_mine > 0 && warp < kE2First) {
         // ---- E1: conv1 accumulators -> conv2's B operand -------------------------------
         const uint32_t p = q * 32u + lane;               // position handled by this thread
-        const float* b1 = reinterpret_cast<const float*>(smem + SM_BLOB + B1_OFF);
         bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
         for (uint32_t m = 0; m < n_mine && ok; m++) {
             const uint32_t s = m & 1u, i = m >> 1, b = i & 1u;
@@ -252,7 +255,7 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                 for (int e = 0; e < 4; e++) {
                     const int c = (j & 3) * 8 + e * 2;
                     const uint32_t a = (j < 4) ? v0[c] : v1[c], bq = (j < 4) ? v0[c + 1] : v1[c + 1];
-                    pk[e] = pack_relu_bf16(a, bq, b1[j * 8 + e * 2], b1[j * 8 + e * 2 + 1]);
+                    pk[e] = pack_relu_bf16(a, bq, b1.v[j * 8 + e * 2], b1.v[j * 8 + e * 2 + 1]);
                 }
                 *reinterpret_cast<uint4*>(hrow + j * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
@@ -399,6 +402,7 @@ int sf_cnn_prepare(sf_slow* s, const float* w1, const float* b1, const float* w2
             memcpy(&W3[c * C2 + k], &bits, 4);
         }
     memcpy(h + B1_OFF, b1, C1 * 4);
+    memcpy(s->h_cnn_b1, b1, C1 * 4);
     memcpy(h + B2_OFF, b2, C2 * 4);
     memcpy(h + B3_OFF, b3, s->n_cls * 4);
     cudaError_t e = cudaMalloc(&s->d_w1, BLOB_BYTES);
@@ -418,7 +422,7 @@ int sf_cnn_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     uint32_t grid = (uint32_t)ctx->num_sms < capacity ? (uint32_t)ctx->num_sms : capacity;
     sf_time_begin(ctx, SF_T_GEMM, st);
     cnn_fused_kernel<<<grid, kThreads, SM_TOTAL, st>>>(reinterpret_cast<const __nv_bfloat16*>(rows), n_rows_dev,
-                                                     reinterpret_cast<const unsigned char*>(s->d_w1), s->n_cls,
+                                                     reinterpret_cast<const unsigned char*>(s->d_w1), *reinterpret_cast<const Bias1*>(s->h_cnn_b1), s->n_cls,
                                                      logits, label, ctx->d_state);
     sf_time_end(ctx, SF_T_GEMM, st);
     SF_LAUNCH_CHECK("cnn_fused_kernel");

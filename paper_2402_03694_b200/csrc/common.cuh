@@ -71,6 +71,7 @@ struct sf_slow {
     uint32_t L, Cin, C1, C2, k, n_cls;
     void* d_w1; void* d_w2; void* d_w3;      // re-laid-out bf16 operands
     float* d_b1; float* d_b2; float* d_b3;
+    float h_cnn_b1[64];                      // conv1 bias, handed to the fused kernel as a launch parameter
 };
 
 // ---- helpers ---------------------------------------------------------------
