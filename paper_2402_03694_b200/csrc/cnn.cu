@@ -199,9 +199,9 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
                         umma_bf16(tmem_base + TM_D2, dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4),
                                   bh + (((2u * k) * H1_COL + t * 32u) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
                 }
-                umma_commit(&bars->h1_empty[b]);
+                mbar_arrive(&bars->c2_issued);                  // conv1 of pair i + 2 may follow in the queue
                 umma_commit(&bars->d2_full);
-                mbar_arrive(&bars->c2_issued);
+                umma_commit(&bars->h1_empty[b]);
             }
         }
     } else if (warp == 2) {
@@ -211,21 +211,28 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             const uint64_t dX = make_smem_desc(sbase + SM_X, 16, 128, 0);
             const uint64_t dW1 = make_smem_desc(sbase + SM_BLOB + W1_OFF, C1 * 16u, 128, 0);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
-            for (uint32_t m = 0; m < n_mine && ok; m++) {
-                const uint32_t xs = m % XS, xph = (m / XS) & 1u, s = m & 1u, i = m >> 1;
-                // pairs 0 and 1 go ahead; pair i + 2 waits until conv2 of pair i is in the pipe's queue, so that it
-                // runs while the E2 warps empty conv2's accumulator
-                if (s == 0 && i >= 2 && !mbar_wait(&bars->c2_issued, i & 1u, abort_flag)) break;
-                if (!mbar_wait(&bars->x_full[xs], xph, abort_flag)) break;
-                if (!mbar_wait(&bars->d1_empty[s], (i & 1u) ^ 1u, abort_flag)) break;
+            for (uint32_t i = 0; i < n_pairs && ok; i++) {
+                const uint32_t n_fl = (2u * i + 1u < n_mine) ? 2u : 1u;
+                // everything this pair's MMAs need is ready long before their turn: check it first ...
+                for (uint32_t s = 0; s < n_fl && ok; s++) {
+                    const uint32_t m = 2u * i + s, xs = m % XS, xph = (m / XS) & 1u;
+                    ok = mbar_wait(&bars->x_full[xs], xph, abort_flag) && mbar_wait(&bars->d1_empty[s], (i & 1u) ^ 1u, abort_flag);
+                }
+                // ... then take the turn: pairs 0 and 1 go ahead, pair i waits until conv2 of pair i - 2 is in the pipe's
+                // queue, so that these MMAs run while the E2 warps empty conv2's accumulator
+                if (ok && i >= 2) ok = mbar_wait(&bars->c2_issued, i & 1u, abort_flag);
+                if (!ok) break;
                 tc_fence_after();
-                const uint64_t ax = dX + (uint64_t)((xs * X_STAGE) >> 4);
+                for (uint32_t s = 0; s < n_fl; s++) {
+                    const uint32_t xs = (2u * i + s) % XS;
+                    const uint64_t ax = dX + (uint64_t)((xs * X_STAGE) >> 4);
 #pragma unroll
-                for (uint32_t k = 0; k < 3; k++)             // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
-                    umma_bf16(tmem_base + TM_D1 + s * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4), idesc1,
-                              k != 0 ? 1u : 0u);
-                umma_commit(&bars->x_empty[xs]);
-                umma_commit(&bars->d1_full[s]);
+                    for (uint32_t k = 0; k < 3; k++)         // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
+                        umma_bf16(tmem_base + TM_D1 + s * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4), idesc1,
+                                  k != 0 ? 1u : 0u);
+                    umma_commit(&bars->d1_full[s]);
+                    umma_commit(&bars->x_empty[xs]);
+                }
             }
         }
     } else if (n_mine > 0 && warp < kE2First) {
@@ -273,30 +280,27 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
         const float bias = ok ? reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF)[ch] : 0.0f;
         for (uint32_t i = 0; i < n_pairs && ok; i++) {
             const uint32_t b = i & 1u;
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->d2_full, i & 1u, abort_flag));
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->d2_full, i & 1u, abort_flag));     // on the critical path: poll without backing off
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D2 + g * 64u;
-            uint32_t v[32], pk[16];
-            tmem_ld32(taddr, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 16; j++)                  // columns 2j, 2j+1 = position 32g+j of flows 0, 1
-                pk[j] = relu_bf16x2(__uint_as_float(v[2 * j + 1]) + bias, __uint_as_float(v[2 * j]) + bias);
-            tmem_ld32(taddr + 32, v);
+            uint32_t v0[32], v1[32];
+            tmem_ld32(taddr, v0);
+            tmem_ld32(taddr + 32, v1);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->d2_empty);         // the accumulator is in registers: conv2 may reuse it
             float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-            for (int j = 0; j < 16; j++) {
-                s0 += __uint_as_float(pk[j] << 16);
-                s1 += __uint_as_float(pk[j] & 0xFFFF0000u);
+            for (int j = 0; j < 16; j++) {                // columns 2j, 2j+1 = position 32g+j of flows 0, 1
+                const uint32_t h = relu_bf16x2(__uint_as_float(v0[2 * j + 1]) + bias, __uint_as_float(v0[2 * j]) + bias);
+                s0 += __uint_as_float(h << 16);
+                s1 += __uint_as_float(h & 0xFFFF0000u);
             }
 #pragma unroll
             for (int j = 0; j < 16; j++) {
-                const uint32_t h = relu_bf16x2(__uint_as_float(v[2 * j + 1]) + bias, __uint_as_float(v[2 * j]) + bias);
+                const uint32_t h = relu_bf16x2(__uint_as_float(v1[2 * j + 1]) + bias, __uint_as_float(v1[2 * j]) + bias);
                 s0 += __uint_as_float(h << 16);
                 s1 += __uint_as_float(h & 0xFFFF0000u);
             }
