@@ -355,7 +355,8 @@ def test_cnn_tap_alignment_with_delta_kernels(env):
         sf.sf_slow_destroy(h)
 
 
-@pytest.mark.parametrize("n_rows,cap,n_cls", [(1, 1, 16), (300, 333, 16), (1000, 1000, 7)])
+# 6,001 rows: about 40 flows (20 pairs, some odd counts) per persistent block, so every ring and barrier phase wraps several times
+@pytest.mark.parametrize("n_rows,cap,n_cls", [(1, 1, 16), (2, 2, 16), (300, 333, 16), (1000, 1000, 7), (6001, 6100, 16)])
 def test_cnn_within_tolerance(env, n_rows, cap, n_cls):
     sf, hz, ctx = env
     m = flowgen.gen_cnn(73, 128, 8, 64, 128, 5, n_cls)
