@@ -147,15 +147,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // W = fields per packet (16: size, L, dir, 13 header bytes; 8: size, L, dir, 5 header bytes)
-template <int W, bool BF16>
+// HW: the header plane starts on a 4-byte boundary, so a packet's NH header bytes are fetched as the
+// aligned 32-bit words that contain them (4 loads instead of 13 for the 16-field row) and moved into
+// place with funnel shifts; only the plane's last, partial word is assembled from byte loads.
+template <int W, bool BF16, bool HW>
 __global__ void __launch_bounds__(256)
 gather_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__ n_esc_dev,
               const uint16_t* __restrict__ size, const uint32_t* __restrict__ iat,
               const uint32_t* __restrict__ dir_bits, const uint8_t* __restrict__ hdr,
-              const uint8_t* __restrict__ n_valid, uint32_t pitch, uint32_t hdr_bytes,
+              const uint8_t* __restrict__ n_valid, uint32_t pitch, uint32_t hdr_bytes, size_t hdr_total,
               uint32_t P, uint32_t P_real, void* __restrict__ rows)
 {
     constexpr int NH = W - 3;
+    constexpr int NW = (NH + 6) / 4;             // words that can hold NH bytes starting at any byte of the first
     const uint32_t n_esc = *n_esc_dev;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
@@ -171,9 +175,32 @@ gather_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__
                 v[0] = __fmul_rn(__uint2float_rn((uint32_t)size[row0 + i]), 0x1p-11f);
                 v[1] = __fmul_rn(__uint2float_rn(ilog4(iat[row0 + i])), 0x1p-7f);
                 v[2] = (float)((dir_bits[(size_t)f * words + (i >> 5)] >> (i & 31)) & 1u);
-                const uint8_t* h = hdr + (row0 + i) * hdr_bytes;
+                if (HW) {
+                    const size_t boff = (row0 + i) * hdr_bytes;
+                    const size_t w0 = boff >> 2;
+                    const uint32_t sh = (uint32_t)(boff & 3) * 8u;
+                    uint32_t raw[NW + 1];
 #pragma unroll
-                for (int k = 0; k < NH; k++) v[3 + k] = __fmul_rn(__uint2float_rn((uint32_t)h[k]), 0x1p-8f);
+                    for (int j = 0; j < NW; j++) {
+                        const size_t a = (w0 + j) * 4;
+                        if (a + 4 <= hdr_total) {
+                            raw[j] = __ldg(reinterpret_cast<const uint32_t*>(hdr) + w0 + j);
+                        } else {                         // the plane's last bytes: never read past its end
+                            raw[j] = 0;
+                            for (uint32_t b = 0; b < 4; b++) if (a + b < hdr_total) raw[j] |= (uint32_t)hdr[a + b] << (8 * b);
+                        }
+                    }
+                    raw[NW] = 0;
+#pragma unroll
+                    for (int k = 0; k < NH; k++) {
+                        const uint32_t al = __funnelshift_r(raw[k / 4], raw[k / 4 + 1], sh);      // bytes k/4*4 .. +3 of the packet's header
+                        v[3 + k] = __fmul_rn(__uint2float_rn((al >> (8 * (k % 4))) & 0xFFu), 0x1p-8f);
+                    }
+                } else {
+                    const uint8_t* h = hdr + (row0 + i) * hdr_bytes;
+#pragma unroll
+                    for (int k = 0; k < NH; k++) v[3 + k] = __fmul_rn(__uint2float_rn((uint32_t)h[k]), 0x1p-8f);
+                }
             } else {
 #pragma unroll
                 for (int k = 0; k < W; k++) v[k] = 0.0f;
@@ -289,8 +316,10 @@ int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wid
     uint32_t blocks = (capacity + 7) / 8;
     uint32_t max_blocks = (uint32_t)ctx->num_sms * 32;
     if (blocks > max_blocks) blocks = max_blocks;
-#define SF_GATHER2(Wv, BF) gather_kernel<Wv, BF><<<blocks, 256, 0, st>>>(ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, \
-        wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, P, P_real, rows)
+    const size_t hdr_total = (size_t)wide->n_flows * wide->pitch_pkts * wide->hdr_bytes;
+    const bool hdr_words = ((uintptr_t)wide->hdr & 3) == 0;
+#define SF_GATHER2(Wv, BF) do { if (hdr_words) gather_kernel<Wv, BF, true><<<blocks, 256, 0, st>>>(ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows); \
+        else gather_kernel<Wv, BF, false><<<blocks, 256, 0, st>>>(ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows); } while (0)
     if (cfg->wide_layout == SF_MLP16) { if (cfg->row_dtype == SF_BF16) SF_GATHER2(16, true); else SF_GATHER2(16, false); }
     else                              { if (cfg->row_dtype == SF_BF16) SF_GATHER2(8, true);  else SF_GATHER2(8, false); }
 #undef SF_GATHER2
@@ -338,9 +367,11 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
         uint32_t max_blocks = (uint32_t)ctx->num_sms * 32;
         if (blocks > max_blocks) blocks = max_blocks;
         const uint32_t* cnt = &ctx->d_state->scan_total;
+        const size_t hdr_total = (size_t)wide->n_flows * wide->pitch_pkts * wide->hdr_bytes;
+        const bool hdr_words = ((uintptr_t)wide->hdr & 3) == 0;
         sf_time_begin(ctx, SF_T_GATHER, st);
-#define SF_GATHER(Wv, BF) gather_kernel<Wv, BF><<<blocks, 256, 0, st>>>(esc_ids, cnt, wide->size, wide->iat_us, wide->dir_bits, \
-            wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, P, P_real, rows)
+#define SF_GATHER(Wv, BF) do { if (hdr_words) gather_kernel<Wv, BF, true><<<blocks, 256, 0, st>>>(esc_ids, cnt, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows); \
+        else gather_kernel<Wv, BF, false><<<blocks, 256, 0, st>>>(esc_ids, cnt, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows); } while (0)
         if (cfg->wide_layout == SF_MLP16) { if (cfg->row_dtype == SF_BF16) SF_GATHER(16, true); else SF_GATHER(16, false); }
         else                              { if (cfg->row_dtype == SF_BF16) SF_GATHER(8, true);  else SF_GATHER(8, false); }
 #undef SF_GATHER
