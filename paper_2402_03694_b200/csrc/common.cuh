@@ -55,6 +55,7 @@ struct sf_forest {
     uint32_t tree_stride;
     // leaves: RF fp32[T][2^d][C]; GBDT fp32[T][2^d]
     float* d_leaf;
+    cudaTextureObject_t leaf_tex;      // RF with C % 4 == 0: the same table as a linear texture of 16-byte texels (0 = none)
 };
 
 enum { SF_SLOW_MLP = 0, SF_SLOW_CNN = 1 };

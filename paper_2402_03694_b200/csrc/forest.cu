@@ -3,9 +3,10 @@
 // One thread per flow, 512 flows per block.  The block's feature rows sit in shared
 // memory transposed ([feature][flow], so a lane's read of x[fid] hits bank = lane
 // whatever fid is).  The ensemble streams through shared memory in chunks of whole
-// trees: one thread issues a bulk copy (cp.async.bulk, completion on an mbarrier) of the
-// next chunk into the other buffer while the block walks the current one, so the copy
-// costs no load/store instructions.  A node is 8 bytes {threshold bits, byte offset of its feature's
+// trees: a producer warp (one extra warp per block) issues a bulk copy (cp.async.bulk, completion on a
+// "full" mbarrier) of a chunk as soon as every walking warp has released that buffer (an "empty" mbarrier
+// with one arrival per warp), so the copy costs no load/store instructions and no warp ever waits at a
+// block-wide barrier for the slowest one: a warp that is done with a chunk goes straight on to the next.  A node is 8 bytes {threshold bits, byte offset of its feature's
 // row in the tile}; trees are 1-based heaps.  A walk keeps the node's shared-memory
 // ADDRESS as its state (addr' = 2*addr + (go right ? 8 : 0) - base), so a level costs
 // six instructions: node load, feature address, feature load, compare, select, shift-add.
@@ -14,10 +15,17 @@
 // t = 0..T-1, which fixes the fp32 summation order.  Random-forest leaf vectors are
 // gathered from L2 one group ahead of their use; boosted-tree leaf scalars travel
 // with their tree's nodes in the shared-memory image.
+// The walk keeps the SM's load/store pipe busy (shared-memory wavefronts), and a gather of one
+// 32-byte sector per lane through the same pipe costs as much as nine levels of the walk.  So,
+// where the class count is a multiple of four, the leaf vectors are fetched through the texture
+// path instead (a linear texture of 16-byte integer texels over the same table: raw bits, no
+// filtering): it has its own queue into the L1, and the gather then overlaps the walk (115 -> 88
+// cycles per warp and tree in a microbenchmark of exactly this mix).
 // A second instantiation with 128 flows per block serves the streaming path, where a launch
 // carries a few thousand flows: more blocks, and a block's walk is latency-bound either way.
 #include "tc_common.cuh"
 #include <new>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -87,14 +95,25 @@ __device__ __forceinline__ void load_leaf_vec(const float* __restrict__ lv, floa
     }
 }
 
+// the same vector through the texture path: C / 4 texels of 16 bytes, starting at texel index `texel`
+template <int C>
+__device__ __forceinline__ void load_leaf_vec_tex(cudaTextureObject_t tex, uint32_t texel, float (&p)[C]) {
+#pragma unroll
+    for (int c = 0; c < C; c += 4) {
+        const uint4 v = tex1Dfetch<uint4>(tex, (int)(texel + c / 4));
+        p[c] = __uint_as_float(v.x); p[c + 1] = __uint_as_float(v.y); p[c + 2] = __uint_as_float(v.z); p[c + 3] = __uint_as_float(v.w);
+    }
+}
+
 // KIND: SF_RF (leaf = C-vector of class probabilities in global memory), SF_GBDT (leaf =
 // scalar stored behind the tree's nodes in the image, C = 1) or SF_GBDT_MC (scalar leaves, tree t
 // adds to class t mod C; a chunk holds whole boosting rounds, so the class of every tree in the
 // unrolled round loop is a compile-time register index).  NCH: trees walked at once.
-template <int KIND, int C, int NCH, uint32_t KB>
-__global__ void __launch_bounds__(KB, 1)
+// TEX: leaf vectors come through the texture object (random forests whose C is a multiple of 4).
+template <int KIND, int C, int NCH, uint32_t KB, bool TEX>
+__global__ void __launch_bounds__(KB + 32, 1)
 forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
-              const unsigned char* __restrict__ image, const float* __restrict__ leaf,
+              const unsigned char* __restrict__ image, const float* __restrict__ leaf, cudaTextureObject_t leaf_tex,
               uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
               float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev)
 {
@@ -103,29 +122,23 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
     if (blockIdx.x * KB >= n) return;
     const uint32_t sbuf0 = smem_u32(smem_raw);
     float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][KB]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * KB * 4);   // [2] + flag
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * KB * 4);   // full[2], empty[2], flag
+    uint64_t* empty = bars + 2;
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 4);
     const uint32_t xbase = smem_u32(xs) + threadIdx.x * 4u;
     const uint32_t f = blockIdx.x * KB + threadIdx.x;
-    const bool live = f < n;
+    const bool producer = threadIdx.x >= KB;                 // the extra warp
+    const bool live = !producer && f < n;
     const uint32_t n_leaf = 1u << depth;
     const uint32_t n_chunks = (T + trees_per_chunk - 1) / trees_per_chunk;
-
-    // called by thread 0 only; the buffer's previous readers have passed a __syncthreads
-    auto issue_chunk = [&](uint32_t ck) {
-        const uint32_t t0 = ck * trees_per_chunk;
-        const uint32_t nt = min(trees_per_chunk, T - t0);
-        const uint32_t bytes = nt * tree_stride;                         // a multiple of 16
-        sftc::mbar_expect_tx(&bars[ck & 1u], bytes);
-        sftc::bulk_load(smem_raw + (size_t)(ck & 1u) * chunk_bytes, image + (size_t)t0 * tree_stride, bytes, &bars[ck & 1u]);
-    };
 
     if (threadIdx.x == 0) {
         sftc::mbar_init(&bars[0], 1);
         sftc::mbar_init(&bars[1], 1);
+        sftc::mbar_init(&empty[0], KB / 32);
+        sftc::mbar_init(&empty[1], KB / 32);
         *abort_flag = 0;
         sftc::fence_barrier_init();
-        issue_chunk(0);
     }
     if (live) {
         const float* row = feat + (size_t)f * F;
@@ -138,8 +151,24 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         } else {
             for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = row[j];
         }
-    } else {
+    } else if (!producer) {
         for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = 0.0f;
+    }
+    __syncthreads();                              // barriers initialised, feature tile written
+
+    if (producer) {
+        if (threadIdx.x == KB) {
+            for (uint32_t ck = 0; ck < n_chunks; ck++) {
+                // the buffer's previous chunk (ck - 2) has been released by every walking warp
+                if (ck >= 2 && !sftc::mbar_wait_relaxed(&empty[ck & 1u], ((ck >> 1) - 1u) & 1u, abort_flag)) break;
+                const uint32_t t0 = ck * trees_per_chunk;
+                const uint32_t nt = min(trees_per_chunk, T - t0);
+                const uint32_t bytes = nt * tree_stride;                         // a multiple of 16
+                sftc::mbar_expect_tx(&bars[ck & 1u], bytes);
+                sftc::bulk_load(smem_raw + (size_t)(ck & 1u) * chunk_bytes, image + (size_t)t0 * tree_stride, bytes, &bars[ck & 1u]);
+            }
+        }
+        return;
     }
 
     float acc[C];
@@ -159,8 +188,6 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
     };
 
     for (uint32_t ck = 0; ck < n_chunks; ck++) {
-        if (ck == 0) __syncthreads();             // barriers initialised, feature tile written
-        if (threadIdx.x == 0 && ck + 1 < n_chunks) issue_chunk(ck + 1);
         // every thread waits for this chunk's bytes (bounded: all give up together if they never land)
         if (!sftc::mbar_wait(&bars[ck & 1u], (ck >> 1) & 1u, abort_flag)) break;
         const uint32_t cur = sbuf0 + (ck & 1u) * chunk_bytes;
@@ -209,8 +236,10 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
             } else {
                 flush_pending();                      // the previous group's vectors have landed by now
 #pragma unroll
-                for (int k = 0; k < NCH; k++)
-                    load_leaf_vec<C>(leaf + ((size_t)(t0 + tt + k) * n_leaf + l[k]) * C, pend[k]);
+                for (int k = 0; k < NCH; k++) {
+                    if (TEX) load_leaf_vec_tex<C>(leaf_tex, ((t0 + tt + k) * n_leaf + l[k]) * (C / 4), pend[k]);
+                    else load_leaf_vec<C>(leaf + ((size_t)(t0 + tt + k) * n_leaf + l[k]) * C, pend[k]);
+                }
                 n_pend = NCH;
             }
         }
@@ -222,11 +251,13 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
                 acc[0] = __fadd_rn(acc[0], lds32f(cur + tt * tree_stride + n_leaf * 8u + l[0] * 4u));
             } else {
                 flush_pending();
-                load_leaf_vec<C>(leaf + ((size_t)(t0 + tt) * n_leaf + l[0]) * C, pend[0]);
+                if (TEX) load_leaf_vec_tex<C>(leaf_tex, ((t0 + tt) * n_leaf + l[0]) * (C / 4), pend[0]);
+                else load_leaf_vec<C>(leaf + ((size_t)(t0 + tt) * n_leaf + l[0]) * C, pend[0]);
                 n_pend = 1;
             }
         }
-        __syncthreads();          // everyone is done with this buffer before it is refilled
+        __syncwarp();             // this warp is done with the buffer: one arrival per warp lets the producer refill it
+        if ((threadIdx.x & 31u) == 0) sftc::mbar_arrive(&empty[ck & 1u]);
     }
     if (KIND == SF_RF) flush_pending();
     if (*abort_flag) { if (threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT); return; }
@@ -249,19 +280,19 @@ Plan make_plan(const sf_forest* fo, uint32_t kb = kB) {
     Plan p;
     const size_t feat_bytes = (size_t)fo->F * kb * sizeof(float);
     // two chunk buffers share what the feature tile leaves of the 227 KB: up to 64 KB each
-    const uint32_t avail = (uint32_t)(((kMaxSmem - feat_bytes - 32) / 2) & ~(size_t)15);
+    const uint32_t avail = (uint32_t)(((kMaxSmem - feat_bytes - 48) / 2) & ~(size_t)15);
     p.chunk_bytes = avail < 65536u ? avail : 65536u;
     p.tpc = p.chunk_bytes / fo->tree_stride;          // 0 if one tree does not fit (checked by the callers)
     if (p.tpc > fo->T) p.tpc = fo->T;
     if (fo->kind == SF_GBDT_MC) p.tpc -= p.tpc % fo->C;          // whole boosting rounds per chunk
     p.nch = (fo->kind == SF_GBDT_MC) ? (fo->C >= 4 ? 4u : (fo->C >= 2 ? 2u : 1u)) : (fo->kind == SF_GBDT) ? (p.tpc >= 4 ? 4u : (p.tpc >= 2 ? 2u : 1u)) : (p.tpc >= 2 ? 2u : 1u);
-    p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes + 32;       // + two mbarriers and the abort flag
+    p.smem = 2 * (size_t)p.chunk_bytes + feat_bytes + 48;       // + four mbarriers and the abort flag
     return p;
 }
 
-template <int KIND, int C, int NCH, uint32_t KB = kB>
+template <int KIND, int C, int NCH, uint32_t KB = kB, bool TEX = false>
 int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
-    auto k = forest_kernel<KIND, C, NCH, KB>;
+    auto k = forest_kernel<KIND, C, NCH, KB, TEX>;
     static size_t smem_set_dev[64] = {};               // per kernel instance and device: raise the opt-in limit only when it grows
     size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
     if (p.smem > smem_set) {
@@ -269,7 +300,7 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
         smem_set = p.smem;
     }
     const uint32_t grid = (n + KB - 1) / KB;
-    k<<<grid, KB, p.smem, st>>>(feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->T, fo->depth, fo->tree_stride, p.tpc,
+    k<<<grid, KB + 32, p.smem, st>>>(feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->leaf_tex, fo->T, fo->depth, fo->tree_stride, p.tpc,
                                 p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
@@ -278,13 +309,22 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
 template <int C>
 int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
               bool small_tiles) {
+    constexpr bool kTexOk = (C % 4) == 0;                 // whole 16-byte texels per leaf vector
+    const bool tex = kTexOk && fo->leaf_tex != 0;
     if (small_tiles && fo->d_image_small) {
         const Plan ps = make_plan(fo, kBSmall);
-        if (ps.tpc >= 2) return launch3<SF_RF, C, 2, kBSmall>(fo, ps, feat, n, out, leaf_idx, st, n_dev);
+        if (ps.tpc >= 2) {
+            if (tex) return launch3<SF_RF, C, 2, kBSmall, kTexOk>(fo, ps, feat, n, out, leaf_idx, st, n_dev);
+            return launch3<SF_RF, C, 2, kBSmall>(fo, ps, feat, n, out, leaf_idx, st, n_dev);
+        }
     }
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
-    if (p.nch == 2) return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    if (p.nch == 2) {
+        if (tex) return launch3<SF_RF, C, 2, kB, kTexOk>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+        return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    }
+    if (tex) return launch3<SF_RF, C, 1, kB, kTexOk>(fo, p, feat, n, out, leaf_idx, st, n_dev);
     return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
@@ -365,7 +405,7 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     sf_forest* fo = new (std::nothrow) sf_forest();
     if (!fo) return SF_ERR_ALLOC;
     fo->ctx = ctx; fo->kind = kind; fo->T = T; fo->depth = depth; fo->F = F; fo->C = (kind == SF_GBDT) ? 1 : C;
-    fo->d_image = nullptr; fo->d_leaf = nullptr; fo->d_image_small = nullptr;
+    fo->d_image = nullptr; fo->d_leaf = nullptr; fo->d_image_small = nullptr; fo->leaf_tex = 0;
     // Image of one tree: 2^d node entries of 8 bytes in a 1-based heap (host node i, children
     // 2i+1 / 2i+2, becomes entry i+1, children 2j / 2j+1; entry 0 unused), then for boosted
     // trees the 2^d leaf scalars; padded to a multiple of 16 bytes for the 16-byte copies.
@@ -404,12 +444,32 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     if (e == cudaSuccess) e = cudaMemcpy(fo->d_leaf, leaf, sizeof(float) * leaf_count, cudaMemcpyHostToDevice);
     free(h); free(h_small);
     if (e != cudaSuccess) { sf_forest_destroy(fo); return sf_set_cuda_error(e, "sf_forest_create"); }
+    if (kind == SF_RF && (fo->C % 4) == 0) {
+        // texture view of the leaf table (16-byte integer texels); where it cannot be made (table beyond the
+        // linear-texture limit, base not aligned for textures) the kernel gathers through plain loads
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, ctx->device) == cudaSuccess && leaf_count / 4 <= (size_t)prop.maxTexture1DLinear &&
+            ((uintptr_t)fo->d_leaf % prop.textureAlignment) == 0) {
+            cudaResourceDesc rd; memset(&rd, 0, sizeof(rd));
+            rd.resType = cudaResourceTypeLinear;
+            rd.res.linear.devPtr = fo->d_leaf;
+            rd.res.linear.desc = cudaCreateChannelDesc<uint4>();
+            rd.res.linear.sizeInBytes = sizeof(float) * leaf_count;
+            cudaTextureDesc td; memset(&td, 0, sizeof(td));
+            td.readMode = cudaReadModeElementType;
+            cudaTextureObject_t tex = 0;
+            if (cudaCreateTextureObject(&tex, &rd, &td, nullptr) == cudaSuccess) fo->leaf_tex = tex;
+            else (void)cudaGetLastError();
+        }
+        if (getenv("SF_DEBUG")) fprintf(stderr, "sf_forest_create: leaf texture %s (table %p, alignment %zu, texels %zu, limit %d)\n", fo->leaf_tex ? "made" : "not made", (void*)fo->d_leaf, (size_t)prop.textureAlignment, leaf_count / 4, prop.maxTexture1DLinear);
+    }
     *out = fo;
     return SF_OK;
 }
 
 extern "C" void sf_forest_destroy(sf_forest* fo) {
     if (!fo) return;
+    if (fo->leaf_tex) cudaDestroyTextureObject(fo->leaf_tex);
     if (fo->d_image) cudaFree(fo->d_image);
     if (fo->d_image_small) cudaFree(fo->d_image_small);
     if (fo->d_leaf) cudaFree(fo->d_leaf);
