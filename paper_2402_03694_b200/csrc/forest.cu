@@ -140,21 +140,7 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         *abort_flag = 0;
         sftc::fence_barrier_init();
     }
-    if (live) {
-        const float* row = feat + (size_t)f * F;
-        if ((F & 3) == 0) {
-            for (uint32_t j = 0; j < F; j += 4) {
-                float4 v = __ldg(reinterpret_cast<const float4*>(row + j));
-                xs[(j + 0) * KB + threadIdx.x] = v.x; xs[(j + 1) * KB + threadIdx.x] = v.y;
-                xs[(j + 2) * KB + threadIdx.x] = v.z; xs[(j + 3) * KB + threadIdx.x] = v.w;
-            }
-        } else {
-            for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = row[j];
-        }
-    } else if (!producer) {
-        for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = 0.0f;
-    }
-    __syncthreads();                              // barriers initialised, feature tile written
+    __syncthreads();                              // barriers initialised: the producer starts streaming trees right away
 
     if (producer) {
         if (threadIdx.x == KB) {
@@ -170,6 +156,22 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         }
         return;
     }
+
+    if (live) {
+        const float* row = feat + (size_t)f * F;
+        if ((F & 3) == 0) {
+            for (uint32_t j = 0; j < F; j += 4) {
+                float4 v = __ldg(reinterpret_cast<const float4*>(row + j));
+                xs[(j + 0) * KB + threadIdx.x] = v.x; xs[(j + 1) * KB + threadIdx.x] = v.y;
+                xs[(j + 2) * KB + threadIdx.x] = v.z; xs[(j + 3) * KB + threadIdx.x] = v.w;
+            }
+        } else {
+            for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = row[j];
+        }
+    } else {
+        for (uint32_t j = 0; j < F; j++) xs[j * KB + threadIdx.x] = 0.0f;
+    }
+    // the feature tile is read by its own thread only (column threadIdx.x of every row): no barrier needed
 
     float acc[C];
     float pend[NCH][C];
