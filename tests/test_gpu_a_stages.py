@@ -191,6 +191,35 @@ def test_route_absmargin_and_cnn_layout(env):
     sf.sf_ctx_poll(ctx, reset=True)
 
 
+@pytest.mark.parametrize("layout,H,P,n,shift", [(0, 13, 9, 7, 0), (0, 13, 9, 7, 1), (0, 13, 9, 7, 2), (1, 13, 11, 5, 0), (1, 5, 7, 3, 3)])
+def test_route_header_bytes_odd_planes(env, layout, H, P, n, shift):
+    """The gather reads a packet's header bytes as the aligned 32-bit words that contain them.  Planes whose
+    size is not a multiple of four (the last word is partial), a header stride wider than the bytes used, and a
+    header plane that does not start on a 4-byte boundary (byte loads instead) must all give the oracle's rows."""
+    sf, hz, ctx = env
+    C = 4
+    rng = np.random.default_rng(41 + shift)
+    prob = rng.dirichlet([0.5] * C, size=n).astype(np.float32)
+    tau = np.full(C, -1.0, np.float32)                     # every flow is assigned
+    wide = flowgen.gen_packets(42, n, P, H)
+    t = {k: hz.dev(wide[k]) for k in ("size", "iat_us", "dir_bits")}
+    buf = torch.zeros(n * P * H + 8, dtype=torch.uint8, device="cuda")
+    hv = buf[shift:shift + n * P * H].view(n, P, H)
+    hv.copy_(hz.dev(wide["hdr"]))
+    assert hv.data_ptr() % 4 == shift % 4
+    st = sf.make_packets(t["size"], t["iat_us"], t["dir_bits"], hv, None)
+    W = 16 if layout == 0 else 8
+    cfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16 if layout == 0 else sf.SF_CNN8, sf.SF_BF16, P, n)
+    ids = torch.zeros(n, dtype=torch.uint32, device="cuda")
+    n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    rows = torch.zeros((n, P * W), dtype=torch.bfloat16, device="cuda")
+    sf.sf_route(ctx, cfg, hz.dev(prob), n, C, st, ids, n_esc, rows)
+    assert int(n_esc.cpu().numpy()[0]) == n
+    ref_rows = oracle.wide_rows(layout, np.arange(n, dtype=np.uint32), wide, P, True)
+    assert np.array_equal(bits(rows.float().cpu().numpy()), bits(ref_rows))
+    sf.sf_ctx_poll(ctx, reset=True)
+
+
 def test_route_zero_padding_and_empty_and_overflow(env):
     sf, hz, ctx = env
     n, C = 3000, 4
