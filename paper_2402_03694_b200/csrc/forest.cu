@@ -25,7 +25,6 @@
 // carries a few thousand flows: more blocks, and a block's walk is latency-bound either way.
 #include "tc_common.cuh"
 #include <new>
-#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -463,7 +462,6 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
             if (cudaCreateTextureObject(&tex, &rd, &td, nullptr) == cudaSuccess) fo->leaf_tex = tex;
             else (void)cudaGetLastError();
         }
-        if (getenv("SF_DEBUG")) fprintf(stderr, "sf_forest_create: leaf texture %s (table %p, alignment %zu, texels %zu, limit %d)\n", fo->leaf_tex ? "made" : "not made", (void*)fo->d_leaf, (size_t)prop.textureAlignment, leaf_count / 4, prop.maxTexture1DLinear);
     }
     *out = fo;
     return SF_OK;
