@@ -1,7 +1,7 @@
-"""Config 2 at its full size (1,000,000 flows) in the launch configuration the benchmark
-times: features, fast-model probabilities, routing and the assigned-id list are compared
-with the oracle on ALL flows (bit-exact); wide rows and slow-model logits on sampled rows
-that include the first and the last GEMM row tile."""
+"""Configs 2, 3 and 4 at their full sizes in the launch configuration the benchmark times:
+features, fast-model outputs, routing and the assigned-id list are compared with the oracle
+on ALL flows (bit-exact); wide rows and slow-model logits on sampled rows that include the
+first and the last row tile."""
 import numpy as np
 import pytest
 
@@ -17,19 +17,22 @@ def bits(a):
     return np.ascontiguousarray(a, np.float32).view(np.uint32)
 
 
-def test_config2_full_size_against_oracle():
+@pytest.mark.parametrize("c", [2, 3, 4])
+def test_config_full_size_against_oracle(c):
+    """Configs 2, 3 and 4 at their full sizes (1,000,000 / 4,000,000 / 1,000,000 flows), as bench.py launches them."""
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2402_03694_b200 import build, binding as sf, harness as hz
     build.build()
-    cfg = flowgen.get_config(2)
+    cfg = flowgen.get_config(c)
     n = cfg.n
     wl = make_workload(cfg, n=n, threads=16)
     feat = oracle.extract_features(wl["fast"], cfg.N, cfg.F, threads=16)
-    prob = oracle.forest_infer(wl["forest"], feat, threads=16)
-    rt = oracle.route_lc(prob, wl["tau"])
+    fast_out = oracle.forest_infer(wl["forest"], feat, threads=16)
+    rt = oracle.route_lc(fast_out, wl["tau"]) if cfg.kind == "rf" else oracle.route_absmargin(fast_out)
     k = rt["n_esc"]
-    assert 0.2 < k / n < 0.28
+    assert 0.2 < k / n < 0.4
+    Cf = 1 if cfg.kind == "gbdt" else cfg.C
 
     ctx = sf.sf_ctx_create(0, 0)
     forest = hz.make_forest(ctx, wl["forest"])
@@ -42,11 +45,11 @@ def test_config2_full_size_against_oracle():
     n_esc = torch.zeros(1, dtype=torch.uint32, device="cuda")
     sf.sf_serve_batch(ctx, forest, slow, fast_d["struct"], cfg.N, cfg.F, wide_d["struct"], rcfg, label, stage, n_esc)
     torch.cuda.synchronize()
-    c = sf.sf_ctx_poll(ctx, reset=True)
-    assert c.device_error == 0 and int(n_esc.cpu().numpy()[0]) == k and c.n_slow_done == k
+    cnt = sf.sf_ctx_poll(ctx, reset=True)
+    assert cnt.device_error == 0 and int(n_esc.cpu().numpy()[0]) == k and cnt.n_slow_done == k
     p = sf.sf_serve_batch_intermediates(ctx)
     assert np.array_equal(bits(hz.ptr_tensor(p["feat"], (n, cfg.F), torch.float32).cpu().numpy()), bits(feat))
-    assert np.array_equal(bits(hz.ptr_tensor(p["fast_out"], (n, cfg.C), torch.float32).cpu().numpy()), bits(prob))
+    assert np.array_equal(bits(hz.ptr_tensor(p["fast_out"], (n, Cf), torch.float32).cpu().numpy().reshape(fast_out.shape)), bits(fast_out))
     assert np.array_equal(hz.ptr_tensor(p["esc_ids"], (k,), torch.uint32).cpu().numpy(), rt["esc_ids"])
     st = stage.cpu().numpy()
     assert np.array_equal(st, 1 + rt["decision"])
@@ -55,10 +58,14 @@ def test_config2_full_size_against_oracle():
     # sampled rows: first tile, last (ragged) tile, and a random spread
     rng = np.random.default_rng(0)
     sel = np.unique(np.concatenate([np.arange(128), np.arange(k - 128, k), rng.integers(0, k, 256)]))
-    rows_ref = oracle.wide_rows(0, rt["esc_ids"][sel], wl["wide"], cfg.P, True, threads=16)
+    layout = 0 if cfg.slow == "mlp" else 1
+    rows_ref = oracle.wide_rows(layout, rt["esc_ids"][sel], wl["wide"], cfg.P, True, threads=16)
     rows_gpu = hz.ptr_tensor(p["rows"], (k, cfg.D), torch.bfloat16)[torch.from_numpy(sel).cuda()].float().cpu().numpy()
     assert np.array_equal(bits(rows_gpu), bits(rows_ref))
-    logits_ref, label_ref = oracle.mlp(wl["slow"], rows_ref, True, threads=16)
+    if cfg.slow == "mlp":
+        logits_ref, label_ref = oracle.mlp(wl["slow"], rows_ref, True, threads=16)
+    else:
+        logits_ref, label_ref = oracle.cnn(wl["slow"], rows_ref, True, threads=16)
     logits_gpu = hz.ptr_tensor(p["logits"], (k, cfg.n_slow_classes), torch.float32).cpu().numpy()[sel]
     assert np.max(np.abs(logits_gpu - logits_ref)) <= 2e-2
     s = np.sort(logits_ref, axis=1)
