@@ -103,6 +103,91 @@ def test_stream_matches_sequential_reference(env, shape):
     sf.sf_forest_destroy(forest_h)
 
 
+def test_stream_config5_full_size(env):
+    """Config 5 at its full size: 10,000,000 keys, a 2^25-slot table, 64K-packet batches, config 2's forest on
+    8 packets and its MLP on 64 packets.  The packet-by-packet reference is too slow here, so the expected values
+    come from what the method fixes for any stream: a flow fires the fast model with its 8th packet and, if
+    assigned, the slow model with its 64th; its answers are the batch oracle's on its first 8 / 64 packets in
+    arrival order; packets after a flow's answer are dropped.  All counters are compared; flow records on samples
+    (every flow that reached the slow model, random answered and unanswered flows)."""
+    sf, hz, ctx = env
+    cfg = flowgen.get_config(5)
+    n_batches, m = 48, 65536
+    fast_pkts, slow_pkts, P_model = cfg.N, cfg.P, 128
+    w = flowgen.gen_packets(cfg.seed_data, 65536, fast_pkts, 0)
+    feat = oracle.extract_features(w, fast_pkts, cfg.F, threads=16)
+    forest = flowgen.gen_forest(cfg.seed_model, "rf", cfg.T, cfg.depth, cfg.F, cfg.C, feat)
+    u = oracle.route_lc(oracle.forest_infer(forest, feat, threads=16), 2.0)["score"]
+    tau = np.full(cfg.C, oracle.universal_thresholds(u, [cfg.q_percent])[0], np.float32)
+    slow = flowgen.gen_mlp(cfg.seed_model, cfg.dims)
+    src = flowgen.StreamSource(cfg.seed_data, cfg.n, 1.1)
+    batches = [src.batch(b, m) for b in range(n_batches)]
+
+    # expected values, vectorised over the whole stream
+    cat = {k: np.concatenate([b[k] for b in batches]) for k in ("flow", "size", "iat_us", "dir", "hdr")}
+    order = np.argsort(cat["flow"], kind="stable")                  # packets grouped by flow, arrival order kept
+    flows, start, count = np.unique(cat["flow"][order], return_index=True, return_counts=True)
+    fired = np.nonzero(count >= fast_pkts)[0]
+    idx8 = order[start[fired][:, None] + np.arange(fast_pkts)[None, :]]
+    dirb = (cat["dir"][idx8].astype(np.uint32) & 1) << np.arange(fast_pkts, dtype=np.uint32)[None, :]
+    planes8 = {"size": cat["size"][idx8], "iat_us": cat["iat_us"][idx8], "dir_bits": dirb.sum(1, dtype=np.uint32)[:, None]}
+    rt = oracle.route_lc(oracle.forest_infer(forest, oracle.extract_features(planes8, fast_pkts, cfg.F, threads=16), threads=16), tau)
+    assigned = rt["decision"].astype(bool)
+    slow_sel = np.nonzero(assigned & (count[fired] >= slow_pkts))[0]            # rows of `fired`
+    idx64 = order[start[fired][slow_sel][:, None] + np.arange(slow_pkts)[None, :]]
+    d64 = cat["dir"][idx64].astype(np.uint32) & 1
+    dirw = np.stack([(d64[:, 32 * j:32 * j + 32] << np.arange(32, dtype=np.uint32)[None, :]).sum(1, dtype=np.uint32)
+                     for j in range(slow_pkts // 32)], axis=1)
+    planes64 = {"size": cat["size"][idx64], "iat_us": cat["iat_us"][idx64], "dir_bits": dirw, "hdr": cat["hdr"][idx64]}
+    rows = oracle.wide_rows(0, np.arange(len(slow_sel), dtype=np.uint32), planes64, P_model, True, P_real=slow_pkts, threads=16)
+    logits, label_slow = oracle.mlp(slow, rows, True, threads=16)
+    done_fast = ~assigned
+    exp = {"new_flows": len(flows), "fast_fired": len(fired), "fast_done": int(done_fast.sum()), "escalated": int(assigned.sum()),
+           "slow_fired": len(slow_sel),
+           "dropped_after_decision": int((count[fired][done_fast] - fast_pkts).sum() + (count[fired][slow_sel] - slow_pkts).sum())}
+    assert exp["slow_fired"] > 20 and exp["fast_fired"] > 5000
+
+    forest_h = hz.make_forest(ctx, forest)
+    slow_h = sf.sf_mlp_create(ctx, sf.SF_BF16, slow["dims"], slow["W"], slow["b"])
+    table = sf.sf_table_create(ctx, 25, fast_pkts, slow_pkts, 1 << 18)
+    rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
+    sf.sf_ctx_poll(ctx, reset=True)
+    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, cfg.F, slow_h, rcfg)
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert got["missed"] == 0 and c.device_error == 0
+    for k in exp:
+        assert got[k] == exp[k], (k, got[k], exp[k])
+    assert c.n_flows == exp["fast_fired"] and c.n_escalated == exp["escalated"] and c.n_slow_done == exp["slow_fired"]
+
+    # flow records on samples
+    rng = np.random.default_rng(5)
+    unfired = np.nonzero(count < fast_pkts)[0]
+    sample_f = np.unique(np.concatenate([slow_sel, rng.integers(0, len(fired), 1500)]))          # rows of `fired`
+    sample_u = unfired[rng.integers(0, len(unfired), 500)]                                     # rows of `flows`
+    kk = src.keys
+    def keys_of(rows_of_flows):
+        r = flows[rows_of_flows]
+        return [(int(kk["src"][i]), int(kk["dst"][i]), int(kk["sport"][i]), int(kk["dport"][i]), int(kk["proto"][i])) for i in r]
+    res = _lookup(sf, hz, ctx, table, keys_of(fired[sample_f]) + keys_of(sample_u))
+    slow_row = {int(r): j for j, r in enumerate(slow_sel)}
+    for i, r in enumerate(sample_f):
+        g = res[i]
+        stage = 1 if done_fast[r] else (3 if int(r) in slow_row else 2)
+        assert g["found"] == 1 and g["n_pkts"] == count[fired[r]] and g["stage"] == stage, (r, g)
+        assert g["label_fast"] == rt["label"][r]
+        assert np.float32(g["score"]).view(np.uint32) == np.float32(rt["score"][r]).view(np.uint32)
+        if stage == 3:
+            lg = np.sort(logits[slow_row[int(r)]])
+            if lg[-1] - lg[-2] >= 4e-2:
+                assert g["label_slow"] == label_slow[slow_row[int(r)]]
+    for i, r in enumerate(sample_u):
+        g = res[len(sample_f) + i]
+        assert g["found"] == 1 and g["n_pkts"] == count[r] and g["stage"] == 0
+    sf.sf_table_destroy(table)
+    sf.sf_slow_destroy(slow_h)
+    sf.sf_forest_destroy(forest_h)
+
+
 def test_full_table_is_reported_not_fatal(env):
     sf, hz, ctx = env
     forest, tau, slow = _models(24, 4, 4, 4, (1024, 64, 4), 93)
