@@ -24,6 +24,7 @@
 // A second instantiation with 128 flows per block serves the streaming path, where a launch
 // carries a few thousand flows: more blocks, and a block's walk is latency-bound either way.
 #include "tc_common.cuh"
+#include <algorithm>
 #include <new>
 #include <stdlib.h>
 #include <string.h>
@@ -275,6 +276,88 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
     }
 }
 
+// ---- small batches (the streaming path: a few hundred flows fire per batch) ----------------------------------
+// With so few flows a block of the kernel above walks the whole forest on its own, chunk after chunk, with four
+// warps and nothing to hide the latency behind.  Here the trees are spread over the grid as well: a work item is
+// (tile of 128 flows, slice of trees that fits one buffer); persistent blocks take items in turn, walk the slice
+// and write each tree's leaf index.  A second kernel then adds every flow's leaf vectors in tree order
+// t = 0..T-1 (the same fp32 sums, bit for bit, as the fused kernel) and divides by T.
+template <int NCH>
+__global__ void __launch_bounds__(kBSmall, 2)
+forest_leaf_index_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F, const unsigned char* __restrict__ image,
+                         uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_item, uint32_t buf_bytes,
+                         uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (n_dev) n = min(n, *n_dev);
+    float* xs = reinterpret_cast<float*>(smem_raw + buf_bytes);                                  // [F][128]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + buf_bytes + (size_t)F * kBSmall * 4);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bar + 1);
+    const uint32_t n_tiles = (n + kBSmall - 1) / kBSmall, n_slices = (T + trees_per_item - 1) / trees_per_item;
+    const uint32_t n_items = n_tiles * n_slices;
+    if (blockIdx.x >= n_items) return;
+    const uint32_t cur = smem_u32(smem_raw);
+    const uint32_t xbase = smem_u32(xs) + threadIdx.x * 4u;
+    if (threadIdx.x == 0) { sftc::mbar_init(bar, 1); *abort_flag = 0; sftc::fence_barrier_init(); }
+    __syncthreads();
+    uint32_t it = 0, tile_loaded = 0xFFFFFFFFu;
+    for (uint32_t w = blockIdx.x; w < n_items; w += gridDim.x, it++) {
+        const uint32_t tile = w / n_slices, slice = w - tile * n_slices;
+        const uint32_t t0 = slice * trees_per_item, nt = min(trees_per_item, T - t0);
+        if (threadIdx.x == 0) {
+            sftc::mbar_expect_tx(bar, nt * tree_stride);
+            sftc::bulk_load(smem_raw, image + (size_t)t0 * tree_stride, nt * tree_stride, bar);
+        }
+        const uint32_t f = tile * kBSmall + threadIdx.x;
+        const bool live = f < n;
+        if (tile != tile_loaded) {                          // every thread reads its own column only
+            if (live) for (uint32_t j = 0; j < F; j++) xs[j * kBSmall + threadIdx.x] = __ldg(feat + (size_t)f * F + j);
+            else for (uint32_t j = 0; j < F; j++) xs[j * kBSmall + threadIdx.x] = 0.0f;
+            tile_loaded = tile;
+        }
+        if (!sftc::mbar_wait(bar, it & 1u, abort_flag)) break;
+        uint32_t tt = 0;
+        for (; tt + NCH <= nt; tt += NCH) {
+            uint32_t l[NCH];
+            walk<NCH>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
+            if (live) {
+#pragma unroll
+                for (int k = 0; k < NCH; k++) leaf_idx[(size_t)f * T + t0 + tt + k] = (uint16_t)l[k];
+            }
+        }
+        for (; tt < nt; tt++) {
+            uint32_t l[1];
+            walk<1>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
+            if (live) leaf_idx[(size_t)f * T + t0 + tt] = (uint16_t)l[0];
+        }
+        __syncthreads();                                    // the buffer is refilled by the next item
+    }
+    if (*abort_flag && threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT);
+}
+
+// out[f][c] = (sum over t = 0..T-1, in that order, of leaf[t][idx[f][t]][c]) / T; one thread per (flow, class)
+__global__ void __launch_bounds__(256)
+forest_leaf_sum_kernel(const uint16_t* __restrict__ leaf_idx, const float* __restrict__ leaf, uint32_t n, uint32_t T, uint32_t n_leaf,
+                       uint32_t C, float* __restrict__ out, const uint32_t* __restrict__ n_dev)
+{
+    if (n_dev) n = min(n, *n_dev);
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t f = i / C, c = i - f * C;
+    if (f >= n) return;
+    const uint16_t* idx = leaf_idx + (size_t)f * T;
+    float acc = 0.0f;
+    uint32_t t = 0;
+    for (; t + 8 <= T; t += 8) {                            // eight loads in flight, added in tree order
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; k++) v[k] = __ldg(leaf + ((size_t)(t + k) * n_leaf + idx[t + k]) * C + c);
+#pragma unroll
+        for (int k = 0; k < 8; k++) acc = __fadd_rn(acc, v[k]);
+    }
+    for (; t < T; t++) acc = __fadd_rn(acc, __ldg(leaf + ((size_t)t * n_leaf + idx[t]) * C + c));
+    out[(size_t)f * C + c] = __fdiv_rn(acc, __uint2float_rn(T));
+}
+
 struct Plan { uint32_t chunk_bytes, tpc, nch; size_t smem; };
 
 Plan make_plan(const sf_forest* fo, uint32_t kb = kB) {
@@ -344,11 +427,40 @@ int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, ui
     return launch3<SF_GBDT_MC, C, (C >= 4 ? 4 : (C >= 2 ? 2 : 1))>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
+// small batches of a random forest: leaf indices by (tile, tree slice) work items, then the ordered sums.
+// leaf_idx doubles as the scratch between the two kernels.
+int launch_rf_split(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+    const size_t feat_bytes = (size_t)fo->F * kBSmall * sizeof(float);
+    uint32_t buf = 65536u;
+    uint32_t tpi = buf / fo->tree_stride;
+    if (tpi == 0) return SF_ERR_UNSUPPORTED;
+    if (tpi > 8) tpi = 8;                                  // more items rather than longer ones
+    if (tpi > fo->T) tpi = fo->T;
+    buf = tpi * fo->tree_stride;
+    const size_t smem = buf + feat_bytes + 16;
+    static size_t smem_set_dev[64] = {};
+    size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
+    if (smem > smem_set) {
+        SF_CUDA(cudaFuncSetAttribute(forest_leaf_index_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        smem_set = smem;
+    }
+    const uint32_t n_items = ((n + kBSmall - 1) / kBSmall) * ((fo->T + tpi - 1) / tpi);
+    const uint32_t grid = std::min<uint32_t>(n_items, (uint32_t)fo->ctx->num_sms * 2u);
+    forest_leaf_index_kernel<2><<<grid, kBSmall, smem, st>>>(feat, n, fo->F, fo->d_image_small, fo->T, fo->depth, fo->tree_stride, tpi, buf,
+                                                           leaf_idx, fo->ctx->d_state, n_dev);
+    SF_LAUNCH_CHECK("forest_leaf_index_kernel");
+    const uint64_t threads = (uint64_t)n * fo->C;
+    forest_leaf_sum_kernel<<<(uint32_t)((threads + 255) / 256), 256, 0, st>>>(leaf_idx, fo->d_leaf, n, fo->T, 1u << fo->depth, fo->C, out, n_dev);
+    SF_LAUNCH_CHECK("forest_leaf_sum_kernel");
+    return SF_OK;
+}
+
 }  // namespace
 
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
                      bool small_tiles) {
     if (n == 0) return SF_OK;
+    if (small_tiles && leaf_idx && fo->kind == SF_RF && fo->d_image_small) return launch_rf_split(fo, feat, n, out, leaf_idx, st, n_dev);
     if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st, n_dev);
     if (fo->kind == SF_GBDT_MC) {
         switch (fo->C) {

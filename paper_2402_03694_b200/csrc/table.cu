@@ -525,7 +525,7 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     const size_t o_feat = take((size_t)n * F * 4), o_prob = take((size_t)n * fo->C * 4), o_dec = take(n), o_lab = take(n),
                  o_score = take((size_t)n * 4), o_bc = take((size_t)(n / 1024 + 2) * 4),
                  o_rows = take((size_t)n * slow->dims[0] * esz), o_logits = take((size_t)n * Cs * 4), o_slab_lab = take(n),
-                 o_slow = take(sf_slow_scratch_bytes(slow, n));
+                 o_slow = take(sf_slow_scratch_bytes(slow, n)), o_lidx = take((size_t)n * fo->T * 2);
     int rc = sf_ws_reserve(ctx, off);
     if (rc != SF_OK) return rc;
     sf_ws_reset(ctx);
@@ -568,7 +568,8 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     sf_time_end(ctx, SF_T_EXTRACT, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_FOREST, st);
-    rc = sf_launch_forest(fo, feat, n, prob, nullptr, st, &t->counts[0], true);      // a few thousand flows fire per batch
+    // a few hundred flows fire per batch: trees spread over the grid, leaf indices as scratch, then the ordered sums
+    rc = sf_launch_forest(fo, feat, n, prob, reinterpret_cast<uint16_t*>(w + o_lidx), st, &t->counts[0], true);
     sf_time_end(ctx, SF_T_FOREST, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_SCORE, st);
