@@ -147,7 +147,10 @@ __global__ void key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, ui
     idx[i] = i;
 }
 
-// Stable LSD radix sort, 4-bit digits, tiles of 1024 items (256 threads x 4 consecutive items).
+// Stable LSD radix sort, 4-bit digits, tiles of 1024 items (256 threads x 4 consecutive items), two kernels
+// per pass: per-tile digit counts hist[digit][tile] (<= 1024 entries), then a scatter whose blocks turn the
+// counts into global offsets by scanning them themselves (no separate scan launch), rank their tile's items
+// and move them.
 constexpr uint32_t kTile = 1024;
 __global__ void __launch_bounds__(256)
 radix_hist_kernel(const uint32_t* __restrict__ keys, uint32_t n, uint32_t shift, uint32_t* __restrict__ hist, uint32_t nblk)
@@ -163,34 +166,35 @@ radix_hist_kernel(const uint32_t* __restrict__ keys, uint32_t n, uint32_t shift,
     if (threadIdx.x < 16) hist[threadIdx.x * nblk + blockIdx.x] = c[threadIdx.x];
 }
 
-__global__ void __launch_bounds__(1024)
-radix_scan_kernel(uint32_t* __restrict__ hist, uint32_t entries)        // exclusive scan of <= 1024 entries
-{
-    __shared__ uint32_t tot[32];
-    const uint32_t t = threadIdx.x;
-    const uint32_t v = (t < entries) ? hist[t] : 0u;
-    uint32_t x = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
-    if ((t & 31) == 31) tot[t >> 5] = x;
-    __syncthreads();
-    if (t < 32) {
-        uint32_t w = tot[t], z = w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (t >= (uint32_t)o) z += y; }
-        tot[t] = z - w;
-    }
-    __syncthreads();
-    if (t < entries) hist[t] = tot[t >> 5] + x - v;
-}
-
 __global__ void __launch_bounds__(256)
 radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ iin, uint32_t* __restrict__ kout,
                      uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk)
 {
     __shared__ uint32_t cnt[16 * 256];
     __shared__ uint32_t tot[8];
+    __shared__ uint32_t gofs[16];
     const uint32_t t = threadIdx.x;
+    // exclusive scan of the 16 * nblk counts in (digit, tile) order; thread t owns entries [4t, 4t+4)
+    {
+        const uint32_t entries = 16 * nblk;
+        uint32_t v[4], s0 = 0;
+#pragma unroll
+        for (uint32_t e = 0; e < 4; e++) { v[e] = (4 * t + e < entries) ? hist[4 * t + e] : 0u; s0 += v[e]; }
+        uint32_t x = s0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
+        if ((t & 31) == 31) tot[t >> 5] = x;
+        __syncthreads();
+        uint32_t run = x - s0;
+        for (uint32_t w = 0; w < (t >> 5); w++) run += tot[w];
+#pragma unroll
+        for (uint32_t e = 0; e < 4; e++) {
+            const uint32_t ent = 4 * t + e;                     // = digit * nblk + tile
+            if (ent < entries && ent % nblk == blockIdx.x) gofs[ent / nblk] = run;
+            run += v[e];
+        }
+        __syncthreads();
+    }
     const uint32_t j0 = blockIdx.x * kTile + t * 4;
     uint32_t k[4], dg[4];
     uint32_t h[16];
@@ -232,7 +236,7 @@ radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restric
             uint32_t before = 0;                         // earlier items of this thread with the same digit
 #pragma unroll
             for (uint32_t q = 0; q < 4; q++) if (q < e && dg[q] == d) before++;
-            const uint32_t p = hist[d * nblk + blockIdx.x] + (cnt[d * 256 + t] - cnt[d * 256]) + before;
+            const uint32_t p = gofs[d] + (cnt[d * 256 + t] - cnt[d * 256]) + before;
             kout[p] = k[e];
             iout[p] = iin[j0 + e];
         }
@@ -537,15 +541,14 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     const uint32_t blocks = (n + 255) / 256;
     probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->pkt_slot, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("probe_kernel");
+    const uint32_t nblk = (n + kTile - 1) / kTile;
     key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a);
     SF_LAUNCH_CHECK("key_kernel");
     {
         // 16-bit keys: four 4-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
-        const uint32_t nblk = (n + kTile - 1) / kTile;
         uint32_t* kin = t->key_a; uint32_t* iin = t->idx_a; uint32_t* kout = t->key_b; uint32_t* iout = t->idx_b;
         for (uint32_t pass = 0; pass < 4; pass++) {
             radix_hist_kernel<<<nblk, 256, 0, st>>>(kin, n, pass * 4, t->hist, nblk);
-            radix_scan_kernel<<<1, 1024, 0, st>>>(t->hist, 16 * nblk);
             radix_scatter_kernel<<<nblk, 256, 0, st>>>(kin, iin, kout, iout, n, pass * 4, t->hist, nblk);
             SF_LAUNCH_CHECK("radix pass");
             uint32_t* tk = kin; kin = kout; kout = tk;
