@@ -95,7 +95,7 @@ static inline size_t sf_align256(size_t b) { return (b + 255) & ~(size_t)255; }
 int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st,
                       const uint32_t* n_dev = nullptr);   // n_dev: optional device-side flow count (<= pk->n_flows)
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st,
-                     const uint32_t* n_dev = nullptr, bool small_tiles = false);   // small_tiles: 128 flows per block (few flows per launch)
+                     const uint32_t* n_dev = nullptr, bool small_tiles = false);   // small_tiles + leaf_idx (used as scratch): few flows per launch, trees spread over the grid
 // route scratch: block_counts uint32[ceil(n/1024)+1], decision bytes if the caller gave none
 size_t sf_route_scratch_bytes(uint32_t n);
 int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,

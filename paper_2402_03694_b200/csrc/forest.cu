@@ -21,8 +21,8 @@
 // path instead (a linear texture of 16-byte integer texels over the same table: raw bits, no
 // filtering): it has its own queue into the L1, and the gather then overlaps the walk (115 -> 88
 // cycles per warp and tree in a microbenchmark of exactly this mix).
-// A second instantiation with 128 flows per block serves the streaming path, where a launch
-// carries a few thousand flows: more blocks, and a block's walk is latency-bound either way.
+// The streaming path, where a launch carries a few hundred flows, has kernels of its own further down
+// (trees spread over the grid as well as flows).
 #include "tc_common.cuh"
 #include <algorithm>
 #include <new>
@@ -32,7 +32,7 @@
 namespace {
 
 constexpr uint32_t kB = 512;                       // flows (= threads) per block
-constexpr uint32_t kBSmall = 128;                  // ... of the small-batch variant (streaming: a few thousand flows per launch)
+constexpr uint32_t kBSmall = 128;                  // ... of a tile of the small-batch kernels (streaming: a few hundred flows per launch)
 constexpr uint32_t kMaxSmem = 232448;              // 227 KB
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -391,17 +391,9 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
 }
 
 template <int C>
-int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
-              bool small_tiles) {
+int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     constexpr bool kTexOk = (C % 4) == 0;                 // whole 16-byte texels per leaf vector
     const bool tex = kTexOk && fo->leaf_tex != 0;
-    if (small_tiles && fo->d_image_small) {
-        const Plan ps = make_plan(fo, kBSmall);
-        if (ps.tpc >= 2) {
-            if (tex) return launch3<SF_RF, C, 2, kBSmall, kTexOk>(fo, ps, feat, n, out, leaf_idx, st, n_dev);
-            return launch3<SF_RF, C, 2, kBSmall>(fo, ps, feat, n, out, leaf_idx, st, n_dev);
-        }
-    }
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
     if (p.nch == 2) {
@@ -484,22 +476,22 @@ int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* 
         return SF_ERR_UNSUPPORTED;
     }
     switch (fo->C) {
-    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
-    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev, small_tiles);
+    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev);
     }
     return SF_ERR_UNSUPPORTED;
 }
