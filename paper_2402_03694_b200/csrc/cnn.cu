@@ -29,17 +29,18 @@
 //
 // Persistent CTAs, one per SM, loop over pairs of flows.  Warp roles:
 //   warp 0        streams input rows with bulk copies into a ring
-//   warp 1        issues conv2's MMAs, pair after pair
-//   warp 2        issues conv1's MMAs: those of pair i+2 right behind conv2 of pair i
-//   warps 3..6    E1: conv1 accumulators -> bias + ReLU -> bf16 -> conv2's B operand (shared memory)
-//   warps 7..22   E2: conv2 accumulators -> bias + ReLU -> bf16 -> partial sums over 32 positions
-//   warps 23..26  E3: partial sums -> mean -> linear head -> logits, argmax
-// The tensor pipe queues only two or three instructions, so a thread that issues MMAs must not do
-// anything else for long: with one issuing thread the barrier waits of conv1 left the pipe idle for a
-// third of the time.  Hence two issuing threads: while one sits in its waits the other keeps the queue full.
-// conv2's accumulator (256 TMEM columns) is single: the E2 warps pull it into registers first
-// thing and release it, and conv1 of a later pair keeps the pipe busy meanwhile.  conv1's bias reaches the
-// E1 threads as a kernel parameter (constant bank operands: no loads, no registers).  Every wait is
+//   warp 1        issues conv2's MMAs, pair after pair, into alternating accumulators
+//   warp 2        issues conv1's MMAs, three pairs ahead of the pair whose accumulator the epilogue is emptying
+//   warps 3..18   epilogue: conv2 accumulator of pair k -> registers (and released) -> bias + ReLU -> bf16 -> partial
+//                 sums over 32 positions; then conv1 accumulators of pair k+3 -> bias + ReLU -> bf16 -> conv2's B
+//                 operand (shared memory); warp = (TMEM lane quarter, column group)
+//   warps 19..22  partial sums -> mean -> linear head -> logits, argmax
+// The tensor pipe queues only two or three instructions, so a thread that issues MMAs must not do anything
+// else for long: hence one issuing thread per MMA stream.  TMEM holds exactly two conv2 accumulators (2 x 256
+// columns): conv2 of pair k+1 starts the moment conv2 of pair k ends, while the epilogue empties the other
+// accumulator at leisure.  conv1 has no columns of its own: the accumulators of pair k+3 are written into the
+// buffer the epilogue has just emptied (pair k's), are pulled into registers at once, and conv2 of pair k+2 reuses
+// the buffer after that.  conv1's bias reaches the epilogue as a kernel parameter (constant bank).  Every wait is
 // bounded; on a timeout the block records SF_ERR_DEVICE_TIMEOUT and leaves.
 #include "tc_common.cuh"
 #include <stdlib.h>
@@ -49,9 +50,10 @@ namespace {
 using namespace sftc;
 
 constexpr uint32_t L = 128, CIN = 8, C1 = 64, C2 = 128, KW = 5, NCLS_MAX = 16;
-constexpr uint32_t kE1Warps = 4, kE2Warps = 16, kE3Warps = 4;
-constexpr uint32_t kE1First = 3, kE2First = kE1First + kE1Warps, kE3First = kE2First + kE2Warps;
-constexpr uint32_t kThreads = (kE3First + kE3Warps) * 32;       // 864
+constexpr uint32_t kEWarps = 16, kE3Warps = 4;
+constexpr uint32_t kEFirst = 3, kE3First = kEFirst + kEWarps;
+constexpr uint32_t kThreads = (kE3First + kE3Warps) * 32;       // 736
+constexpr uint32_t NH1 = 3;                                 // conv1 output (= conv2 operand) buffers
 constexpr uint32_t XS = 4;                                  // input-row ring depth
 constexpr uint32_t X_STAGE = (2 + L + 3) * 16;              // 2 zero rows, 128 rows, 3 zero rows (tap 5 is a zero tap)
 constexpr uint32_t H1_COL = 2 * (2 + L + 2) * 16;           // one 8-channel column of a PAIR's conv1 output: 264 rows, 4,224 bytes
@@ -69,8 +71,8 @@ constexpr uint32_t B3_OFF = B2_OFF + C2 * 4;                // fp32 [16]
 constexpr uint32_t BLOB_BYTES = B3_OFF + NCLS_MAX * 4;
 // shared memory map
 constexpr uint32_t SM_BLOB = 0;
-constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // 2 pair buffers
-constexpr uint32_t SM_X = SM_H1 + 2 * H1_BYTES;             // XS stages
+constexpr uint32_t SM_H1 = SM_BLOB + BLOB_BYTES;            // NH1 pair buffers
+constexpr uint32_t SM_X = SM_H1 + NH1 * H1_BYTES;           // XS stages
 constexpr uint32_t PART_BYTES = 4 * 2 * C2 * 4;             // fp32 [4 position groups][2 flows][128 channels]
 constexpr uint32_t SM_PART = SM_X + XS * X_STAGE;           // 2 buffers
 constexpr uint32_t SM_PART2 = SM_PART + 2 * PART_BYTES;     // fp32 [4 warps][32] partial logits
@@ -78,16 +80,17 @@ constexpr uint32_t SM_BARS = SM_PART2 + kE3Warps * 32 * 4;
 constexpr uint32_t SM_TOTAL = SM_BARS + 320;
 static_assert(BLOB_BYTES % 16 == 0 && SM_H1 % 16 == 0 && SM_X % 16 == 0 && SM_PART % 16 == 0 && SM_BARS % 8 == 0, "alignment");
 static_assert(SM_TOTAL <= 232448, "shared memory");
-// TMEM columns: conv1 accumulators [2 flows of a pair][64], conv2 [256]
-constexpr uint32_t TM_D1 = 0, TM_D2 = 256;
+// TMEM columns: two conv2 accumulators of 256 columns; conv1's accumulators of a pair (2 x 64 columns) borrow the
+// first half of the conv2 accumulator that is idle at the time
+constexpr uint32_t TM_D2 = 256;                             // columns per conv2 accumulator
 
 struct Bars {
     uint64_t w_full;
     uint64_t x_full[XS], x_empty[XS];
-    uint64_t d1_full[2], d1_empty[2];          // per flow slot of a pair
-    uint64_t h1_full[2], h1_empty[2];          // per pair buffer
-    uint64_t d2_full, d2_empty;
-    uint64_t c2_issued;                        // conv2 of a pair has been handed to the tensor pipe
+    uint64_t d1_full[2], d1_empty[2];          // conv1 accumulators of pair j: index j & 1
+    uint64_t h1_full[NH1], h1_empty[NH1];      // conv2 operand of pair j: index j % NH1
+    uint64_t d2_full[2], d2_empty[2];          // conv2 accumulator of pair p: index p & 1
+    uint64_t c1_issued;                        // conv1 of a pair has been handed to the tensor pipe
     uint64_t part_full[2], part_empty[2];
     uint32_t tmem_base, abort_flag;
 };
@@ -143,18 +146,18 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
 
     // zero everything that acts as padding (and the rest of the activation buffers: the unused
     // slot of an odd last pair is multiplied like any other and must hold finite numbers)
-    for (uint32_t i = threadIdx.x; i < (2 * H1_BYTES + XS * X_STAGE) / 16; i += kThreads)
+    for (uint32_t i = threadIdx.x; i < (NH1 * H1_BYTES + XS * X_STAGE) / 16; i += kThreads)
         reinterpret_cast<uint4*>(smem + SM_H1)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
         mbar_init(&bars->w_full, 1);
         for (uint32_t s = 0; s < XS; s++) { mbar_init(&bars->x_full[s], 1); mbar_init(&bars->x_empty[s], 1); }
         for (uint32_t b = 0; b < 2; b++) {
-            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kE1Warps);
-            mbar_init(&bars->h1_full[b], kE1Warps); mbar_init(&bars->h1_empty[b], 1);
-            mbar_init(&bars->part_full[b], kE2Warps); mbar_init(&bars->part_empty[b], kE3Warps);
+            mbar_init(&bars->d1_full[b], 1); mbar_init(&bars->d1_empty[b], kEWarps);
+            mbar_init(&bars->d2_full[b], 1); mbar_init(&bars->d2_empty[b], kEWarps);
+            mbar_init(&bars->part_full[b], kEWarps); mbar_init(&bars->part_empty[b], kE3Warps);
         }
-        mbar_init(&bars->d2_full, 1); mbar_init(&bars->d2_empty, kE2Warps);
-        mbar_init(&bars->c2_issued, 1);
+        for (uint32_t b = 0; b < NH1; b++) { mbar_init(&bars->h1_full[b], kEWarps); mbar_init(&bars->h1_empty[b], 1); }
+        mbar_init(&bars->c1_issued, 1);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -186,22 +189,30 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             const uint64_t dH1 = make_smem_desc(sbase + SM_H1, H1_COL, 128, 0);
             const uint64_t dW2 = make_smem_desc(sbase + SM_BLOB + W2_OFF, C2 * 16u, 128, 0);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
-            for (uint32_t i = 0; i < n_pairs && ok; i++) {
-                const uint32_t b = i & 1u;
-                if (!mbar_wait(&bars->h1_full[b], (i >> 1) & 1u, abort_flag)) break;
-                if (!mbar_wait(&bars->d2_empty, (i & 1u) ^ 1u, abort_flag)) break;
+            for (uint32_t p = 0; p < n_pairs && ok; p++) {
+                const uint32_t b = p & 1u, hb = p % NH1;
+                if (!mbar_wait(&bars->h1_full[hb], (p / NH1) & 1u, abort_flag)) break;
+                // the accumulator is free once conv1 of pair p + 1, which borrowed it, sits in registers (that conv1 was
+                // itself issued after conv2 of pair p - 2 had been emptied); without a pair p + 1 wait for pair p - 2 directly
+                if (p + 1 < n_pairs) { if (!mbar_wait(&bars->d1_empty[(p + 1) & 1u], ((p + 1) >> 1) & 1u, abort_flag)) break; }
+                else if (p >= 2) { if (!mbar_wait(&bars->d2_empty[b], ((p - 2) >> 1) & 1u, abort_flag)) break; }
                 tc_fence_after();
-                const uint64_t bh = dH1 + (uint64_t)((b * H1_BYTES) >> 4);
+                const uint64_t bh = dH1 + (uint64_t)((hb * H1_BYTES) >> 4);
 #pragma unroll
                 for (uint32_t t = 0; t < KW; t++) {
+                    // Give way once per pair: this thread refills the pipe's short queue the moment a slot frees, and conv1 of
+                    // pair p + 2 (issued by the other thread as soon as the epilogue has emptied the previous accumulator) would
+                    // otherwise get in only after this pair's last MMA - too late for the next pair.  Only a matter of timing:
+                    // no result depends on this wait.
+                    if (t == 4 && p >= 1 && p + 2 < n_pairs && !mbar_wait(&bars->c1_issued, (p + 2) & 1u, abort_flag)) { ok = false; break; }
 #pragma unroll
                     for (uint32_t k = 0; k < C1 / 16; k++)      // the activations two rows per tap further down
-                        umma_bf16(tmem_base + TM_D2, dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4),
+                        umma_bf16(tmem_base + b * TM_D2, dW2 + ((t * ((C1 / 8) * C2 * 16u) + (2u * k) * (C2 * 16u)) >> 4),
                                   bh + (((2u * k) * H1_COL + t * 32u) >> 4), idesc2, (t | k) != 0 ? 1u : 0u);
                 }
-                mbar_arrive(&bars->c2_issued);                  // conv1 of pair i + 2 may follow in the queue
-                umma_commit(&bars->d2_full);
-                umma_commit(&bars->h1_empty[b]);
+                if (!ok) break;
+                umma_commit(&bars->d2_full[b]);
+                umma_commit(&bars->h1_empty[hb]);
             }
         }
     } else if (warp == 2) {
@@ -211,106 +222,111 @@ cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restr
             const uint64_t dX = make_smem_desc(sbase + SM_X, 16, 128, 0);
             const uint64_t dW1 = make_smem_desc(sbase + SM_BLOB + W1_OFF, C1 * 16u, 128, 0);
             bool ok = mbar_wait(&bars->w_full, 0, abort_flag);
-            for (uint32_t i = 0; i < n_pairs && ok; i++) {
-                const uint32_t n_fl = (2u * i + 1u < n_mine) ? 2u : 1u;
-                // everything this pair's MMAs need is ready long before their turn: check it first ...
+            for (uint32_t j = 0; j < n_pairs && ok; j++) {
+                const uint32_t n_fl = (2u * j + 1u < n_mine) ? 2u : 1u;
                 for (uint32_t s = 0; s < n_fl && ok; s++) {
-                    const uint32_t m = 2u * i + s, xs = m % XS, xph = (m / XS) & 1u;
-                    ok = mbar_wait(&bars->x_full[xs], xph, abort_flag) && mbar_wait(&bars->d1_empty[s], (i & 1u) ^ 1u, abort_flag);
+                    const uint32_t m = 2u * j + s;
+                    ok = mbar_wait(&bars->x_full[m % XS], (m / XS) & 1u, abort_flag);
                 }
-                // ... then take the turn: pairs 0 and 1 go ahead, pair i waits until conv2 of pair i - 2 is in the pipe's
-                // queue, so that these MMAs run while the E2 warps empty conv2's accumulator
-                if (ok && i >= 2) ok = mbar_wait(&bars->c2_issued, i & 1u, abort_flag);
+                // the accumulators go into conv2's buffer (j + 1) & 1: pair j - 2's conv1 results must have left it, and so
+                // must conv2 of pair j - 3
+                if (ok && j >= 2) ok = mbar_wait(&bars->d1_empty[j & 1u], ((j - 2) >> 1) & 1u, abort_flag);
+                if (ok && j >= 3) ok = mbar_wait(&bars->d2_empty[(j + 1) & 1u], ((j - 3) >> 1) & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 for (uint32_t s = 0; s < n_fl; s++) {
-                    const uint32_t xs = (2u * i + s) % XS;
+                    const uint32_t xs = (2u * j + s) % XS;
                     const uint64_t ax = dX + (uint64_t)((xs * X_STAGE) >> 4);
 #pragma unroll
                     for (uint32_t k = 0; k < 3; k++)         // taps (2k, 2k+1): rows shifted by 2k, next tap = next row
-                        umma_bf16(tmem_base + TM_D1 + s * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4), idesc1,
-                                  k != 0 ? 1u : 0u);
-                    umma_commit(&bars->d1_full[s]);
+                        umma_bf16(tmem_base + ((j + 1) & 1u) * TM_D2 + s * C1, ax + ((k * 32u) >> 4), dW1 + ((k * 2u * (C1 * 16u)) >> 4),
+                                  idesc1, k != 0 ? 1u : 0u);
                     umma_commit(&bars->x_empty[xs]);
                 }
-            }
-        }
-    } else if (n_mine > 0 && warp < kE2First) {
-        // ---- E1: conv1 accumulators -> conv2's B operand -------------------------------
-        const uint32_t p = q * 32u + lane;               // position handled by this thread
-        bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
-        for (uint32_t m = 0; m < n_mine && ok; m++) {
-            const uint32_t s = m & 1u, i = m >> 1, b = i & 1u;
-            bool w = mbar_wait_relaxed(&bars->d1_full[s], i & 1u, abort_flag);
-            if (s == 0) w = w && mbar_wait_relaxed(&bars->h1_empty[b], ((i >> 1) & 1u) ^ 1u, abort_flag);
-            ok = __all_sync(0xFFFFFFFFu, w);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D1 + s * C1;
-            uint8_t* hrow = smem + SM_H1 + b * H1_BYTES + (2u * (p + 2u) + s) * 16u;
-            uint32_t v0[32], v1[32];
-            tmem_ld32(taddr, v0);
-            tmem_ld32(taddr + 32, v1);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->d1_empty[s]);      // the accumulator is in registers: conv1 may reuse it
-#pragma unroll
-            for (int j = 0; j < 8; j++) {                // 8 columns of 8 channels
-                uint32_t pk[4];
-#pragma unroll
-                for (int e = 0; e < 4; e++) {
-                    const int c = (j & 3) * 8 + e * 2;
-                    const uint32_t a = (j < 4) ? v0[c] : v1[c], bq = (j < 4) ? v0[c + 1] : v1[c + 1];
-                    pk[e] = pack_relu_bf16(a, bq, b1.v[j * 8 + e * 2], b1.v[j * 8 + e * 2 + 1]);
-                }
-                *reinterpret_cast<uint4*>(hrow + j * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-            if (s == 1u || m + 1 == n_mine) {            // the pair is complete
-                fence_proxy_async();                     // activations -> visible to the MMA's shared-memory reads
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->h1_full[b]);
+                umma_commit(&bars->d1_full[j & 1u]);
+                mbar_arrive(&bars->c1_issued);
             }
         }
     } else if (n_mine > 0 && warp < kE3First) {
-        // ---- E2: conv2 accumulators [channel][position, flow] -> sums over 32 positions ----
-        const uint32_t g = (warp - kE2First) >> 2;        // positions 32g .. 32g+31 = columns 64g .. 64g+63
-        const uint32_t ch = q * 32u + lane;
+        // ---- epilogue warps: (TMEM lane quarter q, column group cg) ----
+        const uint32_t cg = (warp - kEFirst) >> 2;
         bool ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->w_full, 0, abort_flag));
-        const float bias = ok ? reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF)[ch] : 0.0f;
-        for (uint32_t i = 0; i < n_pairs && ok; i++) {
-            const uint32_t b = i & 1u;
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->d2_full, i & 1u, abort_flag));     // on the critical path: poll without backing off
-            if (!ok) break;
+        const float bias2 = ok ? reinterpret_cast<const float*>(smem + SM_BLOB + B2_OFF)[q * 32u + lane] : 0.0f;
+
+        // conv1 accumulators of pair j [position = lane][channels 16cg .. 16cg+15] of both flows -> conv2's B operand
+        auto conv1_out = [&](uint32_t j) -> bool {
+            const uint32_t hb = j % NH1, n_fl = (2u * j + 1u < n_mine) ? 2u : 1u;
+            bool w = mbar_wait_relaxed(&bars->d1_full[j & 1u], (j >> 1) & 1u, abort_flag) &&
+                     mbar_wait_relaxed(&bars->h1_empty[hb], ((j / NH1) & 1u) ^ 1u, abort_flag);
+            if (!__all_sync(0xFFFFFFFFu, w)) return false;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + TM_D2 + g * 64u;
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + ((j + 1) & 1u) * TM_D2 + cg * 16u;
+            uint32_t v[2][16];
+            tmem_ld16(taddr, v[0]);
+            if (n_fl > 1) tmem_ld16(taddr + C1, v[1]);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->d1_empty[j & 1u]);     // the accumulators are in registers: the buffer is conv2's again
+            const uint32_t p = q * 32u + lane;                       // position
+#pragma unroll
+            for (int s = 0; s < 2; s++) {
+                if ((uint32_t)s < n_fl) {
+                    uint8_t* hrow = smem + SM_H1 + hb * H1_BYTES + (2u * cg) * H1_COL + (2u * (p + 2u) + s) * 16u;
+#pragma unroll
+                    for (int h = 0; h < 2; h++) {                    // two columns of 8 channels
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; e++)
+                            pk[e] = pack_relu_bf16(v[s][h * 8 + e * 2], v[s][h * 8 + e * 2 + 1], b1.v[cg * 16u + h * 8 + e * 2],
+                                                   b1.v[cg * 16u + h * 8 + e * 2 + 1]);
+                        *reinterpret_cast<uint4*>(hrow + h * H1_COL) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+            }
+            fence_proxy_async();                                 // activations -> visible to the MMA's shared-memory reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->h1_full[hb]);
+            return true;
+        };
+        // conv2 accumulator of pair k [channel = lane][positions 32cg .. 32cg+31 of both flows] -> sums over those positions
+        auto conv2_out = [&](uint32_t k) -> bool {
+            const uint32_t b = k & 1u;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&bars->d2_full[b], (k >> 1) & 1u, abort_flag))) return false;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + b * TM_D2 + cg * 64u;
             uint32_t v0[32], v1[32];
             tmem_ld32(taddr, v0);
             tmem_ld32(taddr + 32, v1);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->d2_empty);         // the accumulator is in registers: conv2 may reuse it
+            if (lane == 0) mbar_arrive(&bars->d2_empty[b]);          // the accumulator is in registers: conv1 of pair k + 3 may borrow it
             float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-            for (int j = 0; j < 16; j++) {                // columns 2j, 2j+1 = position 32g+j of flows 0, 1
-                const uint32_t h = relu_bf16x2(__uint_as_float(v0[2 * j + 1]) + bias, __uint_as_float(v0[2 * j]) + bias);
+            for (int j = 0; j < 16; j++) {                // columns 2j, 2j+1 = position 32cg+j of flows 0, 1
+                const uint32_t h = relu_bf16x2(__uint_as_float(v0[2 * j + 1]) + bias2, __uint_as_float(v0[2 * j]) + bias2);
                 s0 += __uint_as_float(h << 16);
                 s1 += __uint_as_float(h & 0xFFFF0000u);
             }
 #pragma unroll
             for (int j = 0; j < 16; j++) {
-                const uint32_t h = relu_bf16x2(__uint_as_float(v1[2 * j + 1]) + bias, __uint_as_float(v1[2 * j]) + bias);
+                const uint32_t h = relu_bf16x2(__uint_as_float(v1[2 * j + 1]) + bias2, __uint_as_float(v1[2 * j]) + bias2);
                 s0 += __uint_as_float(h << 16);
                 s1 += __uint_as_float(h & 0xFFFF0000u);
             }
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->part_empty[b], ((i >> 1) & 1u) ^ 1u, abort_flag));
-            if (!ok) break;
-            float* part = reinterpret_cast<float*>(smem + SM_PART + b * PART_BYTES) + g * 2u * C2;
-            part[ch] = s0;
-            part[C2 + ch] = s1;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_relaxed(&bars->part_empty[b], ((k >> 1) & 1u) ^ 1u, abort_flag))) return false;
+            float* part = reinterpret_cast<float*>(smem + SM_PART + b * PART_BYTES) + cg * 2u * C2;
+            part[q * 32u + lane] = s0;
+            part[C2 + q * 32u + lane] = s1;
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->part_full[b]);
+            return true;
+        };
+        for (uint32_t j = 0; j < 3 && j < n_pairs && ok; j++) ok = conv1_out(j);
+        for (uint32_t k = 0; k < n_pairs && ok; k++) {
+            ok = conv2_out(k);
+            if (ok && k + 3 < n_pairs) ok = conv1_out(k + 3);
         }
     } else if (n_mine > 0) {
         // ---- E3: partial sums -> mean -> linear head -> logits, argmax -----------------
