@@ -51,7 +51,7 @@ struct sf_forest {
     // per-tree image of tree_stride bytes: 2^depth node entries of 8 bytes {thr bits, byte offset of the
     // feature's row in the kernel's shared-memory tile}, 1-based heap (entry 0 unused), then (GBDT) 2^depth leaf scalars
     unsigned char* d_image;
-    unsigned char* d_image_small;      // same trees with feature offsets for the 128-flow tile (random forests only)
+    unsigned char* d_image_small;      // same trees with feature offsets for the 128-flow tile of the small-batch kernels (random forests only)
     uint32_t tree_stride;
     // leaves: RF fp32[T][2^d][C]; GBDT fp32[T][2^d]
     float* d_leaf;
