@@ -407,12 +407,19 @@ def main():
                                                (4 * (cfg.C if cfg.kind == "rf" else 1) * 32) / 128.0) / 1e9,
                    "Gwavefront/s", SM_COUNT * SM_MAX_MHZ * 1e6 / 1e9),
     }
+    Cf = cfg.C if cfg.kind == "rf" else 1
+    # the two small HBM-bound classes: score + scan + scatter (fast-model output in; decision, label, ids out) and the
+    # MLP's last layer (reads the last hidden activations once)
+    alg["score"] = ("hbm", (n * (4 * Cf + 2) + 4 * k_esc) / 1e9, "GB/s", peaks["hbm_gbs"])
+    if cfg.slow == "mlp" and avg.get("head", 0.0) > 0:
+        alg["head"] = ("hbm", k_esc * (cfg.dims[-2] * esz + 4 * cfg.dims[-1]) / 1e9, "GB/s", peaks["hbm_gbs"])
     roof_all = {}
     for k, (bound, work, unit, peak) in alg.items():
         ach = work / (avg[k] * 1e-3) if avg[k] > 0 else 0.0
         roof_all[k] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "ms": avg[k]}
     dom = max(alg, key=lambda k: avg[k])
-    src = {"gemm": "gemm_tc.cu", "forest": "forest.cu", "extract": "extract.cu", "gather": "route.cu"}[dom]
+    src = {"gemm": "gemm_tc.cu", "forest": "forest.cu", "extract": "extract.cu", "gather": "route.cu", "score": "route.cu",
+           "head": "gemm_tc.cu"}[dom]
     traffic = TRAFFIC_BY_SOURCE.get((dom, cfg.c, src_hash(src)))
     if traffic is not None:
         traffic = traffic["bytes_per_row_per_launch"] * k_esc      # scaled by rows: traffic grows in proportion
