@@ -95,14 +95,22 @@ __device__ __forceinline__ void load_leaf_vec(const float* __restrict__ lv, floa
     }
 }
 
-// the same vector through the texture path: C / 4 texels of 16 bytes, starting at texel index `texel`
+// the same vector through the texture path: C / 4 texels of 16 bytes, starting at texel index `texel`.
+// A vector of 16 classes (four texels per lane) would make the texture queue the bottleneck in its turn, so from
+// C = 16 on the second half of the vector comes through the load/store pipe (one 256-bit load): both paths share the work.
 template <int C>
-__device__ __forceinline__ void load_leaf_vec_tex(cudaTextureObject_t tex, uint32_t texel, float (&p)[C]) {
+__device__ __forceinline__ void load_leaf_vec_tex(cudaTextureObject_t tex, uint32_t texel, const float* __restrict__ lv, float (&p)[C]) {
+    constexpr int CT = (C >= 16 && (C % 16) == 0) ? C / 2 : C;       // classes fetched as texels
 #pragma unroll
-    for (int c = 0; c < C; c += 4) {
+    for (int c = 0; c < CT; c += 4) {
         const uint4 v = tex1Dfetch<uint4>(tex, (int)(texel + c / 4));
         p[c] = __uint_as_float(v.x); p[c + 1] = __uint_as_float(v.y); p[c + 2] = __uint_as_float(v.z); p[c + 3] = __uint_as_float(v.w);
     }
+#pragma unroll
+    for (int c = CT; c < C; c += 8)
+        asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                     : "=f"(p[c]), "=f"(p[c + 1]), "=f"(p[c + 2]), "=f"(p[c + 3]), "=f"(p[c + 4]), "=f"(p[c + 5]), "=f"(p[c + 6]), "=f"(p[c + 7])
+                     : "l"(lv + c));
 }
 
 // KIND: SF_RF (leaf = C-vector of class probabilities in global memory), SF_GBDT (leaf =
@@ -239,7 +247,7 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
                 flush_pending();                      // the previous group's vectors have landed by now
 #pragma unroll
                 for (int k = 0; k < NCH; k++) {
-                    if (TEX) load_leaf_vec_tex<C>(leaf_tex, ((t0 + tt + k) * n_leaf + l[k]) * (C / 4), pend[k]);
+                    if (TEX) load_leaf_vec_tex<C>(leaf_tex, ((t0 + tt + k) * n_leaf + l[k]) * (C / 4), leaf + ((size_t)(t0 + tt + k) * n_leaf + l[k]) * C, pend[k]);
                     else load_leaf_vec<C>(leaf + ((size_t)(t0 + tt + k) * n_leaf + l[k]) * C, pend[k]);
                 }
                 n_pend = NCH;
@@ -253,7 +261,7 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
                 acc[0] = __fadd_rn(acc[0], lds32f(cur + tt * tree_stride + n_leaf * 8u + l[0] * 4u));
             } else {
                 flush_pending();
-                if (TEX) load_leaf_vec_tex<C>(leaf_tex, ((t0 + tt) * n_leaf + l[0]) * (C / 4), pend[0]);
+                if (TEX) load_leaf_vec_tex<C>(leaf_tex, ((t0 + tt) * n_leaf + l[0]) * (C / 4), leaf + ((size_t)(t0 + tt) * n_leaf + l[0]) * C, pend[0]);
                 else load_leaf_vec<C>(leaf + ((size_t)(t0 + tt) * n_leaf + l[0]) * C, pend[0]);
                 n_pend = 1;
             }
