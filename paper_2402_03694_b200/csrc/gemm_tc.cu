@@ -73,6 +73,91 @@ struct GemmBars {
     uint32_t abort_flag;
 };
 
+// ---- a handful of rows (the streaming path: about ten flows reach the slow model per batch) --------------------
+// A 128-row tensor-core tile would be almost empty and its K loop (K/16 dependent MMAs on one SM) takes 8 us per layer
+// whatever the row count.  Up to kSmallRows rows are served by the same kernel on CUDA cores instead (the row count is
+// only known on the device, so the choice is made there, at the top of the kernel): a warp per output column, lanes
+// over K (8 consecutive inputs each per step), the rows' activations staged in shared memory, fp32 accumulation, a
+// fixed shuffle tree over the lanes (deterministic), then bias (+ ReLU + bf16, or the logits and the argmax).
+constexpr uint32_t kSmallRows = 16;
+constexpr uint32_t kSmallMaxK = 4096;                // 16 rows x K bf16 must fit in the kernel's tile ring (>= 180 KB)
+
+__device__ __forceinline__ float warp_rows_reduce16(float (&v)[16], uint32_t lane) {
+#pragma unroll
+    for (int j = 0; j < 16; j++) v[j] += __shfl_xor_sync(0xFFFFFFFFu, v[j], 16);
+#pragma unroll
+    for (int off = 8; off >= 1; off >>= 1) {
+        const bool up = (lane & off) != 0;
+#pragma unroll
+        for (int j = 0; j < off; j++) {
+            const float keep = up ? v[j + off] : v[j];
+            const float send = up ? v[j] : v[j + off];
+            v[j] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
+        }
+    }
+    return v[0];                                     // lanes l and l + 16: total of row l & 15
+}
+
+// HEAD = false: out[r][n] = bf16(ReLU(sum + bias[n])), columns spread over all warps of the grid.
+// HEAD = true (block 0 only, W padded to 16 rows): logits[r][c] = sum + bias[c] for c < C, label[r] = argmax (lowest index on ties).
+template <bool HEAD>
+__device__ void small_rows_layer(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias,
+                                 uint32_t rows, uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out,
+                                 float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C, uint8_t* smem)
+{
+    __shared__ float lg[kSmallRows][16];
+    if (HEAD && blockIdx.x != 0) return;
+    uint4* As = reinterpret_cast<uint4*>(smem);                           // [16 rows][K] bf16, rows past the count zero
+    const uint32_t k16 = K / 8;                                           // 16-byte chunks per row
+    for (uint32_t i = threadIdx.x; i < kSmallRows * k16; i += blockDim.x) {
+        const uint32_t r = i / k16, c = i - r * k16;
+        As[i] = (r < rows) ? __ldg(reinterpret_cast<const uint4*>(A + (size_t)r * K) + c) : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    const uint32_t n_cols = HEAD ? 16u : N;
+    const uint32_t w0 = HEAD ? warp : blockIdx.x * wpb + warp, wstep = HEAD ? wpb : gridDim.x * wpb;
+    for (uint32_t n = w0; n < n_cols; n += wstep) {
+        float acc[kSmallRows];
+#pragma unroll
+        for (int r = 0; r < (int)kSmallRows; r++) acc[r] = 0.0f;
+        const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)n * K);
+        for (uint32_t c = lane; c < k16; c += 32) {
+            const uint4 wv = __ldg(wrow + c);
+            const uint32_t wq[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+            for (int r = 0; r < (int)kSmallRows; r++) {
+                const uint4 av = As[r * k16 + c];
+                const uint32_t aq[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    acc[r] = fmaf(__uint_as_float(aq[e] << 16), __uint_as_float(wq[e] << 16), acc[r]);
+                    acc[r] = fmaf(__uint_as_float(aq[e] & 0xFFFF0000u), __uint_as_float(wq[e] & 0xFFFF0000u), acc[r]);
+                }
+            }
+        }
+        const float tot = warp_rows_reduce16(acc, lane);
+        const uint32_t r = lane & 15u;
+        if (!HEAD) {
+            if (lane < 16 && r < rows) out[(size_t)r * N + n] = __float2bfloat16_rn(fmaxf(tot + bias[n], 0.0f));
+        } else if (lane < 16) {
+            lg[r][n] = (n < C) ? tot + bias[n] : -3.0e38f;
+        }
+    }
+    if (HEAD) {
+        __syncthreads();
+        if (threadIdx.x < rows) {
+            float best = lg[threadIdx.x][0]; uint32_t arg = 0;
+            for (uint32_t c = 0; c < C; c++) {
+                const float v = lg[threadIdx.x][c];
+                logits[(size_t)threadIdx.x * C + c] = v;
+                if (v > best) { best = v; arg = c; }
+            }
+            if (label) label[threadIdx.x] = (uint8_t)arg;
+        }
+    }
+}
+
 // HEAD = false: hidden layer, out = bf16(ReLU(acc + bias)) [rows][N].
 // HEAD = true (BN = 16): last layer, W zero-padded to 16 rows; logits[r][c] = acc + bias for
 // c < C (fp32, no activation) and label[r] = argmax (lowest index on ties).
@@ -81,10 +166,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                            const float* __restrict__ bias, const uint32_t* __restrict__ n_rows_dev,
                            uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out, sf_dev_state* st,
-                           float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C)
+                           float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C, uint32_t small_max,
+                           const __nv_bfloat16* __restrict__ A_raw, const __nv_bfloat16* __restrict__ W_raw)
 {
     using Cfg = GemmCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
+    if (*n_rows_dev <= small_max) {                  // a handful of rows (small_max = 0: never): CUDA cores, same launch
+        if (*n_rows_dev) small_rows_layer<HEAD>(A_raw, W_raw, bias, *n_rows_dev, N, K, out, logits, label, C, smem_raw);
+        return;
+    }
     const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* tiles = smem_raw + (base_u32 - smem_u32(smem_raw));
     GemmBars* bars = reinterpret_cast<GemmBars*>(tiles + Cfg::kStages * Cfg::kStageBytes);
@@ -248,7 +338,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 
 template <uint32_t BN>
 int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, const uint32_t* n_rows_dev,
-                uint32_t capacity, uint32_t N, uint32_t K, void* out, cudaStream_t st)
+                uint32_t capacity, uint32_t N, uint32_t K, void* out, cudaStream_t st, uint32_t small_max)
 {
     using Cfg = GemmCfg<BN>;
     CUtensorMap tmA, tmW;
@@ -263,14 +353,15 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     uint32_t max_tiles = ((capacity + BM - 1) / BM) * (N / BN);
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
-                                                  reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state, nullptr, nullptr, 0);
+                                                  reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state, nullptr, nullptr, 0, small_max,
+                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W));
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel");
     return SF_OK;
 }
 
 // last layer on the tensor cores: one 128 x 16 tile per 128 rows, W padded to 16 rows
 int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bias, const uint32_t* n_rows_dev,
-                   uint32_t capacity, uint32_t K, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
+                   uint32_t capacity, uint32_t K, uint32_t C, float* logits, uint8_t* label, cudaStream_t st, uint32_t small_max)
 {
     using Cfg = GemmCfg<16>;
     CUtensorMap tmA, tmW;
@@ -284,10 +375,12 @@ int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bia
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
     uint32_t max_tiles = (capacity + BM - 1) / BM;
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
-    k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C);
+    k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C, small_max,
+                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16));
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(head)");
     return SF_OK;
 }
+
 
 }  // namespace
 
@@ -298,22 +391,26 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     for (uint32_t l = 1; l < s->n_layers; l++) if (s->dims[l] > maxh) maxh = s->dims[l];
     char* h0 = reinterpret_cast<char*>(scratch);
     char* h1 = h0 + sf_align256((size_t)capacity * maxh * 2);
+    // batches that may hold only a handful of rows (the streaming path) may take the CUDA-core path inside the same kernels
+    bool small = capacity <= 65536;
+    for (uint32_t l = 0; l < s->n_layers; l++) if (s->dims[l] > kSmallMaxK || (s->dims[l] % 8) != 0) small = false;
+    const uint32_t small_max = small ? kSmallRows : 0u;
     const void* in = rows;
     sf_time_begin(ctx, SF_T_GEMM, st);
     for (uint32_t l = 0; l + 1 < s->n_layers; l++) {
         void* out = (l & 1) ? h1 : h0;
         const uint32_t K = s->dims[l], N = s->dims[l + 1];
         int rc;
-        if (N % 256 == 0)      rc = launch_gemm<256>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st);
-        else if (N % 128 == 0) rc = launch_gemm<128>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st);
-        else                   rc = launch_gemm<64>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st);
+        if (N % 256 == 0)      rc = launch_gemm<256>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
+        else if (N % 128 == 0) rc = launch_gemm<128>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
+        else                   rc = launch_gemm<64>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
         if (rc != SF_OK) return rc;
         in = out;
     }
     sf_time_end(ctx, SF_T_GEMM, st);
     const uint32_t L = s->n_layers - 1;
     sf_time_begin(ctx, SF_T_HEAD, st);
-    int rc = launch_head_tc(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st);
+    int rc = launch_head_tc(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st, small_max);
     sf_time_end(ctx, SF_T_HEAD, st);
     return rc;
 }
