@@ -136,43 +136,43 @@ __global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ 
 }
 
 // Sort key of a packet = arrival index of its flow's first packet in this batch: 16 bits,
-// unique per flow; a packet that found no slot is a run of its own.
-__global__ void key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
-                           uint32_t* __restrict__ key, uint32_t* __restrict__ idx)
-{
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    const uint32_t slot = pkt_slot[i];
-    key[i] = (slot < t.n_slots) ? t.first[slot] : i;
-    idx[i] = i;
-}
-
-// Stable LSD radix sort, 4-bit digits, tiles of 1024 items (256 threads x 4 consecutive items), two kernels
-// per pass: per-tile digit counts hist[digit][tile] (<= 1024 entries), then a scatter whose blocks turn the
-// counts into global offsets by scanning them themselves (no separate scan launch), rank their tile's items
-// and move them.
+// unique per flow; a packet that found no slot is a run of its own.  The block also counts its keys' first radix
+// digit (shared-memory counters, then one add per digit into hist0[digit][tile]; the caller zeroed hist0).
 constexpr uint32_t kTile = 1024;
 __global__ void __launch_bounds__(256)
-radix_hist_kernel(const uint32_t* __restrict__ keys, uint32_t n, uint32_t shift, uint32_t* __restrict__ hist, uint32_t nblk)
+key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
+           uint32_t* __restrict__ key, uint32_t* __restrict__ idx, uint32_t* __restrict__ hist0, uint32_t nblk)
 {
     __shared__ uint32_t c[16];
     if (threadIdx.x < 16) c[threadIdx.x] = 0;
     __syncthreads();
-    const uint32_t j0 = blockIdx.x * kTile + threadIdx.x * 4;
-#pragma unroll
-    for (uint32_t e = 0; e < 4; e++)
-        if (j0 + e < n) atomicAdd(&c[(keys[j0 + e] >> shift) & 15u], 1u);
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        const uint32_t slot = pkt_slot[i];
+        const uint32_t k = (slot < t.n_slots) ? t.first[slot] : i;
+        key[i] = k;
+        idx[i] = i;
+        atomicAdd(&c[k & 15u], 1u);
+    }
     __syncthreads();
-    if (threadIdx.x < 16) hist[threadIdx.x * nblk + blockIdx.x] = c[threadIdx.x];
+    if (threadIdx.x < 16 && c[threadIdx.x]) atomicAdd(&hist0[threadIdx.x * nblk + (blockIdx.x * 256u) / kTile], c[threadIdx.x]);
 }
 
+// Stable LSD radix sort, 4-bit digits, tiles of 1024 items (256 threads x 4 consecutive items), one kernel per pass:
+// a block turns the pass's per-tile digit counts hist[digit][tile] (<= 1024 entries) into global offsets by scanning
+// them itself, ranks its tile's items and moves them; while doing so it counts the NEXT pass's digit of every item under
+// the tile the item lands in (shared-memory counters first, then one add per non-zero counter into next_hist, which the
+// caller zeroed), so no pass needs a counting kernel of its own.
 __global__ void __launch_bounds__(256)
 radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ iin, uint32_t* __restrict__ kout,
-                     uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk)
+                     uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk,
+                     uint32_t* __restrict__ next_hist)
 {
     __shared__ uint32_t cnt[16 * 256];
     __shared__ uint32_t tot[8];
     __shared__ uint32_t gofs[16];
+    __shared__ uint32_t nh[16 * 64];                     // next pass: [digit][output tile] (a batch has at most 64 tiles)
+    if (next_hist) for (uint32_t i = threadIdx.x; i < 16 * 64; i += 256) nh[i] = 0;
     const uint32_t t = threadIdx.x;
     // exclusive scan of the 16 * nblk counts in (digit, tile) order; thread t owns entries [4t, 4t+4)
     {
@@ -239,6 +239,14 @@ radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restric
             const uint32_t p = gofs[d] + (cnt[d * 256 + t] - cnt[d * 256]) + before;
             kout[p] = k[e];
             iout[p] = iin[j0 + e];
+            if (next_hist) atomicAdd(&nh[((k[e] >> (shift + 4)) & 15u) * 64u + p / kTile], 1u);
+        }
+    }
+    if (next_hist) {
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < 16 * 64; i += 256) {
+            const uint32_t v = nh[i];
+            if (v) atomicAdd(&next_hist[(i >> 6) * nblk + (i & 63u)], v);
         }
     }
 }
@@ -488,8 +496,9 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     t->rank = carve<uint32_t>(p, kMaxBatch); t->pos = carve<uint32_t>(p, kMaxBatch);
     t->fire1_slot = carve<uint32_t>(p, kMaxBatch); t->fire2_slab = carve<uint32_t>(p, kMaxBatch);
     t->fire2_slot = carve<uint32_t>(p, kMaxBatch);
-    t->counts = carve<uint32_t>(p, 16);
-    t->pkt_slot = carve<uint32_t>(p, kMaxBatch); t->hist = carve<uint32_t>(p, 1024);
+    t->counts = carve<uint32_t>(p, 16 + 4 * 1024);           // counters, then the four passes' digit counts (cleared together)
+    t->hist = t->counts + 16;
+    t->pkt_slot = carve<uint32_t>(p, kMaxBatch);
     d.first = carve<uint32_t>(p, S);
     e = cudaMemset(d.first, 0xFF, S * 4);
     if (e != cudaSuccess) { cudaFree(t->all); delete t; return sf_set_cuda_error(e, "cudaMemset(table)"); }
@@ -537,19 +546,19 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     if (!w) return SF_ERR_ALLOC;
     sf_time_new_record(ctx);
     sf_time_begin(ctx, SF_T_TABLE, st);
-    SF_CUDA(cudaMemsetAsync(t->counts, 0, 64, st));
+    SF_CUDA(cudaMemsetAsync(t->counts, 0, (16 + 4 * 1024) * sizeof(uint32_t), st));
     const uint32_t blocks = (n + 255) / 256;
     probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->pkt_slot, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("probe_kernel");
     const uint32_t nblk = (n + kTile - 1) / kTile;
-    key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a);
+    key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a, t->hist, nblk);
     SF_LAUNCH_CHECK("key_kernel");
     {
         // 16-bit keys: four 4-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
         uint32_t* kin = t->key_a; uint32_t* iin = t->idx_a; uint32_t* kout = t->key_b; uint32_t* iout = t->idx_b;
         for (uint32_t pass = 0; pass < 4; pass++) {
-            radix_hist_kernel<<<nblk, 256, 0, st>>>(kin, n, pass * 4, t->hist, nblk);
-            radix_scatter_kernel<<<nblk, 256, 0, st>>>(kin, iin, kout, iout, n, pass * 4, t->hist, nblk);
+            radix_scatter_kernel<<<nblk, 256, 0, st>>>(kin, iin, kout, iout, n, pass * 4, t->hist + pass * 1024, nblk,
+                                                       pass < 3 ? t->hist + (pass + 1) * 1024 : nullptr);
             SF_LAUNCH_CHECK("radix pass");
             uint32_t* tk = kin; kin = kout; kout = tk;
             uint32_t* ti = iin; iin = iout; iout = ti;
