@@ -109,7 +109,7 @@ int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wid
                      const uint32_t* n_ids_dev, uint32_t capacity, void* rows, cudaStream_t st);
 size_t sf_slow_scratch_bytes(const sf_slow* s, uint32_t capacity);
 int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
-                   float* logits, uint8_t* label, void* scratch, cudaStream_t st);
+                   float* logits, uint8_t* label, void* scratch, cudaStream_t st, bool count_done = true);
 int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t n, const uint32_t* esc_ids,
                     const uint32_t* n_esc, uint32_t capacity, const uint8_t* label_slow,
                     uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value = 2, bool write_fast = true);
@@ -117,6 +117,10 @@ int sf_launch_gather_feat(const float* feat, const uint32_t* ids, const uint32_t
                           float* out, cudaStream_t st);
 int sf_launch_compose_ids(const uint32_t* ids1, const uint32_t* ids2_local, const uint32_t* n_dev, uint32_t n_max,
                           uint32_t* out, cudaStream_t st);
+
+// small batches of a random forest in two steps (forest.cu): leaf indices only; the caller adds the leaf vectors itself
+int sf_launch_forest_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st,
+                                const uint32_t* n_dev);
 
 // bf16 tensor-core layers (gemm_tc.cu)
 int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,

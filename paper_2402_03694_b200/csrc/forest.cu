@@ -427,9 +427,7 @@ int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, ui
     return launch3<SF_GBDT_MC, C, (C >= 4 ? 4 : (C >= 2 ? 2 : 1))>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
-// small batches of a random forest: leaf indices by (tile, tree slice) work items, then the ordered sums.
-// leaf_idx doubles as the scratch between the two kernels.
-int launch_rf_split(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int launch_rf_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
     const size_t feat_bytes = (size_t)fo->F * kBSmall * sizeof(float);
     uint32_t buf = 65536u;
     uint32_t tpi = buf / fo->tree_stride;
@@ -449,6 +447,14 @@ int launch_rf_split(const sf_forest* fo, const float* feat, uint32_t n, float* o
     forest_leaf_index_kernel<2><<<grid, kBSmall, smem, st>>>(feat, n, fo->F, fo->d_image_small, fo->T, fo->depth, fo->tree_stride, tpi, buf,
                                                            leaf_idx, fo->ctx->d_state, n_dev);
     SF_LAUNCH_CHECK("forest_leaf_index_kernel");
+    return SF_OK;
+}
+
+// small batches of a random forest: leaf indices by (tile, tree slice) work items, then the ordered sums.
+// leaf_idx doubles as the scratch between the two kernels.
+int launch_rf_split(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+    int rc = launch_rf_leaf_index(fo, feat, n, leaf_idx, st, n_dev);
+    if (rc != SF_OK) return rc;
     const uint64_t threads = (uint64_t)n * fo->C;
     forest_leaf_sum_kernel<<<(uint32_t)((threads + 255) / 256), 256, 0, st>>>(leaf_idx, fo->d_leaf, n, fo->T, 1u << fo->depth, fo->C, out, n_dev);
     SF_LAUNCH_CHECK("forest_leaf_sum_kernel");
@@ -456,6 +462,13 @@ int launch_rf_split(const sf_forest* fo, const float* feat, uint32_t n, float* o
 }
 
 }  // namespace
+
+int sf_launch_forest_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st,
+                                const uint32_t* n_dev) {
+    if (n == 0) return SF_OK;
+    if (fo->kind != SF_RF || !fo->d_image_small || !leaf_idx) return SF_ERR_UNSUPPORTED;
+    return launch_rf_leaf_index(fo, feat, n, leaf_idx, st, n_dev);
+}
 
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
                      bool small_tiles) {

@@ -101,7 +101,7 @@ size_t sf_slow_scratch_bytes(const sf_slow* s, uint32_t capacity) {
 }
 
 int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
-                   float* logits, uint8_t* label, void* scratch, cudaStream_t st)
+                   float* logits, uint8_t* label, void* scratch, cudaStream_t st, bool count_done)
 {
     if (capacity == 0) return SF_OK;
     int rc;
@@ -135,8 +135,10 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
         rc = SF_OK;
     }
     if (rc != SF_OK) return rc;
-    count_slow_kernel<<<1, 1, 0, st>>>(n_rows_dev, ctx->d_state);
-    SF_LAUNCH_CHECK("count_slow_kernel");
+    if (count_done) {                                  // the streaming path adds the count in its own last kernel
+        count_slow_kernel<<<1, 1, 0, st>>>(n_rows_dev, ctx->d_state);
+        SF_LAUNCH_CHECK("count_slow_kernel");
+    }
     return SF_OK;
 }
 

@@ -306,17 +306,50 @@ __global__ void gather_fast_kernel(TableDev t, const uint32_t* __restrict__ fire
     if (p == 0) c_dir[k] = t.f_dir[slot];
 }
 
-__global__ void apply_route_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const uint32_t* __restrict__ counts,
-                                   const uint8_t* __restrict__ decision, const uint8_t* __restrict__ label,
-                                   const float* __restrict__ score, sf_batch_result* res, sf_dev_state* st)
+// Finishes the fast model for the flows that fired in this batch and applies the assignment, one kernel instead of
+// three (leaf sums, score, application): 16 lanes per flow, lane c < C adds class c's leaf values in tree order
+// t = 0..T-1 and divides by T (the random forest's soft vote, same operations and order as the batch kernels), the group
+// finds the largest probability (lowest class on ties), and its first lane takes the least-confidence decision
+// u = 1 - max > tau[label] and updates the table.
+__global__ void __launch_bounds__(256)
+fast_finish_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const uint32_t* __restrict__ counts,
+                   const uint16_t* __restrict__ leaf_idx, const float* __restrict__ leaf, uint32_t T, uint32_t n_leaf, uint32_t C,
+                   const float* __restrict__ tau, sf_batch_result* res, sf_dev_state* st)
 {
-    const uint32_t k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= counts[0]) return;
+    const uint32_t gi = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t k = gi >> 4, c = gi & 15u;
+    const bool live = k < counts[0];
+    float prob = -1.0f;                                  // below every probability: lanes past C never win
+    if (live && c < C) {
+        const uint16_t* idx = leaf_idx + (size_t)k * T;
+        float acc = 0.0f;
+        uint32_t tt = 0;
+        for (; tt + 8 <= T; tt += 8) {                    // eight loads in flight, added in tree order
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; q++) v[q] = __ldg(leaf + ((size_t)(tt + q) * n_leaf + idx[tt + q]) * C + c);
+#pragma unroll
+            for (int q = 0; q < 8; q++) acc = __fadd_rn(acc, v[q]);
+        }
+        for (; tt < T; tt++) acc = __fadd_rn(acc, __ldg(leaf + ((size_t)tt * n_leaf + idx[tt]) * C + c));
+        prob = __fdiv_rn(acc, __uint2float_rn(T));
+    }
+    float best = prob; uint32_t arg = c;
+#pragma unroll
+    for (int o = 8; o >= 1; o >>= 1) {                    // stays inside the 16-lane group
+        const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+        const uint32_t oa = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+        if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+    }
+    if (!live || c != 0) return;
+    const float u = __fsub_rn(1.0f, best);
+    const uint8_t label_k = (uint8_t)arg;
+    const bool decision_k = u > __ldg(tau + arg);
     const uint32_t slot = fire1_slot[k];
-    t.label_fast[slot] = label[k];
-    t.score[slot] = score[k];
+    t.label_fast[slot] = label_k;
+    t.score[slot] = u;
     atomicAdd(&res->n_fast_fired, 1u);
-    bool assigned = decision[k] != 0;
+    bool assigned = decision_k;
     if (assigned) {
         uint32_t s;
         const int k_free = atomicSub(t.slab_free_n, 1);              // returned slabs first, then never-used ones
@@ -376,9 +409,10 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
 }
 
 __global__ void apply_slow_kernel(TableDev t, const uint32_t* __restrict__ fire2_slot, const uint32_t* __restrict__ counts,
-                                  const uint8_t* __restrict__ label_slow, sf_batch_result* res)
+                                  const uint8_t* __restrict__ label_slow, sf_batch_result* res, sf_dev_state* st)
 {
     const uint32_t k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k == 0) atomicAdd((unsigned long long*)&st->counters.n_slow_done, (unsigned long long)counts[1]);
     if (k >= counts[1]) return;
     const uint32_t slot = fire2_slot[k];
     t.label_slow[slot] = label_slow[k];
@@ -535,10 +569,9 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     const uint32_t Cs = slow->dims[slow->n_layers];
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += sf_align256(bytes); return o; };
-    const size_t o_feat = take((size_t)n * F * 4), o_prob = take((size_t)n * fo->C * 4), o_dec = take(n), o_lab = take(n),
-                 o_score = take((size_t)n * 4), o_bc = take((size_t)(n / 1024 + 2) * 4),
+    const size_t o_feat = take((size_t)n * F * 4), o_lidx = take((size_t)n * fo->T * 2),
                  o_rows = take((size_t)n * slow->dims[0] * esz), o_logits = take((size_t)n * Cs * 4), o_slab_lab = take(n),
-                 o_slow = take(sf_slow_scratch_bytes(slow, n)), o_lidx = take((size_t)n * fo->T * 2);
+                 o_slow = take(sf_slow_scratch_bytes(slow, n));
     int rc = sf_ws_reserve(ctx, off);
     if (rc != SF_OK) return rc;
     sf_ws_reset(ctx);
@@ -574,24 +607,20 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     fpk.size = t->c_size; fpk.iat_us = t->c_iat; fpk.dir_bits = t->c_dir; fpk.hdr = nullptr; fpk.n_valid = nullptr;
     fpk.n_flows = n; fpk.pitch_pkts = d.fast_pkts; fpk.hdr_bytes = 0;
     float* feat = reinterpret_cast<float*>(w + o_feat);
-    float* prob = reinterpret_cast<float*>(w + o_prob);
     sf_time_begin(ctx, SF_T_EXTRACT, st);
     rc = sf_launch_extract(&fpk, d.fast_pkts, F, feat, st, &t->counts[0]);
     sf_time_end(ctx, SF_T_EXTRACT, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_FOREST, st);
-    // a few hundred flows fire per batch: trees spread over the grid, leaf indices as scratch, then the ordered sums
-    rc = sf_launch_forest(fo, feat, n, prob, reinterpret_cast<uint16_t*>(w + o_lidx), st, &t->counts[0], true);
+    // a few hundred flows fire per batch: trees spread over the grid, one leaf index per flow and tree ...
+    rc = sf_launch_forest_leaf_index(fo, feat, n, reinterpret_cast<uint16_t*>(w + o_lidx), st, &t->counts[0]);
     sf_time_end(ctx, SF_T_FOREST, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_SCORE, st);
-    rc = sf_launch_score(cfg, prob, n, fo->C, reinterpret_cast<uint8_t*>(w + o_dec), reinterpret_cast<uint8_t*>(w + o_lab),
-                         reinterpret_cast<float*>(w + o_score), reinterpret_cast<uint32_t*>(w + o_bc), &t->counts[0], st);
-    if (rc != SF_OK) return rc;
-    apply_route_kernel<<<blocks, 256, 0, st>>>(d, t->fire1_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_dec),
-                                               reinterpret_cast<uint8_t*>(w + o_lab), reinterpret_cast<float*>(w + o_score),
-                                               result_dev, ctx->d_state);
-    SF_LAUNCH_CHECK("apply_route_kernel");
+    // ... then leaf sums, score, decision and the table update in one kernel (16 lanes per flow)
+    fast_finish_kernel<<<(n * 16u + 255) / 256, 256, 0, st>>>(d, t->fire1_slot, t->counts, reinterpret_cast<const uint16_t*>(w + o_lidx), fo->d_leaf,
+                                                             fo->T, 1u << fo->depth, fo->C, cfg->tau, result_dev, ctx->d_state);
+    SF_LAUNCH_CHECK("fast_finish_kernel");
     apply2_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire2_slab, t->fire2_slot,
                                           t->counts, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("apply2_kernel");
@@ -607,9 +636,9 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     sf_time_end(ctx, SF_T_GATHER, st);
     if (rc != SF_OK) return rc;
     rc = sf_launch_slow(ctx, slow, w + o_rows, &t->counts[1], n, reinterpret_cast<float*>(w + o_logits),
-                        reinterpret_cast<uint8_t*>(w + o_slab_lab), w + o_slow, st);
+                        reinterpret_cast<uint8_t*>(w + o_slab_lab), w + o_slow, st, false);
     if (rc != SF_OK) return rc;
-    apply_slow_kernel<<<blocks, 256, 0, st>>>(d, t->fire2_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_slab_lab), result_dev);
+    apply_slow_kernel<<<blocks, 256, 0, st>>>(d, t->fire2_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_slab_lab), result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("apply_slow_kernel");
     return SF_OK;
 }
