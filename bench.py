@@ -305,7 +305,7 @@ def run_stream(args, cfg):
             "fraction_answered_at_fast_stage": (fast_done / answered) if answered else None,
             "counts": {"new_flows": new_flows, "fast_fired": fast_fired, "fast_done": fast_done, "escalated": escalated,
                        "slow_fired": slow_fired, "dropped_after_decision": dropped, "missed": missed},
-            "per_batch_stage_ms": stage_ms, "us_per_batch": 1e3 * ms / (n_timed - args.warmup * bps), "gpu_launches": 18 * (n_timed - args.warmup * bps),
+            "per_batch_stage_ms": stage_ms, "us_per_batch": 1e3 * ms / (n_timed - args.warmup * bps), "gpu_launches": 17 * (n_timed - args.warmup * bps),
             "clocks": clocks, "device_error": c.device_error}
     print(json.dumps(line))
 

@@ -93,7 +93,8 @@ static inline size_t sf_align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 // ---- internal launchers (each validates nothing; callers did) ---------------
 int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st,
-                      const uint32_t* n_dev = nullptr);   // n_dev: optional device-side flow count (<= pk->n_flows)
+                      const uint32_t* n_dev = nullptr,    // n_dev: optional device-side flow count (<= pk->n_flows)
+                      const uint32_t* row_ids = nullptr); // row_ids: optional, flow f's packets are row row_ids[f] of the planes
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st,
                      const uint32_t* n_dev = nullptr, bool small_tiles = false);   // small_tiles + leaf_idx (used as scratch): few flows per launch, trees spread over the grid
 // route scratch: block_counts uint32[ceil(n/1024)+1], decision bytes if the caller gave none

@@ -112,7 +112,8 @@ template <int G, bool VEC>
 __global__ void __launch_bounds__(kFlowsPerBlock)
 extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ iat,
                const uint32_t* __restrict__ dir_bits, const uint8_t* __restrict__ n_valid,
-               uint32_t n, uint32_t pitch, uint32_t N, float* __restrict__ feat, const uint32_t* __restrict__ n_dev)
+               uint32_t n, uint32_t pitch, uint32_t N, float* __restrict__ feat, const uint32_t* __restrict__ n_dev,
+               const uint32_t* __restrict__ row_ids)
 {
     constexpr int F = 8 * G;
     constexpr int STRIDE = F + 4;                  // 16-byte aligned rows; 8 lanes x 16 B land in distinct bank groups
@@ -123,19 +124,20 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
     const uint32_t f = f0 + threadIdx.x;
 
     if (f < n) {
+        const size_t fr = row_ids ? row_ids[f] : f;      // optional indirection: flow f's packets sit in row row_ids[f] of the planes
         Acc A[8];
 #pragma unroll
         for (int g = 0; g < 8; g++) acc_init(A[g]);
         uint32_t m = N;
-        if (n_valid) m = min(m, (uint32_t)n_valid[f]);
+        if (n_valid) m = min(m, (uint32_t)n_valid[fr]);
         // N <= 32: all direction bits of the window are in the row's first word
-        const uint32_t dirw = dir_bits[(size_t)f * ((pitch + 31) >> 5)];
+        const uint32_t dirw = dir_bits[fr * ((pitch + 31) >> 5)];
         const uint32_t all_mask = (m >= 32) ? 0xFFFFFFFFu : ((1u << m) - 1u);
         const uint32_t fwd_mask = ~dirw & all_mask;
         const uint32_t bwd_mask = dirw & all_mask;
         const uint32_t turn_mask = (dirw ^ (dirw << 1)) & ~1u & all_mask;        // packet i >= 1 whose direction differs from i-1
-        const uint16_t* srow = size + (size_t)f * pitch;
-        const uint32_t* irow = iat + (size_t)f * pitch;
+        const uint16_t* srow = size + fr * pitch;
+        const uint32_t* irow = iat + fr * pitch;
         if (VEC) {
             // issue every load of the window first (N <= 32: at most four chunks of eight packets), then reduce
             uint4 s4[4], a4[4], b4[4];
@@ -195,32 +197,33 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
 }
 
 template <int G>
-int launch_g(const sf_packets* pk, uint32_t N, float* feat, cudaStream_t st, const uint32_t* n_dev) {
+int launch_g(const sf_packets* pk, uint32_t N, float* feat, cudaStream_t st, const uint32_t* n_dev, const uint32_t* row_ids) {
     const uint32_t n = pk->n_flows;
     const bool vec = (pk->pitch_pkts % 8 == 0) && (((uintptr_t)pk->size & 15) == 0) && (((uintptr_t)pk->iat_us & 15) == 0);
     const size_t smem = (size_t)kFlowsPerBlock * (8 * G + 4) * sizeof(float);
     const uint32_t grid = (n + kFlowsPerBlock - 1) / kFlowsPerBlock;
     if (vec)
-        extract_kernel<G, true><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev);
+        extract_kernel<G, true><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev, row_ids);
     else
-        extract_kernel<G, false><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev);
+        extract_kernel<G, false><<<grid, kFlowsPerBlock, smem, st>>>(pk->size, pk->iat_us, pk->dir_bits, pk->n_valid, n, pk->pitch_pkts, N, feat, n_dev, row_ids);
     SF_LAUNCH_CHECK("extract_kernel");
     return SF_OK;
 }
 
 }  // namespace
 
-int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st, const uint32_t* n_dev) {
+int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st, const uint32_t* n_dev,
+                      const uint32_t* row_ids) {
     if (pk->n_flows == 0) return SF_OK;
     switch (F / 8) {
-    case 1: return launch_g<1>(pk, N, feat, st, n_dev);
-    case 2: return launch_g<2>(pk, N, feat, st, n_dev);
-    case 3: return launch_g<3>(pk, N, feat, st, n_dev);
-    case 4: return launch_g<4>(pk, N, feat, st, n_dev);
-    case 5: return launch_g<5>(pk, N, feat, st, n_dev);
-    case 6: return launch_g<6>(pk, N, feat, st, n_dev);
-    case 7: return launch_g<7>(pk, N, feat, st, n_dev);
-    case 8: return launch_g<8>(pk, N, feat, st, n_dev);
+    case 1: return launch_g<1>(pk, N, feat, st, n_dev, row_ids);
+    case 2: return launch_g<2>(pk, N, feat, st, n_dev, row_ids);
+    case 3: return launch_g<3>(pk, N, feat, st, n_dev, row_ids);
+    case 4: return launch_g<4>(pk, N, feat, st, n_dev, row_ids);
+    case 5: return launch_g<5>(pk, N, feat, st, n_dev, row_ids);
+    case 6: return launch_g<6>(pk, N, feat, st, n_dev, row_ids);
+    case 7: return launch_g<7>(pk, N, feat, st, n_dev, row_ids);
+    case 8: return launch_g<8>(pk, N, feat, st, n_dev, row_ids);
     }
     return SF_ERR_UNSUPPORTED;
 }

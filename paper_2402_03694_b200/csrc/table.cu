@@ -60,7 +60,6 @@ struct sf_table {
     uint32_t* fire1_slot; uint32_t* fire2_slab; uint32_t* fire2_slot;
     uint32_t* counts;                 // [0] n_fire1, [1] n_fire2
     uint32_t* pkt_slot; uint32_t* hist;
-    uint16_t* c_size; uint32_t* c_iat; uint32_t* c_dir;      // dense fast planes of the fired flows
     void* all;                        // one allocation behind everything above
 };
 
@@ -294,18 +293,6 @@ __global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
     }
 }
 
-__global__ void gather_fast_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const uint32_t* __restrict__ counts,
-                                   uint16_t* __restrict__ c_size, uint32_t* __restrict__ c_iat, uint32_t* __restrict__ c_dir)
-{
-    const uint32_t e = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t k = e / t.fast_pkts, p = e - k * t.fast_pkts;
-    if (k >= counts[0]) return;
-    const uint32_t slot = fire1_slot[k];
-    c_size[e] = t.f_size[(size_t)slot * t.fast_pkts + p];
-    c_iat[e] = t.f_iat[(size_t)slot * t.fast_pkts + p];
-    if (p == 0) c_dir[k] = t.f_dir[slot];
-}
-
 // Finishes the fast model for the flows that fired in this batch and applies the assignment, one kernel instead of
 // three (leaf sums, score, application): 16 lanes per flow, lane c < C adds class c's leaf values in tree order
 // t = 0..T-1 and divides by T (the random forest's soft vote, same operations and order as the batch kernels), the group
@@ -506,8 +493,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     need(B * slow_pkts * 2); need(B * slow_pkts * 4); need(B * W * 4); need(B * slow_pkts * kHdr); need(4);
     need(B * 4); need(4); need(S * 4);
     for (int k = 0; k < 9; k++) need((size_t)kMaxBatch * 4);
-    need(64); need((size_t)kMaxBatch * 4); need(1024 * 4); need(S * 4);
-    need((size_t)kMaxBatch * fast_pkts * 2); need((size_t)kMaxBatch * fast_pkts * 4); need((size_t)kMaxBatch * 4);
+    need((16 + 4 * 1024) * 4); need((size_t)kMaxBatch * 4); need(S * 4);          // counters + digit counts, pkt_slot, first
     cudaError_t e = cudaMalloc(&t->all, total);
     if (e != cudaSuccess) { delete t; sf_set_cuda_error(e, "cudaMalloc(table)"); return SF_ERR_ALLOC; }
     e = cudaMemset(t->all, 0, total);
@@ -534,10 +520,11 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     t->hist = t->counts + 16;
     t->pkt_slot = carve<uint32_t>(p, kMaxBatch);
     d.first = carve<uint32_t>(p, S);
+    if ((size_t)(p - reinterpret_cast<char*>(t->all)) > total) {          // the size list above and the carving must agree
+        cudaFree(t->all); delete t; return SF_ERR_ALLOC;
+    }
     e = cudaMemset(d.first, 0xFF, S * 4);
     if (e != cudaSuccess) { cudaFree(t->all); delete t; return sf_set_cuda_error(e, "cudaMemset(table)"); }
-    t->c_size = carve<uint16_t>(p, (size_t)kMaxBatch * fast_pkts); t->c_iat = carve<uint32_t>(p, (size_t)kMaxBatch * fast_pkts);
-    t->c_dir = carve<uint32_t>(p, kMaxBatch);
     *out = t;
     return SF_OK;
 }
@@ -599,16 +586,15 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     }
     apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts);
     SF_LAUNCH_CHECK("apply1_kernel");
-    gather_fast_kernel<<<(n * d.fast_pkts + 255) / 256, 256, 0, st>>>(d, t->fire1_slot, t->counts, t->c_size, t->c_iat, t->c_dir);
-    SF_LAUNCH_CHECK("gather_fast_kernel");
     sf_time_end(ctx, SF_T_TABLE, st);
-    // S1..S3 on the flows that just completed their fast context (count stays on the device)
+    // S1..S3 on the flows that just completed their fast context (count stays on the device); the feature kernel reads
+    // their packets in place, through the list of their slots
     sf_packets fpk;
-    fpk.size = t->c_size; fpk.iat_us = t->c_iat; fpk.dir_bits = t->c_dir; fpk.hdr = nullptr; fpk.n_valid = nullptr;
+    fpk.size = d.f_size; fpk.iat_us = d.f_iat; fpk.dir_bits = d.f_dir; fpk.hdr = nullptr; fpk.n_valid = nullptr;
     fpk.n_flows = n; fpk.pitch_pkts = d.fast_pkts; fpk.hdr_bytes = 0;
     float* feat = reinterpret_cast<float*>(w + o_feat);
     sf_time_begin(ctx, SF_T_EXTRACT, st);
-    rc = sf_launch_extract(&fpk, d.fast_pkts, F, feat, st, &t->counts[0]);
+    rc = sf_launch_extract(&fpk, d.fast_pkts, F, feat, st, &t->counts[0], t->fire1_slot);
     sf_time_end(ctx, SF_T_EXTRACT, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_FOREST, st);
