@@ -8,51 +8,70 @@
 namespace {
 
 // out[r][o] = act( sum_k in[r][k] * W[o][k] + b[o] ),  r < *n_rows_dev
-// 64x64 output tile, 16-deep K slices, 256 threads with 4x4 register tiles.
-template <bool RELU>
+// (16 * RM) x 64 output tile, 16-deep K slices (the next one prefetched into registers), 256 threads with RM x 4 register
+// tiles.  RM = 4: 64-row tiles; RM = 2: 32-row tiles, twice as many blocks when the batch is small.
+template <bool RELU, int RM>
 __global__ void __launch_bounds__(256)
 dense_f32_kernel(const float* __restrict__ in, const float* __restrict__ W, const float* __restrict__ b,
                  const uint32_t* __restrict__ n_rows_dev, uint32_t K, uint32_t N, float* __restrict__ out)
 {
-    __shared__ float As[16][64 + 4];
+    constexpr uint32_t TR = 16 * RM;               // rows per tile
+    __shared__ float As[16][TR + 4];
     __shared__ float Bs[16][64 + 4];
     const uint32_t n_rows = *n_rows_dev;
-    const uint32_t r0 = blockIdx.x * 64, o0 = blockIdx.y * 64;
+    const uint32_t r0 = blockIdx.x * TR, o0 = blockIdx.y * 64;
     if (r0 >= n_rows) return;
     const uint32_t tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-    float acc[4][4];
+    float acc[RM][4];
 #pragma unroll
-    for (int i = 0; i < 4; i++)
+    for (int i = 0; i < RM; i++)
 #pragma unroll
         for (int j = 0; j < 4; j++) acc[i][j] = 0.0f;
     const uint32_t lr = threadIdx.x >> 2;          // 0..63: tile row loaded by this thread
     const uint32_t lk = (threadIdx.x & 3) * 4;     // 0,4,8,12
+    const uint32_t ra = r0 + lr, ob = o0 + lr;
+    const bool a_row = lr < TR;
+    const bool vec = (K & 3u) == 0;                // rows start on 16-byte boundaries: one 16-byte load per operand and slice
+    // the next K slice is fetched into registers while the current one is multiplied
+    auto fetch = [&](uint32_t k0, float (&a)[4], float (&w)[4]) {
+        const uint32_t k = k0 + lk;
+        if (vec && k < K) {
+            const float4 va = (a_row && ra < n_rows) ? __ldg(reinterpret_cast<const float4*>(in + (size_t)ra * K + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 vw = (ob < N) ? __ldg(reinterpret_cast<const float4*>(W + (size_t)ob * K + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            a[0] = va.x; a[1] = va.y; a[2] = va.z; a[3] = va.w;
+            w[0] = vw.x; w[1] = vw.y; w[2] = vw.z; w[3] = vw.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                a[j] = (a_row && ra < n_rows && k + j < K) ? in[(size_t)ra * K + k + j] : 0.0f;
+                w[j] = (ob < N && k + j < K) ? W[(size_t)ob * K + k + j] : 0.0f;
+            }
+        }
+    };
+    float pa[4], pw[4];
+    fetch(0, pa, pw);
     for (uint32_t k0 = 0; k0 < K; k0 += 16) {
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            uint32_t k = k0 + lk + j;
-            uint32_t r = r0 + lr, o = o0 + lr;
-            As[lk + j][lr] = (r < n_rows && k < K) ? in[(size_t)r * K + k] : 0.0f;
-            Bs[lk + j][lr] = (o < N && k < K) ? W[(size_t)o * K + k] : 0.0f;
-        }
+        for (int j = 0; j < 4; j++) { if (a_row) As[lk + j][lr] = pa[j]; Bs[lk + j][lr] = pw[j]; }
         __syncthreads();
+        if (k0 + 16 < K) fetch(k0 + 16, pa, pw);
 #pragma unroll
         for (int k = 0; k < 16; k++) {
-            float a[4], w[4];
+            float a[RM], w[4];
 #pragma unroll
-            for (int i = 0; i < 4; i++) a[i] = As[k][ty * 4 + i];
+            for (int i = 0; i < RM; i++) a[i] = As[k][ty * RM + i];
 #pragma unroll
             for (int j = 0; j < 4; j++) w[j] = Bs[k][tx * 4 + j];
 #pragma unroll
-            for (int i = 0; i < 4; i++)
+            for (int i = 0; i < RM; i++)
 #pragma unroll
                 for (int j = 0; j < 4; j++) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
         }
         __syncthreads();
     }
 #pragma unroll
-    for (int i = 0; i < 4; i++) {
-        uint32_t r = r0 + ty * 4 + i;
+    for (int i = 0; i < RM; i++) {
+        uint32_t r = r0 + ty * RM + i;
         if (r >= n_rows) continue;
 #pragma unroll
         for (int j = 0; j < 4; j++) {
@@ -120,9 +139,19 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
             const bool last = (l + 1 == s->n_layers);
             if (last) { sf_time_end(ctx, SF_T_GEMM, st); sf_time_begin(ctx, SF_T_HEAD, st); }
             float* out = last ? logits : ((l & 1) ? h1 : h0);
-            dim3 grid((capacity + 63) / 64, (s->dims[l + 1] + 63) / 64);
-            if (last) dense_f32_kernel<false><<<grid, 256, 0, st>>>(in, (const float*)s->d_W[l], s->d_b[l], n_rows_dev, s->dims[l], s->dims[l + 1], out);
-            else      dense_f32_kernel<true><<<grid, 256, 0, st>>>(in, (const float*)s->d_W[l], s->d_b[l], n_rows_dev, s->dims[l], s->dims[l + 1], out);
+            const uint32_t K = s->dims[l], N = s->dims[l + 1];
+            const float* Wl = (const float*)s->d_W[l];
+            // few tiles: 32-row tiles put twice as many blocks on the machine
+            const bool small_tiles = (size_t)((capacity + 63) / 64) * ((N + 63) / 64) < 4u * (size_t)ctx->num_sms;
+            if (small_tiles) {
+                dim3 grid((capacity + 31) / 32, (N + 63) / 64);
+                if (last) dense_f32_kernel<false, 2><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
+                else      dense_f32_kernel<true, 2><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
+            } else {
+                dim3 grid((capacity + 63) / 64, (N + 63) / 64);
+                if (last) dense_f32_kernel<false, 4><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
+                else      dense_f32_kernel<true, 4><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
+            }
             SF_LAUNCH_CHECK("dense_f32_kernel");
             in = out;
         }
