@@ -297,6 +297,10 @@ def test_mlp_fp32(env):
     ((128, 128, 8), 300, 384),            # ragged last tile
     ((256, 256, 256, 2), 130, 1000),      # BN = 256, count far below capacity
     ((192, 320, 64, 16), 515, 600),       # BN = 64 path, K not a power of two
+    ((256, 256, 256, 2), 1, 1000),        # sixteen rows or fewer: served on CUDA cores inside the same launches
+    ((192, 320, 64, 16), 7, 600),
+    ((2048, 1024, 8), 16, 64),
+    ((2048, 1024, 8), 17, 64),            # one row more: back on the tensor cores
 ])
 def test_mlp_bf16_small_integers_are_exact(env, dims, n_rows, cap):
     """Integer-valued bf16 operands with small sums: every product and partial sum is
@@ -327,7 +331,7 @@ def test_mlp_bf16_small_integers_are_exact(env, dims, n_rows, cap):
     sf.sf_slow_destroy(hd)
 
 
-@pytest.mark.parametrize("dims,n_rows", [((1024, 512, 512, 2), 700), ((2048, 1024, 1024, 1024, 8), 400)])
+@pytest.mark.parametrize("dims,n_rows", [((1024, 512, 512, 2), 700), ((2048, 1024, 1024, 1024, 8), 400), ((2048, 1024, 1024, 1024, 8), 11)])
 def test_mlp_bf16_within_tolerance(env, dims, n_rows):
     sf, hz, ctx = env
     m = flowgen.gen_mlp(33, dims)
