@@ -55,15 +55,18 @@ def _lookup(sf, hz, ctx, table, keys):
     return out.cpu().numpy().reshape(-1).view(sf.FLOW_RESULT_DTYPE)
 
 
-@pytest.mark.parametrize("shape", ["config5_models", "small_models"])
+@pytest.mark.parametrize("shape", ["config5_models", "small_models", "odd_models"])
 def test_stream_matches_sequential_reference(env, shape):
     sf, hz, ctx = env
     if shape == "config5_models":       # config 2's forest on 8 packets, config 2's MLP on 64 packets padded to 128
         F, T, depth, C, dims, P_model = 48, 100, 12, 8, (2048, 1024, 1024, 1024, 8), 128
         n_keys, n_batches, m = 1500, 24, 4096
-    else:
+    elif shape == "small_models":
         F, T, depth, C, dims, P_model = 24, 16, 8, 4, (1024, 256, 4), 64
         n_keys, n_batches, m = 4000, 10, 8192 + 37
+    else:                                # tree count not a multiple of the slice, class count not a power of two
+        F, T, depth, C, dims, P_model = 32, 37, 5, 11, (1024, 192, 5), 64
+        n_keys, n_batches, m = 3000, 8, 6000 + 11
     fast_pkts, slow_pkts = 8, 64
     forest, tau, slow = _models(F, T, depth, C, dims, 91)
     src = flowgen.StreamSource(92, n_keys, 1.1)
