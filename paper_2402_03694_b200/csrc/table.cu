@@ -7,13 +7,14 @@
 //   probe     one thread per packet: 128-bit compare-and-swap on the 16-byte key slot
 //             (claims an empty slot or recognises its own key; bounded linear probing)
 //   sort      key = arrival index of the flow's first packet in the batch (16 bits, unique per
-//             flow); stable LSD radix sort (4 passes of 4 bits, tiles of 1024) puts each flow's
-//             packets together in ARRIVAL order; rank = position minus start of the run
+//             flow); stable LSD radix sort (4 passes of 4 bits, tiles of 1024, one kernel per pass)
+//             puts each flow's packets together in ARRIVAL order; rank = position minus start of the run
 //   apply1    packets that fall into a flow's first `fast_pkts` positions are written to its
 //             fast context; flows that just reached fast_pkts packets are listed
-//   fast path the listed flows' contexts are copied into dense planes and run through the
-//             same S1 / S2 / S3 kernels as the batch path (flow count read on the device)
-//   route     answered flows are marked; assigned flows get a slab for their slow context
+//   fast path S1 reads the listed flows' packets in place (through the slot list), S2 runs as the
+//             tree-sliced leaf-index kernel for small batches (flow count read on the device)
+//   finish    leaf sums in tree order, least-confidence score and decision, then the table update:
+//             answered flows are marked, assigned flows get a slab for their slow context
 //   apply2    later packets go to the slab of an assigned flow (or are counted as arriving
 //             after the decision); flows that just reached slow_pkts packets are listed
 //   slow path wide rows of the listed slabs (zero-padded to the model's width) -> S4 -> labels
