@@ -329,43 +329,50 @@ fast_finish_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const ui
         const uint32_t oa = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
         if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
     }
-    if (!live || c != 0) return;
-    const float u = __fsub_rn(1.0f, best);
-    const uint8_t label_k = (uint8_t)arg;
-    const bool decision_k = u > __ldg(tau + arg);
-    const uint32_t slot = fire1_slot[k];
-    t.label_fast[slot] = label_k;
-    t.score[slot] = u;
-    atomicAdd(&res->n_fast_fired, 1u);
-    bool assigned = decision_k;
-    if (assigned) {
-        uint32_t s;
-        const int k_free = atomicSub(t.slab_free_n, 1);              // returned slabs first, then never-used ones
-        if (k_free >= 1) s = t.slab_free[k_free - 1];
-        else { atomicAdd(t.slab_free_n, 1); s = atomicAdd(t.slab_next, 1u); if (s >= t.slow_slabs) atomicSub(t.slab_next, 1u); }
-        if (s < t.slow_slabs) {
-            t.slab[slot] = s;
-            const uint32_t words = (t.slow_pkts + 31) / 32;
-            for (uint32_t p = 0; p < t.fast_pkts; p++) {
-                t.s_size[(size_t)s * t.slow_pkts + p] = t.f_size[(size_t)slot * t.fast_pkts + p];
-                t.s_iat[(size_t)s * t.slow_pkts + p] = t.f_iat[(size_t)slot * t.fast_pkts + p];
-                const uint8_t* src = t.f_hdr + ((size_t)slot * t.fast_pkts + p) * kHdr;
-                uint8_t* dst = t.s_hdr + ((size_t)s * t.slow_pkts + p) * kHdr;
-                for (uint32_t q = 0; q < kHdr; q++) dst[q] = src[q];
+    // the group's first lane decides and books the flow; all 16 lanes then copy its fast context into the slab
+    const bool lead = live && c == 0;
+    uint32_t slot = 0, slab = kMiss;
+    if (lead) {
+        const float u = __fsub_rn(1.0f, best);
+        bool assigned = u > __ldg(tau + arg);
+        slot = fire1_slot[k];
+        t.label_fast[slot] = (uint8_t)arg;
+        t.score[slot] = u;
+        atomicAdd(&res->n_fast_fired, 1u);
+        if (assigned) {
+            uint32_t sl;
+            const int k_free = atomicSub(t.slab_free_n, 1);              // returned slabs first, then never-used ones
+            if (k_free >= 1) sl = t.slab_free[k_free - 1];
+            else { atomicAdd(t.slab_free_n, 1); sl = atomicAdd(t.slab_next, 1u); if (sl >= t.slow_slabs) atomicSub(t.slab_next, 1u); }
+            if (sl < t.slow_slabs) {
+                t.slab[slot] = sl;
+                slab = sl;
+            } else {
+                // no slab left: the flow keeps its fast answer and is counted as missed by the slow path
+                assigned = false;
+                atomicAdd(&res->n_missed, 1u);
+                atomicAdd((unsigned long long*)&st->counters.n_missed, 1ull);
+                sf_dev_set_error(st, SF_ERR_TABLE_FULL);
             }
-            atomicOr(&t.s_dir[(size_t)s * words], t.f_dir[slot]);
-        } else {
-            // no slab left: the flow keeps its fast answer and is counted as missed by the slow path
-            assigned = false;
-            atomicAdd(&res->n_missed, 1u);
-            atomicAdd((unsigned long long*)&st->counters.n_missed, 1ull);
-            sf_dev_set_error(st, SF_ERR_TABLE_FULL);
         }
+        t.stage[slot] = assigned ? 2 : 1;
+        if (assigned) { atomicAdd(&res->n_escalated, 1u); atomicAdd((unsigned long long*)&st->counters.n_escalated, 1ull); }
+        else          { atomicAdd(&res->n_fast_done, 1u); atomicAdd((unsigned long long*)&st->counters.n_fast_done, 1ull); }
+        atomicAdd((unsigned long long*)&st->counters.n_flows, 1ull);
     }
-    t.stage[slot] = assigned ? 2 : 1;
-    if (assigned) { atomicAdd(&res->n_escalated, 1u); atomicAdd((unsigned long long*)&st->counters.n_escalated, 1ull); }
-    else          { atomicAdd(&res->n_fast_done, 1u); atomicAdd((unsigned long long*)&st->counters.n_fast_done, 1ull); }
-    atomicAdd((unsigned long long*)&st->counters.n_flows, 1ull);
+    const uint32_t lead_lane = (threadIdx.x & 31u) & 16u;
+    slot = __shfl_sync(0xFFFFFFFFu, slot, lead_lane);
+    slab = __shfl_sync(0xFFFFFFFFu, slab, lead_lane);
+    if (slab != kMiss) {                                  // one element or byte per lane and step: the loads of a step are all in flight at once
+        for (uint32_t p = c; p < t.fast_pkts; p += 16) {
+            t.s_size[(size_t)slab * t.slow_pkts + p] = t.f_size[(size_t)slot * t.fast_pkts + p];
+            t.s_iat[(size_t)slab * t.slow_pkts + p] = t.f_iat[(size_t)slot * t.fast_pkts + p];
+        }
+        const uint8_t* src = t.f_hdr + (size_t)slot * t.fast_pkts * kHdr;
+        uint8_t* dst = t.s_hdr + (size_t)slab * t.slow_pkts * kHdr;
+        for (uint32_t i = c; i < t.fast_pkts * kHdr; i += 16) dst[i] = src[i];
+        if (c == 0) atomicOr(&t.s_dir[(size_t)slab * ((t.slow_pkts + 31) / 32)], t.f_dir[slot]);
+    }
 }
 
 __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
