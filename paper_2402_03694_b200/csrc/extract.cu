@@ -13,7 +13,7 @@
 
 namespace {
 
-constexpr int kFlowsPerBlock = 128;
+constexpr int kFlowsPerBlock = 32;       // one warp per block: small blocks schedule better here than 64- or 128-flow ones (measured)
 
 // Integer accumulators of one (quantity, subset) group.  Counts, first and last come from
 // the subset's bit mask (popcount / lowest / highest set bit), so the per-packet work is
