@@ -15,6 +15,13 @@
  *    are skipped when NULL.
  *  - Calls enqueue work on the caller's stream (a cudaStream_t passed as void*,
  *    NULL = the default stream) and do not synchronise, except where stated.
+ *  - A context serves ONE stream at a time.  Every compute call on a context uses the
+ *    context's single device workspace (grown, when a call needs more, by a synchronising
+ *    free + allocate) and its device-side count of assigned flows, so calls on one context
+ *    must be ordered on one stream, or by events, and must not be issued from two threads
+ *    at once; calls that overlap on the GPU race on the intermediates.  The pointers that
+ *    sf_serve_batch_intermediates returns are valid until the next compute call on that
+ *    context.  Use one context per stream for concurrent work.
  *  - Handles (sf_ctx, sf_forest, sf_slow, sf_table) are owned by the library,
  *    built from HOST arrays that are copied and re-laid-out inside, and released
  *    by the matching *_destroy.  A handle belongs to the device of its context.
@@ -212,7 +219,8 @@ int  sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* prob_or_margin,
  * so this call takes no context.
  *
  * It does what sf_route does up to the list of assigned flows - score, fast label,
- * strict threshold, ascending ids, count - and gathers no wide rows.  The per-block
+ * strict threshold, ascending ids, count, under any of sf_route's four rules - and
+ * gathers no wide rows.  The per-block
  * counts and, when decision_out is NULL, the per-flow decisions go to a fixed array
  * built into the library image (about 4 MB; every GPU that loads the library keeps it
  * until the process ends), so n may be at most SF_NOALLOC_MAX_FLOWS; a larger n is
@@ -227,6 +235,7 @@ int  sf_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* prob_or_margin,
  *
  * The first call on a device looks up the array's device address (a one-time set-up
  * with that device current); make that first call before starting any stream capture.
+ * First calls made by several threads at once are harmless (each stores the same address).
  * All calls on a device share the one array and it keeps the previous call's contents
  * (the call clears the part that must start at zero), so two calls whose GPU work
  * overlaps - different streams, or different threads - race; run them one after the
@@ -289,7 +298,9 @@ void sf_slow_destroy(sf_slow* slow);
  * count, read by the kernels: no host round trip) of rows[capacity][D] (bf16 or
  * fp32 as the model's dtype).  logits_out fp32[capacity][n_cls]; label_out
  * uint8[capacity] (nullable) = argmax, lowest index on ties.  Rows at or beyond
- * the count are not written. */
+ * the count are not written.  A count above `capacity` is treated as `capacity`
+ * (nothing is read or written beyond the buffers) and SF_ERR_CAPACITY is recorded in
+ * the error word. */
 int  sf_slow_infer(sf_ctx* ctx, const sf_slow* slow, const void* rows, const uint32_t* n_rows_dev,
                    uint32_t capacity, float* logits_out, uint8_t* label_out, void* stream);
 
@@ -368,7 +379,8 @@ typedef struct {
  * flow id, escalations) replaced by one device hash table keyed by the 5-tuple:
  * 2^log2_slots slots, linear probing with a bounded probe count; every flow keeps
  * its first fast_pkts packets; flows assigned to the slow model get one of
- * `slow_slabs` slabs holding slow_pkts packets. */
+ * `slow_slabs` slabs holding slow_pkts packets.  fast_pkts in 1..32, fast_pkts < slow_pkts
+ * <= 128 (the slow model must see more packets than the fast one, else SF_ERR_ARG). */
 int  sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_pkts, uint32_t slow_pkts,
                      uint32_t slow_slabs, sf_table** out);
 void sf_table_destroy(sf_table* table);

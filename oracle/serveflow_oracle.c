@@ -14,9 +14,9 @@
  * the synthetic stand-in workload; those readings are stated beside each function.
  *
  * Parity status: every function below is pinned by tests that do not re-use its
- * own formula (hand-computed values, closed forms, brute force, invariants),
- * except sfo_sigmoid, which is a derived convenience output compared by tolerance
- * only ("parity unpinned" for bits; routing never uses it).
+ * own formula (hand-computed values, closed forms, brute force, invariants).
+ * sfo_sigmoid is a derived convenience output (closed-form pins: 0 -> 1/2, ln 3 -> 3/4,
+ * symmetry); routing never uses it.
  *
  * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC (no FMA
  * contraction, so every fp32 operation rounds once).

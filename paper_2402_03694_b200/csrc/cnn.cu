@@ -132,14 +132,14 @@ struct Bias1 { float v[C1]; };
 __global__ void __launch_bounds__(kThreads, 1)
 cnn_fused_kernel(const __nv_bfloat16* __restrict__ rows, const uint32_t* __restrict__ n_rows_dev,
                  const unsigned char* __restrict__ blob, const __grid_constant__ Bias1 b1, uint32_t n_cls,
-                 float* __restrict__ logits, uint8_t* __restrict__ label, sf_dev_state* st)
+                 float* __restrict__ logits, uint8_t* __restrict__ label, sf_dev_state* st, uint32_t capacity)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     Bars* bars = reinterpret_cast<Bars*>(smem + SM_BARS);
     volatile uint32_t* abort_flag = &bars->abort_flag;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t n_rows = *n_rows_dev;
+    const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);      // the caller's word, bounded by what the buffers hold
     // flows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; flow m of the CTA is slot (m & 1) of pair (m >> 1)
     const uint32_t n_mine = (n_rows > blockIdx.x) ? (n_rows - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const uint32_t n_pairs = (n_mine + 1) >> 1;
@@ -443,7 +443,7 @@ int sf_cnn_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     sf_time_begin(ctx, SF_T_GEMM, st);
     cnn_fused_kernel<<<grid, kThreads, SM_TOTAL, st>>>(reinterpret_cast<const __nv_bfloat16*>(rows), n_rows_dev,
                                                      reinterpret_cast<const unsigned char*>(s->d_w1), *reinterpret_cast<const Bias1*>(s->h_cnn_b1), s->n_cls,
-                                                     logits, label, ctx->d_state);
+                                                     logits, label, ctx->d_state, capacity);
     sf_time_end(ctx, SF_T_GEMM, st);
     SF_LAUNCH_CHECK("cnn_fused_kernel");
     return SF_OK;

@@ -135,3 +135,11 @@ int sf_cnn_prepare(sf_slow* s, const float* w1, const float* b1, const float* w2
 __device__ __forceinline__ void sf_dev_set_error(sf_dev_state* st, int code) {
     atomicCAS(&st->counters.device_error, 0, code);
 }
+
+// A row count that lives in device memory is the caller's word: the slow-model kernels take at most
+// `capacity` rows (what the buffers hold) and record SF_ERR_CAPACITY when the word said more.
+__device__ __forceinline__ uint32_t sf_clamp_rows(uint32_t n_rows, uint32_t capacity, sf_dev_state* st) {
+    if (n_rows <= capacity) return n_rows;
+    if (st && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_CAPACITY);
+    return capacity;
+}

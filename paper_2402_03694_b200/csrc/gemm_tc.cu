@@ -167,12 +167,14 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                            const float* __restrict__ bias, const uint32_t* __restrict__ n_rows_dev,
                            uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out, sf_dev_state* st,
                            float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C, uint32_t small_max,
-                           const __nv_bfloat16* __restrict__ A_raw, const __nv_bfloat16* __restrict__ W_raw)
+                           const __nv_bfloat16* __restrict__ A_raw, const __nv_bfloat16* __restrict__ W_raw, uint32_t capacity)
 {
     using Cfg = GemmCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
-    if (*n_rows_dev <= small_max) {                  // a handful of rows (small_max = 0: never): CUDA cores, same launch
-        if (*n_rows_dev) small_rows_layer<HEAD>(A_raw, W_raw, bias, *n_rows_dev, N, K, out, logits, label, C, smem_raw);
+    // the count is the caller's device word: never trust it beyond the rows the buffers hold
+    const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);
+    if (n_rows <= small_max) {                       // a handful of rows (small_max = 0: never): CUDA cores, same launch
+        if (n_rows) small_rows_layer<HEAD>(A_raw, W_raw, bias, n_rows, N, K, out, logits, label, C, smem_raw);
         return;
     }
     const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -181,7 +183,6 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t n_rows = *n_rows_dev;
     const uint32_t tiles_m = (n_rows + BM - 1) / BM;
     const uint32_t tiles_n = N / BN;
     const uint32_t n_tiles = tiles_m * tiles_n;
@@ -354,7 +355,7 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
                                                   reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state, nullptr, nullptr, 0, small_max,
-                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W));
+                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity);
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel");
     return SF_OK;
 }
@@ -376,7 +377,7 @@ int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bia
     uint32_t max_tiles = (capacity + BM - 1) / BM;
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C, small_max,
-                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16));
+                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16), capacity);
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(head)");
     return SF_OK;
 }

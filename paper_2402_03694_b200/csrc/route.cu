@@ -455,14 +455,15 @@ extern "C" int sf_route_noalloc(int device, const sf_route_cfg* cfg, const float
                                 uint8_t* label_fast_out, float* score_out, int32_t* status_out, void* stream)
 {
     if (!cfg || !fast_out || !esc_ids_out || !n_esc_out || !cfg->tau) return SF_ERR_ARG;
-    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT) return SF_ERR_ARG;
-    if (cfg->rule == SF_LC_GT && (C < 1 || C > 256)) return SF_ERR_ARG;
+    if (cfg->rule != SF_LC_GT && cfg->rule != SF_ABSMARGIN_LT && cfg->rule != SF_ENTROPY_GT && cfg->rule != SF_SOFTMAX_LC_GT) return SF_ERR_ARG;
+    if (cfg->rule != SF_ABSMARGIN_LT && (C < 1 || C > 256)) return SF_ERR_ARG;
     if (device < 0 || device >= kMaxDevices) return SF_ERR_ARG;
     if (n > SF_NOALLOC_MAX_FLOWS) return SF_ERR_STATIC_LIMIT;
     SF_CUDA(cudaSetDevice(device));
     if (!g_noalloc_ptr[device]) {
         // In host code the array's name is only a handle; the device address has to be asked for,
-        // once per device, with that device current.
+        // once per device, with that device current.  Two threads that make their first call on a device
+        // at the same time both store the same address here, so the unsynchronised write is harmless.
         void* p = nullptr;
         SF_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
         g_noalloc_ptr[device] = reinterpret_cast<NoAllocScratch*>(p);
@@ -476,6 +477,10 @@ extern "C" int sf_route_noalloc(int device, const sf_route_cfg* cfg, const float
     if (n > 0) {
         if (cfg->rule == SF_ABSMARGIN_LT)
             score_kernel<SF_ABSMARGIN_LT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast_out, score_out, sc->block_counts);
+        else if (cfg->rule == SF_ENTROPY_GT)
+            score_kernel<SF_ENTROPY_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast_out, score_out, sc->block_counts);
+        else if (cfg->rule == SF_SOFTMAX_LC_GT)
+            score_kernel<SF_SOFTMAX_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast_out, score_out, sc->block_counts);
         else
             score_kernel<SF_LC_GT><<<nb, kScoreBlock, 0, st>>>(fast_out, n, C, cfg->tau, dec, label_fast_out, score_out, sc->block_counts);
         SF_LAUNCH_CHECK("score_kernel");

@@ -13,12 +13,13 @@ namespace {
 template <bool RELU, int RM>
 __global__ void __launch_bounds__(256)
 dense_f32_kernel(const float* __restrict__ in, const float* __restrict__ W, const float* __restrict__ b,
-                 const uint32_t* __restrict__ n_rows_dev, uint32_t K, uint32_t N, float* __restrict__ out)
+                 const uint32_t* __restrict__ n_rows_dev, uint32_t K, uint32_t N, float* __restrict__ out,
+                 uint32_t capacity, sf_dev_state* st)
 {
     constexpr uint32_t TR = 16 * RM;               // rows per tile
     __shared__ float As[16][TR + 4];
     __shared__ float Bs[16][64 + 4];
-    const uint32_t n_rows = *n_rows_dev;
+    const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);
     const uint32_t r0 = blockIdx.x * TR, o0 = blockIdx.y * 64;
     if (r0 >= n_rows) return;
     const uint32_t tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
@@ -85,9 +86,9 @@ dense_f32_kernel(const float* __restrict__ in, const float* __restrict__ W, cons
 }
 
 __global__ void argmax_kernel(const float* __restrict__ logits, const uint32_t* __restrict__ n_rows_dev,
-                              uint32_t C, uint8_t* __restrict__ label)
+                              uint32_t C, uint8_t* __restrict__ label, uint32_t capacity)
 {
-    const uint32_t n_rows = *n_rows_dev;
+    const uint32_t n_rows = min(*n_rows_dev, capacity);
     for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < n_rows; r += gridDim.x * blockDim.x) {
         const float* p = logits + (size_t)r * C;
         uint32_t a = 0; float mx = p[0];
@@ -96,8 +97,8 @@ __global__ void argmax_kernel(const float* __restrict__ logits, const uint32_t* 
     }
 }
 
-__global__ void count_slow_kernel(const uint32_t* __restrict__ n_rows_dev, sf_dev_state* st) {
-    atomicAdd((unsigned long long*)&st->counters.n_slow_done, (unsigned long long)*n_rows_dev);
+__global__ void count_slow_kernel(const uint32_t* __restrict__ n_rows_dev, uint32_t capacity, sf_dev_state* st) {
+    atomicAdd((unsigned long long*)&st->counters.n_slow_done, (unsigned long long)min(*n_rows_dev, capacity));
 }
 
 void f32_to_bf16_host(const float* src, uint16_t* dst, size_t n) {
@@ -145,19 +146,19 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
             const bool small_tiles = (size_t)((capacity + 63) / 64) * ((N + 63) / 64) < 4u * (size_t)ctx->num_sms;
             if (small_tiles) {
                 dim3 grid((capacity + 31) / 32, (N + 63) / 64);
-                if (last) dense_f32_kernel<false, 2><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
-                else      dense_f32_kernel<true, 2><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
+                if (last) dense_f32_kernel<false, 2><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out, capacity, ctx->d_state);
+                else      dense_f32_kernel<true, 2><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out, capacity, ctx->d_state);
             } else {
                 dim3 grid((capacity + 63) / 64, (N + 63) / 64);
-                if (last) dense_f32_kernel<false, 4><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
-                else      dense_f32_kernel<true, 4><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out);
+                if (last) dense_f32_kernel<false, 4><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out, capacity, ctx->d_state);
+                else      dense_f32_kernel<true, 4><<<grid, 256, 0, st>>>(in, Wl, s->d_b[l], n_rows_dev, K, N, out, capacity, ctx->d_state);
             }
             SF_LAUNCH_CHECK("dense_f32_kernel");
             in = out;
         }
         if (label) {
             uint32_t blocks = (capacity + 255) / 256; if (blocks > 1184) blocks = 1184;
-            argmax_kernel<<<blocks, 256, 0, st>>>(logits, n_rows_dev, s->dims[s->n_layers], label);
+            argmax_kernel<<<blocks, 256, 0, st>>>(logits, n_rows_dev, s->dims[s->n_layers], label, capacity);
             SF_LAUNCH_CHECK("argmax_kernel");
         }
         sf_time_end(ctx, SF_T_HEAD, st);
@@ -165,7 +166,7 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
     }
     if (rc != SF_OK) return rc;
     if (count_done) {                                  // the streaming path adds the count in its own last kernel
-        count_slow_kernel<<<1, 1, 0, st>>>(n_rows_dev, ctx->d_state);
+        count_slow_kernel<<<1, 1, 0, st>>>(n_rows_dev, capacity, ctx->d_state);
         SF_LAUNCH_CHECK("count_slow_kernel");
     }
     return SF_OK;

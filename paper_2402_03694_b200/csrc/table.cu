@@ -487,7 +487,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
 {
     if (!ctx || !out) return SF_ERR_ARG;
     if (log2_slots < 4 || log2_slots > 28) return SF_ERR_ARG;
-    if (fast_pkts < 1 || fast_pkts > 32 || slow_pkts < fast_pkts || slow_pkts > 128 || slow_slabs < 1) return SF_ERR_ARG;
+    if (fast_pkts < 1 || fast_pkts > 32 || slow_pkts <= fast_pkts || slow_pkts > 128 || slow_slabs < 1) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
     sf_table* t = new (std::nothrow) sf_table();
     if (!t) return SF_ERR_ALLOC;

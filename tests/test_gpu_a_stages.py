@@ -351,6 +351,45 @@ def test_mlp_bf16_within_tolerance(env, dims, n_rows):
     sf.sf_slow_destroy(hd)
 
 
+@pytest.mark.parametrize("arch", ["mlp_f32", "mlp_bf16", "cnn"])
+def test_slow_model_row_count_above_capacity_is_clamped(env, arch):
+    """The row count is a device word of the caller.  A value above `capacity` must not make the
+    kernels read or write past the buffers: the first `capacity` rows are answered, nothing
+    beyond them is touched, and the context reports SF_ERR_CAPACITY."""
+    sf, hz, ctx = env
+    cap, guard = 150, 64
+    if arch == "cnn":
+        m = flowgen.gen_cnn(5, 128, 8, 64, 128, 5, 16)
+        rows = _cnn_rows(cap + guard, 9)
+        ref, _ = oracle.cnn(m, rows[:cap], True, threads=8)
+        h = sf.sf_cnn_create(ctx, sf.SF_BF16, m)
+        rt, n_cls, tol = hz.dev(rows).to(torch.bfloat16), 16, TOL_BF16
+    else:
+        bf = arch == "mlp_bf16"
+        dims = (256, 128, 128, 4)
+        m = flowgen.gen_mlp(6, dims)
+        rows = np.random.default_rng(4).uniform(0, 1, size=(cap + guard, dims[0])).astype(np.float32)
+        if bf:
+            rows = torch.from_numpy(rows).to(torch.bfloat16).float().numpy()      # exactly representable inputs
+        ref, _ = oracle.mlp(m, rows[:cap], bf, threads=8)
+        h = sf.sf_mlp_create(ctx, sf.SF_BF16 if bf else sf.SF_F32, m["dims"], m["W"], m["b"])
+        rt = hz.dev(rows).to(torch.bfloat16) if bf else hz.dev(rows)
+        n_cls, tol = 4, (TOL_BF16 if bf else TOL_F32)
+    cnt = hz.dev(np.array([cap + 5], np.uint32))
+    logits = torch.full((cap + guard, n_cls), float("nan"), dtype=torch.float32, device="cuda")
+    label = torch.full((cap + guard,), 255, dtype=torch.uint8, device="cuda")
+    sf.sf_ctx_poll(ctx, reset=True)
+    sf.sf_slow_infer(ctx, h, rt, cnt, cap, logits, label)
+    torch.cuda.synchronize()
+    c = sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    assert c.device_error == sf.SF_ERR_CAPACITY and c.n_slow_done == cap
+    lg, lb = logits.cpu().numpy(), label.cpu().numpy()
+    assert np.max(np.abs(lg[:cap] - ref)) <= tol
+    assert np.all(np.isnan(lg[cap:])) and np.all(lb[cap:] == 255)
+    assert sf.sf_ctx_poll(ctx).device_error == 0
+    sf.sf_slow_destroy(h)
+
+
 def test_create_rejects_unsupported_shapes(env):
     sf, hz, ctx = env
     W = [np.zeros((48, 100), np.float32), np.zeros((4, 48), np.float32)]
@@ -560,7 +599,7 @@ def test_route_softmax_least_confidence_within_tolerance(env):
 @pytest.mark.parametrize("kind", ["rf", "gbdt", "gbdt_mc"])
 def test_forest_threshold_edge_cases_bit_exact(env, kind):
     """Values equal to thresholds, one float apart from them, signed zeros, infinities and negative values:
-    the kernel compares through integer keys with a 26-bit fast path, so these are the cases that matter."""
+    the cases where a comparison that is not the plain fp32 `x <= thr` of the definition would go wrong."""
     sf, hz, ctx = env
     rng = np.random.default_rng(77)
     base = np.concatenate([rng.normal(size=40) * 10.0 ** rng.integers(-3, 9, 40), [0.0, -0.0, 1.0, -1.0, 40.0, 1500.0, 3e38, -3e38,

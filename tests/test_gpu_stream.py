@@ -211,6 +211,17 @@ def test_full_table_is_reported_not_fatal(env):
     sf.sf_forest_destroy(forest_h)
 
 
+def test_table_needs_a_slow_context_longer_than_the_fast_one(env):
+    """A slow model that fires at the packet count at which the fast model fires could never fire (the
+    decision is taken at that very packet): such a shape is refused instead of silently parking flows."""
+    sf, hz, ctx = env
+    for fast_pkts, slow_pkts in ((8, 8), (8, 7), (0, 8), (33, 64), (8, 129)):
+        with pytest.raises(sf.SfError) as e:
+            sf.sf_table_create(ctx, 6, fast_pkts, slow_pkts, 16)
+        assert e.value.status == sf.SF_ERR_ARG
+    sf.sf_table_destroy(sf.sf_table_create(ctx, 6, 8, 9, 16))
+
+
 # ---- table lifecycle: idle timeout, slot and slab reuse, re-arming ----
 def _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg):
     names = ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision", "missed")

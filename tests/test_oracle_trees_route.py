@@ -176,6 +176,20 @@ def test_margin_rule_matches_probability_rule():
         assert abs((1 - max(pp, 1 - pp)) - (0.5 - abs(pp - 0.5))) < 1e-12
 
 
+def test_sigmoid_closed_forms():
+    """The class-1 probability of a boosted binary model: values that are known in closed form, the
+    symmetry sigma(m) + sigma(-m) = 1, and monotonicity (a sign error or a dropped minus fails all three)."""
+    assert oracle.sigmoid(0.0) == 0.5
+    assert abs(oracle.sigmoid(math.log(3.0)) - 0.75) < 1e-15          # 1 / (1 + 1/3)
+    assert abs(oracle.sigmoid(-math.log(3.0)) - 0.25) < 1e-15
+    assert abs(oracle.sigmoid(math.log(7.0 / 3.0)) - 0.7) < 1e-15     # the 0.2 band of the binary rule
+    for m in (-20.0, -3.0, -0.5, 0.25, 2.0, 11.0):
+        assert abs(oracle.sigmoid(m) + oracle.sigmoid(-m) - 1.0) < 1e-15
+    xs = [-8.0, -1.0, -0.1, 0.0, 0.1, 1.0, 8.0]
+    ys = [oracle.sigmoid(x) for x in xs]
+    assert all(a < b for a, b in zip(ys, ys[1:])) and 0.0 < ys[0] and ys[-1] < 1.0
+
+
 def test_bf16_rounding_ties():
     assert oracle.bf16_round(1 + 2 ** -8) == 1.0                 # tie -> even (down)
     assert oracle.bf16_round(1 + 3 * 2 ** -8) == 1 + 2 ** -6     # tie -> even (up)

@@ -76,6 +76,12 @@ def test_noalloc_matches_route_on_two_calls_in_a_row():
             if with_dec:
                 assert np.array_equal(got["dec"], ref["dec"])
             assert int(got["status"][0]) == 0
+            # ... and what the CPU oracle gives (the existing entry point is CUDA too)
+            import oracle
+            o = oracle.route_lc(prob, tau)
+            assert o["n_esc"] == k and np.array_equal(got["ids"][:k], o["esc_ids"])
+            assert np.array_equal(got["lab"], o["label"])
+            assert np.array_equal(got["score"].view(np.uint32), o["score"].view(np.uint32))
         # the capacity error is reported through status_out, and cleared again by the next call
         prob, tau = _inputs(3, 20_000, 8)
         ref = _reference(sf, hz, ctx, prob, tau, 20_000)
@@ -104,3 +110,53 @@ def test_noalloc_rejects_sizes_beyond_its_scratch():
         sf.sf_route_noalloc(0, cfg, dummy, sf.SF_NOALLOC_MAX_FLOWS + 1, 4, ids, ids)
     assert e.value.status == sf.SF_ERR_STATIC_LIMIT
     assert "SF_NOALLOC_MAX_FLOWS" in str(e.value)
+
+
+def test_noalloc_margin_rule_and_empty_batch():
+    """The binary margin rule (|margin| < tau) and a batch of zero flows through the same entry point,
+    against the existing entry point and the oracle."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import oracle
+    from paper_2402_03694_b200 import build, binding as sf, harness as hz
+    build.build()
+    ctx = sf.sf_ctx_create(0, 0)
+    try:
+        n = 70_001
+        margin = (np.random.default_rng(5).normal(size=n) * 2.24).astype(np.float32)
+        tau = hz.dev(np.array([sf.SF_TAU_MARGIN_DEFAULT], np.float32))
+        cfg = sf.make_route_cfg(sf.SF_ABSMARGIN_LT, tau, sf.SF_MLP16, sf.SF_BF16, 64, n)
+        md = hz.dev(margin)
+
+        def buffers():
+            return (torch.full((n,), 0xFFFFFFFF, dtype=torch.uint32, device="cuda"), torch.zeros(1, dtype=torch.uint32, device="cuda"),
+                    torch.zeros(n, dtype=torch.uint8, device="cuda"), torch.zeros(n, dtype=torch.uint8, device="cuda"),
+                    torch.zeros(n, dtype=torch.float32, device="cuda"))
+        ids_r, ne_r, dec_r, lab_r, sc_r = buffers()
+        sf.sf_route(ctx, cfg, md, n, 1, None, ids_r, ne_r, None, dec_r, lab_r, sc_r)
+        ids, ne, dec, lab, sc = buffers()
+        status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
+        sf.sf_route_noalloc(0, cfg, md, n, 1, ids, ne, dec, lab, sc, status)
+        torch.cuda.synchronize()
+        o = oracle.route_absmargin(margin)
+        k = int(ne.cpu().numpy()[0])
+        assert k == o["n_esc"] == int(ne_r.cpu().numpy()[0]) and int(status.cpu().numpy()[0]) == 0
+        assert np.array_equal(ids.cpu().numpy()[:k], o["esc_ids"]) and np.array_equal(ids.cpu().numpy(), ids_r.cpu().numpy())
+        assert np.array_equal(dec.cpu().numpy(), o["decision"]) and np.array_equal(lab.cpu().numpy(), o["label"])
+        assert np.array_equal(sc.cpu().numpy().view(np.uint32), o["score"].view(np.uint32))
+        # zero flows: the count is written (0), nothing else is touched, no error
+        ids, ne, dec, lab, sc = buffers()
+        ne.fill_(9)
+        sf.sf_route_noalloc(0, cfg, md, 0, 1, ids, ne, dec, lab, sc, status)
+        torch.cuda.synchronize()
+        assert int(ne.cpu().numpy()[0]) == 0 and int(status.cpu().numpy()[0]) == 0
+        assert np.all(ids.cpu().numpy() == 0xFFFFFFFF)
+        # zero capacity: every assigned flow overflows, the count saturates at 0 and the status says so
+        cfg0 = sf.make_route_cfg(sf.SF_ABSMARGIN_LT, tau, sf.SF_MLP16, sf.SF_BF16, 64, 0)
+        sf.sf_route_noalloc(0, cfg0, md, n, 1, ids, ne, dec, lab, sc, status)
+        torch.cuda.synchronize()
+        assert int(ne.cpu().numpy()[0]) == 0 and int(status.cpu().numpy()[0]) == sf.SF_ERR_CAPACITY
+        assert np.all(ids.cpu().numpy() == 0xFFFFFFFF)
+        sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    finally:
+        sf.sf_ctx_destroy(ctx)
