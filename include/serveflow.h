@@ -392,6 +392,13 @@ void sf_table_destroy(sf_table* table);
 int  sf_table_ingest(sf_ctx* ctx, sf_table* table, const sf_pkt_batch* batch, const sf_forest* forest,
                      uint32_t F, const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_dev,
                      void* stream);
+/* Same, for a batch in HOST memory (pinned memory makes the copies asynchronous): every plane pointer of
+ * batch_host is a host pointer; the planes are copied to a device staging buffer of the context on
+ * `stream`, the batch is ingested, the counts are copied to *result_host_out (host) and the stream is
+ * synchronised.  cfg->tau stays a DEVICE pointer (thresholds belong to the model, not to the batch). */
+int  sf_table_ingest_host(sf_ctx* ctx, sf_table* table, const sf_pkt_batch* batch_host, const sf_forest* forest,
+                          uint32_t F, const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_host_out,
+                          void* stream);
 int  sf_table_lookup(sf_ctx* ctx, const sf_table* table, const sf_key* keys_dev, uint32_t n,
                      sf_flow_result* out_dev, void* stream);
 

@@ -85,7 +85,7 @@ EXPORTS = [
     "sf_route_noalloc",
     "sf_universal_thresholds", "sf_universal_thresholds_dev", "sf_per_class_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
     "sf_serve_batch", "sf_serve_batch3", "sf_serve_batch_host", "sf_serve_batch_intermediates",
-    "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_lookup", "sf_table_set_time", "sf_table_sweep",
+    "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_ingest_host", "sf_table_lookup", "sf_table_set_time", "sf_table_sweep",
 ]
 
 _L = None
@@ -131,6 +131,7 @@ def _lib():
         L.sf_serve_batch_intermediates.argtypes = [V] + [C.POINTER(V)] * 7
         L.sf_table_create.argtypes = [V, U32, U32, U32, U32, C.POINTER(V)]
         L.sf_table_ingest.argtypes = [V, V, C.POINTER(sf_pkt_batch), V, U32, V, C.POINTER(sf_route_cfg), V, V]
+        L.sf_table_ingest_host.argtypes = L.sf_table_ingest.argtypes
         L.sf_table_lookup.argtypes = [V, V, V, U32, V, V]
         L.sf_table_set_time.argtypes = [V, U32]
         L.sf_table_sweep.argtypes = [V, V, U32, U32, C.c_int, V, V]
@@ -366,6 +367,14 @@ def make_pkt_batch(src, dst, sport, dport, proto, dir_, size, iat_us, hdr, n=Non
 def sf_table_ingest(ctx, table, batch, forest, F, slow, cfg, result_dev, stream=None):
     _check(_lib().sf_table_ingest(ctx, table, C.byref(batch), forest, F, slow, C.byref(cfg), _dp(result_dev),
                                   _stream(stream)), "sf_table_ingest")
+
+
+def sf_table_ingest_host(ctx, table, batch_host, forest, F, slow, cfg, stream=None):
+    """batch_host: sf_pkt_batch of HOST planes (numpy or pinned torch tensors); returns the batch's counts."""
+    res = sf_batch_result()
+    _check(_lib().sf_table_ingest_host(ctx, table, C.byref(batch_host), forest, F, slow, C.byref(cfg), C.addressof(res),
+                                       _stream(stream)), "sf_table_ingest_host")
+    return res
 
 
 SWEEP_FIELDS = ("expired_pending", "expired_assigned", "expired_done", "rearmed", "live")     # first 5 of 8 uint32

@@ -26,6 +26,7 @@
 // Every loop is bounded; a key that finds no slot within the probe limit is counted as missed
 // and SF_ERR_TABLE_FULL is recorded in the context's error word.
 #include "common.cuh"
+#include <algorithm>
 #include <new>
 #include <string.h>
 
@@ -634,6 +635,48 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     if (rc != SF_OK) return rc;
     apply_slow_kernel<<<blocks, 256, 0, st>>>(d, t->fire2_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_slab_lab), result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("apply_slow_kernel");
+    return SF_OK;
+}
+
+// The same with a batch that lives in HOST memory: the nine planes are copied to the context's device
+// staging buffer on the stream (one copy per plane), the batch is ingested, the counts come back.
+extern "C" int sf_table_ingest_host(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bh, const sf_forest* fo, uint32_t F,
+                                    const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_host_out, void* stream)
+{
+    if (!ctx || !t || !bh || !result_host_out) return SF_ERR_ARG;
+    if (bh->n > kMaxBatch) return SF_ERR_ARG;
+    if (bh->n && (!bh->src || !bh->dst || !bh->sport || !bh->dport || !bh->proto || !bh->dir || !bh->size || !bh->iat_us || !bh->hdr))
+        return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = bh->n;
+    const void* src[9] = {bh->src, bh->dst, bh->sport, bh->dport, bh->proto, bh->dir, bh->size, bh->iat_us, bh->hdr};
+    const size_t bytes[9] = {n * 4, n * 4, n * 2, n * 2, n, n, n * 2, n * 4, n * kHdr};
+    size_t off[10], total = 0;
+    for (int i = 0; i < 9; i++) { off[i] = total; total += sf_align256(bytes[i]); }
+    off[9] = total; total += 256;                                        // the counts
+    if (total > ctx->stage_bytes) {
+        SF_CUDA(cudaDeviceSynchronize());
+        if (ctx->stage) { cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
+        const size_t want = std::max(total, (size_t)kMaxBatch * 40 + 4096);     // once: room for the largest batch
+        cudaError_t e = cudaMalloc(&ctx->stage, want);
+        if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(staging)"); return SF_ERR_ALLOC; }
+        ctx->stage_bytes = want;
+    }
+    char* sb = ctx->stage;
+    for (int i = 0; i < 9; i++)
+        if (bytes[i]) SF_CUDA(cudaMemcpyAsync(sb + off[i], src[i], bytes[i], cudaMemcpyHostToDevice, st));
+    sf_pkt_batch bd;
+    bd.src = (const uint32_t*)(sb + off[0]); bd.dst = (const uint32_t*)(sb + off[1]);
+    bd.sport = (const uint16_t*)(sb + off[2]); bd.dport = (const uint16_t*)(sb + off[3]);
+    bd.proto = (const uint8_t*)(sb + off[4]); bd.dir = (const uint8_t*)(sb + off[5]);
+    bd.size = (const uint16_t*)(sb + off[6]); bd.iat_us = (const uint32_t*)(sb + off[7]);
+    bd.hdr = (const uint8_t*)(sb + off[8]); bd.n = bh->n;
+    sf_batch_result* res_dev = reinterpret_cast<sf_batch_result*>(sb + off[9]);
+    int rc = sf_table_ingest(ctx, t, &bd, fo, F, slow, cfg, res_dev, stream);
+    if (rc != SF_OK) return rc;
+    SF_CUDA(cudaMemcpyAsync(result_host_out, res_dev, sizeof(sf_batch_result), cudaMemcpyDeviceToHost, st));
+    SF_CUDA(cudaStreamSynchronize(st));
     return SF_OK;
 }
 

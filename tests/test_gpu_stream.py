@@ -31,10 +31,17 @@ def _models(F, T, depth, C, dims, seed):
     return forest, tau, flowgen.gen_mlp(seed, dims)
 
 
-def _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg):
+def _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg, host=False):
     totals = np.zeros(8, np.int64)
     res = torch.zeros(8, dtype=torch.int32, device="cuda")
+    names8 = ("n_new_flows", "n_fast_fired", "n_fast_done", "n_escalated", "n_slow_fired", "n_dropped_after_decision", "n_missed")
     for b in batches:
+        if host:                  # the host-pointer entry point: numpy planes in, counts back
+            h = {k: np.ascontiguousarray(b[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
+            pb = sf.make_pkt_batch(h["src"], h["dst"], h["sport"], h["dport"], h["proto"], h["dir"], h["size"], h["iat_us"], h["hdr"])
+            r = sf.sf_table_ingest_host(ctx, table, pb, forest_h, F, slow_h, rcfg)
+            totals[:7] += np.array([getattr(r, k) for k in names8], np.int64)
+            continue
         d = {k: hz.dev(b[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
         pb = sf.make_pkt_batch(d["src"], d["dst"], d["sport"], d["dport"], d["proto"], d["dir"], d["size"], d["iat_us"], d["hdr"])
         sf.sf_table_ingest(ctx, table, pb, forest_h, F, slow_h, rcfg, res)
@@ -55,9 +62,11 @@ def _lookup(sf, hz, ctx, table, keys):
     return out.cpu().numpy().reshape(-1).view(sf.FLOW_RESULT_DTYPE)
 
 
-@pytest.mark.parametrize("shape", ["config5_models", "small_models", "odd_models"])
+@pytest.mark.parametrize("shape", ["config5_models", "small_models", "odd_models", "small_models_host"])
 def test_stream_matches_sequential_reference(env, shape):
     sf, hz, ctx = env
+    host = shape.endswith("_host")
+    shape = shape.replace("_host", "")
     if shape == "config5_models":       # config 2's forest on 8 packets, config 2's MLP on 64 packets padded to 128
         F, T, depth, C, dims, P_model = 48, 100, 12, 8, (2048, 1024, 1024, 1024, 8), 128
         n_keys, n_batches, m = 1500, 24, 4096
@@ -79,7 +88,7 @@ def test_stream_matches_sequential_reference(env, shape):
     table = sf.sf_table_create(ctx, 13, fast_pkts, slow_pkts, n_keys)
     rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
     sf.sf_ctx_poll(ctx, reset=True)
-    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg)
+    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg, host=host)
     c = sf.sf_ctx_poll(ctx, reset=True)
     assert got["missed"] == 0 and c.device_error == 0
     for k in ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision"):
