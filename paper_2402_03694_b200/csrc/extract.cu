@@ -1,55 +1,116 @@
 // S1: per-flow statistical features of the first N packet headers.
 //
-// One thread per flow.  A thread streams its packets in chunks of 8 (16-byte
-// vector loads of the uint16 sizes and uint32 inter-arrival times when the row
-// pitch allows it), keeps one integer accumulator set per feature group in
-// registers (subset membership, counts, first and last come from bit masks of the
-// direction word), converts once at the end, and the block hands its [flows][F] tile to
+// One thread per flow.  A thread loads its packets in chunks of 8 (16-byte vector loads of
+// the uint16 sizes and uint32 inter-arrival times when the row pitch allows it; the next chunk
+// is fetched while the current one is reduced, and the chunk loop is not unrolled, so that its
+// body stays in the instruction cache and the register count stays below 100) and keeps one
+// integer accumulator set per feature group in registers.  Subset membership (forward,
+// backward, direction change) comes from the direction word: a packet's bit becomes one
+// predicate per word, under which the subset's min, max and sums are updated without selects
+// or branches.  The 96-bit sum of squared inter-arrival times is kept as two 64-bit sums (of
+// the low and of the high words of the 64-bit squares) and joined at the end.  Counts, first
+// and last come from the masks (popcount / lowest / highest set bit).  Sums of the backward
+// subsets are (all - forward): exact, because everything is an integer.
+// Each fp32 value is produced by exactly one rounding (integer -> fp32 RNE) or one IEEE
+// division, so results are reproducible bit for bit.  The block hands its [flows][F] tile to
 // global memory through shared memory so that the stores are fully coalesced.
-// All statistics come from exact integer sums (128-bit for the variance numerator
-// of inter-arrival times); each fp32 value is produced by exactly one rounding
-// (integer -> fp32 RNE) or one IEEE division, so results are reproducible bit for bit.
+// The kernel is bound by integer issue, not by HBM: min/max/add/logic and the multiply-adds run on
+// two half-rate pipes, and a 64-bit accumulation costs three instructions on this target.
 #include "common.cuh"
 
 namespace {
 
 constexpr int kFlowsPerBlock = 32;       // one warp per block: small blocks schedule better here than 64- or 128-flow ones (measured)
 
-// Integer accumulators of one (quantity, subset) group.  Counts, first and last come from
-// the subset's bit mask (popcount / lowest / highest set bit), so the per-packet work is
-// two selects, a min, a max and the exact sums.
+// size groups (g0 all, g2 forward, g6 direction change): 16-bit values, at most 32 of them, so the sum fits 32 bits
+struct SizeAcc { uint32_t mn, mx, s1; uint64_t s2; };
+// inter-arrival groups (g1 all, g4 forward, g7 direction change): 32-bit values; sum of squares = s2a + s2b * 2^32
+struct IatAcc { uint32_t mn, mx; uint64_t s1, s2a, s2b; };
+// backward groups (g3 size, g5 inter-arrival): only min and max are accumulated, the sums are (all - forward)
+struct MinMax { uint32_t mn, mx; };
+
 struct Acc {
-    uint32_t mn, mx;
-    uint64_t s1;        // sum
-    uint64_t s2lo;      // sum of squares, low 64 bits
-    uint32_t s2hi;      // high part (only inter-arrival times can carry into it)
+    SizeAcc z0, z2, z6;
+    IatAcc a1, a4, a7;
+    MinMax m3, m5;
 };
 
-__device__ __forceinline__ void acc_init(Acc& a) { a.mn = 0xFFFFFFFFu; a.mx = 0; a.s1 = 0; a.s2lo = 0; a.s2hi = 0; }
+__device__ __forceinline__ void acc_init(Acc& A) {
+    A.z0 = A.z2 = A.z6 = SizeAcc{0xFFFFFFFFu, 0u, 0u, 0ull};
+    A.a1 = A.a4 = A.a7 = IatAcc{0xFFFFFFFFu, 0u, 0ull, 0ull, 0ull};
+    A.m3 = A.m5 = MinMax{0xFFFFFFFFu, 0u};
+}
 
-// sizes (16 bit): the square fits 32 bits and the sums never carry out of 64 bits
-__device__ __forceinline__ void add_size(Acc& a, uint32_t x, bool take) {
-    const uint32_t x0 = take ? x : 0u, xm = take ? x : 0xFFFFFFFFu;
-    a.mn = min(a.mn, xm);
-    a.mx = max(a.mx, x0);
-    a.s1 += x0;
-    a.s2lo += (uint64_t)(x0 * x0);
+// c + a with a 64-bit c and a 32-bit a, written as the widening multiply-add a * 1 + c
+__device__ __forceinline__ uint64_t add_wide(uint64_t c, uint32_t a) {
+    uint64_t d;
+    asm("mad.wide.u32 %0, %1, 1, %2;" : "=l"(d) : "r"(a), "l"(c));
+    return d;
 }
-// inter-arrival times (32 bit): 64-bit squares, 128-bit sum of squares
-__device__ __forceinline__ void add_iat(Acc& a, uint32_t x, bool take) {
-    const uint32_t x0 = take ? x : 0u, xm = take ? x : 0xFFFFFFFFu;
-    a.mn = min(a.mn, xm);
-    a.mx = max(a.mx, x0);
-    a.s1 += x0;
-    const uint64_t sq = (uint64_t)x0 * (uint64_t)x0;
-    const uint64_t lo = a.s2lo + sq;
-    a.s2hi += (lo < sq) ? 1u : 0u;
-    a.s2lo = lo;
+
+// Masked updates of one packet, one predicate per direction word: p = forward (bit clear) for the direction groups,
+// p = direction change (bit set) for the turn groups; the updates are predicated, nothing is selected or branched.
+#define SZ_UPD(P, mn, mx, s1, s2, x, sq) P " min.u32 " mn ", " mn ", " x ";\n" P " max.u32 " mx ", " mx ", " x ";\n" P " add.u32 " s1 ", " s1 ", " x ";\n" P " mad.wide.u32 " s2 ", " sq ", 1, " s2 ";\n"
+#define IA_UPD(P, mn, mx, s1, s2a, s2b, x, plo, phi) P " min.u32 " mn ", " mn ", " x ";\n" P " max.u32 " mx ", " mx ", " x ";\n" P " mad.wide.u32 " s1 ", " x ", 1, " s1 ";\n" P " mad.wide.u32 " s2a ", " plo ", 1, " s2a ";\n" P " mad.wide.u32 " s2b ", " phi ", 1, " s2b ";\n"
+#define MM_UPD(P, mn, mx, x) P " min.u32 " mn ", " mn ", " x ";\n" P " max.u32 " mx ", " mx ", " x ";\n"
+#define PRED_EQ(word, bit) "{\n.reg .pred p;\n.reg .b32 t;\nand.b32 t, " word ", " bit ";\nsetp.eq.u32 p, t, 0;\n"
+#define PRED_NE(word, bit) "{\n.reg .pred p;\n.reg .b32 t;\nand.b32 t, " word ", " bit ";\nsetp.ne.u32 p, t, 0;\n"
+
+template <int G>
+__device__ __forceinline__ void dir_groups(Acc& A, uint32_t sz, uint32_t sq, uint32_t ia, uint32_t plo, uint32_t phi, uint32_t dirw, uint32_t bit) {
+    if (G >= 6)
+        asm(PRED_EQ("%18", "%19") SZ_UPD("@p", "%0", "%1", "%2", "%3", "%13", "%14") MM_UPD("@!p", "%4", "%5", "%13")
+            IA_UPD("@p", "%6", "%7", "%8", "%9", "%10", "%15", "%16", "%17") MM_UPD("@!p", "%11", "%12", "%15") "}"
+            : "+r"(A.z2.mn), "+r"(A.z2.mx), "+r"(A.z2.s1), "+l"(A.z2.s2), "+r"(A.m3.mn), "+r"(A.m3.mx), "+r"(A.a4.mn), "+r"(A.a4.mx),
+              "+l"(A.a4.s1), "+l"(A.a4.s2a), "+l"(A.a4.s2b), "+r"(A.m5.mn), "+r"(A.m5.mx)
+            : "r"(sz), "r"(sq), "r"(ia), "r"(plo), "r"(phi), "r"(dirw), "r"(bit));
+    else if (G == 5)
+        asm(PRED_EQ("%16", "%17") SZ_UPD("@p", "%0", "%1", "%2", "%3", "%11", "%12") MM_UPD("@!p", "%4", "%5", "%11")
+            IA_UPD("@p", "%6", "%7", "%8", "%9", "%10", "%13", "%14", "%15") "}"
+            : "+r"(A.z2.mn), "+r"(A.z2.mx), "+r"(A.z2.s1), "+l"(A.z2.s2), "+r"(A.m3.mn), "+r"(A.m3.mx), "+r"(A.a4.mn), "+r"(A.a4.mx),
+              "+l"(A.a4.s1), "+l"(A.a4.s2a), "+l"(A.a4.s2b)
+            : "r"(sz), "r"(sq), "r"(ia), "r"(plo), "r"(phi), "r"(dirw), "r"(bit));
+    else if (G == 4)
+        asm(PRED_EQ("%8", "%9") SZ_UPD("@p", "%0", "%1", "%2", "%3", "%6", "%7") MM_UPD("@!p", "%4", "%5", "%6") "}"
+            : "+r"(A.z2.mn), "+r"(A.z2.mx), "+r"(A.z2.s1), "+l"(A.z2.s2), "+r"(A.m3.mn), "+r"(A.m3.mx)
+            : "r"(sz), "r"(sq), "r"(dirw), "r"(bit));
+    else if (G == 3)
+        asm(PRED_EQ("%6", "%7") SZ_UPD("@p", "%0", "%1", "%2", "%3", "%4", "%5") "}"
+            : "+r"(A.z2.mn), "+r"(A.z2.mx), "+r"(A.z2.s1), "+l"(A.z2.s2)
+            : "r"(sz), "r"(sq), "r"(dirw), "r"(bit));
 }
-// min / max only (the sums of the complementary subset come from a subtraction)
-__device__ __forceinline__ void add_minmax(Acc& a, uint32_t x, bool take) {
-    a.mn = min(a.mn, take ? x : 0xFFFFFFFFu);
-    a.mx = max(a.mx, take ? x : 0u);
+template <int G>
+__device__ __forceinline__ void turn_groups(Acc& A, uint32_t sz, uint32_t sq, uint32_t ia, uint32_t plo, uint32_t phi, uint32_t turnw, uint32_t bit) {
+    if (G >= 8)
+        asm(PRED_NE("%14", "%15") SZ_UPD("@p", "%0", "%1", "%2", "%3", "%9", "%10") IA_UPD("@p", "%4", "%5", "%6", "%7", "%8", "%11", "%12", "%13") "}"
+            : "+r"(A.z6.mn), "+r"(A.z6.mx), "+r"(A.z6.s1), "+l"(A.z6.s2), "+r"(A.a7.mn), "+r"(A.a7.mx), "+l"(A.a7.s1), "+l"(A.a7.s2a), "+l"(A.a7.s2b)
+            : "r"(sz), "r"(sq), "r"(ia), "r"(plo), "r"(phi), "r"(turnw), "r"(bit));
+    else if (G == 7)
+        asm(PRED_NE("%6", "%7") SZ_UPD("@p", "%0", "%1", "%2", "%3", "%4", "%5") "}"
+            : "+r"(A.z6.mn), "+r"(A.z6.mx), "+r"(A.z6.s1), "+l"(A.z6.s2)
+            : "r"(sz), "r"(sq), "r"(turnw), "r"(bit));
+}
+#undef SZ_UPD
+#undef IA_UPD
+#undef MM_UPD
+#undef PRED_EQ
+#undef PRED_NE
+
+// One packet of the window.  Groups: g0 size/all, g1 iat/all, g2 size/fwd, g3 size/bwd, g4 iat/fwd, g5 iat/bwd,
+// g6 size/turn, g7 iat/turn.  dirw: bit set = backward packet; turnw: bit set = direction differs from the packet before.
+template <int G>
+__device__ __forceinline__ void packet(Acc& A, uint32_t sz, uint32_t ia, uint32_t dirw, uint32_t turnw, uint32_t bit) {
+    const uint32_t sq = sz * sz;                                  // 16-bit sizes: the square fits 32 bits
+    A.z0.mn = min(A.z0.mn, sz); A.z0.mx = max(A.z0.mx, sz); A.z0.s1 += sz; A.z0.s2 = add_wide(A.z0.s2, sq);
+    uint32_t plo = 0, phi = 0;
+    if (G > 1) {
+        const uint64_t p = (uint64_t)ia * (uint64_t)ia;
+        plo = (uint32_t)p; phi = (uint32_t)(p >> 32);
+        A.a1.mn = min(A.a1.mn, ia); A.a1.mx = max(A.a1.mx, ia);
+        A.a1.s1 = add_wide(A.a1.s1, ia); A.a1.s2a = add_wide(A.a1.s2a, plo); A.a1.s2b = add_wide(A.a1.s2b, phi);
+    }
+    if (G > 2) dir_groups<G>(A, sz, sq, ia, plo, phi, dirw, bit);
+    if (G > 6) turn_groups<G>(A, sz, sq, ia, plo, phi, turnw, bit);
 }
 
 // exact unsigned 128-bit value (hi:lo) -> fp32, round to nearest even.
@@ -67,17 +128,30 @@ __device__ __forceinline__ float u128_to_f32(uint64_t hi, uint64_t lo) {
 }
 
 // eight slots of one group: cnt, sum, min, max, mean, var, first, last
-__device__ __forceinline__ void finish(uint32_t cnt, uint32_t mn, uint32_t mx, uint64_t s1, uint64_t s2lo, uint64_t s2hi,
-                                       uint32_t first, uint32_t last, float* o) {
+__device__ __forceinline__ void store_slots(float* o, float fc, float fs, uint32_t mn, uint32_t mx, float fv, uint32_t cnt,
+                                            uint32_t first, uint32_t last) {
     float4* o4 = reinterpret_cast<float4*>(o);       // 16-byte stores: conflict-free across a quarter warp
-    if (cnt == 0) {
-        o4[0] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        o4[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        return;
-    }
-    const float fc = __uint2float_rn(cnt);
-    const float fs = __ull2float_rn(s1);
-    // V = cnt * S2 - S1^2 as an exact 128-bit integer
+    o4[0] = make_float4(fc, fs, __uint2float_rn(mn), __uint2float_rn(mx));
+    o4[1] = make_float4(__fdiv_rn(fs, fc), __fdiv_rn(fv, __uint2float_rn(cnt * cnt)), __uint2float_rn(first), __uint2float_rn(last));
+}
+__device__ __forceinline__ void store_empty(float* o) {
+    float4* o4 = reinterpret_cast<float4*>(o);
+    o4[0] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    o4[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+}
+// size group: S1 < 2^21 and cnt * S2, S1^2 < 2^42, so the variance numerator V = cnt * S2 - S1^2 is a 64-bit integer
+__device__ __forceinline__ void finish_size(uint32_t cnt, uint32_t mn, uint32_t mx, uint32_t s1, uint64_t s2,
+                                            uint32_t first, uint32_t last, float* o) {
+    if (cnt == 0) { store_empty(o); return; }
+    const uint64_t v = (uint64_t)cnt * s2 - (uint64_t)s1 * (uint64_t)s1;
+    store_slots(o, __uint2float_rn(cnt), __uint2float_rn(s1), mn, mx, __ull2float_rn(v), cnt, first, last);
+}
+// inter-arrival group: S2 = s2a + s2b * 2^32 (up to 2^69), V = cnt * S2 - S1^2 as an exact 128-bit integer
+__device__ __forceinline__ void finish_iat(uint32_t cnt, uint32_t mn, uint32_t mx, uint64_t s1, uint64_t s2a, uint64_t s2b,
+                                           uint32_t first, uint32_t last, float* o) {
+    if (cnt == 0) { store_empty(o); return; }
+    const uint64_t s2lo = s2a + (s2b << 32);
+    const uint64_t s2hi = (s2b >> 32) + ((s2lo < s2a) ? 1ull : 0ull);
     const uint64_t c = cnt;
     const uint64_t p_lo = c * s2lo;
     const uint64_t p_hi = __umul64hi(c, s2lo) + c * s2hi;
@@ -85,25 +159,7 @@ __device__ __forceinline__ void finish(uint32_t cnt, uint32_t mn, uint32_t mx, u
     const uint64_t q_hi = __umul64hi(s1, s1);
     const uint64_t v_lo = p_lo - q_lo;
     const uint64_t v_hi = p_hi - q_hi - ((p_lo < q_lo) ? 1ull : 0ull);
-    o4[0] = make_float4(fc, fs, __uint2float_rn(mn), __uint2float_rn(mx));
-    o4[1] = make_float4(__fdiv_rn(fs, fc), __fdiv_rn(u128_to_f32(v_hi, v_lo), __uint2float_rn(cnt * cnt)),
-                        __uint2float_rn(first), __uint2float_rn(last));
-}
-
-// Groups: g0 size/all, g1 iat/all, g2 size/fwd, g3 size/bwd, g4 iat/fwd, g5 iat/bwd, g6 size/turn, g7 iat/turn.
-// Sums of the backward subsets are (all - forward): exact, because everything is an integer.
-template <int G>
-__device__ __forceinline__ void packet(Acc (&A)[8], uint32_t sz, uint32_t ia, uint32_t i, uint32_t fwd_mask, uint32_t turn_mask) {
-    const bool f = (fwd_mask >> i) & 1u;
-    const bool tn = (turn_mask >> i) & 1u;
-    add_size(A[0], sz, true);
-    if (G > 1) add_iat(A[1], ia, true);
-    if (G > 2) add_size(A[2], sz, f);
-    if (G > 3) add_minmax(A[3], sz, !f);
-    if (G > 4) add_iat(A[4], ia, f);
-    if (G > 5) add_minmax(A[5], ia, !f);
-    if (G > 6) add_size(A[6], sz, tn);
-    if (G > 7) add_iat(A[7], ia, tn);
+    store_slots(o, __uint2float_rn(cnt), __ull2float_rn(s1), mn, mx, u128_to_f32(v_hi, v_lo), cnt, first, last);
 }
 
 // VEC: row pitch is a multiple of 8 packets, so size rows are 16-byte aligned
@@ -125,45 +181,43 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
 
     if (f < n) {
         const size_t fr = row_ids ? row_ids[f] : f;      // optional indirection: flow f's packets sit in row row_ids[f] of the planes
-        Acc A[8];
-#pragma unroll
-        for (int g = 0; g < 8; g++) acc_init(A[g]);
+        Acc A;
+        acc_init(A);
         uint32_t m = N;
         if (n_valid) m = min(m, (uint32_t)n_valid[fr]);
         // N <= 32: all direction bits of the window are in the row's first word
         const uint32_t dirw = dir_bits[fr * ((pitch + 31) >> 5)];
+        const uint32_t turnw = (dirw ^ (dirw << 1)) & ~1u;        // packet i >= 1 whose direction differs from i-1
         const uint32_t all_mask = (m >= 32) ? 0xFFFFFFFFu : ((1u << m) - 1u);
-        const uint32_t fwd_mask = ~dirw & all_mask;
-        const uint32_t bwd_mask = dirw & all_mask;
-        const uint32_t turn_mask = (dirw ^ (dirw << 1)) & ~1u & all_mask;        // packet i >= 1 whose direction differs from i-1
         const uint16_t* srow = size + fr * pitch;
         const uint32_t* irow = iat + fr * pitch;
+        uint32_t done = 0;                             // packets accumulated so far
         if (VEC) {
-            // issue every load of the window first (N <= 32: at most four chunks of eight packets), then reduce
-            uint4 s4[4], a4[4], b4[4];
-#pragma unroll
-            for (int ch = 0; ch < 4; ch++) {
-                if ((uint32_t)ch * 8 < m) {
-                    s4[ch] = __ldg(reinterpret_cast<const uint4*>(srow + ch * 8));
-                    a4[ch] = __ldg(reinterpret_cast<const uint4*>(irow + ch * 8));
-                    b4[ch] = __ldg(reinterpret_cast<const uint4*>(irow + ch * 8 + 4));
-                }
+            const uint32_t n_full = m >> 3;
+            uint4 s4, a4, b4;
+            if (n_full) {
+                s4 = __ldg(reinterpret_cast<const uint4*>(srow)); a4 = __ldg(reinterpret_cast<const uint4*>(irow));
+                b4 = __ldg(reinterpret_cast<const uint4*>(irow + 4));
             }
-#pragma unroll
-            for (int ch = 0; ch < 4; ch++) {
-                if ((uint32_t)ch * 8 < m) {
-                    const uint32_t sz[8] = {s4[ch].x & 0xFFFFu, s4[ch].x >> 16, s4[ch].y & 0xFFFFu, s4[ch].y >> 16,
-                                            s4[ch].z & 0xFFFFu, s4[ch].z >> 16, s4[ch].w & 0xFFFFu, s4[ch].w >> 16};
-                    const uint32_t ia[8] = {a4[ch].x, a4[ch].y, a4[ch].z, a4[ch].w, b4[ch].x, b4[ch].y, b4[ch].z, b4[ch].w};
-#pragma unroll
-                    for (int j = 0; j < 8; j++)
-                        if ((uint32_t)(ch * 8 + j) < m) packet<G>(A, sz[j], ia[j], ch * 8 + j, fwd_mask, turn_mask);
+#pragma unroll 1
+            for (uint32_t ch = 0; ch < n_full; ch++) {
+                const uint4 cs = s4, ca = a4, cb = b4;
+                if (ch + 1 < n_full) {
+                    s4 = __ldg(reinterpret_cast<const uint4*>(srow + (ch + 1) * 8)); a4 = __ldg(reinterpret_cast<const uint4*>(irow + (ch + 1) * 8));
+                    b4 = __ldg(reinterpret_cast<const uint4*>(irow + (ch + 1) * 8 + 4));
                 }
+                const uint32_t sz[8] = {cs.x & 0xFFFFu, cs.x >> 16, cs.y & 0xFFFFu, cs.y >> 16, cs.z & 0xFFFFu, cs.z >> 16, cs.w & 0xFFFFu, cs.w >> 16};
+                const uint32_t ia[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+                const uint32_t dw = dirw >> (8 * ch), tw = turnw >> (8 * ch);
+#pragma unroll
+                for (int j = 0; j < 8; j++) packet<G>(A, sz[j], ia[j], dw, tw, 1u << j);
             }
-        } else {
-            for (uint32_t i = 0; i < m; i++) packet<G>(A, srow[i], irow[i], i, fwd_mask, turn_mask);
+            done = n_full * 8;
         }
+        for (uint32_t i = done; i < m; i++) packet<G>(A, srow[i], irow[i], dirw, turnw, 1u << i);      // ragged end / unaligned rows
+
         float* o = tile + threadIdx.x * STRIDE;
+        const uint32_t fwd_mask = ~dirw & all_mask, bwd_mask = dirw & all_mask, turn_mask = turnw & all_mask;
 #pragma unroll
         for (int g = 0; g < G; g++) {
             const uint32_t mask = (g < 2) ? all_mask : (g == 2 || g == 4) ? fwd_mask : (g == 3 || g == 5) ? bwd_mask : turn_mask;
@@ -175,15 +229,15 @@ extract_kernel(const uint16_t* __restrict__ size, const uint32_t* __restrict__ i
                 first = is_size ? (uint32_t)srow[i0] : irow[i0];
                 last = is_size ? (uint32_t)srow[i1] : irow[i1];
             }
-            uint64_t s1 = A[g].s1, s2lo = A[g].s2lo, s2hi = A[g].s2hi;
-            if (g == 3 || g == 5) {                  // backward = all - forward
-                const Acc& all = A[g == 3 ? 0 : 1];
-                const Acc& fw = A[g == 3 ? 2 : 4];
-                s1 = all.s1 - fw.s1;
-                s2lo = all.s2lo - fw.s2lo;
-                s2hi = (uint64_t)all.s2hi - fw.s2hi - ((all.s2lo < fw.s2lo) ? 1u : 0u);
-            }
-            finish(cnt, A[g].mn, A[g].mx, s1, s2lo, s2hi, first, last, o + 8 * g);
+            float* og = o + 8 * g;
+            if (g == 0) finish_size(cnt, A.z0.mn, A.z0.mx, A.z0.s1, A.z0.s2, first, last, og);
+            else if (g == 1) finish_iat(cnt, A.a1.mn, A.a1.mx, A.a1.s1, A.a1.s2a, A.a1.s2b, first, last, og);
+            else if (g == 2) finish_size(cnt, A.z2.mn, A.z2.mx, A.z2.s1, A.z2.s2, first, last, og);
+            else if (g == 3) finish_size(cnt, A.m3.mn, A.m3.mx, A.z0.s1 - A.z2.s1, A.z0.s2 - A.z2.s2, first, last, og);
+            else if (g == 4) finish_iat(cnt, A.a4.mn, A.a4.mx, A.a4.s1, A.a4.s2a, A.a4.s2b, first, last, og);
+            else if (g == 5) finish_iat(cnt, A.m5.mn, A.m5.mx, A.a1.s1 - A.a4.s1, A.a1.s2a - A.a4.s2a, A.a1.s2b - A.a4.s2b, first, last, og);
+            else if (g == 6) finish_size(cnt, A.z6.mn, A.z6.mx, A.z6.s1, A.z6.s2, first, last, og);
+            else finish_iat(cnt, A.a7.mn, A.a7.mx, A.a7.s1, A.a7.s2a, A.a7.s2b, first, last, og);
         }
     }
     __syncthreads();
