@@ -123,6 +123,11 @@ int sf_launch_compose_ids(const uint32_t* ids1, const uint32_t* ids2_local, cons
 int sf_launch_forest_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st,
                                 const uint32_t* n_dev);
 
+// the same with the features computed inside the kernel from the flows' packets (rows row_ids[0..n) of pk, first N packets);
+// SF_ERR_UNSUPPORTED when the planes are not laid out for it (the caller then runs the two kernels)
+int sf_launch_forest_leaf_index_packets(const sf_forest* fo, const sf_packets* pk, uint32_t N, const uint32_t* row_ids, uint32_t n,
+                                        uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev);
+
 // bf16 tensor-core layers (gemm_tc.cu)
 int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32_t* n_rows_dev, uint32_t capacity,
                         float* logits, uint8_t* label, void* scratch, cudaStream_t st);

@@ -24,6 +24,7 @@
 // The streaming path, where a launch carries a few hundred flows, has kernels of its own further down
 // (trees spread over the grid as well as flows).
 #include "tc_common.cuh"
+#include "extract_device.cuh"
 #include <algorithm>
 #include <new>
 #include <stdlib.h>
@@ -290,11 +291,16 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
 // (tile of 128 flows, slice of trees that fits one buffer); persistent blocks take items in turn, walk the slice
 // and write each tree's leaf index.  A second kernel then adds every flow's leaf vectors in tree order
 // t = 0..T-1 (the same fp32 sums, bit for bit, as the fused kernel) and divides by T.
-template <int NCH>
+// G > 0: the features are not read from `feat` but computed here, straight into the tile, from the flows' packets
+// (8 * G statistics of the first N packets of row row_ids[f] of the planes pk; rows 16-byte aligned, no n_valid):
+// one launch less on a path whose cost is launch latency.
+struct LeafIndexPackets { const uint16_t* size; const uint32_t* iat; const uint32_t* dir_bits; const uint32_t* row_ids; uint32_t pitch, N; };
+
+template <int NCH, int G>
 __global__ void __launch_bounds__(kBSmall, 2)
 forest_leaf_index_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F, const unsigned char* __restrict__ image,
                          uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_item, uint32_t buf_bytes,
-                         uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev)
+                         uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev, LeafIndexPackets pk)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (n_dev) n = min(n, *n_dev);
@@ -319,8 +325,17 @@ forest_leaf_index_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         const uint32_t f = tile * kBSmall + threadIdx.x;
         const bool live = f < n;
         if (tile != tile_loaded) {                          // every thread reads its own column only
-            if (live) for (uint32_t j = 0; j < F; j++) xs[j * kBSmall + threadIdx.x] = __ldg(feat + (size_t)f * F + j);
-            else for (uint32_t j = 0; j < F; j++) xs[j * kBSmall + threadIdx.x] = 0.0f;
+            if (live) {
+                if (G > 0) {
+                    const size_t fr = pk.row_ids ? pk.row_ids[f] : f;
+                    sfx::extract_flow<(G > 0 ? G : 1), true>(pk.size, pk.iat, fr, pk.pitch, pk.N, pk.dir_bits[fr * ((pk.pitch + 31) >> 5)],
+                                                             sfx::ColOut{xs + threadIdx.x, kBSmall});
+                } else {
+                    for (uint32_t j = 0; j < F; j++) xs[j * kBSmall + threadIdx.x] = __ldg(feat + (size_t)f * F + j);
+                }
+            } else {
+                for (uint32_t j = 0; j < F; j++) xs[j * kBSmall + threadIdx.x] = 0.0f;
+            }
             tile_loaded = tile;
         }
         if (!sftc::mbar_wait(bar, it & 1u, abort_flag)) break;
@@ -427,7 +442,9 @@ int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, ui
     return launch3<SF_GBDT_MC, C, (C >= 4 ? 4 : (C >= 2 ? 2 : 1))>(fo, p, feat, n, out, leaf_idx, st, n_dev);
 }
 
-int launch_rf_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+template <int G>
+int launch_rf_leaf_index_g(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
+                           const LeafIndexPackets& pk) {
     const size_t feat_bytes = (size_t)fo->F * kBSmall * sizeof(float);
     uint32_t buf = 65536u;
     uint32_t tpi = buf / fo->tree_stride;
@@ -439,15 +456,19 @@ int launch_rf_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uin
     static size_t smem_set_dev[64] = {};
     size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
     if (smem > smem_set) {
-        SF_CUDA(cudaFuncSetAttribute(forest_leaf_index_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        SF_CUDA(cudaFuncSetAttribute(forest_leaf_index_kernel<2, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         smem_set = smem;
     }
     const uint32_t n_items = ((n + kBSmall - 1) / kBSmall) * ((fo->T + tpi - 1) / tpi);
     const uint32_t grid = std::min<uint32_t>(n_items, (uint32_t)fo->ctx->num_sms * 2u);
-    forest_leaf_index_kernel<2><<<grid, kBSmall, smem, st>>>(feat, n, fo->F, fo->d_image_small, fo->T, fo->depth, fo->tree_stride, tpi, buf,
-                                                           leaf_idx, fo->ctx->d_state, n_dev);
+    forest_leaf_index_kernel<2, G><<<grid, kBSmall, smem, st>>>(feat, n, fo->F, fo->d_image_small, fo->T, fo->depth, fo->tree_stride, tpi, buf,
+                                                              leaf_idx, fo->ctx->d_state, n_dev, pk);
     SF_LAUNCH_CHECK("forest_leaf_index_kernel");
     return SF_OK;
+}
+
+int launch_rf_leaf_index(const sf_forest* fo, const float* feat, uint32_t n, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+    return launch_rf_leaf_index_g<0>(fo, feat, n, leaf_idx, st, n_dev, LeafIndexPackets{});
 }
 
 // small batches of a random forest: leaf indices by (tile, tree slice) work items, then the ordered sums.
@@ -468,6 +489,27 @@ int sf_launch_forest_leaf_index(const sf_forest* fo, const float* feat, uint32_t
     if (n == 0) return SF_OK;
     if (fo->kind != SF_RF || !fo->d_image_small || !leaf_idx) return SF_ERR_UNSUPPORTED;
     return launch_rf_leaf_index(fo, feat, n, leaf_idx, st, n_dev);
+}
+
+// leaf indices of the flows whose packets are rows row_ids[0..n) of the planes pk, features computed inside the kernel
+int sf_launch_forest_leaf_index_packets(const sf_forest* fo, const sf_packets* pk, uint32_t N, const uint32_t* row_ids, uint32_t n,
+                                        uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+    if (n == 0) return SF_OK;
+    if (fo->kind != SF_RF || !fo->d_image_small || !leaf_idx) return SF_ERR_UNSUPPORTED;
+    if (pk->n_valid || pk->pitch_pkts % 8 != 0 || ((uintptr_t)pk->size & 15) != 0 || ((uintptr_t)pk->iat_us & 15) != 0) return SF_ERR_UNSUPPORTED;
+    if (fo->F % 8 != 0 || N < 1 || N > 32 || N > pk->pitch_pkts) return SF_ERR_UNSUPPORTED;
+    const LeafIndexPackets lp{pk->size, pk->iat_us, pk->dir_bits, row_ids, pk->pitch_pkts, N};
+    switch (fo->F / 8) {
+    case 1: return launch_rf_leaf_index_g<1>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 2: return launch_rf_leaf_index_g<2>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 3: return launch_rf_leaf_index_g<3>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 4: return launch_rf_leaf_index_g<4>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 5: return launch_rf_leaf_index_g<5>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 6: return launch_rf_leaf_index_g<6>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 7: return launch_rf_leaf_index_g<7>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    case 8: return launch_rf_leaf_index_g<8>(fo, nullptr, n, leaf_idx, st, n_dev, lp);
+    }
+    return SF_ERR_UNSUPPORTED;
 }
 
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,

@@ -1,5 +1,8 @@
 // S4 (bf16 MLP): hidden layers as tcgen05 GEMMs with TMEM accumulators fed by
-// TMA; the narrow last layer (<= 16 classes) runs through the same kernel as a 128 x 16 tile.
+// TMA.  The narrow last layer (<= 16 classes) is folded into the epilogue of the last hidden layer where the
+// batch is large (a CTA then owns whole 128-row panels, its epilogue warps multiply the bf16-rounded activations
+// of every tile with the head's weights on the CUDA cores and the activations are never written); otherwise it
+// runs through the same kernel as a 128 x 16 tile of its own.
 //
 // Hidden layer: out[r][o] = bf16( ReLU( sum_k A[r][k] * W[o][k] + b[o] ) ), r < *n_rows.
 // Persistent kernel, one CTA per SM, tile 128 x BN, K slices of 64 bf16 (one 128-byte
@@ -62,13 +65,19 @@ template <uint32_t BN> struct GemmCfg {
     static constexpr uint32_t kTmemCols = 2 * BN;             // a power of two >= 32
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
                                            kEpiWarps * 2048 /*epilogue staging*/;
+    // fused head: the staging space holds the head's weights [col][8] bf16 (N <= 1024); 16 more KB for [col][16]
+    static constexpr uint32_t kSmemBytesHead16 = kSmemBytes + 16384;
 };
+
+constexpr uint32_t kFusedHeadMaxN = 1024;
+enum { MODE_HIDDEN = 0, MODE_HEAD = 1, MODE_HIDDEN_HEAD = 2 };
 
 struct GemmBars {
     uint64_t full[10];
     uint64_t empty[10];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t head_bar;            // fused head: the four high-half epilogue warps have stored their partial logits
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -161,15 +170,22 @@ __device__ void small_rows_layer(const __nv_bfloat16* __restrict__ A, const __nv
 // HEAD = false: hidden layer, out = bf16(ReLU(acc + bias)) [rows][N].
 // HEAD = true (BN = 16): last layer, W zero-padded to 16 rows; logits[r][c] = acc + bias for
 // c < C (fp32, no activation) and label[r] = argmax (lowest index on ties).
-template <uint32_t BN, bool HEAD>
+// MODE_HIDDEN_HEAD: the last hidden layer with the head folded in.  head_w = the head's weights bf16 [16][N] (rows past C
+// zero), head_b its bias, CH = 8 or 16 = classes kept per row.  A CTA takes whole 128-row panels (all N / BN tiles of
+// a panel in turn), so a row's logits are summed in one place and in one fixed order: column chunks in increasing
+// order inside each of the two epilogue warps that share the row, then (low half + high half) + bias.
+template <uint32_t BN, int MODE, uint32_t CH = 8>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                            const float* __restrict__ bias, const uint32_t* __restrict__ n_rows_dev,
                            uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out, sf_dev_state* st,
                            float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C, uint32_t small_max,
-                           const __nv_bfloat16* __restrict__ A_raw, const __nv_bfloat16* __restrict__ W_raw, uint32_t capacity)
+                           const __nv_bfloat16* __restrict__ A_raw, const __nv_bfloat16* __restrict__ W_raw, uint32_t capacity,
+                           const __nv_bfloat16* __restrict__ head_w, const float* __restrict__ head_b)
 {
     using Cfg = GemmCfg<BN>;
+    constexpr bool HEAD = MODE == MODE_HEAD;
+    constexpr bool FUSED = MODE == MODE_HIDDEN_HEAD;
     extern __shared__ uint8_t smem_raw[];
     // the count is the caller's device word: never trust it beyond the rows the buffers hold
     const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);
@@ -185,16 +201,33 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t tiles_m = (n_rows + BM - 1) / BM;
     const uint32_t tiles_n = N / BN;
-    const uint32_t n_tiles = tiles_m * tiles_n;
     const uint32_t k_blocks = K / BK;
+    // tiles of this CTA, in order: every gridDim.x-th tile of the (row panel, column tile) sequence, or - with the head
+    // folded in - every gridDim.x-th row panel with all its column tiles
+    const uint32_t n_my = FUSED ? ((tiles_m > blockIdx.x) ? ((tiles_m - blockIdx.x + gridDim.x - 1) / gridDim.x) * tiles_n : 0u)
+                                : ((tiles_m * tiles_n > blockIdx.x) ? (tiles_m * tiles_n - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u);
+    auto tile_of = [&](uint32_t it, uint32_t& tm, uint32_t& tn) {
+        if (FUSED) { tm = blockIdx.x + (it / tiles_n) * gridDim.x; tn = it % tiles_n; }
+        else { const uint32_t tile = blockIdx.x + it * gridDim.x; tm = tile / tiles_n; tn = tile - tm * tiles_n; }
+    };
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < Cfg::kStages; s++) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
         for (uint32_t b = 0; b < 2; b++) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], kEpiWarps); }
+        mbar_init(&bars->head_bar, kEpiWarps / 2);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, Cfg::kTmemCols);
+    // fused head: the head's weights, transposed to [column][CH] bf16, where the other modes stage their output
+    uint8_t* const epi_smem = tiles + Cfg::kStages * Cfg::kStageBytes + 256;
+    if constexpr (FUSED) {
+        __nv_bfloat16* whT = reinterpret_cast<__nv_bfloat16*>(epi_smem);
+        for (uint32_t i = threadIdx.x; i < N * CH; i += kGemmThreads) {
+            const uint32_t col = i / CH, c = i - col * CH;
+            whT[i] = head_w[(size_t)c * N + col];                // rows past C are zero in the padded head matrix
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -206,8 +239,9 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             tma_prefetch_desc(&tmW);
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const uint32_t tm = tile / tiles_n, tn = tile - tm * tiles_n;
+            for (uint32_t it = 0; it < n_my && ok; it++) {
+                uint32_t tm, tn;
+                tile_of(it, tm, tn);
                 for (uint32_t kb = 0; kb < k_blocks; kb++) {
                     if (!mbar_wait(&bars->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sA = tiles + stage * Cfg::kStageBytes;
@@ -224,7 +258,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
             uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
             bool ok = true;
-            for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            for (uint32_t it = 0; it < n_my && ok; it++) {
                 if (!mbar_wait(&bars->tmem_empty[buf], bphase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
@@ -252,11 +286,13 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         // 8 epilogue warps: TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
         const uint32_t quarter = warp & 3u;
         const uint32_t half = (warp - 2u) >> 2;
-        uint8_t* stg = tiles + Cfg::kStages * Cfg::kStageBytes + 256 + (warp - 2u) * 2048u;   // 32 rows x 64 B, XOR-swizzled
-        uint32_t buf = 0, bphase = 0;
+        uint8_t* stg = epi_smem + (warp - 2u) * 2048u;   // 32 rows x 64 B, XOR-swizzled
+        uint32_t buf = 0, bphase = 0, hphase = 0;
         bool ok = true;
-        for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const uint32_t tm = tile / tiles_n, tn = tile - tm * tiles_n;
+        float lg[CH];                                     // fused head: this thread's row, partial logits over this warp's columns
+        for (uint32_t it = 0; it < n_my && ok; it++) {
+            uint32_t tm, tn;
+            tile_of(it, tm, tn);
             // the whole warp takes the same way out: the TMEM loads below are warp-collective
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->tmem_full[buf], bphase, abort_flag));
             if (!ok) break;
@@ -281,6 +317,77 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                             }
                         }
                         if (label) label[row] = (uint8_t)a;
+                    }
+                }
+            } else if constexpr (FUSED) {
+                constexpr uint32_t kHalfCols = BN / 2;
+                const uint32_t row = row0 + lane;
+                if (tn == 0) {
+#pragma unroll
+                    for (uint32_t c = 0; c < CH; c++) lg[c] = 0.0f;
+                }
+#pragma unroll 1
+                for (uint32_t c = half * kHalfCols; c < (half + 1) * kHalfCols; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c, v);
+                    tmem_ld_wait();
+                    const float4* b4 = reinterpret_cast<const float4*>(bias + col0 + c);
+                    const uint4* wq = reinterpret_cast<const uint4*>(epi_smem) + (size_t)(col0 + c) * (CH / 8);
+#pragma unroll
+                    for (int pc = 0; pc < 8; pc++) {
+                        const float4 bv = __ldg(b4 + pc);
+                        const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            // bias + ReLU + bf16 rounding exactly as the stored activations would have had
+                            const float x0 = fmaxf(__uint_as_float(v[pc * 4 + e]) + bb[e], 0.0f);
+                            const float x1 = fmaxf(__uint_as_float(v[pc * 4 + e + 1]) + bb[e + 1], 0.0f);
+                            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                            const uint32_t hb = *reinterpret_cast<uint32_t*>(&h);
+                            const float a[2] = {__uint_as_float(hb << 16), __uint_as_float(hb & 0xFFFF0000u)};
+#pragma unroll
+                            for (int q = 0; q < 2; q++) {
+                                const uint4* wp = wq + (size_t)(pc * 4 + e + q) * (CH / 8);      // same address in all lanes: a broadcast
+#pragma unroll
+                                for (uint32_t g = 0; g < CH / 8; g++) {
+                                    const uint4 w = wp[g];
+                                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                                    for (int k = 0; k < 4; k++) {
+                                        lg[g * 8 + 2 * k] = fmaf(a[q], __uint_as_float(ww[k] << 16), lg[g * 8 + 2 * k]);
+                                        lg[g * 8 + 2 * k + 1] = fmaf(a[q], __uint_as_float(ww[k] & 0xFFFF0000u), lg[g * 8 + 2 * k + 1]);
+                                    }
+                                }
+                            }
+                        }
+                    }
+                }
+                if (tn + 1 == tiles_n) {
+                    // the row's two halves meet: the high-half warp leaves its partial sums in the logits row, the low-half warp
+                    // adds (low + high) + bias, writes the logits and the label
+                    if (half == 1) {
+                        if (row < n_rows) {
+#pragma unroll
+                            for (uint32_t c = 0; c < CH; c++) if (c < C) logits[(size_t)row * C + c] = lg[c];
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->head_bar);
+                    } else {
+                        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->head_bar, hphase, abort_flag));
+                        if (!ok) break;
+                        hphase ^= 1u;
+                        if (row < n_rows) {
+                            uint32_t arg = 0; float mx = 0.0f;
+#pragma unroll
+                            for (uint32_t c = 0; c < CH; c++) {
+                                if (c < C) {
+                                    const float x = (lg[c] + logits[(size_t)row * C + c]) + __ldg(head_b + c);
+                                    logits[(size_t)row * C + c] = x;
+                                    if (c == 0 || x > mx) { mx = x; arg = c; }
+                                }
+                            }
+                            if (label) label[row] = (uint8_t)arg;
+                        }
                     }
                 }
             } else {
@@ -347,7 +454,7 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     if (rc != SF_OK) return rc;
     rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
     if (rc != SF_OK) return rc;
-    auto k = gemm_bias_relu_bf16_kernel<BN, false>;
+    auto k = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN>;
     static bool attr_set_dev[64] = {};                 // the opt-in is per device
     bool& attr_set = attr_set_dev[ctx->device & 63];
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
@@ -355,8 +462,33 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
                                                   reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state, nullptr, nullptr, 0, small_max,
-                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity);
+                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity, nullptr, nullptr);
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel");
+    return SF_OK;
+}
+
+// last hidden layer with the head folded into its epilogue (no activations written); W16 = the head's weights padded to 16 rows
+template <uint32_t BN, uint32_t CH>
+int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bias, const uint32_t* n_rows_dev, uint32_t capacity,
+                     uint32_t N, uint32_t K, const void* W16, const float* head_bias, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
+{
+    using Cfg = GemmCfg<BN>;
+    constexpr uint32_t kSmem = CH == 8 ? Cfg::kSmemBytes : Cfg::kSmemBytesHead16;
+    CUtensorMap tmA, tmW;
+    int rc = encode_tmap_bf16_2d(&tmA, A, capacity, K, BM, BK);
+    if (rc != SF_OK) return rc;
+    rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
+    if (rc != SF_OK) return rc;
+    auto k = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN_HEAD, CH>;
+    static bool attr_set_dev[64] = {};                 // the opt-in is per device
+    bool& attr_set = attr_set_dev[ctx->device & 63];
+    if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem)); attr_set = true; }
+    const uint32_t panels = (capacity + BM - 1) / BM;
+    const uint32_t grid = (uint32_t)ctx->num_sms < panels ? (uint32_t)ctx->num_sms : panels;
+    k<<<grid, kGemmThreads, kSmem, st>>>(tmA, tmW, bias, n_rows_dev, N, K, nullptr, ctx->d_state, logits, label, C, 0u,
+                                         reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
+                                         reinterpret_cast<const __nv_bfloat16*>(W16), head_bias);
+    SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(hidden + head)");
     return SF_OK;
 }
 
@@ -370,14 +502,14 @@ int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bia
     if (rc != SF_OK) return rc;
     rc = encode_tmap_bf16_2d(&tmW, W16, 16, K, 16, BK);
     if (rc != SF_OK) return rc;
-    auto k = gemm_bias_relu_bf16_kernel<16, true>;
+    auto k = gemm_bias_relu_bf16_kernel<16, MODE_HEAD>;
     static bool attr_set_dev[64] = {};                 // the opt-in is per device
     bool& attr_set = attr_set_dev[ctx->device & 63];
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
     uint32_t max_tiles = (capacity + BM - 1) / BM;
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
     k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C, small_max,
-                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16), capacity);
+                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16), capacity, nullptr, nullptr);
     SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(head)");
     return SF_OK;
 }
@@ -397,19 +529,34 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     for (uint32_t l = 0; l < s->n_layers; l++) if (s->dims[l] > kSmallMaxK || (s->dims[l] % 8) != 0) small = false;
     const uint32_t small_max = small ? kSmallRows : 0u;
     const void* in = rows;
+    const uint32_t L = s->n_layers - 1;                  // the head
+    // Large batches: the head is folded into the last hidden layer (its activations are then never written or re-read).
+    // Not where a launch may see only a handful of rows (those take the CUDA-core path, layer by layer), nor where a
+    // row panel has a single column tile (the epilogue warps' hand-over needs two tiles between two panel ends).
+    const uint32_t Nl = s->dims[L], Cn = s->dims[L + 1];
+    const uint32_t BNl = Nl % 256 == 0 ? 256u : (Nl % 128 == 0 ? 128u : 64u);
+    const bool fuse_head = small_max == 0 && Nl <= kFusedHeadMaxN && Nl / BNl >= 2;
     sf_time_begin(ctx, SF_T_GEMM, st);
     for (uint32_t l = 0; l + 1 < s->n_layers; l++) {
         void* out = (l & 1) ? h1 : h0;
         const uint32_t K = s->dims[l], N = s->dims[l + 1];
         int rc;
-        if (N % 256 == 0)      rc = launch_gemm<256>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
+        if (fuse_head && l + 1 == L) {
+#define SF_FUSED(BNv) (Cn <= 8 ? launch_gemm_head<BNv, 8>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st) \
+                               : launch_gemm_head<BNv, 16>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st))
+            if (N % 256 == 0)      rc = SF_FUSED(256);
+            else if (N % 128 == 0) rc = SF_FUSED(128);
+            else                   rc = SF_FUSED(64);
+#undef SF_FUSED
+        }
+        else if (N % 256 == 0) rc = launch_gemm<256>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
         else if (N % 128 == 0) rc = launch_gemm<128>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
         else                   rc = launch_gemm<64>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
         if (rc != SF_OK) return rc;
         in = out;
     }
     sf_time_end(ctx, SF_T_GEMM, st);
-    const uint32_t L = s->n_layers - 1;
+    if (fuse_head) return SF_OK;
     sf_time_begin(ctx, SF_T_HEAD, st);
     int rc = launch_head_tc(ctx, in, s->d_W[L], s->d_b[L], n_rows_dev, capacity, s->dims[L], s->dims[L + 1], logits, label, st, small_max);
     sf_time_end(ctx, SF_T_HEAD, st);

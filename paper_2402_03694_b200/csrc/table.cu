@@ -7,7 +7,7 @@
 //   probe     one thread per packet: 128-bit compare-and-swap on the 16-byte key slot
 //             (claims an empty slot or recognises its own key; bounded linear probing)
 //   sort      key = arrival index of the flow's first packet in the batch (16 bits, unique per
-//             flow); stable LSD radix sort (4 passes of 4 bits, tiles of 1024, one kernel per pass)
+//             flow); stable LSD radix sort (2 passes of 8 bits, tiles of 1024, one kernel per pass)
 //             puts each flow's packets together in ARRIVAL order; rank = position minus start of the run
 //   apply1    packets that fall into a flow's first `fast_pkts` positions are written to its
 //             fast context; flows that just reached fast_pkts packets are listed
@@ -138,14 +138,16 @@ __global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ 
 
 // Sort key of a packet = arrival index of its flow's first packet in this batch: 16 bits,
 // unique per flow; a packet that found no slot is a run of its own.  The block also counts its keys' first radix
-// digit (shared-memory counters, then one add per digit into hist0[digit][tile]; the caller zeroed hist0).
+// digit (shared-memory counters, then one add per digit into hist0[tile][digit]; the caller zeroed hist0).
 constexpr uint32_t kTile = 1024;
+constexpr uint32_t kMaxTiles = kMaxBatch / kTile;            // 64
+constexpr uint32_t kHistWords = 256 * kMaxTiles;             // one pass: [tile][digit]
 __global__ void __launch_bounds__(256)
 key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
-           uint32_t* __restrict__ key, uint32_t* __restrict__ idx, uint32_t* __restrict__ hist0, uint32_t nblk)
+           uint32_t* __restrict__ key, uint32_t* __restrict__ idx, uint32_t* __restrict__ hist0)
 {
-    __shared__ uint32_t c[16];
-    if (threadIdx.x < 16) c[threadIdx.x] = 0;
+    __shared__ uint32_t c[256];
+    c[threadIdx.x] = 0;
     __syncthreads();
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) {
@@ -153,101 +155,77 @@ key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
         const uint32_t k = (slot < t.n_slots) ? t.first[slot] : i;
         key[i] = k;
         idx[i] = i;
-        atomicAdd(&c[k & 15u], 1u);
+        atomicAdd(&c[k & 255u], 1u);
     }
     __syncthreads();
-    if (threadIdx.x < 16 && c[threadIdx.x]) atomicAdd(&hist0[threadIdx.x * nblk + (blockIdx.x * 256u) / kTile], c[threadIdx.x]);
+    if (c[threadIdx.x]) atomicAdd(&hist0[((blockIdx.x * 256u) / kTile) * 256u + threadIdx.x], c[threadIdx.x]);
 }
 
-// Stable LSD radix sort, 4-bit digits, tiles of 1024 items (256 threads x 4 consecutive items), one kernel per pass:
-// a block turns the pass's per-tile digit counts hist[digit][tile] (<= 1024 entries) into global offsets by scanning
-// them itself, ranks its tile's items and moves them; while doing so it counts the NEXT pass's digit of every item under
-// the tile the item lands in (shared-memory counters first, then one add per non-zero counter into next_hist, which the
+// Stable LSD radix sort of the 16-bit keys: two passes of 8-bit digits, tiles of 1024 items, one kernel per pass.
+// A block turns the pass's per-tile digit counts hist[tile][digit] into the output position of its own tile's first
+// item of every digit (thread d: items of smaller digits in all tiles + items of digit d in earlier tiles), then takes
+// its tile 256 items at a time in index order; an item's place among the items of its digit = (earlier rounds) +
+// (earlier warps of this round) + (lower lanes of its warp with the same digit, by match.any).  While moving the
+// items it counts the NEXT pass's digit of every item under the tile the item lands in (16-bit counters in shared
+// memory, two per word: a block moves at most 1024 items; then one add per non-zero counter into next_hist, which the
 // caller zeroed), so no pass needs a counting kernel of its own.
 __global__ void __launch_bounds__(256)
-radix_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ iin, uint32_t* __restrict__ kout,
-                     uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk,
-                     uint32_t* __restrict__ next_hist)
+radix8_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ iin, uint32_t* __restrict__ kout,
+                      uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk,
+                      uint32_t* __restrict__ next_hist)
 {
-    __shared__ uint32_t cnt[16 * 256];
-    __shared__ uint32_t tot[8];
-    __shared__ uint32_t gofs[16];
-    __shared__ uint32_t nh[16 * 64];                     // next pass: [digit][output tile] (a batch has at most 64 tiles)
-    if (next_hist) for (uint32_t i = threadIdx.x; i < 16 * 64; i += 256) nh[i] = 0;
-    const uint32_t t = threadIdx.x;
-    // exclusive scan of the 16 * nblk counts in (digit, tile) order; thread t owns entries [4t, 4t+4)
+    __shared__ uint32_t base[256];
+    __shared__ uint32_t wc[8][256];
+    __shared__ uint32_t wsum[8];
+    __shared__ uint32_t nh[256 * (kMaxTiles / 2)];       // next pass: [digit][output tile pair]
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    if (next_hist) for (uint32_t i = tid; i < 256 * (kMaxTiles / 2); i += 256) nh[i] = 0;
     {
-        const uint32_t entries = 16 * nblk;
-        uint32_t v[4], s0 = 0;
+        uint32_t tot = 0, part = 0;
+        for (uint32_t t = 0; t < nblk; t++) { const uint32_t v = hist[t * 256u + tid]; tot += v; if (t < blockIdx.x) part += v; }
+        uint32_t x = tot;
 #pragma unroll
-        for (uint32_t e = 0; e < 4; e++) { v[e] = (4 * t + e < entries) ? hist[4 * t + e] : 0u; s0 += v[e]; }
-        uint32_t x = s0;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
-        if ((t & 31) == 31) tot[t >> 5] = x;
+        for (uint32_t o = 1; o < 32; o <<= 1) { const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
+        if (lane == 31) wsum[warp] = x;
         __syncthreads();
-        uint32_t run = x - s0;
-        for (uint32_t w = 0; w < (t >> 5); w++) run += tot[w];
+        uint32_t before = 0;
+        for (uint32_t w = 0; w < warp; w++) before += wsum[w];
+        base[tid] = before + x - tot + part;
+    }
+    const uint32_t t0 = blockIdx.x * kTile;
+    for (uint32_t r = 0; r < kTile / 256; r++) {
 #pragma unroll
-        for (uint32_t e = 0; e < 4; e++) {
-            const uint32_t ent = 4 * t + e;                     // = digit * nblk + tile
-            if (ent < entries && ent % nblk == blockIdx.x) gofs[ent / nblk] = run;
-            run += v[e];
+        for (uint32_t w = 0; w < 8; w++) wc[w][tid] = 0;
+        __syncthreads();
+        const uint32_t i = t0 + r * 256 + tid;
+        const bool valid = i < n;
+        const uint32_t key = valid ? kin[i] : 0u;
+        const uint32_t d = valid ? ((key >> shift) & 255u) : (256u + lane);      // idle lanes match nobody
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
+        const uint32_t below = __popc(peers & ((1u << lane) - 1u));
+        if (valid && below == 0) wc[warp][d] = __popc(peers);
+        __syncthreads();
+        uint32_t acc = base[tid];                               // digit `tid`: this round's warps in order
+#pragma unroll
+        for (uint32_t w = 0; w < 8; w++) { const uint32_t c = wc[w][tid]; wc[w][tid] = acc; acc += c; }
+        base[tid] = acc;
+        __syncthreads();
+        if (valid) {
+            const uint32_t p = wc[warp][d] + below;
+            kout[p] = key;
+            iout[p] = iin[i];
+            if (next_hist) atomicAdd(&nh[((key >> (shift + 8)) & 255u) * (kMaxTiles / 2) + (p >> 11)], 1u << (16u * ((p >> 10) & 1u)));
         }
         __syncthreads();
-    }
-    const uint32_t j0 = blockIdx.x * kTile + t * 4;
-    uint32_t k[4], dg[4];
-    uint32_t h[16];
-#pragma unroll
-    for (int d = 0; d < 16; d++) h[d] = 0;
-#pragma unroll
-    for (uint32_t e = 0; e < 4; e++) {
-        k[e] = (j0 + e < n) ? kin[j0 + e] : 0u;
-        dg[e] = (k[e] >> shift) & 15u;
-        if (j0 + e < n) {
-#pragma unroll
-            for (int d = 0; d < 16; d++) h[d] += (dg[e] == (uint32_t)d) ? 1u : 0u;
-        }
-    }
-#pragma unroll
-    for (int d = 0; d < 16; d++) cnt[d * 256 + t] = h[d];
-    __syncthreads();
-    // exclusive scan of the 4096 counters in (digit, thread) order; thread t owns entries [16t, 16t+16)
-    uint32_t loc[16], s = 0;
-#pragma unroll
-    for (int e = 0; e < 16; e++) { loc[e] = s; s += cnt[t * 16 + e]; }
-    uint32_t x = s;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((t & 31) >= (uint32_t)o) x += y; }
-    if ((t & 31) == 31) tot[t >> 5] = x;
-    __syncthreads();
-    uint32_t wbase = 0;
-    for (uint32_t w = 0; w < (t >> 5); w++) wbase += tot[w];
-    __syncthreads();
-    const uint32_t base = wbase + x - s;
-#pragma unroll
-    for (int e = 0; e < 16; e++) cnt[t * 16 + e] = base + loc[e];
-    __syncthreads();
-    // position = start of (digit, this block) in the output + rank among the block's items of that digit
-#pragma unroll
-    for (uint32_t e = 0; e < 4; e++) {
-        if (j0 + e < n) {
-            const uint32_t d = dg[e];
-            uint32_t before = 0;                         // earlier items of this thread with the same digit
-#pragma unroll
-            for (uint32_t q = 0; q < 4; q++) if (q < e && dg[q] == d) before++;
-            const uint32_t p = gofs[d] + (cnt[d * 256 + t] - cnt[d * 256]) + before;
-            kout[p] = k[e];
-            iout[p] = iin[j0 + e];
-            if (next_hist) atomicAdd(&nh[((k[e] >> (shift + 4)) & 15u) * 64u + p / kTile], 1u);
-        }
     }
     if (next_hist) {
-        __syncthreads();
-        for (uint32_t i = threadIdx.x; i < 16 * 64; i += 256) {
+        for (uint32_t i = tid; i < 256 * (kMaxTiles / 2); i += 256) {
             const uint32_t v = nh[i];
-            if (v) atomicAdd(&next_hist[(i >> 6) * nblk + (i & 63u)], v);
+            if (v) {
+                const uint32_t dg = i / (kMaxTiles / 2), tp = (i % (kMaxTiles / 2)) * 2u;
+                if (v & 0xFFFFu) atomicAdd(&next_hist[tp * 256u + dg], v & 0xFFFFu);
+                if (v >> 16) atomicAdd(&next_hist[(tp + 1u) * 256u + dg], v >> 16);
+            }
         }
     }
 }
@@ -502,7 +480,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     need(B * slow_pkts * 2); need(B * slow_pkts * 4); need(B * W * 4); need(B * slow_pkts * kHdr); need(4);
     need(B * 4); need(4); need(S * 4);
     for (int k = 0; k < 9; k++) need((size_t)kMaxBatch * 4);
-    need((16 + 4 * 1024) * 4); need((size_t)kMaxBatch * 4); need(S * 4);          // counters + digit counts, pkt_slot, first
+    need((16 + 2 * kHistWords) * 4); need((size_t)kMaxBatch * 4); need(S * 4);     // counters + digit counts, pkt_slot, first
     cudaError_t e = cudaMalloc(&t->all, total);
     if (e != cudaSuccess) { delete t; sf_set_cuda_error(e, "cudaMalloc(table)"); return SF_ERR_ALLOC; }
     e = cudaMemset(t->all, 0, total);
@@ -525,7 +503,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     t->rank = carve<uint32_t>(p, kMaxBatch); t->pos = carve<uint32_t>(p, kMaxBatch);
     t->fire1_slot = carve<uint32_t>(p, kMaxBatch); t->fire2_slab = carve<uint32_t>(p, kMaxBatch);
     t->fire2_slot = carve<uint32_t>(p, kMaxBatch);
-    t->counts = carve<uint32_t>(p, 16 + 4 * 1024);           // counters, then the four passes' digit counts (cleared together)
+    t->counts = carve<uint32_t>(p, 16 + 2 * kHistWords);     // counters, then the two passes' digit counts (cleared together)
     t->hist = t->counts + 16;
     t->pkt_slot = carve<uint32_t>(p, kMaxBatch);
     d.first = carve<uint32_t>(p, S);
@@ -575,23 +553,19 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     if (!w) return SF_ERR_ALLOC;
     sf_time_new_record(ctx);
     sf_time_begin(ctx, SF_T_TABLE, st);
-    SF_CUDA(cudaMemsetAsync(t->counts, 0, (16 + 4 * 1024) * sizeof(uint32_t), st));
+    SF_CUDA(cudaMemsetAsync(t->counts, 0, (16 + 2 * kHistWords) * sizeof(uint32_t), st));
     const uint32_t blocks = (n + 255) / 256;
     probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->pkt_slot, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("probe_kernel");
     const uint32_t nblk = (n + kTile - 1) / kTile;
-    key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a, t->hist, nblk);
+    key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a, t->hist);
     SF_LAUNCH_CHECK("key_kernel");
     {
-        // 16-bit keys: four 4-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
-        uint32_t* kin = t->key_a; uint32_t* iin = t->idx_a; uint32_t* kout = t->key_b; uint32_t* iout = t->idx_b;
-        for (uint32_t pass = 0; pass < 4; pass++) {
-            radix_scatter_kernel<<<nblk, 256, 0, st>>>(kin, iin, kout, iout, n, pass * 4, t->hist + pass * 1024, nblk,
-                                                       pass < 3 ? t->hist + (pass + 1) * 1024 : nullptr);
-            SF_LAUNCH_CHECK("radix pass");
-            uint32_t* tk = kin; kin = kout; kout = tk;
-            uint32_t* ti = iin; iin = iout; iout = ti;
-        }
+        // 16-bit keys: two 8-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
+        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_a, t->idx_a, t->key_b, t->idx_b, n, 0, t->hist, nblk, t->hist + kHistWords);
+        SF_LAUNCH_CHECK("radix pass 0");
+        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_b, t->idx_b, t->key_a, t->idx_a, n, 8, t->hist + kHistWords, nblk, nullptr);
+        SF_LAUNCH_CHECK("radix pass 1");
     }
     apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts);
     SF_LAUNCH_CHECK("apply1_kernel");
@@ -602,13 +576,14 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     fpk.size = d.f_size; fpk.iat_us = d.f_iat; fpk.dir_bits = d.f_dir; fpk.hdr = nullptr; fpk.n_valid = nullptr;
     fpk.n_flows = n; fpk.pitch_pkts = d.fast_pkts; fpk.hdr_bytes = 0;
     float* feat = reinterpret_cast<float*>(w + o_feat);
-    sf_time_begin(ctx, SF_T_EXTRACT, st);
-    rc = sf_launch_extract(&fpk, d.fast_pkts, F, feat, st, &t->counts[0], t->fire1_slot);
-    sf_time_end(ctx, SF_T_EXTRACT, st);
-    if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_FOREST, st);
-    // a few hundred flows fire per batch: trees spread over the grid, one leaf index per flow and tree ...
-    rc = sf_launch_forest_leaf_index(fo, feat, n, reinterpret_cast<uint16_t*>(w + o_lidx), st, &t->counts[0]);
+    // a few hundred flows fire per batch: trees spread over the grid, one leaf index per flow and tree; the kernel computes
+    // the fired flows' features itself, in its shared-memory tile, straight from the table's fast contexts ...
+    rc = sf_launch_forest_leaf_index_packets(fo, &fpk, d.fast_pkts, t->fire1_slot, n, reinterpret_cast<uint16_t*>(w + o_lidx), st, &t->counts[0]);
+    if (rc == SF_ERR_UNSUPPORTED) {                        // (planes not laid out for that: features first, then the trees)
+        rc = sf_launch_extract(&fpk, d.fast_pkts, F, feat, st, &t->counts[0], t->fire1_slot);
+        if (rc == SF_OK) rc = sf_launch_forest_leaf_index(fo, feat, n, reinterpret_cast<uint16_t*>(w + o_lidx), st, &t->counts[0]);
+    }
     sf_time_end(ctx, SF_T_FOREST, st);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_SCORE, st);

@@ -301,6 +301,12 @@ def test_mlp_fp32(env):
     ((192, 320, 64, 16), 7, 600),
     ((2048, 1024, 8), 16, 64),
     ((2048, 1024, 8), 17, 64),            # one row more: back on the tensor cores
+    # capacities beyond 65,536 rows: the head is folded into the last hidden layer's epilogue (row panels per CTA)
+    ((256, 512, 512, 8), 777, 66000),     # two 256-column tiles per panel, 8 logits per row
+    ((256, 512, 512, 8), 66000, 66000),   # every panel of every CTA, ragged last panel
+    ((192, 320, 384, 16), 1500, 70000),   # three 128-column tiles per panel, 16 logits per row
+    ((128, 192, 5), 300, 66001),          # three 64-column tiles per panel, odd class count
+    ((128, 256, 3), 300, 66001),          # a single column tile per panel: the head keeps its own launch
 ])
 def test_mlp_bf16_small_integers_are_exact(env, dims, n_rows, cap):
     """Integer-valued bf16 operands with small sums: every product and partial sum is
@@ -331,15 +337,16 @@ def test_mlp_bf16_small_integers_are_exact(env, dims, n_rows, cap):
     sf.sf_slow_destroy(hd)
 
 
-@pytest.mark.parametrize("dims,n_rows", [((1024, 512, 512, 2), 700), ((2048, 1024, 1024, 1024, 8), 400), ((2048, 1024, 1024, 1024, 8), 11)])
-def test_mlp_bf16_within_tolerance(env, dims, n_rows):
+@pytest.mark.parametrize("dims,n_rows,extra", [((1024, 512, 512, 2), 700, 57), ((2048, 1024, 1024, 1024, 8), 400, 57), ((2048, 1024, 1024, 1024, 8), 11, 57),
+                                               ((2048, 1024, 1024, 1024, 8), 3000, 70000), ((1024, 512, 512, 2), 2500, 70000)])
+def test_mlp_bf16_within_tolerance(env, dims, n_rows, extra):
     sf, hz, ctx = env
     m = flowgen.gen_mlp(33, dims)
     wide = flowgen.gen_packets(34, n_rows, dims[0] // 16, 13)
     rows = oracle.wide_rows(0, np.arange(n_rows, dtype=np.uint32), wide, dims[0] // 16, True, threads=4)
     ref, ref_label = oracle.mlp(m, rows, True, threads=8)
     hd = sf.sf_mlp_create(ctx, sf.SF_BF16, m["dims"], m["W"], m["b"])
-    cap = n_rows + 57
+    cap = n_rows + extra             # beyond 65,536 rows of capacity the head runs inside the last hidden layer's launch
     rt = torch.zeros((cap, dims[0]), dtype=torch.bfloat16, device="cuda")
     rt[:n_rows] = hz.dev(rows).to(torch.bfloat16)
     logits, label = _run_slow(sf, hz, ctx, hd, rt, n_rows, cap, dims[-1])
