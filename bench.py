@@ -197,7 +197,7 @@ def kernel_launches_per_step(cfg, capacity):
             slow -= 1                                                         # the head runs inside the last hidden layer's launch
     else:
         slow = 1                                                              # the fused CNN kernel
-    return 1 + 1 + 4 + slow + 1 + 2      # extract, forest, score/scan/scatter/gather, slow, count, merge x2
+    return 1 + 1 + 3 + slow + 1          # extract, forest (takes the decisions itself), scan/scatter/gather, slow, merge
 
 
 def tensor_peak_for(peaks, clocks):
@@ -218,8 +218,8 @@ def rooflines_for(cfg, n, k_esc, avg, peaks, clocks):
     work = {
         "extract": ("hbm", n * (in_b + 4 * cfg.F) / 1e9),
         "gather": ("hbm", k_esc * (per_esc_in + cfg.D * esz) / 1e9),
-        # score + scan + scatter: fast-model output in; decision, label, ids out
-        "score": ("hbm", (n * (4 * Cf + 2) + 4 * k_esc) / 1e9),
+        # scan + scatter (the tree kernel's epilogue took the decisions): decision bytes in, ids out
+        "score": ("hbm", (n + 4 * k_esc) / 1e9),
         "forest": ("alu", (n / 32.0) * cfg.T * (cfg.depth * FOREST_WAVEFRONTS_PER_VISIT + (4 * Cf * 32) / 128.0) / 1e9),
     }
     if cfg.slow_dtype == "bf16":

@@ -302,6 +302,10 @@ int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf
     float* logits = reinterpret_cast<float*>(base + p.logits);
     uint8_t* label_slow = reinterpret_cast<uint8_t*>(base + p.label_slow);
     uint32_t* n_esc_dev = &ctx->d_state->scan_total;
+    // one call for everything, a fast model and rule the tree kernel can score itself, outputs for every flow: fold the
+    // assignment and the first merge into the tree kernel
+    const bool fused = phases == SF_PHASE_ALL && n > 0 &&
+                       ((fo->kind == SF_RF && cfg->rule == SF_LC_GT) || (fo->kind == SF_GBDT && cfg->rule == SF_ABSMARGIN_LT));
 
     if (phases & SF_PHASE_FAST) {
         sf_time_new_record(ctx);
@@ -310,11 +314,23 @@ int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf
         sf_time_end(ctx, SF_T_EXTRACT, st);
         if (rc != SF_OK) return rc;
         sf_time_begin(ctx, SF_T_FOREST, st);
-        rc = sf_launch_forest(fo, feat, n, fast_out, nullptr, st);
-        sf_time_end(ctx, SF_T_FOREST, st);
-        if (rc != SF_OK) return rc;
-        rc = sf_launch_route(ctx, cfg, fast_out, n, fo->C, (phases & SF_PHASE_SLOW) ? wide : nullptr, esc_ids, n_esc_out,
-                             rows, decision, label_fast, nullptr, base + p.route_scratch, st);
+        if (fused) {
+            // the tree kernel takes the decisions in its epilogue (score, label, decision byte, fast label and stage 1 of every
+            // flow, assigned flows per block): no score kernel, no first merge kernel
+            sf_fused_route fr;
+            fr.tau = cfg->tau; fr.rule = cfg->rule; fr.decision = decision; fr.label_fast = label_fast;
+            fr.label_out = label_out; fr.stage_out = stage_out; fr.block_counts = reinterpret_cast<uint32_t*>(base + p.route_scratch);
+            rc = sf_launch_forest(fo, feat, n, fast_out, nullptr, st, nullptr, false, &fr);
+            sf_time_end(ctx, SF_T_FOREST, st);
+            if (rc != SF_OK) return rc;
+            rc = sf_launch_route_after_fused(ctx, cfg, n, wide, esc_ids, n_esc_out, rows, decision, fr.block_counts, st);
+        } else {
+            rc = sf_launch_forest(fo, feat, n, fast_out, nullptr, st);
+            sf_time_end(ctx, SF_T_FOREST, st);
+            if (rc != SF_OK) return rc;
+            rc = sf_launch_route(ctx, cfg, fast_out, n, fo->C, (phases & SF_PHASE_SLOW) ? wide : nullptr, esc_ids, n_esc_out,
+                                 rows, decision, label_fast, nullptr, base + p.route_scratch, st);
+        }
         if (rc != SF_OK) return rc;
         ctx->last_feat = feat; ctx->last_fast_out = fast_out; ctx->last_esc_ids = esc_ids; ctx->last_rows = rows;
         ctx->last_logits = logits; ctx->last_label_fast = label_fast; ctx->last_label_slow = label_slow;
@@ -328,10 +344,11 @@ int serve_on_device(sf_ctx* ctx, const sf_forest* fo, const sf_slow* s, const sf
         sf_time_end(ctx, SF_T_GATHER, st);
         if (rc != SF_OK) return rc;
     }
-    rc = sf_launch_slow(ctx, s, rows, n_esc_dev, cfg->capacity, logits, label_slow, base + p.slow_scratch, st);
+    rc = sf_launch_slow(ctx, s, rows, n_esc_dev, cfg->capacity, logits, label_slow, base + p.slow_scratch, st, !fused);
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_MERGE, st);
-    rc = sf_launch_merge(label_fast, decision, n, esc_ids, n_esc_dev, cfg->capacity, label_slow, label_out, stage_out, st);
+    rc = sf_launch_merge(label_fast, decision, n, esc_ids, n_esc_dev, cfg->capacity, label_slow, label_out, stage_out, st, 2, !fused,
+                         fused ? ctx->d_state : nullptr);
     sf_time_end(ctx, SF_T_MERGE, st);
     if (rc != SF_OK) return rc;
     ctx->last_feat = feat; ctx->last_fast_out = fast_out; ctx->last_esc_ids = esc_ids; ctx->last_rows = rows;

@@ -91,12 +91,27 @@ void  sf_ws_reset(sf_ctx* ctx);
 void* sf_ws_alloc(sf_ctx* ctx, size_t bytes);       // NULL if the reservation was too small
 static inline size_t sf_align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
+// Assignment folded into the tree kernel's epilogue (the composite call on large batches): with tau set, every live flow's
+// fast label, decision byte, final label (= fast label) and stage (= 1) are written by the tree kernel, and
+// block_counts[b] = assigned flows among flows [b * SF_FOREST_BLOCK, (b + 1) * SF_FOREST_BLOCK).
+#define SF_FOREST_BLOCK 512u
+struct sf_fused_route {
+    const float* tau;             // nullptr: not fused
+    int rule;                     // SF_LC_GT (random forest) or SF_ABSMARGIN_LT (binary boosted trees)
+    uint8_t* decision; uint8_t* label_fast; uint8_t* label_out; uint8_t* stage_out;
+    uint32_t* block_counts;
+};
+
 // ---- internal launchers (each validates nothing; callers did) ---------------
 int sf_launch_extract(const sf_packets* pk, uint32_t N, uint32_t F, float* feat, cudaStream_t st,
                       const uint32_t* n_dev = nullptr,    // n_dev: optional device-side flow count (<= pk->n_flows)
                       const uint32_t* row_ids = nullptr); // row_ids: optional, flow f's packets are row row_ids[f] of the planes
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st,
-                     const uint32_t* n_dev = nullptr, bool small_tiles = false);   // small_tiles + leaf_idx (used as scratch): few flows per launch, trees spread over the grid
+                     const uint32_t* n_dev = nullptr, bool small_tiles = false,    // small_tiles + leaf_idx (used as scratch): few flows per launch, trees spread over the grid
+                     const sf_fused_route* fused = nullptr);                       // fused: see sf_fused_route (SF_RF / SF_GBDT, whole batch, n_dev unused)
+// what is left of the assignment after a tree kernel that took the decisions: scan of its block counts, ascending ids, gather
+int sf_launch_route_after_fused(sf_ctx* ctx, const sf_route_cfg* cfg, uint32_t n, const sf_packets* wide, uint32_t* esc_ids,
+                                uint32_t* n_esc, void* rows, const uint8_t* decision, uint32_t* block_counts, cudaStream_t st);
 // route scratch: block_counts uint32[ceil(n/1024)+1], decision bytes if the caller gave none
 size_t sf_route_scratch_bytes(uint32_t n);
 int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out, uint32_t n, uint32_t C,
@@ -113,7 +128,8 @@ int sf_launch_slow(sf_ctx* ctx, const sf_slow* s, const void* rows, const uint32
                    float* logits, uint8_t* label, void* scratch, cudaStream_t st, bool count_done = true);
 int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t n, const uint32_t* esc_ids,
                     const uint32_t* n_esc, uint32_t capacity, const uint8_t* label_slow,
-                    uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value = 2, bool write_fast = true);
+                    uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value = 2, bool write_fast = true,
+                    sf_dev_state* count_slow_done = nullptr);       // count_slow_done: also add the list's length to n_slow_done
 int sf_launch_gather_feat(const float* feat, const uint32_t* ids, const uint32_t* n_dev, uint32_t n_max, uint32_t F,
                           float* out, cudaStream_t st);
 int sf_launch_compose_ids(const uint32_t* ids1, const uint32_t* ids2_local, const uint32_t* n_dev, uint32_t n_max,

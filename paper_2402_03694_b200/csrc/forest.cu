@@ -124,11 +124,15 @@ __global__ void __launch_bounds__(KB + 32, 1)
 forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
               const unsigned char* __restrict__ image, const float* __restrict__ leaf, cudaTextureObject_t leaf_tex,
               uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
-              float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev)
+              float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev,
+              const sf_fused_route fr)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
-    if (blockIdx.x * KB >= n) return;
+    if (blockIdx.x * KB >= n) {
+        if (fr.tau && threadIdx.x == 0) fr.block_counts[blockIdx.x] = 0;
+        return;
+    }
     const uint32_t sbuf0 = smem_u32(smem_raw);
     float* xs = reinterpret_cast<float*>(smem_raw + 2 * (size_t)chunk_bytes);       // [F][KB]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * (size_t)chunk_bytes + (size_t)F * KB * 4);   // full[2], empty[2], flag
@@ -271,17 +275,52 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         if ((threadIdx.x & 31u) == 0) sftc::mbar_arrive(&empty[ck & 1u]);
     }
     if (KIND == SF_RF) flush_pending();
-    if (*abort_flag) { if (threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT); return; }
-    if (!live) return;
-    if (KIND == SF_GBDT) {
-        out[f] = acc[0];
-    } else if (KIND == SF_GBDT_MC) {
+    const bool aborted = *abort_flag != 0;
+    if (aborted && threadIdx.x == 0) sf_dev_set_error(st, SF_ERR_DEVICE_TIMEOUT);
+    bool assigned = false;
+    if (live && !aborted) {
+        if (KIND == SF_GBDT) {
+            out[f] = acc[0];
+            if (fr.tau) {                             // |margin| < tau (the binary rule taken in margin space), label = margin > 0
+                const float m = acc[0];
+                assigned = fabsf(m) < __ldg(fr.tau);
+                const uint8_t a = (m > 0.0f) ? 1 : 0;
+                fr.decision[f] = assigned ? 1 : 0; fr.label_fast[f] = a;
+                if (fr.label_out) fr.label_out[f] = a;
+                if (fr.stage_out) fr.stage_out[f] = 1;
+            }
+        } else if (KIND == SF_GBDT_MC) {
 #pragma unroll
-        for (int c = 0; c < C; c++) out[(size_t)f * C + c] = acc[c];
-    } else {
-        const float fT = __uint2float_rn(T);
+            for (int c = 0; c < C; c++) out[(size_t)f * C + c] = acc[c];
+        } else {
+            const float fT = __uint2float_rn(T);
+            float mx = 0.0f; uint32_t a = 0;
 #pragma unroll
-        for (int c = 0; c < C; c++) out[(size_t)f * C + c] = __fdiv_rn(acc[c], fT);
+            for (int c = 0; c < C; c++) {
+                const float p = __fdiv_rn(acc[c], fT);
+                out[(size_t)f * C + c] = p;
+                if (c == 0 || p > mx) { mx = p; a = c; }      // lowest index on ties
+            }
+            if (fr.tau) {                             // least confidence 1 - max > tau[label], strict
+                assigned = __fsub_rn(1.0f, mx) > __ldg(fr.tau + a);
+                fr.decision[f] = assigned ? 1 : 0; fr.label_fast[f] = (uint8_t)a;
+                if (fr.label_out) fr.label_out[f] = (uint8_t)a;
+                if (fr.stage_out) fr.stage_out[f] = 1;
+            }
+        }
+    }
+    if (fr.tau) {
+        // assigned flows of this block: one count per warp in the warp's own first column of the feature tile (nobody
+        // reads that column any more), then a barrier of the walking warps only (the producer warp has left)
+        const uint32_t b = __ballot_sync(0xFFFFFFFFu, assigned);
+        uint32_t* cnt = reinterpret_cast<uint32_t*>(xs);
+        if ((threadIdx.x & 31u) == 0) cnt[threadIdx.x] = __popc(b);
+        asm volatile("bar.sync 1, %0;" ::"r"(KB) : "memory");
+        if (threadIdx.x == 0) {
+            uint32_t tot = 0;
+            for (uint32_t w = 0; w < KB / 32; w++) tot += cnt[w * 32];
+            fr.block_counts[blockIdx.x] = tot;
+        }
     }
 }
 
@@ -398,7 +437,8 @@ Plan make_plan(const sf_forest* fo, uint32_t kb = kB) {
 }
 
 template <int KIND, int C, int NCH, uint32_t KB = kB, bool TEX = false>
-int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
+            const sf_fused_route& fr) {
     auto k = forest_kernel<KIND, C, NCH, KB, TEX>;
     static size_t smem_set_dev[64] = {};               // per kernel instance and device: raise the opt-in limit only when it grows
     size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
@@ -408,38 +448,38 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
     }
     const uint32_t grid = (n + KB - 1) / KB;
     k<<<grid, KB + 32, p.smem, st>>>(feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->leaf_tex, fo->T, fo->depth, fo->tree_stride, p.tpc,
-                                p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev);
+                                p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev, fr);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
 }
 
 template <int C>
-int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev, const sf_fused_route& fr) {
     constexpr bool kTexOk = (C % 4) == 0;                 // whole 16-byte texels per leaf vector
     const bool tex = kTexOk && fo->leaf_tex != 0;
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
     if (p.nch == 2) {
-        if (tex) return launch3<SF_RF, C, 2, kB, kTexOk>(fo, p, feat, n, out, leaf_idx, st, n_dev);
-        return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+        if (tex) return launch3<SF_RF, C, 2, kB, kTexOk>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+        return launch3<SF_RF, C, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
     }
-    if (tex) return launch3<SF_RF, C, 1, kB, kTexOk>(fo, p, feat, n, out, leaf_idx, st, n_dev);
-    return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    if (tex) return launch3<SF_RF, C, 1, kB, kTexOk>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+    return launch3<SF_RF, C, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
 }
 
-int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev, const sf_fused_route& fr) {
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
-    if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st, n_dev);
-    if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev);
-    return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+    if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+    return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
 }
 
 template <int C>
-int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev) {
+int launch_mc(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev, const sf_fused_route& fr) {
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;           // one boosting round does not fit in a chunk
-    return launch3<SF_GBDT_MC, C, (C >= 4 ? 4 : (C >= 2 ? 2 : 1))>(fo, p, feat, n, out, leaf_idx, st, n_dev);
+    return launch3<SF_GBDT_MC, C, (C >= 4 ? 4 : (C >= 2 ? 2 : 1))>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
 }
 
 template <int G>
@@ -513,48 +553,54 @@ int sf_launch_forest_leaf_index_packets(const sf_forest* fo, const sf_packets* p
 }
 
 int sf_launch_forest(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
-                     bool small_tiles) {
+                     bool small_tiles, const sf_fused_route* fused) {
     if (n == 0) return SF_OK;
+    sf_fused_route fr;
+    memset(&fr, 0, sizeof(fr));
+    if (fused) {
+        if (fo->kind == SF_GBDT_MC || small_tiles || kB != SF_FOREST_BLOCK) return SF_ERR_UNSUPPORTED;
+        fr = *fused;
+    }
     if (small_tiles && leaf_idx && fo->kind == SF_RF && fo->d_image_small) return launch_rf_split(fo, feat, n, out, leaf_idx, st, n_dev);
-    if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st, n_dev);
+    if (fo->kind == SF_GBDT) return launch_gbdt(fo, feat, n, out, leaf_idx, st, n_dev, fr);
     if (fo->kind == SF_GBDT_MC) {
         switch (fo->C) {
-        case 1:  return launch_mc<1>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 2:  return launch_mc<2>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 3:  return launch_mc<3>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 4:  return launch_mc<4>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 5:  return launch_mc<5>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 6:  return launch_mc<6>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 7:  return launch_mc<7>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 8:  return launch_mc<8>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 9:  return launch_mc<9>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 10: return launch_mc<10>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 11: return launch_mc<11>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 12: return launch_mc<12>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 13: return launch_mc<13>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 14: return launch_mc<14>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 15: return launch_mc<15>(fo, feat, n, out, leaf_idx, st, n_dev);
-        case 16: return launch_mc<16>(fo, feat, n, out, leaf_idx, st, n_dev);
+        case 1:  return launch_mc<1>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 2:  return launch_mc<2>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 3:  return launch_mc<3>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 4:  return launch_mc<4>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 5:  return launch_mc<5>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 6:  return launch_mc<6>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 7:  return launch_mc<7>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 8:  return launch_mc<8>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 9:  return launch_mc<9>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 10: return launch_mc<10>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 11: return launch_mc<11>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 12: return launch_mc<12>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 13: return launch_mc<13>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 14: return launch_mc<14>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 15: return launch_mc<15>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+        case 16: return launch_mc<16>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
         }
         return SF_ERR_UNSUPPORTED;
     }
     switch (fo->C) {
-    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev);
-    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev);
+    case 1:  return launch_rf<1>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 2:  return launch_rf<2>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 3:  return launch_rf<3>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 4:  return launch_rf<4>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 5:  return launch_rf<5>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 6:  return launch_rf<6>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 7:  return launch_rf<7>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 8:  return launch_rf<8>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 9:  return launch_rf<9>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 10: return launch_rf<10>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 11: return launch_rf<11>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 12: return launch_rf<12>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 13: return launch_rf<13>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 14: return launch_rf<14>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 15: return launch_rf<15>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
+    case 16: return launch_rf<16>(fo, feat, n, out, leaf_idx, st, n_dev, fr);
     }
     return SF_ERR_UNSUPPORTED;
 }

@@ -108,20 +108,23 @@ scan_kernel(uint32_t* __restrict__ block_counts, uint32_t nb, uint32_t n, uint32
     }
 }
 
-__global__ void __launch_bounds__(kScoreBlock)
+// B = flows per block = the granularity of the block counts (1024 after score_kernel, 512 after a tree kernel that took
+// the decisions itself)
+template <int B>
+__global__ void __launch_bounds__(B)
 scatter_kernel(const uint8_t* __restrict__ decision, uint32_t n, const uint32_t* __restrict__ block_offsets,
                uint32_t capacity, uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__ n_dev = nullptr)
 {
     if (n_dev) n = min(n, *n_dev);
-    __shared__ uint32_t warp_off[kScoreBlock / 32];
-    const uint32_t f = blockIdx.x * kScoreBlock + threadIdx.x;
+    __shared__ uint32_t warp_off[32];
+    const uint32_t f = blockIdx.x * B + threadIdx.x;
     const bool esc = (f < n) && decision[f] != 0;
     const uint32_t b = __ballot_sync(0xFFFFFFFFu, esc);
     const uint32_t lane = threadIdx.x & 31;
     if (lane == 0) warp_off[threadIdx.x >> 5] = __popc(b);
     __syncthreads();
     if (threadIdx.x < 32) {
-        uint32_t w = warp_off[threadIdx.x], z = w;
+        uint32_t w = (threadIdx.x < B / 32) ? warp_off[threadIdx.x] : 0u, z = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (threadIdx.x >= o) z += y; }
         warp_off[threadIdx.x] = z - w;
@@ -232,9 +235,11 @@ __global__ void merge_fast_kernel(const uint8_t* __restrict__ label_fast, const 
 
 __global__ void merge_slow_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__ n_esc_dev,
                                   const uint8_t* __restrict__ label_slow, uint8_t* __restrict__ label,
-                                  uint8_t* __restrict__ stage, uint8_t stage_value)
+                                  uint8_t* __restrict__ stage, uint8_t stage_value, sf_dev_state* count_slow_done)
 {
     const uint32_t n_esc = *n_esc_dev;
+    if (count_slow_done && blockIdx.x == 0 && threadIdx.x == 0)
+        atomicAdd((unsigned long long*)&count_slow_done->counters.n_slow_done, (unsigned long long)n_esc);
     for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r < n_esc; r += gridDim.x * blockDim.x) {
         uint32_t f = esc_ids[r];
         if (label) label[f] = label_slow[r];
@@ -328,7 +333,7 @@ int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wid
 }
 
 size_t sf_route_scratch_bytes(uint32_t n) {
-    size_t nb = ((size_t)n + kScoreBlock - 1) / kScoreBlock;
+    size_t nb = ((size_t)n + SF_FOREST_BLOCK - 1) / SF_FOREST_BLOCK;               // the finer of the two block-count granularities
     return sf_align256((nb + 1) * sizeof(uint32_t)) + sf_align256((size_t)n);      // block counts + decision bytes
 }
 
@@ -356,7 +361,7 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
     scan_kernel<<<1, 1024, 0, st>>>(block_counts, nb, n, cfg->capacity, n_esc, ctx->d_state, n_dev);
     SF_LAUNCH_CHECK("scan_kernel");
     if (n > 0) {
-        scatter_kernel<<<nb, kScoreBlock, 0, st>>>(dec, n, block_counts, cfg->capacity, esc_ids, n_dev);
+        scatter_kernel<kScoreBlock><<<nb, kScoreBlock, 0, st>>>(dec, n, block_counts, cfg->capacity, esc_ids, n_dev);
         SF_LAUNCH_CHECK("scatter_kernel");
     }
     sf_time_end(ctx, SF_T_SCORE, st);
@@ -381,9 +386,30 @@ int sf_launch_route(sf_ctx* ctx, const sf_route_cfg* cfg, const float* fast_out,
     return SF_OK;
 }
 
+int sf_launch_route_after_fused(sf_ctx* ctx, const sf_route_cfg* cfg, uint32_t n, const sf_packets* wide, uint32_t* esc_ids,
+                                uint32_t* n_esc, void* rows, const uint8_t* decision, uint32_t* block_counts, cudaStream_t st)
+{
+    const uint32_t nb = (n + SF_FOREST_BLOCK - 1) / SF_FOREST_BLOCK;
+    sf_time_begin(ctx, SF_T_SCORE, st);
+    scan_kernel<<<1, 1024, 0, st>>>(block_counts, nb, n, cfg->capacity, n_esc, ctx->d_state, nullptr);
+    SF_LAUNCH_CHECK("scan_kernel");
+    if (n > 0) {
+        scatter_kernel<(int)SF_FOREST_BLOCK><<<nb, SF_FOREST_BLOCK, 0, st>>>(decision, n, block_counts, cfg->capacity, esc_ids, nullptr);
+        SF_LAUNCH_CHECK("scatter_kernel");
+    }
+    sf_time_end(ctx, SF_T_SCORE, st);
+    if (wide && rows && n > 0 && cfg->capacity > 0) {
+        sf_time_begin(ctx, SF_T_GATHER, st);
+        int rc = sf_launch_gather(ctx, cfg, wide, esc_ids, &ctx->d_state->scan_total, cfg->capacity, rows, st);
+        sf_time_end(ctx, SF_T_GATHER, st);
+        if (rc != SF_OK) return rc;
+    }
+    return SF_OK;
+}
+
 int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t n, const uint32_t* esc_ids,
                     const uint32_t* n_esc, uint32_t capacity, const uint8_t* label_slow,
-                    uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value, bool write_fast)
+                    uint8_t* label, uint8_t* stage, cudaStream_t st, uint8_t stage_value, bool write_fast, sf_dev_state* count_slow_done)
 {
     if (n == 0) return SF_OK;
     if (write_fast)
@@ -392,7 +418,7 @@ int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t
     uint32_t blocks = (capacity + 255) / 256;
     if (blocks > 1184) blocks = 1184;
     if (blocks > 0) {
-        merge_slow_kernel<<<blocks, 256, 0, st>>>(esc_ids, n_esc, label_slow, label, stage, stage_value);
+        merge_slow_kernel<<<blocks, 256, 0, st>>>(esc_ids, n_esc, label_slow, label, stage, stage_value, count_slow_done);
         SF_LAUNCH_CHECK("merge_slow_kernel");
     }
     return SF_OK;
@@ -488,7 +514,7 @@ extern "C" int sf_route_noalloc(int device, const sf_route_cfg* cfg, const float
     scan_kernel<<<1, 1024, 0, st>>>(sc->block_counts, nb, n, cfg->capacity, n_esc_out, &sc->state);
     SF_LAUNCH_CHECK("scan_kernel");
     if (n > 0) {
-        scatter_kernel<<<nb, kScoreBlock, 0, st>>>(dec, n, sc->block_counts, cfg->capacity, esc_ids_out);
+        scatter_kernel<kScoreBlock><<<nb, kScoreBlock, 0, st>>>(dec, n, sc->block_counts, cfg->capacity, esc_ids_out);
         SF_LAUNCH_CHECK("scatter_kernel");
     }
     if (status_out) {

@@ -69,6 +69,22 @@ def run_and_check(sf, hz, ctx, wl, capacity=None):
     clear = (s[:, -1] - s[:, -2]) >= 2 * tol
     assert np.array_equal(lab[ref["esc_ids"]][clear], ref["label_slow"][clear])
     assert np.array_equal(lab[ref["esc_ids"]], hz.ptr_tensor(p["label_slow"], (k,), torch.uint8).cpu().numpy())
+    # the composite call folds the assignment into the tree kernel: the staged calls must give the same bits
+    lab_fast = hz.ptr_tensor(p["label_fast"], (n,), torch.uint8).cpu().numpy()
+    feat_s = torch.empty((n, cfg.F), dtype=torch.float32, device="cuda")
+    fo_s = torch.empty((n, Cf), dtype=torch.float32, device="cuda")
+    ids_s = torch.full((max(cap, 1),), 0xFFFFFFFF, dtype=torch.uint32, device="cuda")
+    ne_s = torch.zeros(1, dtype=torch.uint32, device="cuda")
+    dec_s = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    lab_s = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    sf.sf_extract_features(ctx, fast_d["struct"], cfg.N, cfg.F, feat_s)
+    sf.sf_fast_infer(ctx, forest, feat_s, n, fo_s)
+    sf.sf_route(ctx, rcfg, fo_s, n, Cf if cfg.kind != "gbdt" else 1, None, ids_s, ne_s, None, dec_s, lab_s, None)
+    torch.cuda.synchronize()
+    sf.sf_ctx_poll(ctx, reset=True)
+    assert np.array_equal(bits(fo_s.cpu().numpy().reshape(fo.shape)), bits(fo))
+    assert int(ne_s.cpu().numpy()[0]) == k and np.array_equal(ids_s.cpu().numpy()[:k], ids)
+    assert np.array_equal(dec_s.cpu().numpy(), (st >= 2).astype(np.uint8)) and np.array_equal(lab_s.cpu().numpy(), lab_fast)
     # host-pointer entry point gives the same answers
     fast_h = hz.pinned_packets(wl["fast"], with_hdr=False)
     wide_h = hz.pinned_packets(wl["wide"])
