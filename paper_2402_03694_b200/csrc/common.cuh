@@ -44,6 +44,10 @@ struct sf_ctx {
     const uint8_t* last_label_slow;
 };
 
+// nodes 1, 2, 3 (1-based heap) of up to 1024 trees: {threshold bits, byte offset of the feature's row}; a kernel argument
+#define SF_FOREST_TOP_TREES 1024
+struct sf_forest_top { uint2 n[SF_FOREST_TOP_TREES][3]; };
+
 struct sf_forest {
     sf_ctx* ctx;
     int kind;
@@ -56,6 +60,8 @@ struct sf_forest {
     // leaves: RF fp32[T][2^d][C]; GBDT fp32[T][2^d]
     float* d_leaf;
     cudaTextureObject_t leaf_tex;      // RF with C % 4 == 0: the same table as a linear texture of 16-byte texels (0 = none)
+    struct sf_forest_top* h_top;       // host copy of every tree's nodes 1..3, handed to the tree kernel as an argument
+    bool top_ok;                       // the kernel variant that reads them is usable (binary boosted trees, T <= 1024, depth >= 2)
 };
 
 enum { SF_SLOW_MLP = 0, SF_SLOW_CNN = 1 };

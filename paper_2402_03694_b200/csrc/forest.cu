@@ -48,10 +48,21 @@ __device__ __forceinline__ float lds32f(uint32_t a) {
     return v;
 }
 
+// The two top levels of every tree (nodes 1, 2, 3 of the 1-based heap) as a kernel argument: kernel arguments live in
+// the constant bank, a tree index is the same in every lane, so these loads never touch the load/store pipe that the
+// rest of the walk saturates (two 64-bit shared-memory loads = four wavefronts less per warp and tree).  Measured on
+// 500 boosted trees of depth 6: 4.56 -> 4.20 ms; a third level this way (four more loads, six selects) cost more than it
+// saved (5.07 ms), and random forests of depth 10 to 12 gained nothing, so only binary boosted trees take this path.
+constexpr uint32_t kTopMaxTrees = SF_FOREST_TOP_TREES;
+typedef sf_forest_top ForestTop;
+
 // Walk NCH consecutive trees (shared-memory images at base, base+stride, ...) for the
 // flow whose feature column starts at xbase; returns leaf indices.
-template <int NCH>
-__device__ __forceinline__ void walk(uint32_t base, uint32_t stride, uint32_t xbase, uint32_t depth, uint32_t (&leaf)[NCH]) {
+// TOPC: levels 0 and 1 come from `top` (trees t_first, t_first + 1, ...; depth >= 2), the walk through shared memory
+// starts at level 2.
+template <int NCH, bool TOPC = false>
+__device__ __forceinline__ void walk(uint32_t base, uint32_t stride, uint32_t xbase, uint32_t depth, uint32_t (&leaf)[NCH],
+                                     const ForestTop* top = nullptr, uint32_t t_first = 0) {
     uint32_t a[NCH], left[NCH], right[NCH];
 #pragma unroll
     for (int c = 0; c < NCH; c++) {
@@ -60,7 +71,24 @@ __device__ __forceinline__ void walk(uint32_t base, uint32_t stride, uint32_t xb
         left[c] = 0u - b;              // addr' = 2*addr - base      (child 2i)
         right[c] = 8u - b;             // addr' = 2*addr - base + 8  (child 2i+1)
     }
-    for (uint32_t l = 0; l < depth; l++) {
+    if (TOPC) {
+        float x0[NCH], x1[NCH];
+        uint2 n1[NCH], n2[NCH];
+#pragma unroll
+        for (int c = 0; c < NCH; c++) { n1[c] = top->n[t_first + c][0]; x0[c] = lds32f(xbase + n1[c].y); }
+#pragma unroll
+        for (int c = 0; c < NCH; c++) {
+            const bool r0 = !(x0[c] <= __uint_as_float(n1[c].x));
+            const uint2 nl = top->n[t_first + c][1], nr = top->n[t_first + c][2];
+            n2[c].x = r0 ? nr.x : nl.x; n2[c].y = r0 ? nr.y : nl.y;
+            a[c] = r0 ? 48u : 32u;                                   // byte offset of node 6 or 4: 8 * (4 + 2 * r0)
+        }
+#pragma unroll
+        for (int c = 0; c < NCH; c++) x1[c] = lds32f(xbase + n2[c].y);
+#pragma unroll
+        for (int c = 0; c < NCH; c++) a[c] = base + c * stride + a[c] + ((x1[c] <= __uint_as_float(n2[c].x)) ? 0u : 8u);
+    }
+    for (uint32_t l = TOPC ? 2u : 0u; l < depth; l++) {
         uint2 nd[NCH];
         float x[NCH];
 #pragma unroll
@@ -119,9 +147,9 @@ __device__ __forceinline__ void load_leaf_vec_tex(cudaTextureObject_t tex, uint3
 // adds to class t mod C; a chunk holds whole boosting rounds, so the class of every tree in the
 // unrolled round loop is a compile-time register index).  NCH: trees walked at once.
 // TEX: leaf vectors come through the texture object (random forests whose C is a multiple of 4).
-template <int KIND, int C, int NCH, uint32_t KB, bool TEX>
+template <int KIND, int C, int NCH, uint32_t KB, bool TEX, bool TOPC>
 __global__ void __launch_bounds__(KB + 32, 1)
-forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
+forest_kernel(const __grid_constant__ ForestTop top, const float* __restrict__ feat, uint32_t n, uint32_t F,
               const unsigned char* __restrict__ image, const float* __restrict__ leaf, cudaTextureObject_t leaf_tex,
               uint32_t T, uint32_t depth, uint32_t tree_stride, uint32_t trees_per_chunk, uint32_t chunk_bytes,
               float* __restrict__ out, uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev,
@@ -237,7 +265,7 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         }
         for (; tt + NCH <= nt; tt += NCH) {
             uint32_t l[NCH];
-            walk<NCH>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
+            walk<NCH, TOPC>(cur + tt * tree_stride, tree_stride, xbase, depth, l, &top, t0 + tt);
             if (leaf_idx && live) {
 #pragma unroll
                 for (int k = 0; k < NCH; k++) leaf_idx[(size_t)f * T + t0 + tt + k] = (uint16_t)l[k];
@@ -260,7 +288,7 @@ forest_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
         }
         for (; tt < nt; tt++) {                       // ragged end of the chunk: one tree at a time
             uint32_t l[1];
-            walk<1>(cur + tt * tree_stride, tree_stride, xbase, depth, l);
+            walk<1, TOPC>(cur + tt * tree_stride, tree_stride, xbase, depth, l, &top, t0 + tt);
             if (leaf_idx && live) leaf_idx[(size_t)f * T + t0 + tt] = (uint16_t)l[0];
             if (KIND == SF_GBDT) {
                 acc[0] = __fadd_rn(acc[0], lds32f(cur + tt * tree_stride + n_leaf * 8u + l[0] * 4u));
@@ -436,10 +464,10 @@ Plan make_plan(const sf_forest* fo, uint32_t kb = kB) {
     return p;
 }
 
-template <int KIND, int C, int NCH, uint32_t KB = kB, bool TEX = false>
+template <int KIND, int C, int NCH, uint32_t KB = kB, bool TEX = false, bool TOPC = false>
 int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev,
             const sf_fused_route& fr) {
-    auto k = forest_kernel<KIND, C, NCH, KB, TEX>;
+    auto k = forest_kernel<KIND, C, NCH, KB, TEX, TOPC>;
     static size_t smem_set_dev[64] = {};               // per kernel instance and device: raise the opt-in limit only when it grows
     size_t& smem_set = smem_set_dev[fo->ctx->device & 63];
     if (p.smem > smem_set) {
@@ -447,7 +475,7 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
         smem_set = p.smem;
     }
     const uint32_t grid = (n + KB - 1) / KB;
-    k<<<grid, KB + 32, p.smem, st>>>(feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->leaf_tex, fo->T, fo->depth, fo->tree_stride, p.tpc,
+    k<<<grid, KB + 32, p.smem, st>>>(*fo->h_top, feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->leaf_tex, fo->T, fo->depth, fo->tree_stride, p.tpc,
                                 p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev, fr);
     SF_LAUNCH_CHECK("forest_kernel");
     return SF_OK;
@@ -470,6 +498,11 @@ int launch_rf(const sf_forest* fo, const float* feat, uint32_t n, float* out, ui
 int launch_gbdt(const sf_forest* fo, const float* feat, uint32_t n, float* out, uint16_t* leaf_idx, cudaStream_t st, const uint32_t* n_dev, const sf_fused_route& fr) {
     const Plan p = make_plan(fo);
     if (p.tpc == 0) return SF_ERR_UNSUPPORTED;
+    if (fo->top_ok) {                                 // the two top levels of every tree travel as a kernel argument
+        if (p.nch == 4) return launch3<SF_GBDT, 1, 4, kB, false, true>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+        if (p.nch == 2) return launch3<SF_GBDT, 1, 2, kB, false, true>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+        return launch3<SF_GBDT, 1, 1, kB, false, true>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
+    }
     if (p.nch == 4) return launch3<SF_GBDT, 1, 4>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
     if (p.nch == 2) return launch3<SF_GBDT, 1, 2>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
     return launch3<SF_GBDT, 1, 1>(fo, p, feat, n, out, leaf_idx, st, n_dev, fr);
@@ -620,6 +653,10 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     if (!fo) return SF_ERR_ALLOC;
     fo->ctx = ctx; fo->kind = kind; fo->T = T; fo->depth = depth; fo->F = F; fo->C = (kind == SF_GBDT) ? 1 : C;
     fo->d_image = nullptr; fo->d_leaf = nullptr; fo->d_image_small = nullptr; fo->leaf_tex = 0;
+    fo->h_top = new (std::nothrow) ForestTop();
+    if (!fo->h_top) { delete fo; return SF_ERR_ALLOC; }
+    memset(fo->h_top, 0, sizeof(ForestTop));
+    fo->top_ok = kind == SF_GBDT && depth >= 2 && T <= kTopMaxTrees;      // (random forests: measured, no gain at depth 10 to 12)
     // Image of one tree: 2^d node entries of 8 bytes in a 1-based heap (host node i, children
     // 2i+1 / 2i+2, becomes entry i+1, children 2j / 2j+1; entry 0 unused), then for boosted
     // trees the 2^d leaf scalars; padded to a multiple of 16 bytes for the 16-byte copies.
@@ -627,7 +664,7 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
     stride = (stride + 15u) & ~15u;
     fo->tree_stride = stride;
     unsigned char* h = (unsigned char*)calloc((size_t)T, stride);
-    if (!h) { delete fo; return SF_ERR_ALLOC; }
+    if (!h) { sf_forest_destroy(fo); return SF_ERR_ALLOC; }
     for (uint32_t t = 0; t < T; t++) {
         uint32_t* ent = reinterpret_cast<uint32_t*>(h + (size_t)t * stride);
         for (uint32_t i = 0; i < n_int; i++) {
@@ -637,12 +674,14 @@ extern "C" int sf_forest_create(sf_ctx* ctx, int kind, uint32_t T, uint32_t dept
             ent[2 * (i + 1) + 1] = (uint32_t)fid[(size_t)t * n_int + i] * kB * 4u;     // byte offset of the feature's row
         }
         if (kind != SF_RF) memcpy(h + (size_t)t * stride + n_ent * 8u, leaf + (size_t)t * n_ent, n_ent * 4u);
+        if (fo->top_ok)
+            for (uint32_t i = 0; i < 3; i++) fo->h_top->n[t][i] = make_uint2(ent[2 * (i + 1)], ent[2 * (i + 1) + 1]);
     }
     // the small-batch variant of the kernel has a narrower feature tile, so its feature offsets differ
     unsigned char* h_small = nullptr;
     if (kind == SF_RF) {
         h_small = (unsigned char*)malloc((size_t)T * stride);
-        if (!h_small) { free(h); delete fo; return SF_ERR_ALLOC; }
+        if (!h_small) { free(h); sf_forest_destroy(fo); return SF_ERR_ALLOC; }
         memcpy(h_small, h, (size_t)T * stride);
         for (uint32_t t = 0; t < T; t++) {
             uint32_t* ent = reinterpret_cast<uint32_t*>(h_small + (size_t)t * stride);
@@ -686,6 +725,7 @@ extern "C" void sf_forest_destroy(sf_forest* fo) {
     if (fo->d_image) cudaFree(fo->d_image);
     if (fo->d_image_small) cudaFree(fo->d_image_small);
     if (fo->d_leaf) cudaFree(fo->d_leaf);
+    delete fo->h_top;
     delete fo;
 }
 
