@@ -65,7 +65,7 @@ template <uint32_t BN> struct GemmCfg {
     static constexpr uint32_t kTmemCols = 2 * BN;             // a power of two >= 32
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
                                            kEpiWarps * 2048 /*epilogue staging*/;
-    // fused head: the staging space holds the head's weights [col][8] bf16 (N <= 1024); 16 more KB for [col][16]
+    // fused head: the head's weights (N <= 1024 columns x 32 bytes) take the staging space and 16 KB more
     static constexpr uint32_t kSmemBytesHead16 = kSmemBytes + 16384;
 };
 
@@ -222,10 +222,13 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     // fused head: the head's weights, transposed to [column][CH] bf16, where the other modes stage their output
     uint8_t* const epi_smem = tiles + Cfg::kStages * Cfg::kStageBytes + 256;
     if constexpr (FUSED) {
-        __nv_bfloat16* whT = reinterpret_cast<__nv_bfloat16*>(epi_smem);
+        // up to 8 classes: fp32 [column][8] (the bf16 values widened once here instead of once per row in the epilogue, whose
+        // integer pipe is the busy one); up to 16: bf16 [column][16]; 32 KB either way
         for (uint32_t i = threadIdx.x; i < N * CH; i += kGemmThreads) {
             const uint32_t col = i / CH, c = i - col * CH;
-            whT[i] = head_w[(size_t)c * N + col];                // rows past C are zero in the padded head matrix
+            const __nv_bfloat16 w = head_w[(size_t)c * N + col];                // rows past C are zero in the padded head matrix
+            if (CH == 8) reinterpret_cast<float*>(epi_smem)[i] = __bfloat162float(w);
+            else reinterpret_cast<__nv_bfloat16*>(epi_smem)[i] = w;
         }
     }
     tc_fence_before();
@@ -332,7 +335,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                     tmem_ld32(taddr + c, v);
                     tmem_ld_wait();
                     const float4* b4 = reinterpret_cast<const float4*>(bias + col0 + c);
-                    const uint4* wq = reinterpret_cast<const uint4*>(epi_smem) + (size_t)(col0 + c) * (CH / 8);
+                    const uint4* wq = reinterpret_cast<const uint4*>(epi_smem) + (size_t)(col0 + c) * 2;     // 32 bytes per column
 #pragma unroll
                     for (int pc = 0; pc < 8; pc++) {
                         const float4 bv = __ldg(b4 + pc);
@@ -347,15 +350,19 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                             const float a[2] = {__uint_as_float(hb << 16), __uint_as_float(hb & 0xFFFF0000u)};
 #pragma unroll
                             for (int q = 0; q < 2; q++) {
-                                const uint4* wp = wq + (size_t)(pc * 4 + e + q) * (CH / 8);      // same address in all lanes: a broadcast
+                                const uint4* wp = wq + (size_t)(pc * 4 + e + q) * 2;      // same address in all lanes: a broadcast
 #pragma unroll
-                                for (uint32_t g = 0; g < CH / 8; g++) {
+                                for (uint32_t g = 0; g < 2; g++) {
                                     const uint4 w = wp[g];
                                     const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                                     for (int k = 0; k < 4; k++) {
-                                        lg[g * 8 + 2 * k] = fmaf(a[q], __uint_as_float(ww[k] << 16), lg[g * 8 + 2 * k]);
-                                        lg[g * 8 + 2 * k + 1] = fmaf(a[q], __uint_as_float(ww[k] & 0xFFFF0000u), lg[g * 8 + 2 * k + 1]);
+                                        if (CH == 8) {
+                                            lg[g * 4 + k] = fmaf(a[q], __uint_as_float(ww[k]), lg[g * 4 + k]);
+                                        } else {
+                                            lg[g * 8 + 2 * k] = fmaf(a[q], __uint_as_float(ww[k] << 16), lg[g * 8 + 2 * k]);
+                                            lg[g * 8 + 2 * k + 1] = fmaf(a[q], __uint_as_float(ww[k] & 0xFFFF0000u), lg[g * 8 + 2 * k + 1]);
+                                        }
                                     }
                                 }
                             }
@@ -473,7 +480,7 @@ int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bia
                      uint32_t N, uint32_t K, const void* W16, const float* head_bias, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
 {
     using Cfg = GemmCfg<BN>;
-    constexpr uint32_t kSmem = CH == 8 ? Cfg::kSmemBytes : Cfg::kSmemBytesHead16;
+    constexpr uint32_t kSmem = Cfg::kSmemBytesHead16;        // 32 KB of head weights where the other modes stage 16 KB of output
     CUtensorMap tmA, tmW;
     int rc = encode_tmap_bf16_2d(&tmA, A, capacity, K, BM, BK);
     if (rc != SF_OK) return rc;
