@@ -60,6 +60,7 @@ struct sf_table {
     // per-batch scratch with fixed addresses
     uint32_t* key_a; uint32_t* key_b; uint32_t* idx_a; uint32_t* idx_b; uint32_t* rank; uint32_t* pos;
     uint32_t* fire1_slot; uint32_t* fire2_slab; uint32_t* fire2_slot;
+    uint32_t* run0;                   // [key] position where the run of the flow with that sort key starts in the sorted batch
     uint32_t* counts;                 // [0] n_fire1, [1] n_fire2
     uint32_t* pkt_slot; uint32_t* hist;
     void* all;                        // one allocation behind everything above
@@ -101,15 +102,17 @@ __global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ 
                              sf_batch_result* res, sf_dev_state* st)
 {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= b.n) return;
-    uint64_t lo, hi;
-    make_key(b.src[i], b.dst[i], b.sport[i], b.dport[i], b.proto[i], lo, hi);
+    const bool valid = i < b.n;                      // every lane stays to the end: the counters are added up per warp
+    const uint32_t lane = threadIdx.x & 31u;
+    uint64_t lo = 0, hi = 0;
+    if (valid) make_key(b.src[i], b.dst[i], b.sport[i], b.dport[i], b.proto[i], lo, hi);
     uint32_t slot = t.n_slots;                       // "missed" sorts after every real slot
+    bool is_new = false;
     // Walk the whole probe chain: the key may sit behind a tombstone.  If it is absent, claim the
     // first tombstone seen, else the empty slot that ends the chain.  Every thread with this key
     // walks the same chain and slots only ever change from free to taken during a batch, so all
     // of them end at one slot.  A lost race against another key restarts the walk (bounded).
-    for (uint32_t attempt = 0; attempt < 16 && slot == t.n_slots; attempt++) {
+    for (uint32_t attempt = 0; valid && attempt < 16 && slot == t.n_slots; attempt++) {
         uint32_t h = hash_key(lo, hi, t.mask), cand = t.n_slots;
         bool cand_tomb = false;
         for (uint32_t p = 0; p < kProbeLimit; p++) {
@@ -124,16 +127,23 @@ __global__ void probe_kernel(TableDev t, sf_pkt_batch b, uint32_t* __restrict__ 
         uint64_t olo, ohi;
         const uint64_t c = cand_tomb ? kTomb : 0ull;
         cas128(&t.keys[cand], c, c, lo, hi, olo, ohi);
-        if (olo == c && ohi == c) { slot = cand; atomicAdd(&res->n_new_flows, 1u); }
+        if (olo == c && ohi == c) { slot = cand; is_new = true; }
         else if (olo == lo && ohi == hi) slot = cand;
     }
-    if (slot == t.n_slots) {
-        atomicAdd(&res->n_missed, 1u);
-        atomicAdd((unsigned long long*)&st->counters.n_missed, 1ull);
+    // One atomic per warp and counter, and one atomicMin per warp and flow: a heavy flow puts thousands of packets of a
+    // batch on one slot, and same-address atomics are served one after the other.
+    const bool missed = valid && slot == t.n_slots;
+    const uint32_t m_new = __ballot_sync(0xFFFFFFFFu, is_new), m_miss = __ballot_sync(0xFFFFFFFFu, missed);
+    if (lane == 0 && m_new) atomicAdd(&res->n_new_flows, (uint32_t)__popc(m_new));
+    if (lane == 0 && m_miss) {
+        atomicAdd(&res->n_missed, (uint32_t)__popc(m_miss));
+        atomicAdd((unsigned long long*)&st->counters.n_missed, (unsigned long long)__popc(m_miss));
         sf_dev_set_error(st, SF_ERR_TABLE_FULL);
     }
-    else atomicMin(&t.first[slot], i);
-    pkt_slot[i] = slot;
+    // lanes hold consecutive arrival indices, so the lowest lane among those with the same slot holds their minimum
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, (valid && !missed) ? slot : (0xFFFFFFC0u + lane));
+    if (valid && !missed && (peers & ((1u << lane) - 1u)) == 0) atomicMin(&t.first[slot], i);
+    if (valid) pkt_slot[i] = slot;
 }
 
 // Sort key of a packet = arrival index of its flow's first packet in this batch: 16 bits,
@@ -172,7 +182,7 @@ key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
 __global__ void __launch_bounds__(256)
 radix8_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ iin, uint32_t* __restrict__ kout,
                       uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk,
-                      uint32_t* __restrict__ next_hist)
+                      uint32_t* __restrict__ next_hist, uint32_t* __restrict__ run_start_of)
 {
     __shared__ uint32_t base[256];
     __shared__ uint32_t wc[8][256];
@@ -212,8 +222,12 @@ radix8_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restri
         __syncthreads();
         if (valid) {
             const uint32_t p = wc[warp][d] + below;
+            const uint32_t id = iin[i];
             kout[p] = key;
-            iout[p] = iin[i];
+            iout[p] = id;
+            // last pass: a key is the arrival index of its flow's first packet, so the item whose index equals its key opens
+            // the flow's run in the sorted order
+            if (run_start_of && id == key) run_start_of[key] = p;
             if (next_hist) atomicAdd(&nh[((key >> (shift + 8)) & 255u) * (kMaxTiles / 2) + (p >> 11)], 1u << (16u * ((p >> 10) & 1u)));
         }
         __syncthreads();
@@ -228,12 +242,6 @@ radix8_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restri
             }
         }
     }
-}
-
-__device__ __forceinline__ uint32_t run_start(const uint32_t* __restrict__ s_key, uint32_t n, uint32_t key) {
-    uint32_t lo = 0, hi = n;                             // first position whose key is >= key
-    while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (s_key[mid] < key) lo = mid + 1; else hi = mid; }
-    return lo;
 }
 
 __device__ __forceinline__ void store_packet(uint16_t* sz, uint32_t* ia, uint32_t* dirw, uint8_t* hd, uint32_t row,
@@ -256,6 +264,7 @@ __device__ __forceinline__ void release_slab(const TableDev& t, uint32_t s) {
 }
 
 __global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
+                              const uint32_t* __restrict__ run_start_of,
                               const uint32_t* __restrict__ pkt_slot, uint32_t* __restrict__ rank, uint32_t* __restrict__ pos_out,
                               uint32_t* __restrict__ fire1_slot, uint32_t* __restrict__ counts)
 {
@@ -263,7 +272,7 @@ __global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
     if (j >= b.n) return;
     const uint32_t slot = pkt_slot[s_idx[j]];
     if (slot >= t.n_slots) { pos_out[j] = kMiss; rank[j] = 0; return; }
-    const uint32_t rk = j - run_start(s_key, b.n, s_key[j]);     // arrival rank among the flow's packets of this batch
+    const uint32_t rk = j - run_start_of[s_key[j]];              // arrival rank among the flow's packets of this batch
     rank[j] = rk;
     const uint32_t pos = t.cnt[slot] + rk;
     pos_out[j] = pos;
@@ -283,15 +292,25 @@ fast_finish_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const ui
                    const uint16_t* __restrict__ leaf_idx, const float* __restrict__ leaf, uint32_t T, uint32_t n_leaf, uint32_t C,
                    const float* __restrict__ tau, sf_batch_result* res, sf_dev_state* st)
 {
-    const uint32_t gi = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t k = gi >> 4, c = gi & 15u;
-    const bool live = k < counts[0];
+    const uint32_t c = threadIdx.x & 15u;
+    const uint32_t n_fired = counts[0];
+    // a few hundred flows fire per batch, the batch could hold 65,536: a small grid walks over the fired flows
+    for (uint32_t k0 = blockIdx.x * (blockDim.x >> 4); k0 < n_fired; k0 += gridDim.x * (blockDim.x >> 4)) {
+    const uint32_t k = k0 + (threadIdx.x >> 4);
+    const bool live = k < n_fired;
     float prob = -1.0f;                                  // below every probability: lanes past C never win
     if (live && c < C) {
         const uint16_t* idx = leaf_idx + (size_t)k * T;
         float acc = 0.0f;
         uint32_t tt = 0;
-        for (; tt + 8 <= T; tt += 8) {                    // eight loads in flight, added in tree order
+        for (; tt + 32 <= T; tt += 32) {                  // 32 loads in flight (the kernel lives on their latency), added in tree order
+            float v[32];
+#pragma unroll
+            for (int q = 0; q < 32; q++) v[q] = __ldg(leaf + ((size_t)(tt + q) * n_leaf + idx[tt + q]) * C + c);
+#pragma unroll
+            for (int q = 0; q < 32; q++) acc = __fadd_rn(acc, v[q]);
+        }
+        for (; tt + 8 <= T; tt += 8) {
             float v[8];
 #pragma unroll
             for (int q = 0; q < 8; q++) v[q] = __ldg(leaf + ((size_t)(tt + q) * n_leaf + idx[tt + q]) * C + c);
@@ -352,6 +371,7 @@ fast_finish_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const ui
         for (uint32_t i = c; i < t.fast_pkts * kHdr; i += 16) dst[i] = src[i];
         if (c == 0) atomicOr(&t.s_dir[(size_t)slab * ((t.slow_pkts + 31) / 32)], t.f_dir[slot]);
     }
+    }
 }
 
 __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __restrict__ s_key, const uint32_t* __restrict__ s_idx,
@@ -360,11 +380,11 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
                               uint32_t* __restrict__ counts, sf_batch_result* res, sf_dev_state* st)
 {
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= b.n) return;
-    const uint32_t slot = pkt_slot[s_idx[j]];
-    if (slot >= t.n_slots) return;
-    const uint32_t pos = pos_in[j];
-    if (pos >= t.fast_pkts) {
+    const uint32_t slot = (j < b.n) ? pkt_slot[s_idx[j]] : t.n_slots;
+    const bool live = slot < t.n_slots;              // every lane stays to the end: the counter is added up per warp
+    bool dropped = false;
+    const uint32_t pos = live ? pos_in[j] : 0u;
+    if (live && pos >= t.fast_pkts) {
         const uint32_t stg = t.stage[slot];
         if (stg == 2 && pos < t.slow_pkts) {
             const uint32_t s = t.slab[slot];
@@ -374,10 +394,15 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
                 fire2_slab[k] = s; fire2_slot[k] = slot;
             }
         } else {
-            atomicAdd(&res->n_dropped_after_decision, 1u);
-            atomicAdd((unsigned long long*)&st->counters.n_dropped_after_decision, 1ull);
+            dropped = true;
         }
     }
+    const uint32_t m_drop = __ballot_sync(0xFFFFFFFFu, dropped);
+    if ((threadIdx.x & 31u) == 0 && m_drop) {
+        atomicAdd(&res->n_dropped_after_decision, (uint32_t)__popc(m_drop));
+        atomicAdd((unsigned long long*)&st->counters.n_dropped_after_decision, (unsigned long long)__popc(m_drop));
+    }
+    if (!live) return;
     // the last packet of the flow's run in this batch advances the flow's packet counter
     if (j + 1 == b.n || s_key[j + 1] != s_key[j]) { t.cnt[slot] += rank[j] + 1; t.first[slot] = 0xFFFFFFFFu; t.last_seen[slot] = t.now; }
 }
@@ -479,7 +504,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     need(S * fast_pkts * 2); need(S * fast_pkts * 4); need(S * 4); need(S * fast_pkts * kHdr);
     need(B * slow_pkts * 2); need(B * slow_pkts * 4); need(B * W * 4); need(B * slow_pkts * kHdr); need(4);
     need(B * 4); need(4); need(S * 4);
-    for (int k = 0; k < 9; k++) need((size_t)kMaxBatch * 4);
+    for (int k = 0; k < 10; k++) need((size_t)kMaxBatch * 4);
     need((16 + 2 * kHistWords) * 4); need((size_t)kMaxBatch * 4); need(S * 4);     // counters + digit counts, pkt_slot, first
     cudaError_t e = cudaMalloc(&t->all, total);
     if (e != cudaSuccess) { delete t; sf_set_cuda_error(e, "cudaMalloc(table)"); return SF_ERR_ALLOC; }
@@ -503,6 +528,7 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     t->rank = carve<uint32_t>(p, kMaxBatch); t->pos = carve<uint32_t>(p, kMaxBatch);
     t->fire1_slot = carve<uint32_t>(p, kMaxBatch); t->fire2_slab = carve<uint32_t>(p, kMaxBatch);
     t->fire2_slot = carve<uint32_t>(p, kMaxBatch);
+    t->run0 = carve<uint32_t>(p, kMaxBatch);
     t->counts = carve<uint32_t>(p, 16 + 2 * kHistWords);     // counters, then the two passes' digit counts (cleared together)
     t->hist = t->counts + 16;
     t->pkt_slot = carve<uint32_t>(p, kMaxBatch);
@@ -562,12 +588,12 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     SF_LAUNCH_CHECK("key_kernel");
     {
         // 16-bit keys: two 8-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
-        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_a, t->idx_a, t->key_b, t->idx_b, n, 0, t->hist, nblk, t->hist + kHistWords);
+        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_a, t->idx_a, t->key_b, t->idx_b, n, 0, t->hist, nblk, t->hist + kHistWords, nullptr);
         SF_LAUNCH_CHECK("radix pass 0");
-        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_b, t->idx_b, t->key_a, t->idx_a, n, 8, t->hist + kHistWords, nblk, nullptr);
+        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_b, t->idx_b, t->key_a, t->idx_a, n, 8, t->hist + kHistWords, nblk, nullptr, t->run0);
         SF_LAUNCH_CHECK("radix pass 1");
     }
-    apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts);
+    apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->run0, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts);
     SF_LAUNCH_CHECK("apply1_kernel");
     sf_time_end(ctx, SF_T_TABLE, st);
     // S1..S3 on the flows that just completed their fast context (count stays on the device); the feature kernel reads
@@ -588,7 +614,7 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_SCORE, st);
     // ... then leaf sums, score, decision and the table update in one kernel (16 lanes per flow)
-    fast_finish_kernel<<<(n * 16u + 255) / 256, 256, 0, st>>>(d, t->fire1_slot, t->counts, reinterpret_cast<const uint16_t*>(w + o_lidx), fo->d_leaf,
+    fast_finish_kernel<<<std::min<uint32_t>((n * 16u + 255) / 256, (uint32_t)ctx->num_sms * 2u), 256, 0, st>>>(d, t->fire1_slot, t->counts, reinterpret_cast<const uint16_t*>(w + o_lidx), fo->d_leaf,
                                                              fo->T, 1u << fo->depth, fo->C, cfg->tau, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("fast_finish_kernel");
     apply2_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire2_slab, t->fire2_slot,
