@@ -220,7 +220,9 @@ def rooflines_for(cfg, n, k_esc, avg, peaks, clocks):
         "gather": ("hbm", k_esc * (per_esc_in + cfg.D * esz) / 1e9),
         # scan + scatter (the tree kernel's epilogue took the decisions): decision bytes in, ids out
         "score": ("hbm", (n + 4 * k_esc) / 1e9),
-        "forest": ("alu", (n / 32.0) * cfg.T * (cfg.depth * FOREST_WAVEFRONTS_PER_VISIT + (4 * Cf * 32) / 128.0) / 1e9),
+        # (binary boosted trees take the node of their two top levels from the constant bank: two 64-bit loads less per tree)
+        "forest": ("alu", (n / 32.0) * cfg.T * (cfg.depth * FOREST_WAVEFRONTS_PER_VISIT - (4 if cfg.kind == "gbdt" and cfg.depth >= 2 and cfg.T <= 1024 else 0) +
+                                               (4 * Cf * 32) / 128.0) / 1e9),
     }
     if cfg.slow_dtype == "bf16":
         work["gemm"] = ("tensor", k_esc * hidden_flops_per_row(cfg) / 1e12)
