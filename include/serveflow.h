@@ -346,7 +346,8 @@ int  sf_serve_batch_intermediates(sf_ctx* ctx, const float** feat, const float**
                                   const uint8_t** label_slow);
 
 /* ---- streaming: device-resident per-flow state table ----------------------- */
-/* One batch of interleaved packets, struct of arrays (device), n <= 65536. */
+/* One batch of interleaved packets, struct of arrays (device).  More than 65,536 packets in one call are
+ * ingested as consecutive pieces of 65,536 (the table ends as if each piece had come in its own call). */
 typedef struct {
     const uint32_t* src; const uint32_t* dst;     /* addresses */
     const uint16_t* sport; const uint16_t* dport; /* ports */

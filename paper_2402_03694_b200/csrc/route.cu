@@ -172,7 +172,14 @@ gather_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__
         uint32_t m = P_real;
         if (n_valid) m = min(m, (uint32_t)n_valid[f]);
         const size_t row0 = (size_t)f * pitch;
-        for (uint32_t i = lane; i < P; i += 32) {
+        // PPL packets per lane so that a lane writes 32 contiguous bytes of bf16 (one packet of 16 fields, two of 8): a warp pass
+        // then covers 1 KB of the row whatever the layout
+        constexpr int PPL = (BF16 && W == 8) ? 2 : 1;
+        for (uint32_t i0 = lane * PPL; i0 < P; i0 += 32 * PPL) {
+#pragma unroll
+          for (int q = 0; q < PPL; q++) {
+            const uint32_t i = i0 + q;
+            if (PPL > 1 && i >= P) break;
             float v[W];
             if (i < m) {
                 v[0] = __fmul_rn(__uint2float_rn((uint32_t)size[row0 + i]), 0x1p-11f);
@@ -211,14 +218,15 @@ gather_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__
             if (BF16) {
                 uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(rows) + ((size_t)r * P + i) * W);
 #pragma unroll
-                for (int q = 0; q < W / 8; q++)
-                    dst[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
-                                        pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+                for (int q4 = 0; q4 < W / 8; q4++)
+                    dst[q4] = make_uint4(pack_bf16(v[8 * q4], v[8 * q4 + 1]), pack_bf16(v[8 * q4 + 2], v[8 * q4 + 3]),
+                                         pack_bf16(v[8 * q4 + 4], v[8 * q4 + 5]), pack_bf16(v[8 * q4 + 6], v[8 * q4 + 7]));
             } else {
                 float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(rows) + ((size_t)r * P + i) * W);
 #pragma unroll
-                for (int q = 0; q < W / 4; q++) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                for (int q4 = 0; q4 < W / 4; q4++) dst[q4] = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
             }
+          }
         }
     }
 }

@@ -548,10 +548,34 @@ extern "C" void sf_table_destroy(sf_table* t) {
     delete t;
 }
 
+namespace {
+int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_forest* fo, uint32_t F,
+                 const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_dev, void* stream, bool zero_result);
+}
+
+// A batch of more than 65,536 packets (the sort keys are 16-bit arrival indices) is ingested as consecutive pieces of at most
+// 65,536 packets on the same stream: the table sees the packets in the same order as if they had come in separate calls,
+// and the pieces' counts add up in *result_dev.
 extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_forest* fo, uint32_t F,
                                const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_dev, void* stream)
 {
     if (!ctx || !t || !batch || !fo || !slow || !cfg || !result_dev || !cfg->tau) return SF_ERR_ARG;
+    if (batch->n <= kMaxBatch) return ingest_chunk(ctx, t, batch, fo, F, slow, cfg, result_dev, stream, true);
+    for (uint32_t o = 0; o < batch->n; o += kMaxBatch) {
+        sf_pkt_batch part = *batch;
+        part.src += o; part.dst += o; part.sport += o; part.dport += o; part.proto += o; part.dir += o; part.size += o;
+        part.iat_us += o; part.hdr += (size_t)o * kHdr;
+        part.n = std::min<uint32_t>(kMaxBatch, batch->n - o);
+        const int rc = ingest_chunk(ctx, t, &part, fo, F, slow, cfg, result_dev, stream, o == 0);
+        if (rc != SF_OK) return rc;
+    }
+    return SF_OK;
+}
+
+namespace {
+int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_forest* fo, uint32_t F,
+                 const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_dev, void* stream, bool zero_result)
+{
     if (batch->n > kMaxBatch) return SF_ERR_ARG;
     if (!batch->src || !batch->dst || !batch->sport || !batch->dport || !batch->proto || !batch->dir || !batch->size ||
         !batch->iat_us || !batch->hdr) return SF_ERR_ARG;
@@ -561,7 +585,7 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     SF_CUDA(cudaSetDevice(ctx->device));
     cudaStream_t st = (cudaStream_t)stream;
     const uint32_t n = batch->n;
-    SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_batch_result), st));
+    if (zero_result) SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_batch_result), st));
     if (n == 0) return SF_OK;
     const TableDev& d = t->d;
     // workspace: features, probabilities, decisions, wide rows and slow-model scratch for at most n flows
@@ -638,6 +662,7 @@ extern "C" int sf_table_ingest(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* bat
     SF_LAUNCH_CHECK("apply_slow_kernel");
     return SF_OK;
 }
+}  // namespace
 
 // The same with a batch that lives in HOST memory: the nine planes are copied to the context's device
 // staging buffer on the stream (one copy per plane), the batch is ingested, the counts come back.
@@ -645,7 +670,6 @@ extern "C" int sf_table_ingest_host(sf_ctx* ctx, sf_table* t, const sf_pkt_batch
                                     const sf_slow* slow, const sf_route_cfg* cfg, sf_batch_result* result_host_out, void* stream)
 {
     if (!ctx || !t || !bh || !result_host_out) return SF_ERR_ARG;
-    if (bh->n > kMaxBatch) return SF_ERR_ARG;
     if (bh->n && (!bh->src || !bh->dst || !bh->sport || !bh->dport || !bh->proto || !bh->dir || !bh->size || !bh->iat_us || !bh->hdr))
         return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));

@@ -115,6 +115,45 @@ def test_stream_matches_sequential_reference(env, shape):
     sf.sf_forest_destroy(forest_h)
 
 
+@pytest.mark.parametrize("host", [False, True])
+def test_batch_larger_than_the_sort_window_is_ingested_in_pieces(env, host):
+    """A batch of more than 65,536 packets in ONE call: the table must end as if the packets had arrived in
+    consecutive pieces of 65,536 (the reference is fed exactly those pieces), and the call's counts are the
+    pieces' sums."""
+    sf, hz, ctx = env
+    F, T, depth, C, dims, P_model = 24, 16, 8, 4, (1024, 256, 4), 64
+    n_keys, m = 6000, 2 * 65536 + 18939
+    fast_pkts, slow_pkts = 8, 64
+    forest, tau, slow = _models(F, T, depth, C, dims, 93)
+    big = flowgen.StreamSource(94, n_keys, 1.1).batch(0, m)
+    planes = ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")
+    pieces = [{k: (v[o:o + 65536] if k in planes else v) for k, v in big.items()} for o in range(0, m, 65536)]
+    per, cnt = simulate_stream(pieces, fast_pkts, slow_pkts, F, forest, tau, slow, P_model, True, threads=8)
+    assert cnt["slow_fired"] > 5 and cnt["fast_done"] > 50 and cnt["dropped_after_decision"] > 0
+
+    forest_h = hz.make_forest(ctx, forest)
+    slow_h = sf.sf_mlp_create(ctx, sf.SF_BF16, slow["dims"], slow["W"], slow["b"])
+    table = sf.sf_table_create(ctx, 14, fast_pkts, slow_pkts, n_keys)
+    rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
+    sf.sf_ctx_poll(ctx, reset=True)
+    got = _ingest_all(sf, hz, ctx, table, [big], forest_h, F, slow_h, rcfg, host=host)
+    c = sf.sf_ctx_poll(ctx, reset=True)
+    assert got["missed"] == 0 and c.device_error == 0
+    for k in ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision"):
+        assert got[k] == cnt[k], k
+    keys = list(per.keys())
+    res = _lookup(sf, hz, ctx, table, keys)
+    for i, k in enumerate(keys):
+        r, g = per[k], res[i]
+        assert g["found"] == 1 and g["n_pkts"] == r["n_pkts"] and g["stage"] == r["stage"], k
+        if r["stage"] >= 1:
+            assert g["label_fast"] == r["label_fast"]
+            assert np.float32(g["score"]).view(np.uint32) == np.float32(r["score"]).view(np.uint32)
+    sf.sf_table_destroy(table)
+    sf.sf_slow_destroy(slow_h)
+    sf.sf_forest_destroy(forest_h)
+
+
 def test_stream_config5_full_size(env):
     """Config 5 at its full size: 10,000,000 keys, a 2^25-slot table, 64K-packet batches, config 2's forest on
     8 packets and its MLP on 64 packets.  The packet-by-packet reference is too slow here, so the expected values
