@@ -57,11 +57,13 @@ constexpr uint32_t BK = 64;
 constexpr uint32_t kEpiWarps = 8;
 constexpr uint32_t kGemmThreads = 64 + kEpiWarps * 32;
 
-template <uint32_t BN> struct GemmCfg {
+// PAIR: two CTAs (a cluster of two, on the two SMs of one TPC) share every MMA: the tile is 256 rows x BN, each CTA loads its
+// 128 rows of A and its BN / 2 rows of W per stage (a third less shared-memory and L2 traffic per flop, two more stages)
+template <uint32_t BN, bool PAIR = false> struct GemmCfg {
     static constexpr uint32_t kStageBytesA = BM * BK * 2;
-    static constexpr uint32_t kStageBytesB = BN * BK * 2;
+    static constexpr uint32_t kStageBytesB = (PAIR ? BN / 2 : BN) * BK * 2;
     static constexpr uint32_t kStageBytes = kStageBytesA + kStageBytesB;
-    static constexpr uint32_t kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : (BN == 64 ? 8 : 10));
+    static constexpr uint32_t kStages = PAIR ? 6 : ((BN == 256) ? 4 : (BN == 128 ? 6 : (BN == 64 ? 8 : 10)));
     static constexpr uint32_t kTmemCols = 2 * BN;             // a power of two >= 32
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ +
                                            kEpiWarps * 2048 /*epilogue staging*/;
@@ -174,7 +176,14 @@ __device__ void small_rows_layer(const __nv_bfloat16* __restrict__ A, const __nv
 // zero), head_b its bias, CH = 8 or 16 = classes kept per row.  A CTA takes whole 128-row panels (all N / BN tiles of
 // a panel in turn), so a row's logits are summed in one place and in one fixed order: column chunks in increasing
 // order inside each of the two epilogue warps that share the row, then (low half + high half) + bias.
-template <uint32_t BN, int MODE, uint32_t CH = 8>
+//
+// PAIR (launched as clusters of two CTAs, BN = 256): CTA rank 0 of a pair is the leader.  Both producers wait on their own
+// `empty` barriers and load into their own shared memory, the bytes of both counted on the LEADER's `full` barrier; one thread
+// of the leader issues the pair MMAs and commits to `empty` and `tmem_full` in both CTAs; each CTA's epilogue warps read their
+// own TMEM (rows rank * 128 ... of the 256-row tile) and release the accumulator on the leader's `tmem_empty`.  No CTA leaves
+// while its partner may still touch its shared memory: the producers first see every stage released, then the pair meets
+// at a cluster barrier that every thread reaches (all waits before it are bounded).
+template <uint32_t BN, int MODE, uint32_t CH = 8, bool PAIR = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                            const float* __restrict__ bias, const uint32_t* __restrict__ n_rows_dev,
@@ -183,13 +192,15 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                            const __nv_bfloat16* __restrict__ A_raw, const __nv_bfloat16* __restrict__ W_raw, uint32_t capacity,
                            const __nv_bfloat16* __restrict__ head_w, const float* __restrict__ head_b)
 {
-    using Cfg = GemmCfg<BN>;
+    using Cfg = GemmCfg<BN, PAIR>;
     constexpr bool HEAD = MODE == MODE_HEAD;
     constexpr bool FUSED = MODE == MODE_HIDDEN_HEAD;
+    static_assert(!PAIR || (BN == 256 && !HEAD), "pairs: 256-column tiles of a hidden layer");
+    constexpr uint32_t BMT = PAIR ? 2 * BM : BM;       // rows of a tile
     extern __shared__ uint8_t smem_raw[];
     // the count is the caller's device word: never trust it beyond the rows the buffers hold
     const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);
-    if (n_rows <= small_max) {                       // a handful of rows (small_max = 0: never): CUDA cores, same launch
+    if (n_rows <= small_max) {                       // a handful of rows (small_max = 0: never): CUDA cores, same launch (pairs: both CTAs alike)
         if (n_rows) small_rows_layer<HEAD>(A_raw, W_raw, bias, n_rows, N, K, out, logits, label, C, smem_raw);
         return;
     }
@@ -199,26 +210,29 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t tiles_m = (n_rows + BM - 1) / BM;
+    const uint32_t tiles_m = (n_rows + BMT - 1) / BMT;
     const uint32_t tiles_n = N / BN;
     const uint32_t k_blocks = K / BK;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;                   // 0 = the pair's leader
+    const uint32_t unit = PAIR ? blockIdx.x >> 1 : blockIdx.x;             // this CTA's (pair's) place among ...
+    const uint32_t n_units = PAIR ? gridDim.x >> 1 : gridDim.x;            // ... the CTAs (pairs) that share the tiles
     // tiles of this CTA, in order: every gridDim.x-th tile of the (row panel, column tile) sequence, or - with the head
     // folded in - every gridDim.x-th row panel with all its column tiles
-    const uint32_t n_my = FUSED ? ((tiles_m > blockIdx.x) ? ((tiles_m - blockIdx.x + gridDim.x - 1) / gridDim.x) * tiles_n : 0u)
-                                : ((tiles_m * tiles_n > blockIdx.x) ? (tiles_m * tiles_n - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u);
+    const uint32_t n_my = FUSED ? ((tiles_m > unit) ? ((tiles_m - unit + n_units - 1) / n_units) * tiles_n : 0u)
+                                : ((tiles_m * tiles_n > unit) ? (tiles_m * tiles_n - unit + n_units - 1) / n_units : 0u);
     auto tile_of = [&](uint32_t it, uint32_t& tm, uint32_t& tn) {
-        if (FUSED) { tm = blockIdx.x + (it / tiles_n) * gridDim.x; tn = it % tiles_n; }
-        else { const uint32_t tile = blockIdx.x + it * gridDim.x; tm = tile / tiles_n; tn = tile - tm * tiles_n; }
+        if (FUSED) { tm = unit + (it / tiles_n) * n_units; tn = it % tiles_n; }
+        else { const uint32_t tile = unit + it * n_units; tm = tile / tiles_n; tn = tile - tm * tiles_n; }
     };
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < Cfg::kStages; s++) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        for (uint32_t b = 0; b < 2; b++) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], kEpiWarps); }
+        for (uint32_t b = 0; b < 2; b++) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], PAIR ? 2 * kEpiWarps : kEpiWarps); }
         mbar_init(&bars->head_bar, kEpiWarps / 2);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(&bars->tmem_base, Cfg::kTmemCols);
+    if (warp == 1) { if constexpr (PAIR) tmem_alloc_pair(&bars->tmem_base, Cfg::kTmemCols); else tmem_alloc(&bars->tmem_base, Cfg::kTmemCols); }
     // fused head: the head's weights, transposed to [column][CH] bf16, where the other modes stage their output
     uint8_t* const epi_smem = tiles + Cfg::kStages * Cfg::kStageBytes + 256;
     if constexpr (FUSED) {
@@ -233,6 +247,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();          // the partner's barriers are initialised before anything reaches them
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
@@ -249,16 +264,30 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                     if (!mbar_wait(&bars->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sA = tiles + stage * Cfg::kStageBytes;
                     uint8_t* sB = sA + Cfg::kStageBytesA;
-                    mbar_expect_tx(&bars->full[stage], Cfg::kStageBytes);
-                    tma_load_2d(sA, &tmA, (int32_t)(kb * BK), (int32_t)(tm * BM), &bars->full[stage]);
-                    tma_load_2d(sB, &tmW, (int32_t)(kb * BK), (int32_t)(tn * BN), &bars->full[stage]);
+                    if constexpr (PAIR) {
+                        const uint32_t full_leader = map_to_cta(smem_u32(&bars->full[stage]), 0);
+                        if (rank == 0) mbar_expect_tx(&bars->full[stage], 2 * Cfg::kStageBytes);
+                        tma_load_2d_pair(sA, &tmA, (int32_t)(kb * BK), (int32_t)(tm * BMT + rank * BM), full_leader);
+                        tma_load_2d_pair(sB, &tmW, (int32_t)(kb * BK), (int32_t)(tn * BN + rank * (BN / 2)), full_leader);
+                    } else {
+                        mbar_expect_tx(&bars->full[stage], Cfg::kStageBytes);
+                        tma_load_2d(sA, &tmA, (int32_t)(kb * BK), (int32_t)(tm * BM), &bars->full[stage]);
+                        tma_load_2d(sB, &tmW, (int32_t)(kb * BK), (int32_t)(tn * BN), &bars->full[stage]);
+                    }
+                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if constexpr (PAIR) {
+                // every stage's last use released: no arrival from the leader is still on its way to this CTA's barriers
+                for (uint32_t s = 0; s < Cfg::kStages && ok; s++) {
+                    if (!mbar_wait(&bars->empty[stage], phase ^ 1u, abort_flag)) ok = false;
                     if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BMT, BN);
             uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
             bool ok = true;
             for (uint32_t it = 0; it < n_my && ok; it++) {
@@ -275,13 +304,16 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                         // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row
                         const uint64_t adesc = make_smem_desc(aaddr + k * 32u, 16, 1024, 2);
                         const uint64_t bdesc = make_smem_desc(baddr + k * 32u, 16, 1024, 2);
-                        umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        if constexpr (PAIR) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        else umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    umma_commit(&bars->empty[stage]);            // stage reusable once these MMAs retire
+                    // stage reusable once these MMAs retire
+                    if constexpr (PAIR) umma_commit_pair(&bars->empty[stage]); else umma_commit(&bars->empty[stage]);
                     if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(&bars->tmem_full[buf]);              // accumulator complete
+                // accumulator complete
+                if constexpr (PAIR) umma_commit_pair(&bars->tmem_full[buf]); else umma_commit(&bars->tmem_full[buf]);
                 buf ^= 1u; if (buf == 0) bphase ^= 1u;
             }
         }
@@ -300,7 +332,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->tmem_full[buf], bphase, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t row0 = tm * BM + quarter * 32u;
+            const uint32_t row0 = tm * BMT + rank * BM + quarter * 32u;
             const uint32_t col0 = tn * BN;
             const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BN;
             if constexpr (HEAD) {
@@ -435,7 +467,10 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->tmem_empty[buf]), 0));
+                else mbar_arrive(&bars->tmem_empty[buf]);
+            }
             buf ^= 1u; if (buf == 0) bphase ^= 1u;
         }
     }
@@ -447,8 +482,24 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         __nanosleep(200000);
         __syncthreads();
     }
+    if constexpr (PAIR) cluster_sync_all();          // the partner is done with this CTA's shared memory and barriers
     tc_fence_after();
-    if (warp == 1) { __syncwarp(); tmem_dealloc(tmem_base, Cfg::kTmemCols); }
+    if (warp == 1) {
+        __syncwarp();
+        if constexpr (PAIR) tmem_dealloc_pair(tmem_base, Cfg::kTmemCols); else tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+}
+
+// launch as clusters of two CTAs
+template <typename Kern, typename... Args>
+cudaError_t launch_pairs(Kern k, uint32_t grid, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid); lc.blockDim = dim3(kGemmThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, k, args...);
 }
 
 template <uint32_t BN>
@@ -461,6 +512,23 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     if (rc != SF_OK) return rc;
     rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
     if (rc != SF_OK) return rc;
+    if constexpr (BN == 256) {
+        if (small_max == 0) {                          // large batches: CTA pairs on 256 x 256 tiles
+            using CfgP = GemmCfg<BN, true>;
+            rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN / 2, BK);
+            if (rc != SF_OK) return rc;
+            auto kp = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN, 8, true>;
+            static bool attr_set_dev[64] = {};
+            bool& attr_set = attr_set_dev[ctx->device & 63];
+            if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CfgP::kSmemBytes)); attr_set = true; }
+            const uint32_t pair_tiles = ((capacity + 2 * BM - 1) / (2 * BM)) * (N / BN);
+            const uint32_t grid = 2u * std::min<uint32_t>((uint32_t)ctx->num_sms / 2u, pair_tiles);
+            SF_CUDA(launch_pairs(kp, grid, CfgP::kSmemBytes, st, tmA, tmW, bias, n_rows_dev, N, K, reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state,
+                                 (float*)nullptr, (uint8_t*)nullptr, 0u, 0u, reinterpret_cast<const __nv_bfloat16*>(A),
+                                 reinterpret_cast<const __nv_bfloat16*>(W), capacity, (const __nv_bfloat16*)nullptr, (const float*)nullptr));
+            return SF_OK;
+        }
+    }
     auto k = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN>;
     static bool attr_set_dev[64] = {};                 // the opt-in is per device
     bool& attr_set = attr_set_dev[ctx->device & 63];
@@ -486,6 +554,21 @@ int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bia
     if (rc != SF_OK) return rc;
     rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);
     if (rc != SF_OK) return rc;
+    if constexpr (BN == 256) {                         // CTA pairs: a pair owns whole 256-row panels
+        constexpr uint32_t kSmemP = GemmCfg<BN, true>::kSmemBytesHead16;
+        rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN / 2, BK);
+        if (rc != SF_OK) return rc;
+        auto kp = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN_HEAD, CH, true>;
+        static bool attr_set_dev[64] = {};
+        bool& attr_set = attr_set_dev[ctx->device & 63];
+        if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP)); attr_set = true; }
+        const uint32_t pair_panels = (capacity + 2 * BM - 1) / (2 * BM);
+        const uint32_t grid = 2u * std::min<uint32_t>((uint32_t)ctx->num_sms / 2u, pair_panels);
+        SF_CUDA(launch_pairs(kp, grid, kSmemP, st, tmA, tmW, bias, n_rows_dev, N, K, (__nv_bfloat16*)nullptr, ctx->d_state, logits, label, C, 0u,
+                             reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
+                             reinterpret_cast<const __nv_bfloat16*>(W16), head_bias));
+        return SF_OK;
+    }
     auto k = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN_HEAD, CH>;
     static bool attr_set_dev[64] = {};                 // the opt-in is per device
     bool& attr_set = attr_set_dev[ctx->device & 63];
