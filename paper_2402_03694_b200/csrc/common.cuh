@@ -86,6 +86,30 @@ int  sf_set_cuda_error(cudaError_t e, const char* where);      // records text, 
 #define SF_CUDA(call) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) return sf_set_cuda_error(e__, #call); } while (0)
 #define SF_LAUNCH_CHECK(name) do { cudaError_t e__ = cudaGetLastError(); if (e__ != cudaSuccess) return sf_set_cuda_error(e__, name); } while (0)
 
+// ---- chained launches ---------------------------------------------------------
+// A kernel launched with sf_launch_chained may be scheduled while the previous kernel of the stream is still draining (programmatic
+// stream serialisation): its blocks are set up early and the gap between two short dependent kernels shrinks.  Such a kernel's FIRST
+// statement, before any return and any access to global memory, must be sf_chain_enter(): it lets the kernel after it be set up
+// early in turn, then waits until every earlier kernel of the stream has completed and its writes are visible.  Launched the plain
+// way the same kernel runs unchanged (both instructions are no-ops then).
+#ifdef __CUDACC__
+__device__ __forceinline__ void sf_chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void sf_chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void sf_chain_enter() { sf_chain_release(); sf_chain_wait(); }
+// (A kernel may instead call sf_chain_release() first and sf_chain_wait() later, in every thread that goes on to touch global
+// memory other than constant model data: what it does in between - barrier set-up, loading weights - overlaps its predecessor.)
+template <typename... KArgs, typename... Args>
+inline cudaError_t sf_launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = smem; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kernel, args...);
+}
+#endif
+
 // timing: sf_time_new_record at the start of a public compute call, begin/end around kernels
 void sf_time_new_record(sf_ctx* ctx);
 void sf_time_begin(sf_ctx* ctx, int slot, cudaStream_t st);

@@ -156,8 +156,12 @@ forest_kernel(const __grid_constant__ ForestTop top, const float* __restrict__ f
               const sf_fused_route fr)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    if (n_dev) n = min(n, *n_dev);               // optional device-side flow count (streaming path)
+    // a chained launch: barrier set-up and the first tree chunks (model data) overlap the previous kernel's tail; every thread waits
+    // for that kernel before it reads a count or a feature, or writes anything
+    sf_chain_release();
+    if (n_dev) { sf_chain_wait(); n = min(n, *n_dev); }     // optional device-side flow count (streaming path)
     if (blockIdx.x * KB >= n) {
+        sf_chain_wait();
         if (fr.tau && threadIdx.x == 0) fr.block_counts[blockIdx.x] = 0;
         return;
     }
@@ -198,6 +202,7 @@ forest_kernel(const __grid_constant__ ForestTop top, const float* __restrict__ f
         return;
     }
 
+    sf_chain_wait();
     if (live) {
         const float* row = feat + (size_t)f * F;
         if ((F & 3) == 0) {
@@ -370,6 +375,7 @@ forest_leaf_index_kernel(const float* __restrict__ feat, uint32_t n, uint32_t F,
                          uint16_t* __restrict__ leaf_idx, sf_dev_state* st, const uint32_t* __restrict__ n_dev, LeafIndexPackets pk)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    sf_chain_enter();
     if (n_dev) n = min(n, *n_dev);
     float* xs = reinterpret_cast<float*>(smem_raw + buf_bytes);                                  // [F][128]
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + buf_bytes + (size_t)F * kBSmall * 4);
@@ -475,9 +481,9 @@ int launch3(const sf_forest* fo, const Plan& p, const float* feat, uint32_t n, f
         smem_set = p.smem;
     }
     const uint32_t grid = (n + KB - 1) / KB;
-    k<<<grid, KB + 32, p.smem, st>>>(*fo->h_top, feat, n, fo->F, KB == kB ? fo->d_image : fo->d_image_small, fo->d_leaf, fo->leaf_tex, fo->T, fo->depth, fo->tree_stride, p.tpc,
-                                p.chunk_bytes, out, leaf_idx, fo->ctx->d_state, n_dev, fr);
-    SF_LAUNCH_CHECK("forest_kernel");
+    SF_CUDA(sf_launch_chained(k, grid, KB + 32, p.smem, st, *fo->h_top, feat, n, fo->F, (const unsigned char*)(KB == kB ? fo->d_image : fo->d_image_small),
+                              (const float*)fo->d_leaf, fo->leaf_tex, fo->T, fo->depth, fo->tree_stride, p.tpc, p.chunk_bytes, out, leaf_idx,
+                              fo->ctx->d_state, n_dev, fr));
     return SF_OK;
 }
 
@@ -534,9 +540,8 @@ int launch_rf_leaf_index_g(const sf_forest* fo, const float* feat, uint32_t n, u
     }
     const uint32_t n_items = ((n + kBSmall - 1) / kBSmall) * ((fo->T + tpi - 1) / tpi);
     const uint32_t grid = std::min<uint32_t>(n_items, (uint32_t)fo->ctx->num_sms * 2u);
-    forest_leaf_index_kernel<2, G><<<grid, kBSmall, smem, st>>>(feat, n, fo->F, fo->d_image_small, fo->T, fo->depth, fo->tree_stride, tpi, buf,
-                                                              leaf_idx, fo->ctx->d_state, n_dev, pk);
-    SF_LAUNCH_CHECK("forest_leaf_index_kernel");
+    SF_CUDA(sf_launch_chained(forest_leaf_index_kernel<2, G>, grid, kBSmall, smem, st, feat, n, fo->F, (const unsigned char*)fo->d_image_small, fo->T,
+                              fo->depth, fo->tree_stride, tpi, buf, leaf_idx, fo->ctx->d_state, n_dev, pk));
     return SF_OK;
 }
 

@@ -198,6 +198,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     static_assert(!PAIR || (BN == 256 && !HEAD), "pairs: 256-column tiles of a hidden layer");
     constexpr uint32_t BMT = PAIR ? 2 * BM : BM;       // rows of a tile
     extern __shared__ uint8_t smem_raw[];
+    sf_chain_enter();
     // the count is the caller's device word: never trust it beyond the rows the buffers hold
     const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);
     if (n_rows <= small_max) {                       // a handful of rows (small_max = 0: never): CUDA cores, same launch (pairs: both CTAs alike)
@@ -495,10 +496,12 @@ template <typename Kern, typename... Args>
 cudaError_t launch_pairs(Kern k, uint32_t grid, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(grid); lc.blockDim = dim3(kGemmThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    lc.attrs = at; lc.numAttrs = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;       // a chained launch (the kernel starts with sf_chain_enter)
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = 2;
     return cudaLaunchKernelEx(&lc, k, args...);
 }
 
@@ -535,10 +538,9 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
     uint32_t max_tiles = ((capacity + BM - 1) / BM) * (N / BN);
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
-    k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, N, K,
-                                                  reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state, nullptr, nullptr, 0, small_max,
-                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity, nullptr, nullptr);
-    SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel");
+    SF_CUDA(sf_launch_chained(k, grid, kGemmThreads, Cfg::kSmemBytes, st, tmA, tmW, bias, n_rows_dev, N, K, reinterpret_cast<__nv_bfloat16*>(out),
+                              ctx->d_state, (float*)nullptr, (uint8_t*)nullptr, 0u, small_max, reinterpret_cast<const __nv_bfloat16*>(A),
+                              reinterpret_cast<const __nv_bfloat16*>(W), capacity, (const __nv_bfloat16*)nullptr, (const float*)nullptr));
     return SF_OK;
 }
 
@@ -575,10 +577,9 @@ int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bia
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem)); attr_set = true; }
     const uint32_t panels = (capacity + BM - 1) / BM;
     const uint32_t grid = (uint32_t)ctx->num_sms < panels ? (uint32_t)ctx->num_sms : panels;
-    k<<<grid, kGemmThreads, kSmem, st>>>(tmA, tmW, bias, n_rows_dev, N, K, nullptr, ctx->d_state, logits, label, C, 0u,
-                                         reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
-                                         reinterpret_cast<const __nv_bfloat16*>(W16), head_bias);
-    SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(hidden + head)");
+    SF_CUDA(sf_launch_chained(k, grid, kGemmThreads, kSmem, st, tmA, tmW, bias, n_rows_dev, N, K, (__nv_bfloat16*)nullptr, ctx->d_state, logits, label, C, 0u,
+                              reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
+                              reinterpret_cast<const __nv_bfloat16*>(W16), head_bias));
     return SF_OK;
 }
 
@@ -598,9 +599,9 @@ int launch_head_tc(sf_ctx* ctx, const void* A, const void* W16, const float* bia
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes)); attr_set = true; }
     uint32_t max_tiles = (capacity + BM - 1) / BM;
     uint32_t grid = (uint32_t)ctx->num_sms < max_tiles ? (uint32_t)ctx->num_sms : max_tiles;
-    k<<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, bias, n_rows_dev, 16, K, nullptr, ctx->d_state, logits, label, C, small_max,
-                                                  reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16), capacity, nullptr, nullptr);
-    SF_LAUNCH_CHECK("gemm_bias_relu_bf16_kernel(head)");
+    SF_CUDA(sf_launch_chained(k, grid, kGemmThreads, Cfg::kSmemBytes, st, tmA, tmW, bias, n_rows_dev, 16u, K, (__nv_bfloat16*)nullptr, ctx->d_state, logits, label,
+                              C, small_max, reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W16), capacity,
+                              (const __nv_bfloat16*)nullptr, (const float*)nullptr));
     return SF_OK;
 }
 

@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(1024)
 scan_kernel(uint32_t* __restrict__ block_counts, uint32_t nb, uint32_t n, uint32_t capacity,
             uint32_t* __restrict__ n_esc, sf_dev_state* __restrict__ st, const uint32_t* __restrict__ n_dev = nullptr)
 {
+    sf_chain_enter();
     if (n_dev) n = min(n, *n_dev);               // flows actually scored (blocks past the count contributed zeros)
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry_s;
@@ -115,6 +116,7 @@ __global__ void __launch_bounds__(B)
 scatter_kernel(const uint8_t* __restrict__ decision, uint32_t n, const uint32_t* __restrict__ block_offsets,
                uint32_t capacity, uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__ n_dev = nullptr)
 {
+    sf_chain_enter();
     if (n_dev) n = min(n, *n_dev);
     __shared__ uint32_t warp_off[32];
     const uint32_t f = blockIdx.x * B + threadIdx.x;
@@ -163,6 +165,7 @@ gather_kernel(const uint32_t* __restrict__ esc_ids, const uint32_t* __restrict__
 {
     constexpr int NH = W - 3;
     constexpr int NW = (NH + 6) / 4;             // words that can hold NH bytes starting at any byte of the first
+    sf_chain_enter();
     const uint32_t n_esc = *n_esc_dev;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
@@ -245,6 +248,7 @@ __global__ void merge_slow_kernel(const uint32_t* __restrict__ esc_ids, const ui
                                   const uint8_t* __restrict__ label_slow, uint8_t* __restrict__ label,
                                   uint8_t* __restrict__ stage, uint8_t stage_value, sf_dev_state* count_slow_done)
 {
+    sf_chain_enter();
     const uint32_t n_esc = *n_esc_dev;
     if (count_slow_done && blockIdx.x == 0 && threadIdx.x == 0)
         atomicAdd((unsigned long long*)&count_slow_done->counters.n_slow_done, (unsigned long long)n_esc);
@@ -331,8 +335,8 @@ int sf_launch_gather(sf_ctx* ctx, const sf_route_cfg* cfg, const sf_packets* wid
     if (blocks > max_blocks) blocks = max_blocks;
     const size_t hdr_total = (size_t)wide->n_flows * wide->pitch_pkts * wide->hdr_bytes;
     const bool hdr_words = ((uintptr_t)wide->hdr & 3) == 0;
-#define SF_GATHER2(Wv, BF) do { if (hdr_words) gather_kernel<Wv, BF, true><<<blocks, 256, 0, st>>>(ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows); \
-        else gather_kernel<Wv, BF, false><<<blocks, 256, 0, st>>>(ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows); } while (0)
+#define SF_GATHER2(Wv, BF) do { if (hdr_words) SF_CUDA(sf_launch_chained(gather_kernel<Wv, BF, true>, blocks, 256, 0, st, ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows)); \
+        else SF_CUDA(sf_launch_chained(gather_kernel<Wv, BF, false>, blocks, 256, 0, st, ids, n_ids_dev, wide->size, wide->iat_us, wide->dir_bits, wide->hdr, wide->n_valid, wide->pitch_pkts, wide->hdr_bytes, hdr_total, P, P_real, rows)); } while (0)
     if (cfg->wide_layout == SF_MLP16) { if (cfg->row_dtype == SF_BF16) SF_GATHER2(16, true); else SF_GATHER2(16, false); }
     else                              { if (cfg->row_dtype == SF_BF16) SF_GATHER2(8, true);  else SF_GATHER2(8, false); }
 #undef SF_GATHER2
@@ -399,12 +403,10 @@ int sf_launch_route_after_fused(sf_ctx* ctx, const sf_route_cfg* cfg, uint32_t n
 {
     const uint32_t nb = (n + SF_FOREST_BLOCK - 1) / SF_FOREST_BLOCK;
     sf_time_begin(ctx, SF_T_SCORE, st);
-    scan_kernel<<<1, 1024, 0, st>>>(block_counts, nb, n, cfg->capacity, n_esc, ctx->d_state, nullptr);
-    SF_LAUNCH_CHECK("scan_kernel");
-    if (n > 0) {
-        scatter_kernel<(int)SF_FOREST_BLOCK><<<nb, SF_FOREST_BLOCK, 0, st>>>(decision, n, block_counts, cfg->capacity, esc_ids, nullptr);
-        SF_LAUNCH_CHECK("scatter_kernel");
-    }
+    SF_CUDA(sf_launch_chained(scan_kernel, 1, 1024, 0, st, block_counts, nb, n, cfg->capacity, n_esc, ctx->d_state, (const uint32_t*)nullptr));
+    if (n > 0)
+        SF_CUDA(sf_launch_chained(scatter_kernel<(int)SF_FOREST_BLOCK>, nb, SF_FOREST_BLOCK, 0, st, decision, n, (const uint32_t*)block_counts, cfg->capacity,
+                                  esc_ids, (const uint32_t*)nullptr));
     sf_time_end(ctx, SF_T_SCORE, st);
     if (wide && rows && n > 0 && cfg->capacity > 0) {
         sf_time_begin(ctx, SF_T_GATHER, st);
@@ -426,8 +428,7 @@ int sf_launch_merge(const uint8_t* label_fast, const uint8_t* decision, uint32_t
     uint32_t blocks = (capacity + 255) / 256;
     if (blocks > 1184) blocks = 1184;
     if (blocks > 0) {
-        merge_slow_kernel<<<blocks, 256, 0, st>>>(esc_ids, n_esc, label_slow, label, stage, stage_value, count_slow_done);
-        SF_LAUNCH_CHECK("merge_slow_kernel");
+        SF_CUDA(sf_launch_chained(merge_slow_kernel, blocks, 256, 0, st, esc_ids, n_esc, label_slow, label, stage, stage_value, count_slow_done));
     }
     return SF_OK;
 }

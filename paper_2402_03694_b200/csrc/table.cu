@@ -156,6 +156,7 @@ __global__ void __launch_bounds__(256)
 key_kernel(TableDev t, const uint32_t* __restrict__ pkt_slot, uint32_t n,
            uint32_t* __restrict__ key, uint32_t* __restrict__ idx, uint32_t* __restrict__ hist0)
 {
+    sf_chain_enter();
     __shared__ uint32_t c[256];
     c[threadIdx.x] = 0;
     __syncthreads();
@@ -184,6 +185,7 @@ radix8_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restri
                       uint32_t* __restrict__ iout, uint32_t n, uint32_t shift, const uint32_t* __restrict__ hist, uint32_t nblk,
                       uint32_t* __restrict__ next_hist, uint32_t* __restrict__ run_start_of)
 {
+    sf_chain_enter();
     __shared__ uint32_t base[256];
     __shared__ uint32_t wc[8][256];
     __shared__ uint32_t wsum[8];
@@ -268,6 +270,7 @@ __global__ void apply1_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
                               const uint32_t* __restrict__ pkt_slot, uint32_t* __restrict__ rank, uint32_t* __restrict__ pos_out,
                               uint32_t* __restrict__ fire1_slot, uint32_t* __restrict__ counts)
 {
+    sf_chain_enter();
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= b.n) return;
     const uint32_t slot = pkt_slot[s_idx[j]];
@@ -292,6 +295,7 @@ fast_finish_kernel(TableDev t, const uint32_t* __restrict__ fire1_slot, const ui
                    const uint16_t* __restrict__ leaf_idx, const float* __restrict__ leaf, uint32_t T, uint32_t n_leaf, uint32_t C,
                    const float* __restrict__ tau, sf_batch_result* res, sf_dev_state* st)
 {
+    sf_chain_enter();
     const uint32_t c = threadIdx.x & 15u;
     const uint32_t n_fired = counts[0];
     // a few hundred flows fire per batch, the batch could hold 65,536: a small grid walks over the fired flows
@@ -379,6 +383,7 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
                               uint32_t* __restrict__ fire2_slab, uint32_t* __restrict__ fire2_slot,
                               uint32_t* __restrict__ counts, sf_batch_result* res, sf_dev_state* st)
 {
+    sf_chain_enter();
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t slot = (j < b.n) ? pkt_slot[s_idx[j]] : t.n_slots;
     const bool live = slot < t.n_slots;              // every lane stays to the end: the counter is added up per warp
@@ -410,6 +415,7 @@ __global__ void apply2_kernel(TableDev t, sf_pkt_batch b, const uint32_t* __rest
 __global__ void apply_slow_kernel(TableDev t, const uint32_t* __restrict__ fire2_slot, const uint32_t* __restrict__ counts,
                                   const uint8_t* __restrict__ label_slow, sf_batch_result* res, sf_dev_state* st)
 {
+    sf_chain_enter();
     const uint32_t k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k == 0) atomicAdd((unsigned long long*)&st->counters.n_slow_done, (unsigned long long)counts[1]);
     if (k >= counts[1]) return;
@@ -608,17 +614,16 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->pkt_slot, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("probe_kernel");
     const uint32_t nblk = (n + kTile - 1) / kTile;
-    key_kernel<<<blocks, 256, 0, st>>>(d, t->pkt_slot, n, t->key_a, t->idx_a, t->hist);
-    SF_LAUNCH_CHECK("key_kernel");
+    // from here on every kernel of the batch is a chained launch (set up while its predecessor drains)
+    SF_CUDA(sf_launch_chained(key_kernel, blocks, 256, 0, st, d, t->pkt_slot, n, t->key_a, t->idx_a, t->hist));
     {
         // 16-bit keys: two 8-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
-        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_a, t->idx_a, t->key_b, t->idx_b, n, 0, t->hist, nblk, t->hist + kHistWords, nullptr);
-        SF_LAUNCH_CHECK("radix pass 0");
-        radix8_scatter_kernel<<<nblk, 256, 0, st>>>(t->key_b, t->idx_b, t->key_a, t->idx_a, n, 8, t->hist + kHistWords, nblk, nullptr, t->run0);
-        SF_LAUNCH_CHECK("radix pass 1");
+        SF_CUDA(sf_launch_chained(radix8_scatter_kernel, nblk, 256, 0, st, t->key_a, t->idx_a, t->key_b, t->idx_b, n, 0u, t->hist, nblk,
+                                  t->hist + kHistWords, (uint32_t*)nullptr));
+        SF_CUDA(sf_launch_chained(radix8_scatter_kernel, nblk, 256, 0, st, t->key_b, t->idx_b, t->key_a, t->idx_a, n, 8u, t->hist + kHistWords, nblk,
+                                  (uint32_t*)nullptr, t->run0));
     }
-    apply1_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->run0, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts);
-    SF_LAUNCH_CHECK("apply1_kernel");
+    SF_CUDA(sf_launch_chained(apply1_kernel, blocks, 256, 0, st, d, *batch, t->key_a, t->idx_a, t->run0, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts));
     sf_time_end(ctx, SF_T_TABLE, st);
     // S1..S3 on the flows that just completed their fast context (count stays on the device); the feature kernel reads
     // their packets in place, through the list of their slots
@@ -638,12 +643,11 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     if (rc != SF_OK) return rc;
     sf_time_begin(ctx, SF_T_SCORE, st);
     // ... then leaf sums, score, decision and the table update in one kernel (16 lanes per flow)
-    fast_finish_kernel<<<std::min<uint32_t>((n * 16u + 255) / 256, (uint32_t)ctx->num_sms * 2u), 256, 0, st>>>(d, t->fire1_slot, t->counts, reinterpret_cast<const uint16_t*>(w + o_lidx), fo->d_leaf,
-                                                             fo->T, 1u << fo->depth, fo->C, cfg->tau, result_dev, ctx->d_state);
-    SF_LAUNCH_CHECK("fast_finish_kernel");
-    apply2_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire2_slab, t->fire2_slot,
-                                          t->counts, result_dev, ctx->d_state);
-    SF_LAUNCH_CHECK("apply2_kernel");
+    SF_CUDA(sf_launch_chained(fast_finish_kernel, std::min<uint32_t>((n * 16u + 255) / 256, (uint32_t)ctx->num_sms * 2u), 256, 0, st, d, t->fire1_slot,
+                              t->counts, reinterpret_cast<const uint16_t*>(w + o_lidx), fo->d_leaf, fo->T, 1u << fo->depth, fo->C, cfg->tau,
+                              result_dev, ctx->d_state));
+    SF_CUDA(sf_launch_chained(apply2_kernel, blocks, 256, 0, st, d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire2_slab,
+                              t->fire2_slot, t->counts, result_dev, ctx->d_state));
     sf_time_end(ctx, SF_T_SCORE, st);
     // S4 on the flows that just completed their slow context
     sf_packets spk;
@@ -658,8 +662,8 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     rc = sf_launch_slow(ctx, slow, w + o_rows, &t->counts[1], n, reinterpret_cast<float*>(w + o_logits),
                         reinterpret_cast<uint8_t*>(w + o_slab_lab), w + o_slow, st, false);
     if (rc != SF_OK) return rc;
-    apply_slow_kernel<<<blocks, 256, 0, st>>>(d, t->fire2_slot, t->counts, reinterpret_cast<uint8_t*>(w + o_slab_lab), result_dev, ctx->d_state);
-    SF_LAUNCH_CHECK("apply_slow_kernel");
+    SF_CUDA(sf_launch_chained(apply_slow_kernel, blocks, 256, 0, st, d, t->fire2_slot, t->counts, reinterpret_cast<const uint8_t*>(w + o_slab_lab),
+                              result_dev, ctx->d_state));
     return SF_OK;
 }
 }  // namespace
