@@ -173,7 +173,7 @@ __device__ void small_rows_layer(const __nv_bfloat16* __restrict__ A, const __nv
 // HEAD = true (BN = 16): last layer, W zero-padded to 16 rows; logits[r][c] = acc + bias for
 // c < C (fp32, no activation) and label[r] = argmax (lowest index on ties).
 // MODE_HIDDEN_HEAD: the last hidden layer with the head folded in.  head_w = the head's weights bf16 [16][N] (rows past C
-// zero), head_b its bias, CH = 8 or 16 = classes kept per row.  A CTA takes whole 128-row panels (all N / BN tiles of
+// zero), head_b its bias, CH = 2, 4, 8 or 16 = classes kept per row.  A CTA takes whole 128-row panels (all N / BN tiles of
 // a panel in turn), so a row's logits are summed in one place and in one fixed order: column chunks in increasing
 // order inside each of the two epilogue warps that share the row, then (low half + high half) + bias.
 //
@@ -237,12 +237,12 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     // fused head: the head's weights, transposed to [column][CH] bf16, where the other modes stage their output
     uint8_t* const epi_smem = tiles + Cfg::kStages * Cfg::kStageBytes + 256;
     if constexpr (FUSED) {
-        // up to 8 classes: fp32 [column][8] (the bf16 values widened once here instead of once per row in the epilogue, whose
-        // integer pipe is the busy one); up to 16: bf16 [column][16]; 32 KB either way
+        // CH = 2, 4 or 8 classes kept: fp32 [column][CH] (the bf16 values widened once here instead of once per row in the
+        // epilogue, whose integer pipe is the busy one); 16: bf16 [column][16]; at most 32 KB
         for (uint32_t i = threadIdx.x; i < N * CH; i += kGemmThreads) {
             const uint32_t col = i / CH, c = i - col * CH;
             const __nv_bfloat16 w = head_w[(size_t)c * N + col];                // rows past C are zero in the padded head matrix
-            if (CH == 8) reinterpret_cast<float*>(epi_smem)[i] = __bfloat162float(w);
+            if (CH <= 8) reinterpret_cast<float*>(epi_smem)[i] = __bfloat162float(w);
             else reinterpret_cast<__nv_bfloat16*>(epi_smem)[i] = w;
         }
     }
@@ -368,7 +368,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                     tmem_ld32(taddr + c, v);
                     tmem_ld_wait();
                     const float4* b4 = reinterpret_cast<const float4*>(bias + col0 + c);
-                    const uint4* wq = reinterpret_cast<const uint4*>(epi_smem) + (size_t)(col0 + c) * 2;     // 32 bytes per column
+                    const uint8_t* wq = epi_smem + (size_t)(col0 + c) * (CH <= 8 ? CH * 4 : 32);     // this chunk's first column
 #pragma unroll
                     for (int pc = 0; pc < 8; pc++) {
                         const float4 bv = __ldg(b4 + pc);
@@ -383,18 +383,30 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                             const float a[2] = {__uint_as_float(hb << 16), __uint_as_float(hb & 0xFFFF0000u)};
 #pragma unroll
                             for (int q = 0; q < 2; q++) {
-                                const uint4* wp = wq + (size_t)(pc * 4 + e + q) * 2;      // same address in all lanes: a broadcast
+                                // this column's head weights: the same address in all lanes, a broadcast
+                                if constexpr (CH == 16) {
+                                    const uint4* wp = reinterpret_cast<const uint4*>(wq) + (size_t)(pc * 4 + e + q) * 2;
 #pragma unroll
-                                for (uint32_t g = 0; g < 2; g++) {
-                                    const uint4 w = wp[g];
-                                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                                    for (uint32_t g = 0; g < 2; g++) {
+                                        const uint4 w = wp[g];
+                                        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                                    for (int k = 0; k < 4; k++) {
-                                        if (CH == 8) {
-                                            lg[g * 4 + k] = fmaf(a[q], __uint_as_float(ww[k]), lg[g * 4 + k]);
-                                        } else {
+                                        for (int k = 0; k < 4; k++) {
                                             lg[g * 8 + 2 * k] = fmaf(a[q], __uint_as_float(ww[k] << 16), lg[g * 8 + 2 * k]);
                                             lg[g * 8 + 2 * k + 1] = fmaf(a[q], __uint_as_float(ww[k] & 0xFFFF0000u), lg[g * 8 + 2 * k + 1]);
+                                        }
+                                    }
+                                } else {
+                                    const float2* wp = reinterpret_cast<const float2*>(wq) + (size_t)(pc * 4 + e + q) * (CH / 2);
+                                    if constexpr (CH == 2) {
+                                        const float2 w = wp[0];
+                                        lg[0] = fmaf(a[q], w.x, lg[0]); lg[1] = fmaf(a[q], w.y, lg[1]);
+                                    } else {
+#pragma unroll
+                                        for (uint32_t g = 0; g < CH / 4; g++) {
+                                            const float4 w = reinterpret_cast<const float4*>(wp)[g];
+                                            lg[g * 4 + 0] = fmaf(a[q], w.x, lg[g * 4 + 0]); lg[g * 4 + 1] = fmaf(a[q], w.y, lg[g * 4 + 1]);
+                                            lg[g * 4 + 2] = fmaf(a[q], w.z, lg[g * 4 + 2]); lg[g * 4 + 3] = fmaf(a[q], w.w, lg[g * 4 + 3]);
                                         }
                                     }
                                 }
@@ -633,12 +645,13 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
         const uint32_t K = s->dims[l], N = s->dims[l + 1];
         int rc;
         if (fuse_head && l + 1 == L) {
-#define SF_FUSED(BNv) (Cn <= 8 ? launch_gemm_head<BNv, 8>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st) \
-                               : launch_gemm_head<BNv, 16>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st))
+#define SF_FUSED_CH(BNv, CHv) launch_gemm_head<BNv, CHv>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st)
+#define SF_FUSED(BNv) (Cn <= 2 ? SF_FUSED_CH(BNv, 2) : (Cn <= 4 ? SF_FUSED_CH(BNv, 4) : (Cn <= 8 ? SF_FUSED_CH(BNv, 8) : SF_FUSED_CH(BNv, 16))))
             if (N % 256 == 0)      rc = SF_FUSED(256);
             else if (N % 128 == 0) rc = SF_FUSED(128);
             else                   rc = SF_FUSED(64);
 #undef SF_FUSED
+#undef SF_FUSED_CH
         }
         else if (N % 256 == 0) rc = launch_gemm<256>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);
         else if (N % 128 == 0) rc = launch_gemm<128>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, out, st, small_max);

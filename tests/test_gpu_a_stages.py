@@ -306,6 +306,9 @@ def test_mlp_fp32(env):
     ((256, 512, 512, 8), 66000, 66000),   # every panel of every CTA, ragged last panel
     ((192, 320, 384, 16), 1500, 70000),   # three 128-column tiles per panel, 16 logits per row
     ((128, 192, 5), 300, 66001),          # three 64-column tiles per panel, odd class count
+    ((256, 512, 512, 4), 900, 66000),     # four logits kept per row
+    ((256, 512, 512, 3), 515, 66000),     # three classes in the four-logit form
+    ((256, 512, 512, 2), 515, 66000),     # two logits kept per row
     ((128, 256, 3), 300, 66001),          # a single column tile per panel: the head keeps its own launch
 ])
 def test_mlp_bf16_small_integers_are_exact(env, dims, n_rows, cap):
