@@ -169,6 +169,16 @@ __device__ void small_rows_layer(const __nv_bfloat16* __restrict__ A, const __nv
     }
 }
 
+// (d0, d1) += a * (w0, w1): two IEEE fp32 fused multiply-adds in one instruction
+__device__ __forceinline__ void fma_pair(float& d0, float& d1, float a, float w0, float w1) {
+    uint64_t d, aa, ww;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(d0), "f"(d1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(aa) : "f"(a));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ww) : "f"(w0), "f"(w1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(aa), "l"(ww));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+}
+
 // HEAD = false: hidden layer, out = bf16(ReLU(acc + bias)) [rows][N].
 // HEAD = true (BN = 16): last layer, W zero-padded to 16 rows; logits[r][c] = acc + bias for
 // c < C (fp32, no activation) and label[r] = argmax (lowest index on ties).
@@ -405,8 +415,8 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 #pragma unroll
                                         for (uint32_t g = 0; g < CH / 4; g++) {
                                             const float4 w = reinterpret_cast<const float4*>(wp)[g];
-                                            lg[g * 4 + 0] = fmaf(a[q], w.x, lg[g * 4 + 0]); lg[g * 4 + 1] = fmaf(a[q], w.y, lg[g * 4 + 1]);
-                                            lg[g * 4 + 2] = fmaf(a[q], w.z, lg[g * 4 + 2]); lg[g * 4 + 3] = fmaf(a[q], w.w, lg[g * 4 + 3]);
+                                            fma_pair(lg[g * 4 + 0], lg[g * 4 + 1], a[q], w.x, w.y);
+                                            fma_pair(lg[g * 4 + 2], lg[g * 4 + 3], a[q], w.z, w.w);
                                         }
                                     }
                                 }
