@@ -179,6 +179,14 @@ __device__ __forceinline__ void fma_pair(float& d0, float& d1, float a, float w0
     asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
 }
 
+// bf16x2( ReLU(v0 + b0), ReLU(v1 + b1) ), first value in the low half: the conversion clamps at zero itself
+__device__ __forceinline__ uint32_t bias_relu_bf16x2(uint32_t v0, uint32_t v1, float b0, float b1) {
+    const float x0 = __uint_as_float(v0) + b0, x1 = __uint_as_float(v1) + b1;
+    uint32_t h;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(h) : "f"(x1), "f"(x0));
+    return h;
+}
+
 // HEAD = false: hidden layer, out = bf16(ReLU(acc + bias)) [rows][N].
 // HEAD = true (BN = 16): last layer, W zero-padded to 16 rows; logits[r][c] = acc + bias for
 // c < C (fp32, no activation) and label[r] = argmax (lowest index on ties).
@@ -386,10 +394,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 #pragma unroll
                         for (int e = 0; e < 4; e += 2) {
                             // bias + ReLU + bf16 rounding exactly as the stored activations would have had
-                            const float x0 = fmaxf(__uint_as_float(v[pc * 4 + e]) + bb[e], 0.0f);
-                            const float x1 = fmaxf(__uint_as_float(v[pc * 4 + e + 1]) + bb[e + 1], 0.0f);
-                            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
-                            const uint32_t hb = *reinterpret_cast<uint32_t*>(&h);
+                            const uint32_t hb = bias_relu_bf16x2(v[pc * 4 + e], v[pc * 4 + e + 1], bb[e], bb[e + 1]);
                             const float a[2] = {__uint_as_float(hb << 16), __uint_as_float(hb & 0xFFFF0000u)};
 #pragma unroll
                             for (int q = 0; q < 2; q++) {
@@ -469,10 +474,7 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
                         uint32_t pk[4];
 #pragma unroll
                         for (int e = 0; e < 4; e++) {
-                            float x0 = fmaxf(__uint_as_float(v[pc * 8 + 2 * e]) + bv[2 * e], 0.0f);
-                            float x1 = fmaxf(__uint_as_float(v[pc * 8 + 2 * e + 1]) + bv[2 * e + 1], 0.0f);
-                            __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
-                            pk[e] = *reinterpret_cast<uint32_t*>(&h);
+                            pk[e] = bias_relu_bf16x2(v[pc * 8 + 2 * e], v[pc * 8 + 2 * e + 1], bv[2 * e], bv[2 * e + 1]);
                         }
                         *reinterpret_cast<uint4*>(stg + lane * 64u + (((uint32_t)pc ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
