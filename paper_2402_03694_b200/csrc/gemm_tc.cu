@@ -14,7 +14,9 @@
 //               32 x 32 block through shared memory so that global stores are whole 64-byte
 //               row segments (8 rows per instruction)
 // Two accumulator buffers in TMEM (2 x BN columns) let the MMAs of tile i+1 overlap
-// the epilogue of tile i.  The row count lives in device memory, so routing and the
+// the epilogue of tile i.  Large batches of 256-column layers run the same kernel on CTA pairs (clusters of two, one
+// tcgen05.mma.cta_group::2 per K step for a 256 x 256 tile): a third less operand traffic per flop, which is what counts
+// on a part whose tensor pipe is power-limited.  The row count lives in device memory, so routing and the
 // slow model need no host round trip; tiles past the count are never scheduled and
 // rows past it are never stored.  Every barrier wait is bounded: on a timeout the
 // block records SF_ERR_DEVICE_TIMEOUT, lets its copies land, frees TMEM and returns.
@@ -515,6 +517,26 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     }
 }
 
+// Can this device co-schedule two-CTA clusters of this kernel at all?  Asked once per kernel and device (the smem opt-in must
+// already be set); where the answer is no, or the query fails, the single-CTA kernel serves the layer instead.
+template <typename Kern>
+bool pairs_supported(Kern k, size_t smem, int device, int (&cache)[64]) {
+    int& c = cache[device & 63];                       // 0 unknown, 1 yes, -1 no
+    if (c == 0) {
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(2); lc.blockDim = dim3(kGemmThreads); lc.dynamicSmemBytes = smem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        int n = 0;
+        const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, k, &lc);
+        if (e != cudaSuccess) (void)cudaGetLastError();
+        c = (e == cudaSuccess && n > 0) ? 1 : -1;
+    }
+    return c > 0;
+}
+
 // launch as clusters of two CTAs
 template <typename Kern, typename... Args>
 cudaError_t launch_pairs(Kern k, uint32_t grid, size_t smem, cudaStream_t st, Args... args) {
@@ -548,12 +570,17 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
             static bool attr_set_dev[64] = {};
             bool& attr_set = attr_set_dev[ctx->device & 63];
             if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CfgP::kSmemBytes)); attr_set = true; }
+            static int pairs_ok[64] = {};
             const uint32_t pair_tiles = ((capacity + 2 * BM - 1) / (2 * BM)) * (N / BN);
             const uint32_t grid = 2u * std::min<uint32_t>((uint32_t)ctx->num_sms / 2u, pair_tiles);
+            if (pairs_supported(kp, CfgP::kSmemBytes, ctx->device, pairs_ok)) {
             SF_CUDA(launch_pairs(kp, grid, CfgP::kSmemBytes, st, tmA, tmW, bias, n_rows_dev, N, K, reinterpret_cast<__nv_bfloat16*>(out), ctx->d_state,
                                  (float*)nullptr, (uint8_t*)nullptr, 0u, 0u, reinterpret_cast<const __nv_bfloat16*>(A),
                                  reinterpret_cast<const __nv_bfloat16*>(W), capacity, (const __nv_bfloat16*)nullptr, (const float*)nullptr));
             return SF_OK;
+            }
+            rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);      // back to the single-CTA tile
+            if (rc != SF_OK) return rc;
         }
     }
     auto k = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN>;
@@ -588,12 +615,17 @@ int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bia
         static bool attr_set_dev[64] = {};
         bool& attr_set = attr_set_dev[ctx->device & 63];
         if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP)); attr_set = true; }
+        static int pairs_ok[64] = {};
         const uint32_t pair_panels = (capacity + 2 * BM - 1) / (2 * BM);
         const uint32_t grid = 2u * std::min<uint32_t>((uint32_t)ctx->num_sms / 2u, pair_panels);
+        if (pairs_supported(kp, kSmemP, ctx->device, pairs_ok)) {
         SF_CUDA(launch_pairs(kp, grid, kSmemP, st, tmA, tmW, bias, n_rows_dev, N, K, (__nv_bfloat16*)nullptr, ctx->d_state, logits, label, C, 0u,
                              reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
                              reinterpret_cast<const __nv_bfloat16*>(W16), head_bias));
         return SF_OK;
+        }
+        rc = encode_tmap_bf16_2d(&tmW, W, N, K, BN, BK);          // back to the single-CTA tile
+        if (rc != SF_OK) return rc;
     }
     auto k = gemm_bias_relu_bf16_kernel<BN, MODE_HIDDEN_HEAD, CH>;
     static bool attr_set_dev[64] = {};                 // the opt-in is per device
