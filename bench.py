@@ -193,7 +193,7 @@ def kernel_launches_per_step(cfg, capacity):
         slow = (len(cfg.dims) - 1) + (1 if cfg.slow_dtype == "f32" else 0)    # layers (+ argmax for fp32)
         nl = cfg.dims[-2]
         bn = 256 if nl % 256 == 0 else (128 if nl % 128 == 0 else 64)
-        if cfg.slow_dtype == "bf16" and capacity > 65536 and nl <= 1024 and nl // bn >= 2:
+        if cfg.slow_dtype == "bf16" and nl <= 1024 and nl // bn >= 2:
             slow -= 1                                                         # the head runs inside the last hidden layer's launch
     else:
         slow = 1                                                              # the fused CNN kernel
@@ -581,7 +581,7 @@ def bench_stream(cfg, args, env, with_e2e, with_cpu, cpu_budget_s, steps):
     return out
 
 
-STREAM_LAUNCHES_PER_BATCH = 14
+STREAM_LAUNCHES_PER_BATCH = 13
 
 
 def oracle_stream_baseline(cfg, n_keys, m, budget_s):

@@ -12,7 +12,8 @@
 struct sf_dev_state {
     sf_counters counters;
     uint32_t    scan_total;      // number of assigned flows found by the last route
-    uint32_t    pad[15];
+    uint32_t    blocks_done;     // blocks of the running few-rows layer that have stored their columns (the last one puts it back to zero)
+    uint32_t    pad[14];
 };
 
 struct sf_ctx {

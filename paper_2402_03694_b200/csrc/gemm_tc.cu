@@ -112,40 +112,61 @@ __device__ __forceinline__ float warp_rows_reduce16(float (&v)[16], uint32_t lan
 }
 
 // HEAD = false: out[r][n] = bf16(ReLU(sum + bias[n])), columns spread over all warps of the grid.
-// HEAD = true (block 0 only, W padded to 16 rows): logits[r][c] = sum + bias[c] for c < C, label[r] = argmax (lowest index on ties).
-template <bool HEAD>
+// HEAD = true (one block: block 0, or whichever block calls it with ANY_BLOCK; W padded to 16 rows): logits[r][c] = sum + bias[c]
+// for c < C, label[r] = argmax (lowest index on ties).
+template <bool HEAD, bool ANY_BLOCK = false>
 __device__ void small_rows_layer(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias,
                                  uint32_t rows, uint32_t N, uint32_t K, __nv_bfloat16* __restrict__ out,
                                  float* __restrict__ logits, uint8_t* __restrict__ label, uint32_t C, uint8_t* smem)
 {
     __shared__ float lg[kSmallRows][16];
-    if (HEAD && blockIdx.x != 0) return;
+    if (HEAD && !ANY_BLOCK && blockIdx.x != 0) return;
     uint4* As = reinterpret_cast<uint4*>(smem);                           // [16 rows][K] bf16, rows past the count zero
     const uint32_t k16 = K / 8;                                           // 16-byte chunks per row
-    for (uint32_t i = threadIdx.x; i < kSmallRows * k16; i += blockDim.x) {
-        const uint32_t r = i / k16, c = i - r * k16;
-        As[i] = (r < rows) ? __ldg(reinterpret_cast<const uint4*>(A + (size_t)r * K) + c) : make_uint4(0, 0, 0, 0);
-    }
-    __syncthreads();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
     const uint32_t n_cols = HEAD ? 16u : N;
     const uint32_t w0 = HEAD ? warp : blockIdx.x * wpb + warp, wstep = HEAD ? wpb : gridDim.x * wpb;
+    // A lane holds kPF 16-byte pieces of a weight row at a time (K up to 2048 in one go): the loads are all in flight before the
+    // first is used, so a column costs one trip to L2 instead of one per piece.  The first column's pieces are asked for before
+    // the activations are staged, and travel meanwhile.
+    constexpr int kPF = 8;
+    uint4 wv[kPF];
+    auto fetch = [&](uint32_t n, uint32_t c0) {
+        const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)n * K);
+#pragma unroll
+        for (int j = 0; j < kPF; j++) {
+            const uint32_t c = c0 + lane + 32u * j;
+            wv[j] = (c < k16) ? __ldg(wrow + c) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    if (w0 < n_cols) fetch(w0, 0);
+    for (uint32_t i = threadIdx.x; i < kSmallRows * k16; i += blockDim.x) {
+        const uint32_t r = i / k16, c = i - r * k16;
+        // (from L2: with the head in the same launch these activations were written by other blocks a moment ago)
+        As[i] = (r < rows) ? __ldcg(reinterpret_cast<const uint4*>(A + (size_t)r * K) + c) : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
     for (uint32_t n = w0; n < n_cols; n += wstep) {
         float acc[kSmallRows];
 #pragma unroll
         for (int r = 0; r < (int)kSmallRows; r++) acc[r] = 0.0f;
-        const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)n * K);
-        for (uint32_t c = lane; c < k16; c += 32) {
-            const uint4 wv = __ldg(wrow + c);
-            const uint32_t wq[4] = {wv.x, wv.y, wv.z, wv.w};
+        for (uint32_t c0 = 0; c0 < k16; c0 += 32u * kPF) {
+            if (n != w0 || c0 != 0) fetch(n, c0);
 #pragma unroll
-            for (int r = 0; r < (int)kSmallRows; r++) {
-                const uint4 av = As[r * k16 + c];
-                const uint32_t aq[4] = {av.x, av.y, av.z, av.w};
+            for (int j = 0; j < kPF; j++) {
+                const uint32_t c = c0 + lane + 32u * j;
+                if (c < k16) {
+                    const uint32_t wq[4] = {wv[j].x, wv[j].y, wv[j].z, wv[j].w};
 #pragma unroll
-                for (int e = 0; e < 4; e++) {
-                    acc[r] = fmaf(__uint_as_float(aq[e] << 16), __uint_as_float(wq[e] << 16), acc[r]);
-                    acc[r] = fmaf(__uint_as_float(aq[e] & 0xFFFF0000u), __uint_as_float(wq[e] & 0xFFFF0000u), acc[r]);
+                    for (int r = 0; r < (int)kSmallRows; r++) {
+                        const uint4 av = As[r * k16 + c];
+                        const uint32_t aq[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+                        for (int e = 0; e < 4; e++) {
+                            acc[r] = fmaf(__uint_as_float(aq[e] << 16), __uint_as_float(wq[e] << 16), acc[r]);
+                            acc[r] = fmaf(__uint_as_float(aq[e] & 0xFFFF0000u), __uint_as_float(wq[e] & 0xFFFF0000u), acc[r]);
+                        }
+                    }
                 }
             }
         }
@@ -222,7 +243,27 @@ gemm_bias_relu_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     // the count is the caller's device word: never trust it beyond the rows the buffers hold
     const uint32_t n_rows = sf_clamp_rows(*n_rows_dev, capacity, st);
     if (n_rows <= small_max) {                       // a handful of rows (small_max = 0: never): CUDA cores, same launch (pairs: both CTAs alike)
-        if (n_rows) small_rows_layer<HEAD>(A_raw, W_raw, bias, n_rows, N, K, out, logits, label, C, smem_raw);
+        if constexpr (FUSED) {
+            // hidden layer into the caller's 16-row scratch (`out`), then the head by whichever block stores its columns last:
+            // nobody waits for anybody (an arrival counter in device memory; the last block puts it back to zero)
+            __shared__ uint32_t is_last;
+            if (n_rows) {
+                small_rows_layer<false>(A_raw, W_raw, bias, n_rows, N, K, out, nullptr, nullptr, 0, smem_raw);
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    __threadfence();
+                    is_last = (atomicAdd(&st->blocks_done, 1u) == gridDim.x - 1u) ? 1u : 0u;
+                }
+                __syncthreads();
+                if (is_last) {
+                    if (threadIdx.x == 0) st->blocks_done = 0;
+                    __threadfence();
+                    small_rows_layer<true, true>(out, head_w, head_b, n_rows, 16, N, nullptr, logits, label, C, smem_raw);
+                }
+            }
+        } else {
+            if (n_rows) small_rows_layer<HEAD>(A_raw, W_raw, bias, n_rows, N, K, out, logits, label, C, smem_raw);
+        }
         return;
     }
     const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -598,7 +639,8 @@ int launch_gemm(sf_ctx* ctx, const void* A, const void* W, const float* bias, co
 // last hidden layer with the head folded into its epilogue (no activations written); W16 = the head's weights padded to 16 rows
 template <uint32_t BN, uint32_t CH>
 int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bias, const uint32_t* n_rows_dev, uint32_t capacity,
-                     uint32_t N, uint32_t K, const void* W16, const float* head_bias, uint32_t C, float* logits, uint8_t* label, cudaStream_t st)
+                     uint32_t N, uint32_t K, const void* W16, const float* head_bias, uint32_t C, float* logits, uint8_t* label, cudaStream_t st,
+                     uint32_t small_max, void* small_scratch /* bf16 [16][N]: the hidden layer of a few-rows batch */)
 {
     using Cfg = GemmCfg<BN>;
     constexpr uint32_t kSmem = Cfg::kSmemBytesHead16;        // 32 KB of head weights where the other modes stage 16 KB of output
@@ -619,7 +661,7 @@ int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bia
         const uint32_t pair_panels = (capacity + 2 * BM - 1) / (2 * BM);
         const uint32_t grid = 2u * std::min<uint32_t>((uint32_t)ctx->num_sms / 2u, pair_panels);
         if (pairs_supported(kp, kSmemP, ctx->device, pairs_ok)) {
-        SF_CUDA(launch_pairs(kp, grid, kSmemP, st, tmA, tmW, bias, n_rows_dev, N, K, (__nv_bfloat16*)nullptr, ctx->d_state, logits, label, C, 0u,
+        SF_CUDA(launch_pairs(kp, grid, kSmemP, st, tmA, tmW, bias, n_rows_dev, N, K, reinterpret_cast<__nv_bfloat16*>(small_scratch), ctx->d_state, logits, label, C, small_max,
                              reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
                              reinterpret_cast<const __nv_bfloat16*>(W16), head_bias));
         return SF_OK;
@@ -633,7 +675,7 @@ int launch_gemm_head(sf_ctx* ctx, const void* A, const void* W, const float* bia
     if (!attr_set) { SF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem)); attr_set = true; }
     const uint32_t panels = (capacity + BM - 1) / BM;
     const uint32_t grid = (uint32_t)ctx->num_sms < panels ? (uint32_t)ctx->num_sms : panels;
-    SF_CUDA(sf_launch_chained(k, grid, kGemmThreads, kSmem, st, tmA, tmW, bias, n_rows_dev, N, K, (__nv_bfloat16*)nullptr, ctx->d_state, logits, label, C, 0u,
+    SF_CUDA(sf_launch_chained(k, grid, kGemmThreads, kSmem, st, tmA, tmW, bias, n_rows_dev, N, K, reinterpret_cast<__nv_bfloat16*>(small_scratch), ctx->d_state, logits, label, C, small_max,
                               reinterpret_cast<const __nv_bfloat16*>(A), reinterpret_cast<const __nv_bfloat16*>(W), capacity,
                               reinterpret_cast<const __nv_bfloat16*>(W16), head_bias));
     return SF_OK;
@@ -677,19 +719,19 @@ int sf_mlp_bf16_forward(sf_ctx* ctx, const sf_slow* s, const void* rows, const u
     const uint32_t small_max = small ? kSmallRows : 0u;
     const void* in = rows;
     const uint32_t L = s->n_layers - 1;                  // the head
-    // Large batches: the head is folded into the last hidden layer (its activations are then never written or re-read).
-    // Not where a launch may see only a handful of rows (those take the CUDA-core path, layer by layer), nor where a
-    // row panel has a single column tile (the epilogue warps' hand-over needs two tiles between two panel ends).
+    // The head is folded into the last hidden layer (its activations are then never written or re-read; a few-rows batch
+    // keeps them in a 16-row scratch and the block that finishes last adds the head): one launch less either way.
+    // Not where a row panel has a single column tile (the epilogue warps' hand-over needs two tiles between two panel ends).
     const uint32_t Nl = s->dims[L], Cn = s->dims[L + 1];
     const uint32_t BNl = Nl % 256 == 0 ? 256u : (Nl % 128 == 0 ? 128u : 64u);
-    const bool fuse_head = small_max == 0 && Nl <= kFusedHeadMaxN && Nl / BNl >= 2;
+    const bool fuse_head = Nl <= kFusedHeadMaxN && Nl / BNl >= 2;
     sf_time_begin(ctx, SF_T_GEMM, st);
     for (uint32_t l = 0; l + 1 < s->n_layers; l++) {
         void* out = (l & 1) ? h1 : h0;
         const uint32_t K = s->dims[l], N = s->dims[l + 1];
         int rc;
         if (fuse_head && l + 1 == L) {
-#define SF_FUSED_CH(BNv, CHv) launch_gemm_head<BNv, CHv>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st)
+#define SF_FUSED_CH(BNv, CHv) launch_gemm_head<BNv, CHv>(ctx, in, s->d_W[l], s->d_b[l], n_rows_dev, capacity, N, K, s->d_W[L], s->d_b[L], Cn, logits, label, st, small_max, out)
 #define SF_FUSED(BNv) (Cn <= 2 ? SF_FUSED_CH(BNv, 2) : (Cn <= 4 ? SF_FUSED_CH(BNv, 4) : (Cn <= 8 ? SF_FUSED_CH(BNv, 8) : SF_FUSED_CH(BNv, 16))))
             if (N % 256 == 0)      rc = SF_FUSED(256);
             else if (N % 128 == 0) rc = SF_FUSED(128);
