@@ -47,7 +47,7 @@ FOREST_WAVEFRONTS_PER_VISIT = 3
 # DRAM bytes per launch measured with ncu for the dominant kernel class of a config, with the hash of the
 # kernel's source at capture time: the figure turns null as soon as the kernel changes
 # (profiles/gemm_traffic_config2_524288_flows.md).
-TRAFFIC_BY_SOURCE = {("gemm", 2): {"src_hash": "d6be8276c57016a9", "bytes_per_row_per_launch": 1458944000 / 3 / 123679}}
+TRAFFIC_BY_SOURCE = {("gemm", 2): {"src_hash": "159f94d817c7cda2", "bytes_per_row_per_launch": 1468544768 / 3 / 123679}}
 PAPER_CONTEXT = ("paper: over 48.5k new flows/s on a 16-core CPU server; 76.3% of flows inferred in under 16 ms "
                  "(other hardware, real traffic; not comparable)")
 
