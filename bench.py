@@ -610,6 +610,56 @@ def oracle_stream_baseline(cfg, n_keys, m, budget_s):
                       "(model stages on %d threads), %.1f s" % (nb, m, threads, dt)}
 
 
+def slow_model_sustained(cfg, seconds, env):
+    """Diagnostic, not a bench line: the slow model alone, back to back for `seconds`, with the SM clock and the board power
+    sampled every 25 ms - shows what the tensor pipe sustains under the power limit next to a short burst."""
+    torch, sf, hz, ctx = env["torch"], env["sf"], env["hz"], env["ctx"]
+    if cfg.slow != "mlp" or cfg.slow_dtype != "bf16":
+        raise SystemExit("--slow-sustained: a bf16 MLP config (2, 3 or 5)")
+    rows_n = int(min(cfg.n, 4_000_000) * ((100 - cfg.q_percent) / 100.0 if cfg.q_percent else 0.3))   # about the assigned share
+    model = flowgen.gen_mlp(cfg.seed_model, cfg.dims)
+    h = sf.sf_mlp_create(ctx, sf.SF_BF16, model["dims"], model["W"], model["b"])
+    g = torch.Generator(device="cuda").manual_seed(cfg.seed_data)
+    x = (torch.randn(rows_n, cfg.dims[0], device="cuda", generator=g) * 0.5).to(torch.bfloat16)
+    nd = torch.tensor([rows_n], dtype=torch.int32, device="cuda")
+    logits = torch.zeros(rows_n, cfg.dims[-1], device="cuda")
+    lab = torch.zeros(rows_n, dtype=torch.uint8, device="cuda")
+    flops = rows_n * hidden_flops_per_row(cfg)
+    for _ in range(3):
+        sf.sf_slow_infer(ctx, h, x, nd, rows_n, logits, lab)
+    torch.cuda.synchronize()
+    time.sleep(1.0)
+    f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+    p = subprocess.Popen(["nvidia-smi", "-i", str(env["local"]), "--query-gpu=clocks.sm,power.draw,clocks_event_reasons.sw_power_cap",
+                          "--format=csv,noheader,nounits", "-lms", "25"], stdout=f, stderr=subprocess.DEVNULL)
+    ev = [torch.cuda.Event(enable_timing=True)]
+    ev[0].record()
+    t0 = time.perf_counter()
+    while time.perf_counter() - t0 < seconds and len(ev) < 20000:
+        for _ in range(10):
+            sf.sf_slow_infer(ctx, h, x, nd, rows_n, logits, lab)
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        ev.append(e)
+        if len(ev) % 8 == 0:
+            ev[-1].synchronize()                            # keep the launch queue short so that the wall clock bounds the loop
+    torch.cuda.synchronize()
+    p.terminate()
+    p.wait()
+    ms = np.array([ev[i].elapsed_time(ev[i + 1]) / 10 for i in range(len(ev) - 1)])
+    rows = [r.split(",") for r in open(f.name).read().strip().splitlines() if r.count(",") >= 2]
+    os.unlink(f.name)
+    half = rows[len(rows) // 2:]
+    out = {"diagnostic": "slow model alone, back to back", "workload": cfg.name, "rows": rows_n, "seconds": seconds,
+           "forwards": 10 * (len(ev) - 1), "first_10_forwards_tflops": flops / ms[0] / 1e9,
+           "second_half_tflops": flops / float(np.mean(ms[len(ms) // 2:])) / 1e9,
+           "second_half_sm_mhz_median": float(np.median([float(r[0]) for r in half])) if half else None,
+           "second_half_power_w_median": float(np.median([float(r[1]) for r in half])) if half else None,
+           "sw_power_cap_active_share": float(np.mean([r[2].strip().lower().startswith("active") for r in rows])) if rows else None}
+    sf.sf_slow_destroy(h)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -625,6 +675,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="only the headline config (no `configs` object)")
     ap.add_argument("--batches-per-step", type=int, default=16)
+    ap.add_argument("--slow-sustained", type=float, default=0.0,
+                    help="diagnostic: loop the config's bf16 MLP alone for this many seconds and print clocks, power and TFLOP/s")
     args = ap.parse_args()
     cfg = flowgen.get_config(args.config)
     if args.impl == "reference":
@@ -654,6 +706,10 @@ def main():
     peaks, peak_kind = load_peaks()
     env = {"torch": torch, "sf": sf, "hz": hz, "ctx": ctx, "rank": rank, "world": world, "local": local, "dist": dist,
            "peaks": peaks, "peak_kind": peak_kind}
+    if args.slow_sustained > 0:
+        if rank == 0:
+            print(json.dumps(slow_model_sustained(cfg, args.slow_sustained, env)))
+        return
     t_start = time.time()
     with_e2e, with_cpu = not args.no_e2e, not args.no_cpu_baseline
     if cfg.c == 5:
