@@ -116,15 +116,14 @@ __device__ __forceinline__ float transpose_reduce32(float (&v)[32], uint32_t lan
     return v[0];
 }
 
-__device__ __forceinline__ uint32_t pack_relu_bf16(uint32_t a, uint32_t b, float ba, float bb) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(__uint_as_float(a) + ba, 0.0f), fmaxf(__uint_as_float(b) + bb, 0.0f));
-    return *reinterpret_cast<uint32_t*>(&h);
-}
 // {high half: bf16(max(hi, 0)), low half: bf16(max(lo, 0))}, round to nearest even
 __device__ __forceinline__ uint32_t relu_bf16x2(float hi, float lo) {
     uint32_t d;
     asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
+}
+__device__ __forceinline__ uint32_t pack_relu_bf16(uint32_t a, uint32_t b, float ba, float bb) {
+    return relu_bf16x2(__uint_as_float(b) + bb, __uint_as_float(a) + ba);     // a in the low half
 }
 
 struct Bias1 { float v[C1]; };
