@@ -481,7 +481,8 @@ def bench_stream(cfg, args, env, with_e2e, with_cpu, cpu_budget_s, steps):
     prof_b = 8                                             # extra batches, run with the per-kernel timing ring on
     e2e_b = 32 if with_e2e else 0                          # extra batches, ingested from pinned host memory
     n_warm, n_meas = args.warmup * bps, steps * bps
-    n_batches = n_warm + n_meas + prof_b + e2e_b
+    n_seq = n_meas                                         # the same number of batches once more, ingested without the pipelining
+    n_batches = n_warm + n_meas + n_seq + prof_b + e2e_b
     log2_slots = max(10, int(np.ceil(np.log2(n_keys / 0.3))))
     src = flowgen.StreamSource(cfg.seed_data, n_keys, 1.1)
     # models of config 2 (forest on 8 packets with the 48-feature definition, 2048-wide MLP on 64 packets + zero padding)
@@ -516,30 +517,46 @@ def bench_stream(cfg, args, env, with_e2e, with_cpu, cpu_budget_s, steps):
             h = {k: torch.from_numpy(np.ascontiguousarray(hb[k])).pin_memory() for k in names}
             host_batches.append(sf.make_pkt_batch(*[h[k] for k in names]))
     res = torch.zeros((n_batches, 8), dtype=torch.int32, device="cuda")
+    # the timed region: pipelined ingest (look-up + sort of batch b+1 under the model work of batch b), flushed before the
+    # closing event so that every batch's work lies inside the region
+    sf.sf_table_set_pipelined(ctx, table, True)
     for b in range(n_warm):
         sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
+    sf.sf_table_flush(ctx, table)
     torch.cuda.synchronize()
+    b0 = n_warm
     sampler = ClockSampler(device_index(env["local"]))
     sampler.start(); time.sleep(0.3)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    for b in range(n_warm, n_warm + n_meas):
+    for b in range(b0, b0 + n_meas):
         sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
+    sf.sf_table_flush(ctx, table)
     ev1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
     ms = ev0.elapsed_time(ev1)
+    sf.sf_table_set_pipelined(ctx, table, False)
     c = sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
+    # for comparison, the following batches one after the other on one stream
+    es0, es1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    es0.record()
+    for b in range(b0 + n_meas, b0 + n_meas + n_seq):
+        sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
+    es1.record()
+    torch.cuda.synchronize()
+    ms_seq = es0.elapsed_time(es1)
+    sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
     # per-kernel-class times from a few more batches with the event ring on (the events cost time themselves)
     sf.sf_ctx_set_timing(ctx, True)
-    for b in range(n_warm + n_meas, n_warm + n_meas + prof_b):
+    for b in range(b0 + n_meas + n_seq, b0 + n_meas + n_seq + prof_b):
         sf.sf_table_ingest(ctx, table, dev_batches[b], forest, cfg.F, slow, rcfg, res[b])
     torch.cuda.synchronize()
     recs = [sf.sf_ctx_get_timing(ctx, back) for back in range(prof_b)]
     sf.sf_ctx_set_timing(ctx, False)
     sf.sf_ctx_poll(ctx, reset=True, raise_on_error=False)
     stage_ms = {k: float(np.mean([x[k] for x in recs])) for k in recs[0]}
-    r = res[n_warm:n_warm + n_meas].cpu().numpy().astype(np.int64).sum(0)
+    r = res[b0:b0 + n_meas].cpu().numpy().astype(np.int64).sum(0)
     new_flows, fast_fired, fast_done, escalated, slow_fired, dropped, missed = [int(x) for x in r[:7]]
     secs = ms * 1e-3
     pk = n_meas * m
@@ -568,7 +585,9 @@ def bench_stream(cfg, args, env, with_e2e, with_cpu, cpu_budget_s, steps):
            "fraction_answered_at_fast_stage": (fast_done / answered) if answered else None,
            "counts": {"new_flows": new_flows, "fast_fired": fast_fired, "fast_done": fast_done, "escalated": escalated,
                       "slow_fired": slow_fired, "dropped_after_decision": dropped, "missed": missed},
-           "per_batch_stage_ms": stage_ms, "us_per_batch": 1e3 * ms / n_meas,
+           "per_batch_stage_ms": stage_ms, "us_per_batch": 1e3 * ms / n_meas, "us_per_batch_unpipelined": 1e3 * ms_seq / n_seq,
+           "pipelined": "sf_table_set_pipelined: look-up and sort of batch b+1 on the caller's stream under the model work of batch b on "
+                        "the table's stream; flushed inside the timed region",
            "launches_per_batch": STREAM_LAUNCHES_PER_BATCH, "gpu_launches": STREAM_LAUNCHES_PER_BATCH * n_meas,
            "sector_traffic_gbs": pk * 200 / secs / 1e9,
            "e2e": e2e, "clocks": clocks, "device_error": c.device_error}

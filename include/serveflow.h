@@ -402,6 +402,18 @@ int  sf_table_ingest_host(sf_ctx* ctx, sf_table* table, const sf_pkt_batch* batc
                           void* stream);
 int  sf_table_lookup(sf_ctx* ctx, const sf_table* table, const sf_key* keys_dev, uint32_t n,
                      sf_flow_result* out_dev, void* stream);
+/* Pipelined ingest (off by default; the paper's server likewise keeps packet collection and inference in separate consumers,
+ * Sec. 4.1).  With it on, sf_table_ingest enqueues the look-up and the sort of the batch on the caller's stream and everything
+ * from the context update on (S1-S4, table updates, the counts in *result_dev) on a stream of the table's own, so that the next
+ * batch's look-up and sort overlap this batch's model work.  Results are the same as without it.  What changes for the caller:
+ * *result_dev, the context's counters and the table's state are complete on the caller's stream only after sf_table_flush
+ * (sf_table_lookup, sf_table_sweep and sf_table_ingest_host flush by themselves); a batch's input planes and its result_dev
+ * must stay untouched until then; every call on the table uses the same stream; the context serves this table only while
+ * batches are in flight (its workspace is the model phase's scratch).  Turning it on allocates a second set of per-batch
+ * scratch (about 2 MB + 4 bytes per slot) and synchronises the device; turning it off waits for the table's stream. */
+int  sf_table_set_pipelined(sf_ctx* ctx, sf_table* table, int on);
+/* Makes `stream` wait for the model work of every batch ingested so far (no-op unless pipelined). */
+int  sf_table_flush(sf_ctx* ctx, sf_table* table, void* stream);
 
 /* Table lifecycle.  Sec. 3.1 and 4.1: data that waits without a match is discarded after a
  * timeout; the QoE task of Sec. 5.1 needs a monitored flow to be inferred again and again.

@@ -85,7 +85,7 @@ EXPORTS = [
     "sf_route_noalloc",
     "sf_universal_thresholds", "sf_universal_thresholds_dev", "sf_per_class_thresholds", "sf_mlp_create", "sf_cnn_create", "sf_slow_destroy", "sf_slow_infer",
     "sf_serve_batch", "sf_serve_batch3", "sf_serve_batch_host", "sf_serve_batch_intermediates",
-    "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_ingest_host", "sf_table_lookup", "sf_table_set_time", "sf_table_sweep",
+    "sf_table_create", "sf_table_destroy", "sf_table_ingest", "sf_table_ingest_host", "sf_table_lookup", "sf_table_set_time", "sf_table_sweep", "sf_table_set_pipelined", "sf_table_flush",
 ]
 
 _L = None
@@ -133,6 +133,8 @@ def _lib():
         L.sf_table_ingest.argtypes = [V, V, C.POINTER(sf_pkt_batch), V, U32, V, C.POINTER(sf_route_cfg), V, V]
         L.sf_table_ingest_host.argtypes = L.sf_table_ingest.argtypes
         L.sf_table_lookup.argtypes = [V, V, V, U32, V, V]
+        L.sf_table_set_pipelined.argtypes = [V, V, I]
+        L.sf_table_flush.argtypes = [V, V, V]
         L.sf_table_set_time.argtypes = [V, U32]
         L.sf_table_sweep.argtypes = [V, V, U32, U32, C.c_int, V, V]
         _L = L
@@ -387,6 +389,14 @@ def sf_table_set_time(table, now):
 def sf_table_sweep(ctx, table, now, idle_timeout, rearm, result_dev, stream=None):
     _check(_lib().sf_table_sweep(ctx, table, now & 0xFFFFFFFF, idle_timeout, int(bool(rearm)), _dp(result_dev), _stream(stream)),
            "sf_table_sweep")
+
+
+def sf_table_set_pipelined(ctx, table, on):
+    _check(_lib().sf_table_set_pipelined(ctx, table, int(on)), "sf_table_set_pipelined")
+
+
+def sf_table_flush(ctx, table, stream=None):
+    _check(_lib().sf_table_flush(ctx, table, _stream(stream)), "sf_table_flush")
 
 
 def sf_table_lookup(ctx, table, keys_dev, n, out_dev, stream=None):

@@ -64,6 +64,17 @@ struct sf_table {
     uint32_t* counts;                 // [0] n_fire1, [1] n_fire2
     uint32_t* pkt_slot; uint32_t* hist;
     void* all;                        // one allocation behind everything above
+    // Pipelined ingest (off by default): the look-up and sort of batch b+1 (caller's stream) overlap the fast / slow model work
+    // of batch b (the table's own stream).  What the two halves of consecutive batches would share exists twice and is used in
+    // turn: sort keys, indices, run starts, packet slots, digit counts, and the per-slot `first` array.
+    struct SortSet { uint32_t* key_a; uint32_t* key_b; uint32_t* idx_a; uint32_t* idx_b; uint32_t* run0; uint32_t* pkt_slot; uint32_t* hist; uint32_t* first; };
+    SortSet set[2];
+    void* all2;                       // the second set's allocation
+    int pipelined;
+    uint64_t n_batches;               // batches ingested in pipelined mode (selects the set)
+    cudaStream_t model_stream;
+    cudaEvent_t ev_sorted[2], ev_done[2];
+    bool outstanding;                 // model-phase work may still be running on model_stream
 };
 
 namespace {
@@ -544,12 +555,70 @@ extern "C" int sf_table_create(sf_ctx* ctx, uint32_t log2_slots, uint32_t fast_p
     }
     e = cudaMemset(d.first, 0xFF, S * 4);
     if (e != cudaSuccess) { cudaFree(t->all); delete t; return sf_set_cuda_error(e, "cudaMemset(table)"); }
+    t->set[0] = sf_table::SortSet{t->key_a, t->key_b, t->idx_a, t->idx_b, t->run0, t->pkt_slot, t->hist, d.first};
     *out = t;
+    return SF_OK;
+}
+
+// Makes `stream` wait for the model-phase work of every batch ingested so far (pipelined mode; nothing to do otherwise).
+extern "C" int sf_table_flush(sf_ctx* ctx, sf_table* t, void* stream)
+{
+    if (!ctx || !t) return SF_ERR_ARG;
+    if (!t->pipelined || !t->outstanding) return SF_OK;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    // the model stream runs the batches in order: the last recorded "done" event covers all of them
+    const uint32_t last = (uint32_t)((t->n_batches - 1) & 1u);
+    SF_CUDA(cudaStreamWaitEvent((cudaStream_t)stream, t->ev_done[last], 0));
+    return SF_OK;
+}
+
+extern "C" int sf_table_set_pipelined(sf_ctx* ctx, sf_table* t, int on)
+{
+    if (!ctx || !t) return SF_ERR_ARG;
+    SF_CUDA(cudaSetDevice(ctx->device));
+    if (!on) {
+        if (t->pipelined) { SF_CUDA(cudaStreamSynchronize(t->model_stream)); t->outstanding = false; }
+        t->pipelined = 0;
+        return SF_OK;
+    }
+    if (t->pipelined) return SF_OK;
+    if (!t->all2) {
+        const size_t S = t->d.n_slots;
+        size_t total = 0;
+        for (int k = 0; k < 6; k++) total += sf_align256((size_t)kMaxBatch * 4);
+        total += sf_align256((size_t)2 * kHistWords * 4) + sf_align256(S * 4);
+        cudaError_t e = cudaMalloc(&t->all2, total);
+        if (e != cudaSuccess) { sf_set_cuda_error(e, "cudaMalloc(table, second sort set)"); return SF_ERR_ALLOC; }
+        char* p = reinterpret_cast<char*>(t->all2);
+        sf_table::SortSet& s1 = t->set[1];
+        s1.key_a = carve<uint32_t>(p, kMaxBatch); s1.key_b = carve<uint32_t>(p, kMaxBatch);
+        s1.idx_a = carve<uint32_t>(p, kMaxBatch); s1.idx_b = carve<uint32_t>(p, kMaxBatch);
+        s1.run0 = carve<uint32_t>(p, kMaxBatch); s1.pkt_slot = carve<uint32_t>(p, kMaxBatch);
+        s1.hist = carve<uint32_t>(p, 2 * kHistWords);
+        s1.first = carve<uint32_t>(p, S);
+        SF_CUDA(cudaMemset(t->all2, 0, total));
+        SF_CUDA(cudaMemset(s1.first, 0xFF, S * 4));
+        SF_CUDA(cudaStreamCreateWithFlags(&t->model_stream, cudaStreamNonBlocking));
+        for (int k = 0; k < 2; k++) {
+            SF_CUDA(cudaEventCreateWithFlags(&t->ev_sorted[k], cudaEventDisableTiming));
+            SF_CUDA(cudaEventCreateWithFlags(&t->ev_done[k], cudaEventDisableTiming));
+        }
+    }
+    SF_CUDA(cudaDeviceSynchronize());                     // whatever ran the plain way so far is done
+    t->pipelined = 1;
+    t->n_batches = 0;
+    t->outstanding = false;
     return SF_OK;
 }
 
 extern "C" void sf_table_destroy(sf_table* t) {
     if (!t) return;
+    if (t->all2) {
+        cudaStreamSynchronize(t->model_stream);
+        for (int k = 0; k < 2; k++) { cudaEventDestroy(t->ev_sorted[k]); cudaEventDestroy(t->ev_done[k]); }
+        cudaStreamDestroy(t->model_stream);
+        cudaFree(t->all2);
+    }
     if (t->all) cudaFree(t->all);
     delete t;
 }
@@ -589,11 +658,19 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     if (slow->arch != SF_SLOW_MLP || cfg->wide_layout != SF_MLP16 || cfg->row_dtype != slow->dtype) return SF_ERR_UNSUPPORTED;
     if (cfg->P * 16 != slow->dims[0] || cfg->P < t->d.slow_pkts) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
-    cudaStream_t st = (cudaStream_t)stream;
+    cudaStream_t ss = (cudaStream_t)stream;                   // look-up and sort: the caller's stream
     const uint32_t n = batch->n;
-    if (zero_result) SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_batch_result), st));
+    if (zero_result) SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_batch_result), ss));
     if (n == 0) return SF_OK;
-    const TableDev& d = t->d;
+    // Pipelined: this batch uses sort set b & 1 and hands over to the table's stream for everything from apply1 on; the set (and
+    // its `first` array) is free again when the model phase of batch b - 2 has ended.
+    const bool pipe = t->pipelined != 0;
+    const uint32_t si = pipe ? (uint32_t)(t->n_batches & 1u) : 0u;
+    const sf_table::SortSet& S = t->set[si];
+    cudaStream_t st = pipe ? t->model_stream : ss;            // the model phase
+    if (pipe && t->n_batches >= 2) SF_CUDA(cudaStreamWaitEvent(ss, t->ev_done[si], 0));
+    TableDev d = t->d;
+    d.first = S.first;
     // workspace: features, probabilities, decisions, wide rows and slow-model scratch for at most n flows
     const size_t esz = slow->dtype == SF_BF16 ? 2 : 4;
     const uint32_t Cs = slow->dims[slow->n_layers];
@@ -608,22 +685,33 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     char* w = reinterpret_cast<char*>(sf_ws_alloc(ctx, off));
     if (!w) return SF_ERR_ALLOC;
     sf_time_new_record(ctx);
-    sf_time_begin(ctx, SF_T_TABLE, st);
-    SF_CUDA(cudaMemsetAsync(t->counts, 0, (16 + 2 * kHistWords) * sizeof(uint32_t), st));
+    sf_time_begin(ctx, SF_T_TABLE, ss);
+    if (!pipe) {
+        SF_CUDA(cudaMemsetAsync(t->counts, 0, (16 + 2 * kHistWords) * sizeof(uint32_t), ss));     // fire counts and digit counts lie together
+    } else {
+        SF_CUDA(cudaMemsetAsync(S.hist, 0, 2 * kHistWords * sizeof(uint32_t), ss));
+    }
     const uint32_t blocks = (n + 255) / 256;
-    probe_kernel<<<blocks, 256, 0, st>>>(d, *batch, t->pkt_slot, result_dev, ctx->d_state);
+    probe_kernel<<<blocks, 256, 0, ss>>>(d, *batch, S.pkt_slot, result_dev, ctx->d_state);
     SF_LAUNCH_CHECK("probe_kernel");
     const uint32_t nblk = (n + kTile - 1) / kTile;
     // from here on every kernel of the batch is a chained launch (set up while its predecessor drains)
-    SF_CUDA(sf_launch_chained(key_kernel, blocks, 256, 0, st, d, t->pkt_slot, n, t->key_a, t->idx_a, t->hist));
+    SF_CUDA(sf_launch_chained(key_kernel, blocks, 256, 0, ss, d, S.pkt_slot, n, S.key_a, S.idx_a, S.hist));
     {
         // 16-bit keys: two 8-bit passes, ping-ponging between the two buffers, end in (key_a, idx_a)
-        SF_CUDA(sf_launch_chained(radix8_scatter_kernel, nblk, 256, 0, st, t->key_a, t->idx_a, t->key_b, t->idx_b, n, 0u, t->hist, nblk,
-                                  t->hist + kHistWords, (uint32_t*)nullptr));
-        SF_CUDA(sf_launch_chained(radix8_scatter_kernel, nblk, 256, 0, st, t->key_b, t->idx_b, t->key_a, t->idx_a, n, 8u, t->hist + kHistWords, nblk,
-                                  (uint32_t*)nullptr, t->run0));
+        SF_CUDA(sf_launch_chained(radix8_scatter_kernel, nblk, 256, 0, ss, S.key_a, S.idx_a, S.key_b, S.idx_b, n, 0u, S.hist, nblk,
+                                  S.hist + kHistWords, (uint32_t*)nullptr));
+        SF_CUDA(sf_launch_chained(radix8_scatter_kernel, nblk, 256, 0, ss, S.key_b, S.idx_b, S.key_a, S.idx_a, n, 8u, S.hist + kHistWords, nblk,
+                                  (uint32_t*)nullptr, S.run0));
     }
-    SF_CUDA(sf_launch_chained(apply1_kernel, blocks, 256, 0, st, d, *batch, t->key_a, t->idx_a, t->run0, t->pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts));
+    if (pipe) {
+        SF_CUDA(cudaEventRecord(t->ev_sorted[si], ss));
+        SF_CUDA(cudaStreamWaitEvent(st, t->ev_sorted[si], 0));
+        SF_CUDA(cudaMemsetAsync(t->counts, 0, 16 * sizeof(uint32_t), st));                       // this batch's fire counts
+        t->n_batches++;
+        t->outstanding = true;
+    }
+    SF_CUDA(sf_launch_chained(apply1_kernel, blocks, 256, 0, st, d, *batch, S.key_a, S.idx_a, S.run0, S.pkt_slot, t->rank, t->pos, t->fire1_slot, t->counts));
     sf_time_end(ctx, SF_T_TABLE, st);
     // S1..S3 on the flows that just completed their fast context (count stays on the device); the feature kernel reads
     // their packets in place, through the list of their slots
@@ -646,7 +734,7 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     SF_CUDA(sf_launch_chained(fast_finish_kernel, std::min<uint32_t>((n * 16u + 255) / 256, (uint32_t)ctx->num_sms * 2u), 256, 0, st, d, t->fire1_slot,
                               t->counts, reinterpret_cast<const uint16_t*>(w + o_lidx), fo->d_leaf, fo->T, 1u << fo->depth, fo->C, cfg->tau,
                               result_dev, ctx->d_state));
-    SF_CUDA(sf_launch_chained(apply2_kernel, blocks, 256, 0, st, d, *batch, t->key_a, t->idx_a, t->pkt_slot, t->rank, t->pos, t->fire2_slab,
+    SF_CUDA(sf_launch_chained(apply2_kernel, blocks, 256, 0, st, d, *batch, S.key_a, S.idx_a, S.pkt_slot, t->rank, t->pos, t->fire2_slab,
                               t->fire2_slot, t->counts, result_dev, ctx->d_state));
     sf_time_end(ctx, SF_T_SCORE, st);
     // S4 on the flows that just completed their slow context
@@ -664,6 +752,7 @@ int ingest_chunk(sf_ctx* ctx, sf_table* t, const sf_pkt_batch* batch, const sf_f
     if (rc != SF_OK) return rc;
     SF_CUDA(sf_launch_chained(apply_slow_kernel, blocks, 256, 0, st, d, t->fire2_slot, t->counts, reinterpret_cast<const uint8_t*>(w + o_slab_lab),
                               result_dev, ctx->d_state));
+    if (pipe) SF_CUDA(cudaEventRecord(t->ev_done[si], st));
     return SF_OK;
 }
 }  // namespace
@@ -704,6 +793,8 @@ extern "C" int sf_table_ingest_host(sf_ctx* ctx, sf_table* t, const sf_pkt_batch
     sf_batch_result* res_dev = reinterpret_cast<sf_batch_result*>(sb + off[9]);
     int rc = sf_table_ingest(ctx, t, &bd, fo, F, slow, cfg, res_dev, stream);
     if (rc != SF_OK) return rc;
+    rc = sf_table_flush(ctx, t, stream);                                 // pipelined mode: the counts are complete after the model phase
+    if (rc != SF_OK) return rc;
     SF_CUDA(cudaMemcpyAsync(result_host_out, res_dev, sizeof(sf_batch_result), cudaMemcpyDeviceToHost, st));
     SF_CUDA(cudaStreamSynchronize(st));
     return SF_OK;
@@ -722,6 +813,7 @@ extern "C" int sf_table_sweep(sf_ctx* ctx, sf_table* t, uint32_t now, uint32_t i
     if (!ctx || !t || !result_dev) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
     cudaStream_t st = (cudaStream_t)stream;
+    { const int rcf = sf_table_flush(ctx, t, stream); if (rcf != SF_OK) return rcf; }
     SF_CUDA(cudaMemsetAsync(result_dev, 0, sizeof(sf_sweep_result), st));
     sweep_kernel<<<(t->d.n_slots + 255) / 256, 256, 0, st>>>(t->d, now, idle_timeout, rearm, result_dev);
     SF_LAUNCH_CHECK("sweep_kernel");
@@ -734,6 +826,7 @@ extern "C" int sf_table_lookup(sf_ctx* ctx, const sf_table* t, const sf_key* key
     if (!ctx || !t || (n && (!keys_dev || !out_dev))) return SF_ERR_ARG;
     SF_CUDA(cudaSetDevice(ctx->device));
     if (n == 0) return SF_OK;
+    { const int rcf = sf_table_flush(ctx, const_cast<sf_table*>(t), stream); if (rcf != SF_OK) return rcf; }
     lookup_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(t->d, keys_dev, n, out_dev);
     SF_LAUNCH_CHECK("lookup_kernel");
     return SF_OK;

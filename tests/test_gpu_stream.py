@@ -31,7 +31,21 @@ def _models(F, T, depth, C, dims, seed):
     return forest, tau, flowgen.gen_mlp(seed, dims)
 
 
-def _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg, host=False):
+def _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg, host=False, pipelined=False):
+    if pipelined:
+        # every batch enqueued back to back (its own planes and its own counts, alive until the flush), one flush at the end
+        keep, results = [], []
+        for b in batches:
+            d = {k: hz.dev(b[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
+            pb = sf.make_pkt_batch(d["src"], d["dst"], d["sport"], d["dport"], d["proto"], d["dir"], d["size"], d["iat_us"], d["hdr"])
+            r = torch.zeros(8, dtype=torch.int32, device="cuda")
+            sf.sf_table_ingest(ctx, table, pb, forest_h, F, slow_h, rcfg, r)
+            keep.append((d, pb)); results.append(r)
+        sf.sf_table_flush(ctx, table)
+        torch.cuda.synchronize()
+        tot = sum(r.cpu().numpy().astype(np.int64) for r in results)
+        names = ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision", "missed")
+        return dict(zip(names, tot[:7].tolist()))
     totals = np.zeros(8, np.int64)
     res = torch.zeros(8, dtype=torch.int32, device="cuda")
     names8 = ("n_new_flows", "n_fast_fired", "n_fast_done", "n_escalated", "n_slow_fired", "n_dropped_after_decision", "n_missed")
@@ -62,11 +76,13 @@ def _lookup(sf, hz, ctx, table, keys):
     return out.cpu().numpy().reshape(-1).view(sf.FLOW_RESULT_DTYPE)
 
 
-@pytest.mark.parametrize("shape", ["config5_models", "small_models", "odd_models", "small_models_host"])
+@pytest.mark.parametrize("shape", ["config5_models", "small_models", "odd_models", "small_models_host", "config5_models_pipelined",
+                                   "small_models_pipelined"])
 def test_stream_matches_sequential_reference(env, shape):
     sf, hz, ctx = env
     host = shape.endswith("_host")
-    shape = shape.replace("_host", "")
+    pipelined = shape.endswith("_pipelined")         # look-up + sort of batch b+1 overlap the model work of batch b: same results
+    shape = shape.replace("_host", "").replace("_pipelined", "")
     if shape == "config5_models":       # config 2's forest on 8 packets, config 2's MLP on 64 packets padded to 128
         F, T, depth, C, dims, P_model = 48, 100, 12, 8, (2048, 1024, 1024, 1024, 8), 128
         n_keys, n_batches, m = 1500, 24, 4096
@@ -88,7 +104,9 @@ def test_stream_matches_sequential_reference(env, shape):
     table = sf.sf_table_create(ctx, 13, fast_pkts, slow_pkts, n_keys)
     rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
     sf.sf_ctx_poll(ctx, reset=True)
-    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg, host=host)
+    if pipelined:
+        sf.sf_table_set_pipelined(ctx, table, True)
+    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, F, slow_h, rcfg, host=host, pipelined=pipelined)
     c = sf.sf_ctx_poll(ctx, reset=True)
     assert got["missed"] == 0 and c.device_error == 0
     for k in ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision"):
@@ -203,7 +221,8 @@ def test_stream_config5_full_size(env):
     table = sf.sf_table_create(ctx, 25, fast_pkts, slow_pkts, 1 << 18)
     rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
     sf.sf_ctx_poll(ctx, reset=True)
-    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, cfg.F, slow_h, rcfg)
+    sf.sf_table_set_pipelined(ctx, table, True)          # as bench.py ingests it: batches back to back, one flush at the end
+    got = _ingest_all(sf, hz, ctx, table, batches, forest_h, cfg.F, slow_h, rcfg, pipelined=True)
     c = sf.sf_ctx_poll(ctx, reset=True)
     assert got["missed"] == 0 and c.device_error == 0
     for k in exp:
@@ -271,18 +290,24 @@ def test_table_needs_a_slow_context_longer_than_the_fast_one(env):
 
 
 # ---- table lifecycle: idle timeout, slot and slab reuse, re-arming ----
-def _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg):
+def _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg, pipelined=False):
     names = ("new_flows", "fast_fired", "fast_done", "escalated", "slow_fired", "dropped_after_decision", "missed")
     totals = np.zeros(8, np.int64)
     sweeps = []
     res = torch.zeros(8, dtype=torch.int32, device="cuda")
     sw = torch.zeros(8, dtype=torch.int32, device="cuda")
+    keep, results = [], []
     for ev in events:
         if ev[0] == "batch":
             b = ev[1]
             sf.sf_table_set_time(table, ev[2])
             d = {k: hz.dev(b[k]) for k in ("src", "dst", "sport", "dport", "proto", "dir", "size", "iat_us", "hdr")}
             pb = sf.make_pkt_batch(d["src"], d["dst"], d["sport"], d["dport"], d["proto"], d["dir"], d["size"], d["iat_us"], d["hdr"])
+            if pipelined:          # no wait between batches: planes and counts stay alive until the table has been flushed
+                r = torch.zeros(8, dtype=torch.int32, device="cuda")
+                sf.sf_table_ingest(ctx, table, pb, forest_h, F, slow_h, rcfg, r)
+                keep.append((d, pb)); results.append(r)
+                continue
             sf.sf_table_ingest(ctx, table, pb, forest_h, F, slow_h, rcfg, res)
             torch.cuda.synchronize()
             totals += res.cpu().numpy().astype(np.int64)
@@ -290,11 +315,16 @@ def _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg):
             sf.sf_table_sweep(ctx, table, ev[1], ev[2], ev[3], sw)
             torch.cuda.synchronize()
             sweeps.append(dict(zip(sf.SWEEP_FIELDS, sw.cpu().numpy()[:5].tolist())))
+    if pipelined:
+        sf.sf_table_flush(ctx, table)
+        torch.cuda.synchronize()
+        for r in results:
+            totals += r.cpu().numpy().astype(np.int64)
     return dict(zip(names, totals[:7].tolist())), sweeps
 
 
-@pytest.mark.parametrize("rearm", [False, True])
-def test_lifecycle_matches_sequential_reference(env, rearm):
+@pytest.mark.parametrize("rearm,pipelined", [(False, False), (True, False), (True, True)])
+def test_lifecycle_matches_sequential_reference(env, rearm, pipelined):
     from oracle.lifecycle import simulate_lifecycle
     sf, hz, ctx = env
     F, T, depth, C, dims, P_model, fast_pkts, slow_pkts = 24, 16, 8, 4, (1024, 256, 4), 64, 8, 64
@@ -321,7 +351,9 @@ def test_lifecycle_matches_sequential_reference(env, rearm):
     table = sf.sf_table_create(ctx, 11, fast_pkts, slow_pkts, 600)
     rcfg = sf.make_route_cfg(sf.SF_LC_GT, hz.dev(tau), sf.SF_MLP16, sf.SF_BF16, P_model, 0, P_real=slow_pkts)
     sf.sf_ctx_poll(ctx, reset=True)
-    got, got_sweeps = _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg)
+    if pipelined:
+        sf.sf_table_set_pipelined(ctx, table, True)
+    got, got_sweeps = _run_events(sf, hz, ctx, table, events, forest_h, F, slow_h, rcfg, pipelined=pipelined)
     c = sf.sf_ctx_poll(ctx, reset=True)
     assert got["missed"] == 0 and c.device_error == 0
     assert tot["escalated"] > 600                      # more assignments than slabs: returned slabs were used again
